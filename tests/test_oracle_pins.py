@@ -1,0 +1,461 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+Nothing here touches the GPU library.  Each test is chosen so that a plausible
+mistake in the oracle (dropped term, wrong sign or index, transposed operand,
+floor instead of round) makes it fail.
+"""
+import itertools
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+from ivit_inputs import ExpParams, Scale, make_config
+from ivit_inputs.gen import dyadic
+from oracle import api as O
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "paper_constants.txt")
+
+
+def golden():
+    out = {}
+    for line in open(GOLDEN):
+        line = line.split("#")[0].split()
+        if len(line) == 2:
+            out[line[0]] = float(line[1])
+    return out
+
+
+# ---------------------------------------------------------------- requantisation (Sec. 3.2)
+
+def exact_round_half_up(a, m, s):
+    return math.floor(Fraction(a * m, 2 ** s) + Fraction(1, 2))
+
+
+def test_rq_equals_exact_rational_rounding_exhaustive():
+    rng = np.random.default_rng(1)
+    pairs = [(2 ** 30, 31), (2 ** 31 - 1, 31), (2 ** 30, 32), (2 ** 31 - 1, 33), (2 ** 30 + 1, 40), (1, 1), (3, 2)]
+    for s in (31, 32, 33, 35, 38, 40, 45, 62):
+        for _ in range(8):
+            pairs.append((int(rng.integers(2 ** 30, 2 ** 31)), s))
+    assert len(pairs) >= 64
+    a = np.arange(-4096, 4097, dtype=np.int64)
+    for m, s in pairs:
+        got = O.rq_array(a, m, s)
+        want = np.array([exact_round_half_up(int(x), m, s) for x in a], dtype=np.int64)
+        assert np.array_equal(got, want), (m, s)
+
+
+def test_rq_ties_and_large_accumulators():
+    # ratio 1/2: ties go up (+0.5 -> 1, -0.5 -> 0)
+    assert O.rq(1, 2 ** 30, 31) == 1 and O.rq(-1, 2 ** 30, 31) == 0
+    assert O.rq(3, 2 ** 30, 31) == 2 and O.rq(-3, 2 ** 30, 31) == -1
+    rng = np.random.default_rng(2)
+    for _ in range(2000):
+        a = int(rng.integers(-2 ** 31 + 1, 2 ** 31))
+        m = int(rng.integers(2 ** 30, 2 ** 31))
+        s = int(rng.integers(31, 63))
+        assert O.rq(a, m, s) == exact_round_half_up(a, m, s)
+
+
+def test_dyadic_from_double_is_normalised_and_close():
+    rng = np.random.default_rng(3)
+    for r in list(np.exp(rng.uniform(math.log(1e-6), math.log(0.9), 300))) + [0.5, 0.25, 1.0 / 3, 0.9999999999]:
+        m, s = O.dyadic_from_double(float(r))
+        assert 2 ** 30 <= m < 2 ** 31
+        assert abs(m / 2 ** s - r) <= r * 2.0 ** -31
+        assert (m, s) == dyadic(float(r))      # the input generator's own conversion agrees
+
+
+# ---------------------------------------------------------------- ShiftExp (Algorithm 1)
+
+def test_log2e_shift_constant():
+    g = golden()
+    # for multiples of 16 no floor is involved: Ip = I * (1.0111)b exactly
+    for I0 in (7, 16, 100):
+        for I in range(-240, 1, 16):
+            Ip = I * 23 // 16
+            assert I * 23 % 16 == 0 and Ip == int(I * g["log2e_shift_value"])
+            # ShiftExp(I) must equal the value built from Ip by hand
+            q, r = divmod(-Ip, I0)
+            Ib = I0 - (r + 1) // 2
+            assert O.shiftexp(I, I0, 20) == (Ib << 20) >> q
+    assert abs(g["log2e_shift_value"] - math.log2(math.e)) / math.log2(math.e) < 0.0037
+
+
+def test_shiftexp_anchor_and_exact_powers():
+    for I0 in (1, 5, 11, 16, 23, 255, 1000):
+        for N in (0, 15, 23):
+            assert O.shiftexp(0, I0, N) == I0 << N
+    # choose I with Ip = -q*I0 exactly: I = -16 j gives Ip = -23 j; with I0 = 23, q = j
+    for j in range(0, 15):
+        assert O.shiftexp(-16 * j, 23, 15) == (23 << 15) >> j
+    # q > N: keeps flooring, reaches 0
+    assert O.shiftexp(-16 * 14, 23, 3) == (23 << 3) >> 14 == 0
+
+
+def test_shiftexp_monotone_and_positive_range():
+    for I0 in range(1, 256):
+        v = [O.shiftexp(I, I0, 15) for I in range(-255, 1)]
+        assert all(b >= a for a, b in zip(v, v[1:])), I0
+        assert v[-1] == I0 << 15 and min(v) >= 0
+
+
+def test_linear_exp_closed_form_error_bound():
+    """2^x ~ 1 + x/2 on (-1, 0]: sup relative error 2/(e ln2) - 1 at x = 1/ln2 - 2 (Eq. (linear))."""
+    g = golden()
+    bound = 2.0 / (math.e * math.log(2.0)) - 1.0
+    assert abs(bound - g["linear_exp_max_rel_err"]) < 1e-6
+    I0, N = 1 << 15, 15
+    worst, at = 0.0, None
+    for I in range(-3 * I0, 1, 7):
+        Ip = I + (I >> 1) - (I >> 4)
+        q, r = divmod(-Ip, I0)
+        approx = O.shiftexp(I, I0, N) / float(I0 << N)
+        exact = 2.0 ** (Ip / I0)
+        rel = abs(approx - exact) / exact
+        assert rel <= 0.0615 + 2.0 ** q / I0     # floor of the final shift costs < 1 unit
+        if q == 0 and rel > worst:
+            worst, at = rel, -(r / I0)
+    assert abs(worst - bound) < 2e-4             # the bound is attained ...
+    assert abs(at - (1.0 / math.log(2.0) - 2.0)) < 5e-3   # ... where the closed form says
+    # exact at both ends of the interval
+    assert O.shiftexp(0, I0, N) == I0 << N
+
+
+@pytest.mark.parametrize("I0,bound", [(5, 0.24), (11, 0.16), (16, 0.145), (20, 0.14), (64, 0.085), (181, 0.07)])
+def test_shiftexp_vs_exp(I0, bound):
+    worst = 0.0
+    for I in range(-255, 1):
+        x = I / I0
+        if x > -13.8:
+            e = O.shiftexp(I, I0, 30) / float(I0 << 30)
+            worst = max(worst, abs(e - math.exp(x)) / math.exp(x))
+    assert worst <= bound
+
+
+# ---------------------------------------------------------------- IntDiv (Eq. (IntDiv))
+
+def test_intdiv_against_exact_quotient():
+    rng = np.random.default_rng(4)
+    for _ in range(3000):
+        I2 = int(rng.integers(1, 2 ** 32))
+        I1 = int(rng.integers(0, I2 + 1))
+        got = O.intdiv(I1, I2, 45, 8)
+        assert got == ((2 ** 45 // I2) * I1) >> 38
+        exact = Fraction(I1 * 128, I2)
+        assert exact - 1 - Fraction(I1, 2 ** 38) <= got <= exact
+    assert O.intdiv(5, 0, 45, 8) == 0
+
+
+# ---------------------------------------------------------------- Shiftmax (Algorithm 1)
+
+def float_softmax(x):
+    e = np.exp(x - x.max(axis=1, keepdims=True))
+    return e / e.sum(axis=1, keepdims=True)
+
+
+@pytest.mark.parametrize("I0", [7, 13, 20])
+def test_shiftmax_brute_force_vs_float_softmax(I0):
+    p = ExpParams(I0, 15)
+    vals = list(range(-24, 25, 3))
+    for d in (2, 3, 4):
+        rows = np.array(list(itertools.product(vals, repeat=d)), dtype=np.int8)
+        out = O.shiftmax(rows, p)
+        err = np.abs(out.astype(np.float64) / 128.0 - float_softmax(rows.astype(np.float64) / I0)).max()
+        assert err <= 0.04, (d, err)
+        s = out.astype(np.int64).sum(axis=1)
+        assert s.min() >= 128 - d and s.max() <= 128
+
+
+def test_shiftmax_invariants_random_rows():
+    rng = np.random.default_rng(5)
+    for d, I0 in [(197, 11), (197, 23), (577, 11), (577, 17), (49, 16), (64, 12)]:
+        rows = np.clip(np.rint(rng.standard_normal((64, d)) * 32), -128, 127).astype(np.int8)
+        p = ExpParams(I0, 15)
+        out = O.shiftmax(rows, p)
+        assert out.min() >= 0 and out.max() <= 127
+        s = out.astype(np.int64).sum(axis=1)
+        assert (s <= 128).all() and (s >= 128 - d).all()
+        err = np.abs(out.astype(np.float64) / 128.0 - float_softmax(rows.astype(np.float64) / I0)).max()
+        assert err <= 0.025
+        # the largest input gets the largest output
+        assert (out[np.arange(64), rows.argmax(axis=1)] == out.max(axis=1)).all()
+        # shift invariance and permutation equivariance
+        narrow = np.clip(rows, -100, 100)
+        assert np.array_equal(O.shiftmax((narrow.astype(np.int64) - 27).astype(np.int8), p), O.shiftmax(narrow, p))
+        perm = rng.permutation(d)
+        assert np.array_equal(O.shiftmax(rows[:, perm], p), out[:, perm])
+
+
+def test_shiftmax_special_rows():
+    for I0 in (11, 16):
+        p = ExpParams(I0, 15)
+        assert O.shiftmax(np.array([[42]], dtype=np.int8), p)[0, 0] == 127     # would be 2^(k-1): clamped
+        for d in (2, 3, 4, 7, 49):
+            o = O.shiftmax(np.full((1, d), -3, dtype=np.int8), p)[0]
+            assert (o == o[0]).all() and o[0] in (128 // d, 128 // d - 1)
+        # one dominant entry takes (almost) everything
+        row = np.full((1, 50), -128, dtype=np.int8)
+        row[0, 17] = 127
+        o = O.shiftmax(row, p)[0]
+        assert o[17] == 127 and o.sum() == 127
+
+
+def test_shiftmax_int32_input_equals_requant_then_int8():
+    rng = np.random.default_rng(6)
+    acc = rng.integers(-40000, 40000, size=(37, 53)).astype(np.int32)
+    bias = rng.integers(-5000, 5000, size=(37, 53)).astype(np.int32)
+    pre = Scale(*dyadic(30.0 / 8192))
+    p = ExpParams(13, 15)
+    x8 = np.array([[max(-128, min(127, exact_round_half_up(int(a) + int(b), pre.mult, pre.shift)))
+                    for a, b in zip(ra, rb)] for ra, rb in zip(acc, bias)], dtype=np.int8)
+    assert np.array_equal(O.shiftmax(acc, p, pre=pre, bias32=bias), O.shiftmax(x8, p))
+
+
+# ---------------------------------------------------------------- ShiftGELU (Algorithm 2)
+
+def test_gelu_shift_constant():
+    g = golden()
+    assert abs(g["gelu_shift_value"] - g["gelu_sigmoid_coeff"]) / g["gelu_sigmoid_coeff"] < 0.0086
+    # I multiple of 16: I_p = 27 I / 16 exactly; checked through the operator's output
+    p = ExpParams(32, 23)
+    post = Scale(2 ** 30, 37)      # 1/128
+    for x in range(-128, 128, 16):
+        row = np.array([[x, 112]], dtype=np.int8)
+        Ip, mx = x * 27 // 16, 112 * 27 // 16
+        e, e1 = O.shiftexp(Ip - mx, 32, 23), O.shiftexp(-mx, 32, 23)
+        div = O.intdiv(e, e + e1, 45, 8)
+        assert O.shiftgelu(row, p, post)[0, 0] == max(-128, min(127, exact_round_half_up(x * div, 2 ** 30, 37)))
+
+
+@pytest.mark.parametrize("I0", [29, 32, 37])
+def test_shiftgelu_brute_force_vs_float_gelu(I0):
+    p = ExpParams(I0, 23)
+    post = Scale(2 ** 30, 30 - 4)            # ratio 1/16: out = x*div/16 would saturate, so measure div through rows
+    worst_erf = worst_sig = 0.0
+    for mxv in (127, 90, 40, 5):
+        xs = np.arange(-128, mxv + 1)
+        # out = sat8(rq(x*div; 1/128 * c)) loses resolution; use the unit ratio on x*div/128 via two runs:
+        row = np.concatenate([xs, [mxv]]).astype(np.int8)[None, :]
+        # ratio 1/128 gives the int8 GELU in input units; compare in real units with +-0.5 step slack
+        out = O.shiftgelu(row, p, Scale(2 ** 30, 37))[0, :-1].astype(np.float64)
+        xr = xs / I0
+        g_erf = xr * 0.5 * (1.0 + np.vectorize(math.erf)(xr / math.sqrt(2.0)))
+        g_sig = xr / (1.0 + np.exp(-1.702 * xr))
+        worst_erf = max(worst_erf, np.abs(out / I0 - g_erf).max())
+        worst_sig = max(worst_sig, np.abs(out / I0 - g_sig).max())
+    half_step = 0.5 / I0
+    assert worst_erf <= 0.05 + half_step, worst_erf
+    assert worst_sig <= 0.035 + half_step, worst_sig
+    del post
+
+
+def test_shiftgelu_invariants():
+    rng = np.random.default_rng(7)
+    p = ExpParams(31, 23)
+    post = Scale(*dyadic(1.0 / (128 * 0.9)))
+    x = np.clip(np.rint(rng.standard_normal((32, 300)) * 31), -128, 127).astype(np.int8)
+    out = O.shiftgelu(x, p, post).astype(np.int64)
+    xs = x.astype(np.int64)
+    assert ((np.sign(out) == np.sign(xs)) | (out == 0)).all()
+    assert (np.abs(out) <= np.abs(xs) / 0.9 + 1).all()
+    # large positive inputs pass through (sigmoid -> 1), large negative ones vanish
+    big = xs >= 100
+    assert (out[big] >= np.minimum(127, xs[big] / 0.9 - 3)).all()
+    assert (out[xs <= -100] == 0).all()
+    # an all-negative row uses max = 0 (both exponents stay non-positive)
+    neg = -np.abs(x) - 1
+    o2 = O.shiftgelu(neg.astype(np.int8), p, post)
+    assert (o2 <= 0).all() and (o2 >= -8).all()
+
+
+# ---------------------------------------------------------------- integer square root (Sec. 3.5)
+
+def test_isqrt_equals_floor_sqrt_below_2_24():
+    n = np.arange(0, 1 << 24, dtype=np.int64)
+    got = O.isqrt_array(n)
+    want = np.floor(np.sqrt(n.astype(np.float64))).astype(np.int64)
+    want -= (want * want > n)
+    want += ((want + 1) * (want + 1) <= n)
+    assert np.array_equal(got, want)
+
+
+def test_isqrt_large_values_and_squares():
+    rng = np.random.default_rng(8)
+    vals = [int(v) for v in rng.integers(0, 2 ** 62, 20000)]
+    vals += [k * k for k in (1, 2, 3, 46340, 2 ** 20, 2 ** 30 - 1)] + [k * k - 1 for k in (2, 3, 4, 46341, 2 ** 20, 2 ** 30)]
+    for n in vals:
+        assert O.isqrt(n) == math.isqrt(n), n
+
+
+def test_isqrt_iteration_as_printed_oscillates():
+    """Ten unguarded iterations end one too high for n = k^2 - 1; the guarded reading does not."""
+    bad = [n for n in (3, 15, 63, 255) if O.isqrt_as_printed(n) != math.isqrt(n)]
+    assert bad, "the unguarded iteration was expected to overshoot for some n = k^2 - 1"
+    for n in (3, 15, 63, 255):
+        assert O.isqrt(n) == math.isqrt(n)
+
+
+# ---------------------------------------------------------------- I-LayerNorm (Sec. 3.5)
+
+@pytest.mark.parametrize("C", [96, 192, 384, 1024])
+def test_layernorm_vs_float(C):
+    rng = np.random.default_rng(9)
+    for sigma in (8, 20, 35):
+        x = np.clip(np.rint(rng.standard_normal((16, C)) * sigma + rng.integers(-20, 20, (16, 1))), -128, 127).astype(np.int8)
+        # unit affine: gamma*target = 32 int8 steps per sigma, beta = 0
+        ratios = np.full(C, 32.0 * math.sqrt(C) / 2.0 ** 20)
+        ms = [dyadic(r) for r in ratios]
+        scale = Scale(np.array([m for m, _ in ms], np.int32), np.array([s for _, s in ms], np.uint8))
+        out = O.layernorm(x, scale, np.zeros(C, np.int32)).astype(np.float64) / 32.0
+        xf = x.astype(np.float64)
+        ref = (xf - xf.mean(1, keepdims=True)) / xf.std(1, keepdims=True)
+        keep = np.abs(ref) < 3.9            # away from int8 saturation
+        srow = xf.std(1, keepdims=True)
+        err = np.abs(out - ref) / 1.0
+        tol = 0.5 / srow + 0.03 + 0.5 / 32.0
+        assert (err[keep] <= np.broadcast_to(tol, err.shape)[keep]).all(), (C, sigma, err[keep].max())
+
+
+def test_layernorm_affine_constant_row_and_int32():
+    rng = np.random.default_rng(10)
+    C = 48
+    ms = [dyadic(r) for r in rng.uniform(2e-4, 6e-4, C)]
+    scale = Scale(np.array([m for m, _ in ms], np.int32), np.array([s for _, s in ms], np.uint8))
+    beta = rng.integers(-20, 20, C).astype(np.int32)
+    const = np.full((2, C), 17, dtype=np.int8)
+    assert np.array_equal(O.layernorm(const, scale, beta), np.broadcast_to(beta.astype(np.int8), (2, C)))
+    # hand computation of one row in Python integers
+    x = rng.integers(-128, 128, (1, C)).astype(np.int8)
+    xs = [int(v) for v in x[0]]
+    S1 = sum(xs)
+    mu = (2 * S1 + C) // (2 * C)
+    V = sum((v - mu) ** 2 for v in xs)
+    F = 2 ** 20 // math.isqrt(V)
+    want = [max(-128, min(127, exact_round_half_up((v - mu) * F, int(scale.mult[i]), int(scale.shift[i])) + int(beta[i])))
+            for i, v in enumerate(xs)]
+    assert O.layernorm(x, scale, beta)[0].tolist() == want
+    assert abs(sum(v - mu for v in xs)) <= C / 2
+    # int32 input path computes the same thing
+    assert np.array_equal(O.layernorm(x.astype(np.int32), scale, beta), O.layernorm(x, scale, beta))
+    # scaling the row by 8 only coarsens the reciprocal F by 8: the result moves by at most one step
+    o = O.layernorm(x.astype(np.int32) * 8, scale, beta)
+    assert np.abs(o.astype(int) - np.array(want)).max() <= 1
+
+
+# ---------------------------------------------------------------- Dense / MatMul (Sec. 3.2)
+
+def test_linear_vs_numpy_and_exact_requant():
+    rng = np.random.default_rng(11)
+    M, N, K = 23, 17, 40
+    A = rng.integers(-128, 128, (M, K)).astype(np.int8)
+    W = rng.integers(-127, 128, (N, K)).astype(np.int8)
+    bias = rng.integers(-3000, 3000, N).astype(np.int32)
+    ms = [dyadic(r) for r in rng.uniform(5e-4, 3e-3, N)]
+    scale = Scale(np.array([m for m, _ in ms], np.int32), np.array([s for _, s in ms], np.uint8))
+    res = rng.integers(-128, 128, (5, N)).astype(np.int8)
+    rs = Scale(*dyadic(0.9))
+    acc = A.astype(np.int64) @ W.astype(np.int64).T + bias[None, :]
+    want = np.empty((M, N), np.int64)
+    for r in range(M):
+        for c in range(N):
+            want[r, c] = exact_round_half_up(int(acc[r, c]), int(scale.mult[c]), int(scale.shift[c])) + \
+                exact_round_half_up(int(res[r % 5, c]), rs.mult, rs.shift)
+    got = O.linear(A, W, bias, scale, res=res, res_scale=rs, res_rows=5)
+    assert np.array_equal(got, np.clip(want, -128, 127).astype(np.int8))
+    got32 = O.linear(A, W, bias, scale, res=res, res_scale=rs, res_rows=5, out_dtype=O.I32)
+    assert np.array_equal(got32, want.astype(np.int32))
+    # output row grouping: rows land at (r // g) * stride + r % g
+    buf = np.full((40, N), 77, dtype=np.int8)
+    O.linear(A[:20], W, bias, scale, out=buf[1:], out_group_rows=4, out_group_stride=7)
+    plain = O.linear(A[:20], W, bias, scale)
+    for r in range(20):
+        assert np.array_equal(buf[1 + (r // 4) * 7 + r % 4], plain[r])
+    untouched = sorted(set(range(40)) - {1 + (r // 4) * 7 + r % 4 for r in range(20)})
+    assert (buf[untouched] == 77).all()
+
+
+def test_matmul_vs_numpy_both_operand_orders():
+    rng = np.random.default_rng(12)
+    nb, Ma, Nb, K = 5, 9, 11, 13
+    A = rng.integers(-128, 128, (nb, Ma, K)).astype(np.int8)
+    Bt = rng.integers(-128, 128, (nb, Nb, K)).astype(np.int8)
+    bias = rng.integers(-2000, 2000, (2, Ma, Nb)).astype(np.int32)
+    sc = Scale(*dyadic(1.0 / 300))
+    acc = np.einsum("bik,bjk->bij", A.astype(np.int64), Bt.astype(np.int64))
+    acc_b = acc + bias[np.arange(nb) % 2]
+    want = np.vectorize(lambda a: max(-128, min(127, exact_round_half_up(int(a), sc.mult, sc.shift))))(acc_b)
+    assert np.array_equal(O.matmul(A, Bt, True, sc, bias32=bias), want.astype(np.int8))
+    Bn = np.ascontiguousarray(Bt.transpose(0, 2, 1))
+    want2 = np.vectorize(lambda a: max(-128, min(127, exact_round_half_up(int(a), sc.mult, sc.shift))))(acc)
+    assert np.array_equal(O.matmul(A, Bn, False, sc), want2.astype(np.int8))
+
+
+# ---------------------------------------------------------------- data movement helpers
+
+def test_patchify_gather_token_mean():
+    rng = np.random.default_rng(13)
+    img = rng.integers(-128, 128, (2, 3, 16, 16)).astype(np.int8)
+    P = 4
+    want = img.reshape(2, 3, 4, P, 4, P).transpose(0, 2, 4, 1, 3, 5).reshape(2 * 16, 3 * P * P)
+    assert np.array_equal(O.patchify(img, P), want)
+    # window-major order, window of 2x2 patches
+    w = O.patchify(img, P, window=2)
+    grid = want.reshape(2, 4, 4, -1)
+    wm = grid.reshape(2, 2, 2, 2, 2, -1).transpose(0, 1, 3, 2, 4, 5).reshape(32, -1)
+    assert np.array_equal(w, wm)
+    idx = rng.integers(0, 32, 50).astype(np.int32)
+    assert np.array_equal(O.gather_rows(want, idx), want[idx])
+    sc = Scale(*dyadic(3.0 / 16))
+    tm = O.token_mean(want, 16, sc)
+    s = want.reshape(2, 16, -1).astype(np.int64).sum(1)
+    ref = np.vectorize(lambda a: max(-128, min(127, exact_round_half_up(int(a), sc.mult, sc.shift))))(s)
+    assert np.array_equal(tm, ref.astype(np.int8))
+
+
+# ---------------------------------------------------------------- block composition (Sec. 3.1)
+
+def test_block_equals_composition_of_ops():
+    blk, X = make_config(0)
+    D, T, h = blk.D, blk.T, blk.heads
+    d = D // h
+    A = O.layernorm(X, blk.ln1_gamma, blk.ln1_beta, blk.M_ln)
+    QKV = O.linear(A, blk.Wqkv, blk.bqkv, blk.qkv_scale)
+    Q = QKV[:, :D].reshape(T, h, d).transpose(1, 0, 2)
+    K = QKV[:, D:2 * D].reshape(T, h, d).transpose(1, 0, 2)
+    V = QKV[:, 2 * D:].reshape(T, h, d).transpose(1, 0, 2)
+    S = O.matmul(Q, K, True, blk.qk_scale)
+    P = O.shiftmax(S.reshape(-1, T), blk.smax).reshape(h, T, T)
+    Oh = O.matmul(P, V, False, blk.pv_scale).transpose(1, 0, 2).reshape(T, D)
+    assert np.array_equal(Oh, O.attention(blk, QKV))
+    Xh = O.linear(Oh, blk.Wo, blk.bo, blk.o_scale, res=X, res_scale=blk.res1_scale)
+    A2 = O.layernorm(Xh, blk.ln2_gamma, blk.ln2_beta, blk.M_ln)
+    G = O.linear(A2, blk.W1, blk.b1, blk.fc1_scale)
+    Hh = O.shiftgelu(G, blk.gelu, blk.gelu_post)
+    Y = O.linear(Hh, blk.W2, blk.b2, blk.fc2_scale, res=Xh, res_scale=blk.res2_scale)
+    assert np.array_equal(Y, O.block_forward(blk, X))
+    # the workload is not degenerate
+    assert 0.02 < (P > 0).mean() < 0.9 and 15 < Y.astype(float).std() < 40
+    assert (np.abs(Y.astype(int)) >= 127).mean() < 0.01 and (np.abs(QKV.astype(int)) >= 127).mean() < 0.01
+
+
+def test_block_tracks_float_shadow_model():
+    """The int8 block output follows a float64 forward of the same block (exact Softmax / GELU / LayerNorm)."""
+    from shadow import block_forward_float
+    blk, X = make_config(0)
+    Y = O.block_forward(blk, X).astype(np.float64)
+    Yf = block_forward_float(blk, X)
+    keep = np.abs(Yf) < 120
+    diff = (Y - Yf)[keep]
+    assert np.sqrt((diff ** 2).mean()) < 2.0
+    corr = np.corrcoef(Y[keep], Yf[keep])[0, 1]
+    assert corr > 0.995
+    # a wrong composition is caught: dropping the residual or swapping Q and K breaks the agreement
+    blk_bad, _ = make_config(0)
+    D = blk.D
+    blk_bad.Wqkv = np.concatenate([blk.Wqkv[D:2 * D], blk.Wqkv[:D], blk.Wqkv[2 * D:]])
+    Yb = block_forward_float(blk_bad, X)
+    assert np.sqrt(((Y - Yb)[keep] ** 2).mean()) > np.sqrt((diff ** 2).mean())
