@@ -1,0 +1,241 @@
+/*
+ * ivit.h - C ABI of the B200 (sm_100a) integer-only ViT encoder library.
+ *
+ * The library implements the integer pipeline of I-ViT ("Integer-only
+ * Quantization for Efficient Vision Transformer Inference"): INT8xINT8->INT32
+ * linear operations with dyadic requantisation (Sec. 3.2), Shiftmax
+ * (Sec. 3.3, Algorithm 1), ShiftGELU (Sec. 3.4, Algorithm 2), I-LayerNorm
+ * (Sec. 3.5) and their composition into an encoder block (Sec. 3.1).
+ * No floating point is used on the device.
+ *
+ * Conventions (all entry points unless stated otherwise)
+ *  - Every call returns IVIT_OK (0) or a negative IVIT_ERR_* code; nothing is
+ *    enqueued when a call fails argument validation.
+ *  - Tensor and parameter-array pointers are DEVICE pointers owned by the
+ *    caller.  The library allocates no memory per call; scratch comes from a
+ *    caller-provided workspace (ivit_*_workspace_bytes).  ivit_ctx_create
+ *    allocates a few hundred KB once (status word, ShiftGELU table cache).
+ *  - Work is enqueued on the CUDA stream held by the context; calls never
+ *    synchronise.  Device-side failures (a bounded wait that ran out) are
+ *    reported by ivit_ctx_poll_status after the stream has been synchronised.
+ *  - Matrices are row-major; leading dimensions (ld*) and strides are in
+ *    elements.  int8 tensors: pointer 16-byte aligned and ld a multiple of 16.
+ *    int32 tensors: pointer 16-byte aligned and ld a multiple of 4.  Otherwise
+ *    IVIT_ERR_ALIGNMENT.  A 197-wide int8 score matrix is therefore stored
+ *    with ld = 208.
+ *  - rq(a; m, s) = floor((a*m + 2^(s-1)) / 2^s) evaluated in 64 bits
+ *    (round-half-up dyadic requantisation, Sec. 3.2 Eq. (I_A)).
+ *    sat8(v) = min(127, max(-128, v)).
+ *  - For every input there is exactly one correct output (integer arithmetic).
+ */
+#ifndef IVIT_H
+#define IVIT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  IVIT_OK = 0,
+  IVIT_ERR_INVALID_ARG = -1,    /* null pointer, negative size, bad enum */
+  IVIT_ERR_ALIGNMENT = -2,      /* pointer or leading dimension not aligned as stated above */
+  IVIT_ERR_RANGE = -3,          /* a quantisation constant violates a stated bound */
+  IVIT_ERR_UNSUPPORTED = -4,    /* shape / dtype combination not built */
+  IVIT_ERR_WORKSPACE = -5,      /* workspace missing, misaligned or too small */
+  IVIT_ERR_CUDA = -6,           /* a CUDA runtime / driver call failed */
+  IVIT_ERR_DEVICE_TIMEOUT = -7  /* a bounded device-side wait ran out (see ivit_ctx_poll_status) */
+};
+
+enum { IVIT_I8 = 0, IVIT_I32 = 1 };
+
+typedef struct ivit_ctx ivit_ctx; /* opaque */
+
+/* Dyadic number b / 2^c of Sec. 3.2 (DN()).  Per-channel when mult_c != NULL:
+ * device arrays of one (mult, shift) per output channel.  Otherwise the
+ * per-tensor pair (mult, shift), passed by value.  Bounds: 0 < mult < 2^31,
+ * 1 <= shift <= 62 (per-channel arrays are checked by ivit_validate_scale at
+ * model-load time; kernels clamp the shift into range). */
+typedef struct {
+  const int32_t* mult_c;
+  const uint8_t* shift_c;
+  int32_t mult;
+  int32_t shift;
+} ivit_scale;
+
+/* Constants of Algorithm 1 / Algorithm 2: I0 = round(1 / S_in); N = the
+ * left pre-shift of ShiftExp (footnote of Algorithm 1); M = width of the
+ * reciprocal in Eq. (IntDiv); k_out = output bit width (only 8 is built).
+ * Bounds (IVIT_ERR_RANGE otherwise): 1 <= I0 <= 2^15, 0 <= N <= 24, M == 45,
+ * k_out == 8; Shiftmax: row_len * I0 * 2^N < 2^32 and I0 * 2^N >= 2^14;
+ * ShiftGELU: 2 * I0 * 2^N < 2^32. */
+typedef struct {
+  int32_t I0, N, M, k_out;
+} ivit_exp_params;
+
+/* ---- context ---- */
+
+/* Creates a context on `device` that enqueues on `cuda_stream` (a
+ * cudaStream_t; NULL = the legacy default stream).  Fails with IVIT_ERR_CUDA
+ * when no usable sm_100 device is present: there is no CPU fallback. */
+int ivit_ctx_create(ivit_ctx** ctx, int device, void* cuda_stream);
+int ivit_ctx_destroy(ivit_ctx* ctx);
+int ivit_ctx_set_stream(ivit_ctx* ctx, void* cuda_stream);
+/* Non-blocking: IVIT_OK, or the last device-side error recorded by a kernel
+ * of this context (cleared by the call). */
+int ivit_ctx_poll_status(ivit_ctx* ctx);
+/* Number of kernels this context has launched since creation. */
+int64_t ivit_ctx_launch_count(const ivit_ctx* ctx);
+/* Selects the GEMM engine: 0 = tcgen05 tensor-core kernels where the shape
+ * qualifies (default), 1 = force the CUDA-core (dp4a) kernels everywhere.
+ * Both are bit-exact; the switch exists for testing and measurement. */
+int ivit_ctx_set_gemm_engine(ivit_ctx* ctx, int engine);
+const char* ivit_strerror(int code);
+
+/* ---- Sec. 3.2: Dense layer with dyadic requantisation ----
+ *   acc        = sum_k A[r,k] * W[c,k] + (bias ? bias[c] : 0)          (int32)
+ *   v          = rq(acc; scale[c]) + (res ? rq(res[r % res_rows, c]; res_scale) : 0)
+ *   out[ro, c] = out_dtype == IVIT_I8 ? sat8(v) : v
+ *   ro         = out_group_rows > 0 ? (r / out_group_rows) * out_group_stride + r % out_group_rows : r
+ * A [M,K] int8, W [N,K] int8 (one row per output channel), bias int32 [N] or
+ * NULL, res int8 [res_rows, N] or NULL (res_scale per-tensor), out int8 or
+ * int32 [*, N].  K <= 65536 so the accumulator cannot overflow; K % 16 == 0.
+ * The output-row grouping lets the patch embedding write token rows 1..T-1 of
+ * every image directly. */
+int ivit_linear(ivit_ctx* ctx, const int8_t* A, int64_t lda, const int8_t* W, int64_t ldw,
+                const int32_t* bias, ivit_scale scale, const int8_t* res, int64_t ldres,
+                int64_t res_rows, ivit_scale res_scale, void* out, int64_t ldo, int32_t out_dtype,
+                int64_t out_group_rows, int64_t out_group_stride, int64_t M, int64_t N, int64_t K);
+
+/* ---- Sec. 3.2: batched MatMul with dyadic requantisation ----
+ * Batch b = bo * batches_inner + bi; operand bases are offset by
+ * bo * s?o + bi * s?i elements (two-level strides address one head of one
+ * image inside a [tokens, 3D] QKV tensor without a copy).
+ *   C_b = sat8( rq( A_b (Ma x K) * op(B_b) + bias32[b % bias_batches]; scale ) )
+ * transB != 0: B_b is [Nb, K] and C = A * B^T (scores Q K^T); transB == 0:
+ * B_b is [K, Nb] (attention times V).  bias32 int32 [bias_batches, Ma, ldbias]
+ * or NULL; scale per-tensor.  All offsets must keep 4-byte alignment
+ * (strides and ld multiples of 4); K arbitrary. */
+int ivit_matmul(ivit_ctx* ctx, const int8_t* A, int64_t lda, int64_t sAo, int64_t sAi,
+                const int8_t* B, int64_t ldb, int64_t sBo, int64_t sBi, int32_t transB,
+                const int32_t* bias32, int64_t ldbias, int64_t bias_batches, ivit_scale scale,
+                int8_t* C, int64_t ldc, int64_t sCo, int64_t sCi, int64_t batches_outer,
+                int64_t batches_inner, int64_t Ma, int64_t Nb, int64_t K);
+
+/* ---- Sec. 3.3, Algorithm 1: Shiftmax over each row ----
+ * in_dtype IVIT_I8: rows of int8 scores.  IVIT_I32: rows of int32
+ * accumulators, x8 = sat8(rq(in32 + bias32[row % bias_rows, :]; pre)) first
+ * (bias32 may be NULL), which is bit-identical to requantising to int8 and
+ * then calling the int8 form.  out int8 in [0, 127], scale 1/128
+ * (Eq. (IntDiv), S_out = 1/2^(k_out-1)).  Columns d .. roundup(d,16)-1 of out
+ * are written as 0.  1 <= d <= 8192. */
+int ivit_shiftmax(ivit_ctx* ctx, const void* in, int32_t in_dtype, int64_t ldin,
+                  const int32_t* bias32, int64_t ldbias, int64_t bias_rows, ivit_scale pre,
+                  ivit_exp_params p, int8_t* out, int64_t ldout, int64_t rows, int64_t d);
+
+/* ---- Sec. 3.4, Algorithm 2: ShiftGELU over each row, then requantisation ----
+ *   I_p = x + (x>>1) + (x>>3) + (x>>4); I_max = max(0, max_row I_p);
+ *   I_div = IntDiv(ShiftExp(I_p - I_max), ShiftExp(I_p - I_max) + ShiftExp(-I_max), k_out)
+ *   out = sat8( rq(x * I_div; post) )            (post per-tensor)
+ * in == out (in place) is allowed.  cols % 16 == 0, cols <= 16384. */
+int ivit_shiftgelu(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_params p,
+                   ivit_scale post, int8_t* out, int64_t ldout, int64_t rows, int64_t cols);
+
+/* ---- Sec. 3.5: I-LayerNorm over each row ----
+ *   mu = floor((2*sum x + C) / (2C)); y = x - mu; V = sum y^2;
+ *   sd = integer sqrt of V by Eq. (iterative) (10 guarded iterations);
+ *   F = sd ? floor(2^M_ln / sd) : 0;
+ *   out[c] = sat8( rq(y[c] * F; gamma_scale[c]) + beta[c] )
+ * gamma_scale per-channel or per-tensor; beta int32 [C] or NULL.
+ * in_dtype IVIT_I8, or IVIT_I32 with |x| <= 2^20.  8 <= M_ln <= 30.
+ * C % 4 == 0, C <= 16384. */
+int ivit_layernorm(ivit_ctx* ctx, const void* in, int32_t in_dtype, int64_t ldin,
+                   ivit_scale gamma_scale, const int32_t* beta, int32_t M_ln, int8_t* out,
+                   int64_t ldout, int64_t rows, int64_t C);
+
+/* ---- Sec. 3.1: one encoder block ----
+ *   X^ = MSA(LayerNorm(X)) + X ;  Y = MLP(LayerNorm(X^)) + X^
+ * with every arrow an int8 tensor: LN -> QKV Dense -> per head
+ * [Q K^T (+attn_bias) -> rq(qk_scale) -> sat8 -> Shiftmax -> P V -> rq(pv_scale) -> sat8]
+ * -> output Dense + rq(X; res1_scale) -> LN -> FC1 -> ShiftGELU -> FC2 + rq(X^; res2_scale).
+ * B images (or attention windows) of T tokens; D = heads * d, d % 16 == 0;
+ * H = MLP width.  Wqkv is [3D, D]: Q | K | V thirds, head-major inside each.
+ * attn_bias int32 [attn_bias_batches, T, T] (row stride T) or NULL; batch
+ * (b*heads + h) uses entry (b*heads + h) % attn_bias_batches. */
+typedef struct {
+  int64_t B, T, D, heads, H;
+  int32_t M_ln;
+  ivit_scale ln1_gamma; const int32_t* ln1_beta;
+  const int8_t* Wqkv; const int32_t* bqkv; ivit_scale qkv_scale;
+  ivit_scale qk_scale; const int32_t* attn_bias; int64_t attn_bias_batches;
+  ivit_exp_params smax; ivit_scale pv_scale;
+  const int8_t* Wo; const int32_t* bo; ivit_scale o_scale; ivit_scale res1_scale;
+  ivit_scale ln2_gamma; const int32_t* ln2_beta;
+  const int8_t* W1; const int32_t* b1; ivit_scale fc1_scale;
+  ivit_exp_params gelu; ivit_scale gelu_post;
+  const int8_t* W2; const int32_t* b2; ivit_scale fc2_scale; ivit_scale res2_scale;
+} ivit_block_params;
+
+size_t ivit_block_workspace_bytes(const ivit_block_params* p);
+/* X, Y: [B*T, D] int8 contiguous (ld = D); X == Y is not allowed.  workspace:
+ * device memory, 256-byte aligned, at least ivit_block_workspace_bytes(p). */
+int ivit_block_forward(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* X, int8_t* Y,
+                       void* workspace, size_t workspace_bytes);
+
+/* Attention core of the block alone (Sec. 3.1 MSA equation without the output
+ * projection): QKV [B*T, 3D] int8 -> O [B*T, D] int8, using the attention
+ * fields of p.  workspace as for ivit_block_forward. */
+int ivit_attention(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* QKV, int8_t* O,
+                   void* workspace, size_t workspace_bytes);
+
+/* ---- full ViT-family forward (patch embedding, class token, blocks, head) ----
+ * The paper does not describe these outer layers; they are Dense / LayerNorm
+ * instances of the operators above:  patches -> Dense(Wpe) + rq(pos) -> rows
+ * 1..T-1 of each image; row 0 = cls; depth blocks; LayerNorm of the class row;
+ * Dense(Whead) -> int32 logits rq(acc + b; head_scale) (not saturated). */
+typedef struct {
+  int64_t B, img, patch, T, D, depth, classes;   /* T = (img/patch)^2 + 1 */
+  const int8_t* Wpe; const int32_t* bpe; ivit_scale pe_scale;   /* [D, 3*patch*patch] */
+  const int8_t* pos; ivit_scale pos_scale;                      /* [T-1, D] */
+  const int8_t* cls;                                            /* [D] */
+  const ivit_block_params* blocks;                              /* HOST array of depth entries */
+  ivit_scale lnf_gamma; const int32_t* lnf_beta;
+  const int8_t* Whead; const int32_t* bhead; ivit_scale head_scale; /* [classes, D] */
+} ivit_vit_params;
+
+size_t ivit_vit_workspace_bytes(const ivit_vit_params* p);
+/* image [B,3,img,img] int8 -> logits [B, classes] int32 (ld = classes). */
+int ivit_vit_forward(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* image, int32_t* logits,
+                     void* workspace, size_t workspace_bytes);
+
+/* ---- data movement helpers (not in the paper; needed by the full models) ---- */
+
+/* img [B,C,Hi,Wi] int8 -> rows [B*(Hi/P)*(Wi/P), C*P*P], column order
+ * (c, py, px).  window > 0: rows of one image are emitted window-major. */
+int ivit_patchify(ivit_ctx* ctx, const int8_t* img, int64_t B, int64_t C, int64_t Hi, int64_t Wi,
+                  int64_t P, int64_t window, int8_t* out, int64_t ldout);
+/* dst[i, 0:width] = src[index[i], 0:width]; width % 16 == 0; index int32 on device. */
+int ivit_gather_rows(ivit_ctx* ctx, const int8_t* src, int64_t ldsrc, const int32_t* index,
+                     int64_t n_rows, int64_t width, int8_t* dst, int64_t lddst);
+/* dst[g * group_stride + 0:width] = src_row[0:width] for g < groups (class-token rows). */
+int ivit_fill_rows(ivit_ctx* ctx, const int8_t* src_row, int64_t width, int8_t* dst,
+                   int64_t group_stride, int64_t groups);
+/* out[g, c] = sat8( rq( sum_{t<T} in[g*T + t, c]; scale ) )  (token pooling, 1/T folded in scale) */
+int ivit_token_mean(ivit_ctx* ctx, const int8_t* in, int64_t ldin, int64_t groups, int64_t T,
+                    int64_t C, ivit_scale scale, int8_t* out, int64_t ldout);
+
+/* ---- host-only helpers (offline) ---- */
+
+/* Sec. 3.2, DN(): ratio > 0 -> mult in [2^30, 2^31), shift in [1, 62]. */
+int ivit_dyadic_from_double(double ratio, int32_t* mult, int32_t* shift);
+/* Checks the bounds listed at ivit_exp_params. */
+int ivit_validate_exp_params(ivit_exp_params p, int64_t row_len, int32_t is_gelu);
+/* Checks a HOST copy of a per-channel scale: 0 < mult, 1 <= shift <= 62. */
+int ivit_validate_scale(const int32_t* mult_host, const uint8_t* shift_host, int64_t n);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* IVIT_H */

@@ -1,0 +1,139 @@
+// Shared device helpers and the context of the integer-only ViT library (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/ivit.h"
+
+namespace ivit {
+
+constexpr int kGeluTableSlots = 16;
+constexpr int kGeluTableBytes = 128 * 256;  // [max(0,row max of x)] [x + 128] -> int8 output
+
+struct GeluKey {
+  int32_t I0, N, M, k_out, mult, shift;
+  bool operator==(const GeluKey& o) const {
+    return I0 == o.I0 && N == o.N && M == o.M && k_out == o.k_out && mult == o.mult && shift == o.shift;
+  }
+};
+
+}  // namespace ivit
+
+struct ivit_ctx {
+  int device;
+  cudaStream_t stream;
+  int* status_host;  // mapped pinned memory: kernels write the first device-side error here
+  int* status_dev;   // device view of the same word
+  int8_t* gelu_tables;  // kGeluTableSlots tables on the device
+  ivit::GeluKey gelu_keys[ivit::kGeluTableSlots];
+  int gelu_used;
+  int gelu_next;
+  int64_t launches;
+  int gemm_engine;
+  int sm_count;
+  void* tmap_encode;  // cuTensorMapEncodeTiled, resolved at context creation
+};
+
+namespace ivit {
+
+__device__ __forceinline__ int sat8(int v) { return max(-128, min(127, v)); }
+
+// Round-half-up dyadic requantisation, Sec. 3.2: floor((a*m + 2^(s-1)) / 2^s) in 64 bits.
+__device__ __forceinline__ int rq(int a, int m, int s) {
+  long long p = (long long)a * (long long)m + (1ll << (s - 1));
+  return (int)(p >> s);
+}
+
+// Same value, for a shift known to be >= 32 (the product's low word only feeds the carry).
+__device__ __forceinline__ int rq_hi(int a, int m, int s) {
+  long long p = (long long)a * (long long)m + (1ll << (s - 1));
+  return (int)(p >> 32) >> (s - 32);
+}
+
+__host__ __device__ __forceinline__ int clamp_shift(int s) { return s < 1 ? 1 : (s > 62 ? 62 : s); }
+
+struct ScaleDev {
+  const int32_t* mult_c;
+  const uint8_t* shift_c;
+  int mult;
+  int shift;
+  __device__ __forceinline__ int m(int c) const { return mult_c ? mult_c[c] : mult; }
+  __device__ __forceinline__ int s(int c) const { return clamp_shift(shift_c ? (int)shift_c[c] : shift); }
+};
+
+inline ScaleDev to_dev(const ivit_scale& s) { return ScaleDev{s.mult_c, s.shift_c, s.mult, s.shift}; }
+
+// Algorithm 1, function ShiftExp, for I <= 0 (32-bit: |I| < 2^15, I0 <= 2^15, N <= 24).
+__device__ __forceinline__ unsigned shiftexp(int I, int I0, int N) {
+  int Ip = I + (I >> 1) - (I >> 4);  // I * log2(e) as (1.0111)b; >> on int is arithmetic in CUDA
+  int negp = -Ip;                    // >= 0
+  int q = negp / I0;                 // floor(Ip / (-I0))
+  int r = negp - q * I0;             // 0 <= r < I0
+  int Ib = I0 - ((r + 1) >> 1);      // ((-r) >> 1) + I0
+  if (q <= N) return (unsigned)Ib << (N - q);
+  int sh = q - N;
+  return sh >= 31 ? 0u : ((unsigned)Ib >> sh);
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+inline bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3) == 0; }
+
+inline bool scale_ok(const ivit_scale& s) {
+  if (s.mult_c) return s.shift_c != nullptr;
+  return s.mult > 0 && s.shift >= 1 && s.shift <= 62;
+}
+
+inline int check_launch(ivit_ctx* ctx, int n = 1) {
+  ctx->launches += n;
+  return cudaGetLastError() == cudaSuccess ? IVIT_OK : IVIT_ERR_CUDA;
+}
+
+// launchers implemented in the kernel files ---------------------------------------------
+
+struct GemmEpilogue {
+  const int32_t* bias;       // [N] (linear) or nullptr
+  const int32_t* bias32;     // [bias_batches, Ma, ldbias] (matmul) or nullptr
+  int64_t ldbias, bias_batches;
+  ScaleDev scale;
+  const int8_t* res;
+  int64_t ldres, res_rows;
+  ScaleDev res_scale;
+  void* out;
+  int64_t ldo;
+  int out_dtype;
+  int64_t group_rows, group_stride;
+};
+
+struct GemmProblem {
+  const int8_t* A; int64_t lda, sAo, sAi;
+  const int8_t* B; int64_t ldb, sBo, sBi;
+  int transB;              // 1: B is [N,K]; 0: B is [K,N]
+  int64_t sCo, sCi;        // batch offsets of out (elements)
+  int64_t batches_outer, batches_inner;
+  int64_t M, N, K;
+  GemmEpilogue epi;
+};
+
+int launch_gemm_simt(ivit_ctx* ctx, const GemmProblem& g);
+// Returns IVIT_ERR_UNSUPPORTED when the shape does not qualify for the tensor-core kernel.
+int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g);
+int launch_gemm(ivit_ctx* ctx, const GemmProblem& g);
+
+int launch_layernorm(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, ScaleDev gs,
+                     const int32_t* beta, int M_ln, int8_t* out, int64_t ldout, int64_t rows, int64_t C);
+int launch_shiftmax(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, const int32_t* bias32,
+                    int64_t ldbias, int64_t bias_rows, ScaleDev pre, ivit_exp_params p, int8_t* out,
+                    int64_t ldout, int64_t rows, int64_t d);
+int launch_shiftgelu(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_params p, ivit_scale post,
+                     int8_t* out, int64_t ldout, int64_t rows, int64_t cols);
+int launch_patchify(ivit_ctx* ctx, const int8_t* img, int64_t B, int64_t C, int64_t Hi, int64_t Wi,
+                    int64_t P, int64_t window, int8_t* out, int64_t ldout);
+int launch_gather_rows(ivit_ctx* ctx, const int8_t* src, int64_t ldsrc, const int32_t* index,
+                       int64_t n_rows, int64_t width, int8_t* dst, int64_t lddst);
+int launch_fill_rows(ivit_ctx* ctx, const int8_t* src_row, int64_t width, int8_t* dst,
+                     int64_t group_stride, int64_t groups);
+int launch_token_mean(ivit_ctx* ctx, const int8_t* in, int64_t ldin, int64_t groups, int64_t T,
+                      int64_t C, ScaleDev scale, int8_t* out, int64_t ldout);
+
+}  // namespace ivit

@@ -1,0 +1,103 @@
+// Data-movement helpers around the encoder (patch extraction, row gathers, class-token rows,
+// token pooling).  Pure permutations / sums; none of them is described in the paper.
+#include "common.cuh"
+
+namespace ivit {
+
+// One thread per 4 output bytes (px .. px+3 of one patch row); P % 4 == 0.
+__global__ void patchify_kernel(const int8_t* __restrict__ img, int64_t B, int C, int Hi, int Wi, int P,
+                                int window, int8_t* __restrict__ out, int64_t ldout, int64_t total_words) {
+  const int gh = Hi / P, gw = Wi / P;
+  const int kw = C * P * P / 4;
+  for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total_words;
+       t += (int64_t)gridDim.x * blockDim.x) {
+    const int w = (int)(t % kw);
+    const int64_t prow = t / kw;  // raster patch index over the batch
+    const int gx = (int)(prow % gw), gy = (int)((prow / gw) % gh);
+    const int64_t b = prow / ((int64_t)gw * gh);
+    const int px = (w * 4) % P, py = ((w * 4) / P) % P, c = (w * 4) / (P * P);
+    const int v = __ldg(reinterpret_cast<const int*>(img + ((b * C + c) * Hi + gy * P + py) * (int64_t)Wi + gx * P + px));
+    int64_t row;
+    if (window > 0) {
+      const int wy = gy / window, wx = gx / window, iy = gy % window, ix = gx % window;
+      row = (int64_t)(wy * (gw / window) + wx) * window * window + iy * window + ix;
+    } else {
+      row = (int64_t)gy * gw + gx;
+    }
+    *reinterpret_cast<int*>(out + (b * gh * gw + row) * ldout + w * 4) = v;
+  }
+}
+
+__global__ void gather_rows_kernel(const int8_t* __restrict__ src, int64_t ldsrc, const int32_t* __restrict__ index,
+                                   int64_t n_rows, int vec_per_row, int8_t* __restrict__ dst, int64_t lddst) {
+  const int64_t total = n_rows * vec_per_row;
+  for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t r = t / vec_per_row;
+    const int v = (int)(t % vec_per_row);
+    const int4 x = __ldg(reinterpret_cast<const int4*>(src + (int64_t)__ldg(index + r) * ldsrc) + v);
+    reinterpret_cast<int4*>(dst + r * lddst)[v] = x;
+  }
+}
+
+__global__ void fill_rows_kernel(const int8_t* __restrict__ src_row, int vec_per_row, int8_t* __restrict__ dst,
+                                 int64_t group_stride, int64_t groups) {
+  const int64_t total = groups * vec_per_row;
+  for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t g = t / vec_per_row;
+    const int v = (int)(t % vec_per_row);
+    reinterpret_cast<int4*>(dst + g * group_stride)[v] = __ldg(reinterpret_cast<const int4*>(src_row) + v);
+  }
+}
+
+__global__ void token_mean_kernel(const int8_t* __restrict__ in, int64_t ldin, int64_t groups, int T, int C,
+                                  ScaleDev scale, int8_t* __restrict__ out, int64_t ldout) {
+  const int64_t total = groups * C;
+  for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t g = t / C;
+    const int c = (int)(t % C);
+    int s = 0;
+    for (int k = 0; k < T; ++k) s += __ldg(in + (g * T + k) * ldin + c);
+    out[g * ldout + c] = (int8_t)sat8(rq(s, scale.mult, clamp_shift(scale.shift)));
+  }
+}
+
+static int grid_for(ivit_ctx* ctx, int64_t items, int threads) {
+  int64_t want = (items + threads - 1) / threads;
+  const int64_t cap = (int64_t)ctx->sm_count * 16;
+  return (int)(want < cap ? (want < 1 ? 1 : want) : cap);
+}
+
+int launch_patchify(ivit_ctx* ctx, const int8_t* img, int64_t B, int64_t C, int64_t Hi, int64_t Wi,
+                    int64_t P, int64_t window, int8_t* out, int64_t ldout) {
+  const int64_t total = B * C * Hi * Wi / 4;
+  if (total == 0) return IVIT_OK;
+  patchify_kernel<<<grid_for(ctx, total, 256), 256, 0, ctx->stream>>>(img, B, (int)C, (int)Hi, (int)Wi, (int)P,
+                                                                       (int)window, out, ldout, total);
+  return check_launch(ctx);
+}
+
+int launch_gather_rows(ivit_ctx* ctx, const int8_t* src, int64_t ldsrc, const int32_t* index,
+                       int64_t n_rows, int64_t width, int8_t* dst, int64_t lddst) {
+  if (n_rows == 0) return IVIT_OK;
+  gather_rows_kernel<<<grid_for(ctx, n_rows * (width / 16), 256), 256, 0, ctx->stream>>>(
+      src, ldsrc, index, n_rows, (int)(width / 16), dst, lddst);
+  return check_launch(ctx);
+}
+
+int launch_fill_rows(ivit_ctx* ctx, const int8_t* src_row, int64_t width, int8_t* dst,
+                     int64_t group_stride, int64_t groups) {
+  if (groups == 0) return IVIT_OK;
+  fill_rows_kernel<<<grid_for(ctx, groups * (width / 16), 256), 256, 0, ctx->stream>>>(
+      src_row, (int)(width / 16), dst, group_stride, groups);
+  return check_launch(ctx);
+}
+
+int launch_token_mean(ivit_ctx* ctx, const int8_t* in, int64_t ldin, int64_t groups, int64_t T,
+                      int64_t C, ScaleDev scale, int8_t* out, int64_t ldout) {
+  if (groups == 0) return IVIT_OK;
+  token_mean_kernel<<<grid_for(ctx, groups * C, 256), 256, 0, ctx->stream>>>(in, ldin, groups, (int)T, (int)C,
+                                                                             scale, out, ldout);
+  return check_launch(ctx);
+}
+
+}  // namespace ivit

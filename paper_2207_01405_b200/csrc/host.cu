@@ -1,0 +1,487 @@
+// Host side of the C ABI: context, argument validation, operator entry points and the
+// composition of one encoder block / one ViT forward out of the kernels (Sec. 3.1).
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+
+using namespace ivit;
+
+namespace {
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+inline int64_t round16(int64_t v) { return (v + 15) / 16 * 16; }
+
+int check_exp(ivit_exp_params p, int64_t row_len, bool gelu) {
+  if (p.I0 < 1 || p.I0 > (1 << 15) || p.N < 0 || p.N > 24 || p.M != 45 || p.k_out != 8) return IVIT_ERR_RANGE;
+  const int64_t top = (int64_t)p.I0 << p.N;
+  if (gelu) {
+    if (2 * top > 4294967295LL) return IVIT_ERR_RANGE;
+  } else {
+    if (row_len * top > 4294967295LL || top < (1 << 14)) return IVIT_ERR_RANGE;
+  }
+  return IVIT_OK;
+}
+
+struct BlockWs {
+  size_t A, QKV, S, P, O, Xh, G, total;
+  int64_t ldS;
+};
+
+BlockWs block_ws(const ivit_block_params* p) {
+  BlockWs w;
+  const size_t M = (size_t)(p->B * p->T), D = (size_t)p->D, H = (size_t)p->H;
+  w.ldS = round16(p->T);
+  const size_t s_bytes = (size_t)(p->B * p->heads * p->T) * (size_t)w.ldS;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  w.A = take(M * D);
+  w.QKV = take(M * 3 * D);
+  w.S = take(s_bytes);
+  w.P = take(s_bytes);
+  w.O = take(M * D);
+  w.Xh = take(M * D);
+  w.G = take(M * H);
+  w.total = off;
+  return w;
+}
+
+int check_block(const ivit_block_params* p) {
+  if (!p || p->B < 0 || p->T < 1 || p->D < 16 || p->heads < 1 || p->H < 16) return IVIT_ERR_INVALID_ARG;
+  if (p->D % p->heads) return IVIT_ERR_INVALID_ARG;
+  const int64_t d = p->D / p->heads;
+  if (d % 16 || p->D % 16 || p->H % 16) return IVIT_ERR_UNSUPPORTED;
+  if (!p->Wqkv || !p->Wo || !p->W1 || !p->W2) return IVIT_ERR_INVALID_ARG;
+  if (p->M_ln < 8 || p->M_ln > 30) return IVIT_ERR_RANGE;
+  const ivit_scale* sc[] = {&p->ln1_gamma, &p->qkv_scale, &p->qk_scale, &p->pv_scale, &p->o_scale, &p->res1_scale,
+                            &p->ln2_gamma, &p->fc1_scale, &p->gelu_post, &p->fc2_scale, &p->res2_scale};
+  for (const ivit_scale* s : sc)
+    if (!scale_ok(*s)) return IVIT_ERR_RANGE;
+  if (p->qk_scale.mult_c || p->pv_scale.mult_c || p->res1_scale.mult_c || p->res2_scale.mult_c || p->gelu_post.mult_c)
+    return IVIT_ERR_INVALID_ARG;
+  if (p->attn_bias && p->attn_bias_batches < 1) return IVIT_ERR_INVALID_ARG;
+  int rc = check_exp(p->smax, p->T, false);
+  if (rc) return rc;
+  return check_exp(p->gelu, p->H, true);
+}
+
+GemmProblem linear_problem(const int8_t* A, int64_t lda, const int8_t* W, int64_t ldw, const int32_t* bias,
+                           ivit_scale scale, const int8_t* res, int64_t ldres, int64_t res_rows,
+                           ivit_scale res_scale, void* out, int64_t ldo, int out_dtype, int64_t group_rows,
+                           int64_t group_stride, int64_t M, int64_t N, int64_t K) {
+  GemmProblem g{};
+  g.A = A; g.lda = lda; g.B = W; g.ldb = ldw; g.transB = 1;
+  g.batches_outer = g.batches_inner = 1;
+  g.M = M; g.N = N; g.K = K;
+  g.epi.bias = bias;
+  g.epi.bias32 = nullptr; g.epi.ldbias = 0; g.epi.bias_batches = 1;
+  g.epi.scale = to_dev(scale);
+  g.epi.res = res; g.epi.ldres = ldres; g.epi.res_rows = res_rows < 1 ? 1 : res_rows;
+  g.epi.res_scale = to_dev(res_scale);
+  g.epi.out = out; g.epi.ldo = ldo; g.epi.out_dtype = out_dtype;
+  g.epi.group_rows = group_rows; g.epi.group_stride = group_stride;
+  return g;
+}
+
+int attention_impl(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* QKV, int8_t* O, char* ws, const BlockWs& w) {
+  const int64_t B = p->B, T = p->T, D = p->D, h = p->heads, d = D / h, ldq = 3 * D, ldS = w.ldS;
+  int8_t* S = reinterpret_cast<int8_t*>(ws + w.S);
+  int8_t* P = reinterpret_cast<int8_t*>(ws + w.P);
+  // scores: Q_i K_i^T (+ bias), requantised to int8; 1/sqrt(d) lives in qk_scale
+  GemmProblem qk{};
+  qk.A = QKV; qk.lda = ldq; qk.sAo = T * ldq; qk.sAi = d;
+  qk.B = QKV + D; qk.ldb = ldq; qk.sBo = T * ldq; qk.sBi = d; qk.transB = 1;
+  qk.sCo = h * T * ldS; qk.sCi = T * ldS;
+  qk.batches_outer = B; qk.batches_inner = h; qk.M = T; qk.N = T; qk.K = d;
+  qk.epi.bias32 = p->attn_bias; qk.epi.ldbias = T; qk.epi.bias_batches = p->attn_bias ? p->attn_bias_batches : 1;
+  qk.epi.scale = to_dev(p->qk_scale); qk.epi.res_rows = 1;
+  qk.epi.out = S; qk.epi.ldo = ldS; qk.epi.out_dtype = IVIT_I8;
+  int rc = launch_gemm(ctx, qk);
+  if (rc) return rc;
+  rc = launch_shiftmax(ctx, S, IVIT_I8, ldS, nullptr, 0, 1, ScaleDev{nullptr, nullptr, 1, 1}, p->smax, P, ldS, B * h * T, T);
+  if (rc) return rc;
+  // Attn_i = P_i V_i, heads concatenated along the feature dimension
+  GemmProblem pv{};
+  pv.A = P; pv.lda = ldS; pv.sAo = h * T * ldS; pv.sAi = T * ldS;
+  pv.B = QKV + 2 * D; pv.ldb = ldq; pv.sBo = T * ldq; pv.sBi = d; pv.transB = 0;
+  pv.sCo = T * D; pv.sCi = d;
+  pv.batches_outer = B; pv.batches_inner = h; pv.M = T; pv.N = d; pv.K = T;
+  pv.epi.bias_batches = 1; pv.epi.res_rows = 1;
+  pv.epi.scale = to_dev(p->pv_scale);
+  pv.epi.out = O; pv.epi.ldo = D; pv.epi.out_dtype = IVIT_I8;
+  return launch_gemm(ctx, pv);
+}
+
+int block_impl(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* X, int8_t* Y, char* ws) {
+  const BlockWs w = block_ws(p);
+  const int64_t M = p->B * p->T, D = p->D, H = p->H;
+  int8_t* A = reinterpret_cast<int8_t*>(ws + w.A);
+  int8_t* QKV = reinterpret_cast<int8_t*>(ws + w.QKV);
+  int8_t* O = reinterpret_cast<int8_t*>(ws + w.O);
+  int8_t* Xh = reinterpret_cast<int8_t*>(ws + w.Xh);
+  int8_t* G = reinterpret_cast<int8_t*>(ws + w.G);
+  const ivit_scale none{nullptr, nullptr, 1, 1};
+  int rc;
+  // X^ = MSA(LayerNorm(X)) + X
+  if ((rc = launch_layernorm(ctx, X, IVIT_I8, D, to_dev(p->ln1_gamma), p->ln1_beta, p->M_ln, A, D, M, D))) return rc;
+  if ((rc = launch_gemm(ctx, linear_problem(A, D, p->Wqkv, D, p->bqkv, p->qkv_scale, nullptr, 0, 1, none, QKV, 3 * D,
+                                            IVIT_I8, 0, 0, M, 3 * D, D)))) return rc;
+  if ((rc = attention_impl(ctx, p, QKV, O, ws, w))) return rc;
+  if ((rc = launch_gemm(ctx, linear_problem(O, D, p->Wo, D, p->bo, p->o_scale, X, D, M, p->res1_scale, Xh, D,
+                                            IVIT_I8, 0, 0, M, D, D)))) return rc;
+  // Y = MLP(LayerNorm(X^)) + X^
+  if ((rc = launch_layernorm(ctx, Xh, IVIT_I8, D, to_dev(p->ln2_gamma), p->ln2_beta, p->M_ln, A, D, M, D))) return rc;
+  if ((rc = launch_gemm(ctx, linear_problem(A, D, p->W1, D, p->b1, p->fc1_scale, nullptr, 0, 1, none, G, H, IVIT_I8,
+                                            0, 0, M, H, D)))) return rc;
+  if ((rc = launch_shiftgelu(ctx, G, H, p->gelu, p->gelu_post, G, H, M, H))) return rc;
+  return launch_gemm(ctx, linear_problem(G, H, p->W2, H, p->b2, p->fc2_scale, Xh, D, M, p->res2_scale, Y, D, IVIT_I8,
+                                         0, 0, M, D, H));
+}
+
+}  // namespace
+
+namespace ivit {
+int launch_gemm(ivit_ctx* ctx, const GemmProblem& g) {
+  if (ctx->gemm_engine == 0) {
+    const int rc = launch_gemm_tc(ctx, g);
+    if (rc != IVIT_ERR_UNSUPPORTED) return rc;
+  }
+  return launch_gemm_simt(ctx, g);
+}
+}  // namespace ivit
+
+extern "C" {
+
+const char* ivit_strerror(int code) {
+  switch (code) {
+    case IVIT_OK: return "ok";
+    case IVIT_ERR_INVALID_ARG: return "invalid argument";
+    case IVIT_ERR_ALIGNMENT: return "pointer or leading dimension not aligned";
+    case IVIT_ERR_RANGE: return "quantisation constant out of range";
+    case IVIT_ERR_UNSUPPORTED: return "shape or dtype combination not supported";
+    case IVIT_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case IVIT_ERR_CUDA: return "CUDA call failed";
+    case IVIT_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+    default: return "unknown error";
+  }
+}
+
+int ivit_ctx_create(ivit_ctx** out, int device, void* cuda_stream) {
+  if (!out) return IVIT_ERR_INVALID_ARG;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return IVIT_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return IVIT_ERR_CUDA;
+  if (prop.major != 10) return IVIT_ERR_CUDA;  // kernels are built for sm_100a only
+  if (cudaSetDevice(device) != cudaSuccess) return IVIT_ERR_CUDA;
+  ivit_ctx* c = new (std::nothrow) ivit_ctx();
+  if (!c) return IVIT_ERR_CUDA;
+  std::memset(c, 0, sizeof(*c));
+  c->device = device;
+  c->stream = (cudaStream_t)cuda_stream;
+  c->sm_count = prop.multiProcessorCount;
+  if (cudaHostAlloc((void**)&c->status_host, sizeof(int), cudaHostAllocMapped) != cudaSuccess) { delete c; return IVIT_ERR_CUDA; }
+  *c->status_host = 0;
+  if (cudaHostGetDevicePointer((void**)&c->status_dev, c->status_host, 0) != cudaSuccess ||
+      cudaMalloc((void**)&c->gelu_tables, (size_t)kGeluTableSlots * kGeluTableBytes) != cudaSuccess) {
+    cudaFreeHost(c->status_host);
+    delete c;
+    return IVIT_ERR_CUDA;
+  }
+  cudaDriverEntryPointQueryResult qres;
+  void* fn = nullptr;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess)
+    fn = nullptr;
+  c->tmap_encode = fn;
+  *out = c;
+  return IVIT_OK;
+}
+
+int ivit_ctx_destroy(ivit_ctx* ctx) {
+  if (!ctx) return IVIT_ERR_INVALID_ARG;
+  cudaSetDevice(ctx->device);
+  cudaFree(ctx->gelu_tables);
+  cudaFreeHost(ctx->status_host);
+  delete ctx;
+  return IVIT_OK;
+}
+
+int ivit_ctx_set_stream(ivit_ctx* ctx, void* cuda_stream) {
+  if (!ctx) return IVIT_ERR_INVALID_ARG;
+  ctx->stream = (cudaStream_t)cuda_stream;
+  ctx->gelu_used = 0;  // tables were built in the order of the old stream
+  ctx->gelu_next = 0;
+  return IVIT_OK;
+}
+
+int ivit_ctx_poll_status(ivit_ctx* ctx) {
+  if (!ctx) return IVIT_ERR_INVALID_ARG;
+  volatile int* s = ctx->status_host;
+  const int v = *s;
+  if (v != 0) { *s = 0; return v; }
+  return IVIT_OK;
+}
+
+int64_t ivit_ctx_launch_count(const ivit_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int ivit_ctx_set_gemm_engine(ivit_ctx* ctx, int engine) {
+  if (!ctx || engine < 0 || engine > 1) return IVIT_ERR_INVALID_ARG;
+  ctx->gemm_engine = engine;
+  return IVIT_OK;
+}
+
+int ivit_linear(ivit_ctx* ctx, const int8_t* A, int64_t lda, const int8_t* W, int64_t ldw,
+                const int32_t* bias, ivit_scale scale, const int8_t* res, int64_t ldres,
+                int64_t res_rows, ivit_scale res_scale, void* out, int64_t ldo, int32_t out_dtype,
+                int64_t out_group_rows, int64_t out_group_stride, int64_t M, int64_t N, int64_t K) {
+  if (!ctx || !A || !W || !out || M < 0 || N < 1 || K < 1) return IVIT_ERR_INVALID_ARG;
+  if (out_dtype != IVIT_I8 && out_dtype != IVIT_I32) return IVIT_ERR_INVALID_ARG;
+  if (K > 65536) return IVIT_ERR_RANGE;
+  if (K % 16) return IVIT_ERR_UNSUPPORTED;
+  if (lda < K || ldw < K || ldo < N) return IVIT_ERR_INVALID_ARG;
+  if (!aligned16(A) || !aligned16(W) || !aligned16(out) || lda % 16 || ldw % 16) return IVIT_ERR_ALIGNMENT;
+  if (ldo % (out_dtype == IVIT_I8 ? 16 : 4)) return IVIT_ERR_ALIGNMENT;
+  if (bias && !aligned16(bias)) return IVIT_ERR_ALIGNMENT;
+  if (!scale_ok(scale)) return IVIT_ERR_RANGE;
+  if (res) {
+    if (!scale_ok(res_scale) || res_scale.mult_c) return IVIT_ERR_RANGE;
+    if (res_rows < 1 || ldres < N) return IVIT_ERR_INVALID_ARG;
+    if (!aligned16(res) || ldres % 16) return IVIT_ERR_ALIGNMENT;
+  }
+  if (out_group_rows > 0 && out_group_stride < out_group_rows) return IVIT_ERR_INVALID_ARG;
+  return launch_gemm(ctx, linear_problem(A, lda, W, ldw, bias, scale, res, ldres, res_rows, res_scale, out, ldo,
+                                         out_dtype, out_group_rows, out_group_stride, M, N, K));
+}
+
+int ivit_matmul(ivit_ctx* ctx, const int8_t* A, int64_t lda, int64_t sAo, int64_t sAi,
+                const int8_t* B, int64_t ldb, int64_t sBo, int64_t sBi, int32_t transB,
+                const int32_t* bias32, int64_t ldbias, int64_t bias_batches, ivit_scale scale,
+                int8_t* C, int64_t ldc, int64_t sCo, int64_t sCi, int64_t batches_outer,
+                int64_t batches_inner, int64_t Ma, int64_t Nb, int64_t K) {
+  if (!ctx || !A || !B || !C || Ma < 0 || Nb < 0 || K < 1 || batches_outer < 0 || batches_inner < 1)
+    return IVIT_ERR_INVALID_ARG;
+  if (K > 65536) return IVIT_ERR_RANGE;
+  if (!scale_ok(scale) || scale.mult_c) return IVIT_ERR_RANGE;
+  if (bias32 && (bias_batches < 1 || ldbias < Nb)) return IVIT_ERR_INVALID_ARG;
+  if (!aligned4(A) || !aligned4(B) || !aligned4(C)) return IVIT_ERR_ALIGNMENT;
+  const int64_t strides[] = {lda, sAo, sAi, ldb, sBo, sBi, ldc, sCo, sCi};
+  for (int64_t s : strides)
+    if (s % 4) return IVIT_ERR_ALIGNMENT;
+  if (lda < K || ldc < Nb || ldb < (transB ? K : Nb)) return IVIT_ERR_INVALID_ARG;
+  GemmProblem g{};
+  g.A = A; g.lda = lda; g.sAo = sAo; g.sAi = sAi;
+  g.B = B; g.ldb = ldb; g.sBo = sBo; g.sBi = sBi; g.transB = transB ? 1 : 0;
+  g.sCo = sCo; g.sCi = sCi; g.batches_outer = batches_outer; g.batches_inner = batches_inner;
+  g.M = Ma; g.N = Nb; g.K = K;
+  g.epi.bias32 = bias32; g.epi.ldbias = ldbias; g.epi.bias_batches = bias32 ? bias_batches : 1;
+  g.epi.scale = to_dev(scale); g.epi.res_rows = 1;
+  g.epi.out = C; g.epi.ldo = ldc; g.epi.out_dtype = IVIT_I8;
+  return launch_gemm(ctx, g);
+}
+
+int ivit_shiftmax(ivit_ctx* ctx, const void* in, int32_t in_dtype, int64_t ldin,
+                  const int32_t* bias32, int64_t ldbias, int64_t bias_rows, ivit_scale pre,
+                  ivit_exp_params p, int8_t* out, int64_t ldout, int64_t rows, int64_t d) {
+  if (!ctx || !in || !out || rows < 0 || d < 1) return IVIT_ERR_INVALID_ARG;
+  if (in_dtype != IVIT_I8 && in_dtype != IVIT_I32) return IVIT_ERR_INVALID_ARG;
+  if (d > 8192) return IVIT_ERR_UNSUPPORTED;
+  if (ldin < d || ldout < round16(d)) return IVIT_ERR_INVALID_ARG;
+  if (!aligned16(in) || !aligned16(out) || ldout % 16 || ldin % (in_dtype == IVIT_I8 ? 16 : 4)) return IVIT_ERR_ALIGNMENT;
+  int rc = check_exp(p, d, false);
+  if (rc) return rc;
+  if (in_dtype == IVIT_I32) {
+    if (!scale_ok(pre) || pre.mult_c) return IVIT_ERR_RANGE;
+    if (bias32 && (bias_rows < 1 || ldbias < d)) return IVIT_ERR_INVALID_ARG;
+    if (bias32 && (!aligned16(bias32) || ldbias % 4)) return IVIT_ERR_ALIGNMENT;
+  }
+  return launch_shiftmax(ctx, in, in_dtype, ldin, bias32, ldbias, bias_rows, to_dev(pre), p, out, ldout, rows, d);
+}
+
+int ivit_shiftgelu(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_params p,
+                   ivit_scale post, int8_t* out, int64_t ldout, int64_t rows, int64_t cols) {
+  if (!ctx || !in || !out || rows < 0 || cols < 1) return IVIT_ERR_INVALID_ARG;
+  if (cols % 16 || cols > 16384) return IVIT_ERR_UNSUPPORTED;
+  if (ldin < cols || ldout < cols) return IVIT_ERR_INVALID_ARG;
+  if (!aligned16(in) || !aligned16(out) || ldin % 16 || ldout % 16) return IVIT_ERR_ALIGNMENT;
+  if (!scale_ok(post) || post.mult_c) return IVIT_ERR_RANGE;
+  int rc = check_exp(p, cols, true);
+  if (rc) return rc;
+  return launch_shiftgelu(ctx, in, ldin, p, post, out, ldout, rows, cols);
+}
+
+int ivit_layernorm(ivit_ctx* ctx, const void* in, int32_t in_dtype, int64_t ldin,
+                   ivit_scale gamma_scale, const int32_t* beta, int32_t M_ln, int8_t* out,
+                   int64_t ldout, int64_t rows, int64_t C) {
+  if (!ctx || !in || !out || rows < 0 || C < 1) return IVIT_ERR_INVALID_ARG;
+  if (in_dtype != IVIT_I8 && in_dtype != IVIT_I32) return IVIT_ERR_INVALID_ARG;
+  if (C % 4 || C > 16384) return IVIT_ERR_UNSUPPORTED;
+  if (M_ln < 8 || M_ln > 30) return IVIT_ERR_RANGE;
+  if (ldin < C || ldout < C) return IVIT_ERR_INVALID_ARG;
+  if (!aligned16(in) || !aligned16(out) || ldout % 16 || ldin % (in_dtype == IVIT_I8 ? 16 : 4)) return IVIT_ERR_ALIGNMENT;
+  if (!scale_ok(gamma_scale)) return IVIT_ERR_RANGE;
+  return launch_layernorm(ctx, in, in_dtype, ldin, to_dev(gamma_scale), beta, M_ln, out, ldout, rows, C);
+}
+
+size_t ivit_block_workspace_bytes(const ivit_block_params* p) {
+  if (check_block(p) != IVIT_OK) return 0;
+  return block_ws(p).total;
+}
+
+int ivit_block_forward(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* X, int8_t* Y,
+                       void* workspace, size_t workspace_bytes) {
+  if (!ctx || !X || !Y || X == Y) return IVIT_ERR_INVALID_ARG;
+  int rc = check_block(p);
+  if (rc) return rc;
+  if (!aligned16(X) || !aligned16(Y)) return IVIT_ERR_ALIGNMENT;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < block_ws(p).total)
+    return IVIT_ERR_WORKSPACE;
+  return block_impl(ctx, p, X, Y, static_cast<char*>(workspace));
+}
+
+int ivit_attention(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* QKV, int8_t* O,
+                   void* workspace, size_t workspace_bytes) {
+  if (!ctx || !QKV || !O) return IVIT_ERR_INVALID_ARG;
+  int rc = check_block(p);
+  if (rc) return rc;
+  if (!aligned16(QKV) || !aligned16(O)) return IVIT_ERR_ALIGNMENT;
+  const BlockWs w = block_ws(p);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < w.total) return IVIT_ERR_WORKSPACE;
+  return attention_impl(ctx, p, QKV, O, static_cast<char*>(workspace), w);
+}
+
+static int check_vit(const ivit_vit_params* p) {
+  if (!p || p->B < 0 || p->depth < 1 || !p->blocks || p->patch < 4 || p->patch % 4 || p->img % p->patch) return IVIT_ERR_INVALID_ARG;
+  const int64_t g = p->img / p->patch;
+  if (p->T != g * g + 1 || p->D % 16 || p->classes < 1) return IVIT_ERR_INVALID_ARG;
+  if (!p->Wpe || !p->pos || !p->cls || !p->Whead) return IVIT_ERR_INVALID_ARG;
+  if (!scale_ok(p->pe_scale) || !scale_ok(p->pos_scale) || p->pos_scale.mult_c || !scale_ok(p->lnf_gamma) || !scale_ok(p->head_scale))
+    return IVIT_ERR_RANGE;
+  for (int64_t l = 0; l < p->depth; ++l) {
+    const ivit_block_params* b = &p->blocks[l];
+    int rc = check_block(b);
+    if (rc) return rc;
+    if (b->B != p->B || b->T != p->T || b->D != p->D) return IVIT_ERR_INVALID_ARG;
+  }
+  return IVIT_OK;
+}
+
+struct VitWs { size_t patches, X, Y, Z, block, total; };
+static VitWs vit_ws(const ivit_vit_params* p) {
+  VitWs w;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  const size_t Kpe = (size_t)(3 * p->patch * p->patch);
+  w.patches = take((size_t)(p->B * (p->T - 1)) * Kpe);
+  w.X = take((size_t)(p->B * p->T * p->D));
+  w.Y = take((size_t)(p->B * p->T * p->D));
+  w.Z = take((size_t)(p->B * p->D));
+  size_t blk = 0;
+  for (int64_t l = 0; l < p->depth; ++l) {
+    const size_t b = block_ws(&p->blocks[l]).total;
+    blk = b > blk ? b : blk;
+  }
+  w.block = take(blk);
+  w.total = off;
+  return w;
+}
+
+size_t ivit_vit_workspace_bytes(const ivit_vit_params* p) {
+  if (check_vit(p) != IVIT_OK) return 0;
+  return vit_ws(p).total;
+}
+
+int ivit_vit_forward(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* image, int32_t* logits,
+                     void* workspace, size_t workspace_bytes) {
+  if (!ctx || !image || !logits) return IVIT_ERR_INVALID_ARG;
+  int rc = check_vit(p);
+  if (rc) return rc;
+  if (!aligned16(image) || !aligned16(logits) || p->classes % 4) return IVIT_ERR_ALIGNMENT;
+  const VitWs w = vit_ws(p);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < w.total) return IVIT_ERR_WORKSPACE;
+  char* ws = static_cast<char*>(workspace);
+  const int64_t B = p->B, T = p->T, D = p->D, np = T - 1, Kpe = 3 * p->patch * p->patch;
+  int8_t* patches = reinterpret_cast<int8_t*>(ws + w.patches);
+  int8_t* X = reinterpret_cast<int8_t*>(ws + w.X);
+  int8_t* Y = reinterpret_cast<int8_t*>(ws + w.Y);
+  int8_t* Z = reinterpret_cast<int8_t*>(ws + w.Z);
+  const ivit_scale none{nullptr, nullptr, 1, 1};
+  if ((rc = launch_patchify(ctx, image, B, 3, p->img, p->img, p->patch, 0, patches, Kpe))) return rc;
+  // patch embedding as a Dense layer; the position embedding enters through the residual port;
+  // patch q of image b lands in token row b*T + 1 + q
+  if ((rc = launch_gemm(ctx, linear_problem(patches, Kpe, p->Wpe, Kpe, p->bpe, p->pe_scale, p->pos, D, np,
+                                            p->pos_scale, X + D, D, IVIT_I8, np, T, B * np, D, Kpe)))) return rc;
+  if ((rc = launch_fill_rows(ctx, p->cls, D, X, T * D, B))) return rc;
+  for (int64_t l = 0; l < p->depth; ++l) {
+    if ((rc = block_impl(ctx, &p->blocks[l], X, Y, ws + w.block))) return rc;
+    int8_t* t = X; X = Y; Y = t;
+  }
+  // final LayerNorm on the class-token rows, then the classifier (int32 logits, not saturated)
+  if ((rc = launch_layernorm(ctx, X, IVIT_I8, T * D, to_dev(p->lnf_gamma), p->lnf_beta, p->blocks[0].M_ln, Z, D, B, D))) return rc;
+  return launch_gemm(ctx, linear_problem(Z, D, p->Whead, D, p->bhead, p->head_scale, nullptr, 0, 1, none, logits,
+                                         p->classes, IVIT_I32, 0, 0, B, p->classes, D));
+}
+
+int ivit_patchify(ivit_ctx* ctx, const int8_t* img, int64_t B, int64_t C, int64_t Hi, int64_t Wi,
+                  int64_t P, int64_t window, int8_t* out, int64_t ldout) {
+  if (!ctx || !img || !out || B < 0 || C < 1 || P < 1) return IVIT_ERR_INVALID_ARG;
+  if (P % 4 || Hi % P || Wi % P) return IVIT_ERR_UNSUPPORTED;
+  if (window > 0 && ((Hi / P) % window || (Wi / P) % window)) return IVIT_ERR_INVALID_ARG;
+  if (ldout < C * P * P) return IVIT_ERR_INVALID_ARG;
+  if (!aligned16(img) || !aligned16(out) || ldout % 4 || Wi % 4) return IVIT_ERR_ALIGNMENT;
+  return launch_patchify(ctx, img, B, C, Hi, Wi, P, window, out, ldout);
+}
+
+int ivit_gather_rows(ivit_ctx* ctx, const int8_t* src, int64_t ldsrc, const int32_t* index,
+                     int64_t n_rows, int64_t width, int8_t* dst, int64_t lddst) {
+  if (!ctx || !src || !index || !dst || n_rows < 0 || width < 1) return IVIT_ERR_INVALID_ARG;
+  if (width % 16) return IVIT_ERR_UNSUPPORTED;
+  if (!aligned16(src) || !aligned16(dst) || ldsrc % 16 || lddst % 16) return IVIT_ERR_ALIGNMENT;
+  return launch_gather_rows(ctx, src, ldsrc, index, n_rows, width, dst, lddst);
+}
+
+int ivit_fill_rows(ivit_ctx* ctx, const int8_t* src_row, int64_t width, int8_t* dst,
+                   int64_t group_stride, int64_t groups) {
+  if (!ctx || !src_row || !dst || groups < 0 || width < 1) return IVIT_ERR_INVALID_ARG;
+  if (width % 16) return IVIT_ERR_UNSUPPORTED;
+  if (!aligned16(src_row) || !aligned16(dst) || group_stride % 16) return IVIT_ERR_ALIGNMENT;
+  return launch_fill_rows(ctx, src_row, width, dst, group_stride, groups);
+}
+
+int ivit_token_mean(ivit_ctx* ctx, const int8_t* in, int64_t ldin, int64_t groups, int64_t T,
+                    int64_t C, ivit_scale scale, int8_t* out, int64_t ldout) {
+  if (!ctx || !in || !out || groups < 0 || T < 1 || C < 1) return IVIT_ERR_INVALID_ARG;
+  if (!scale_ok(scale) || scale.mult_c) return IVIT_ERR_RANGE;
+  if (T > (1 << 23)) return IVIT_ERR_RANGE;
+  return launch_token_mean(ctx, in, ldin, groups, T, C, to_dev(scale), out, ldout);
+}
+
+int ivit_dyadic_from_double(double ratio, int32_t* mult, int32_t* shift) {
+  if (!mult || !shift || !(ratio > 0.0) || !std::isfinite(ratio)) return IVIT_ERR_INVALID_ARG;
+  int e = 0;
+  const double mant = std::frexp(ratio, &e);
+  long long b = std::llround(std::ldexp(mant, 31));
+  int c = 31 - e;
+  if (b == (1ll << 31)) { b = 1ll << 30; c -= 1; }
+  if (c < 1 || c > 62) return IVIT_ERR_RANGE;
+  *mult = (int32_t)b;
+  *shift = c;
+  return IVIT_OK;
+}
+
+int ivit_validate_exp_params(ivit_exp_params p, int64_t row_len, int32_t is_gelu) {
+  if (row_len < 1) return IVIT_ERR_INVALID_ARG;
+  return check_exp(p, row_len, is_gelu != 0);
+}
+
+int ivit_validate_scale(const int32_t* mult_host, const uint8_t* shift_host, int64_t n) {
+  if (!mult_host || !shift_host || n < 0) return IVIT_ERR_INVALID_ARG;
+  for (int64_t i = 0; i < n; ++i)
+    if (mult_host[i] <= 0 || shift_host[i] < 1 || shift_host[i] > 62) return IVIT_ERR_RANGE;
+  return IVIT_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,458 @@
+// I-LayerNorm (Sec. 3.5), Shiftmax (Algorithm 1) and ShiftGELU (Algorithm 2) kernels, sm_100a.
+// One warp owns one row; rows are read once from HBM as coalesced 32-bit words and
+// kept in registers between the reduction and the output pass.
+#include "common.cuh"
+
+namespace ivit {
+
+__device__ __forceinline__ int warp_sum(int v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ unsigned warp_sum_u(unsigned v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ long long warp_sum_ll(long long v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+__device__ __forceinline__ int warp_max(int v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v = max(v, __shfl_xor_sync(0xffffffffu, v, o));
+  return v;
+}
+
+// Eq. (iterative): x_{i+1} = (x_i + floor(n / x_i)) >> 1 from x_0 = 2^floor(bit(n)/2); the first
+// step is taken unconditionally, the following nine only while they decrease (leaving the loop
+// at the first non-decrease gives the same value as holding it for the remaining steps).
+__device__ __forceinline__ unsigned isqrt_u32(unsigned n) {
+  if (n == 0) return 0;
+  int bits = 32 - __clz(n);
+  unsigned x = 1u << (bits >> 1);
+  x = (x + n / x) >> 1;
+#pragma unroll 1
+  for (int i = 1; i < 10; ++i) {
+    unsigned nx = (x + n / x) >> 1;
+    if (nx >= x) break;
+    x = nx;
+  }
+  return x;
+}
+__device__ __forceinline__ unsigned long long isqrt_u64(unsigned long long n) {
+  if (n == 0) return 0;
+  int bits = 64 - __clzll(n);
+  unsigned long long x = 1ull << (bits >> 1);
+  x = (x + n / x) >> 1;
+#pragma unroll 1
+  for (int i = 1; i < 10; ++i) {
+    unsigned long long nx = (x + n / x) >> 1;
+    if (nx >= x) break;
+    x = nx;
+  }
+  return x;
+}
+
+__device__ __forceinline__ int floordiv_pos(int a, int b) {  // b > 0
+  int q = a / b;
+  return (a - q * b < 0) ? q - 1 : q;
+}
+
+// ------------------------------------------------------------------ I-LayerNorm, int8 input
+
+// WPL = 32-bit words of the row held per lane (C <= 128 * WPL).
+template <int WPL>
+__global__ void __launch_bounds__(256) layernorm_i8_kernel(const int8_t* __restrict__ in, int64_t ldin,
+                                                           ScaleDev gs, const int32_t* __restrict__ beta,
+                                                           int M_ln, int8_t* __restrict__ out, int64_t ldout,
+                                                           int64_t rows, int C) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  const int nwords = C >> 2;
+  for (int64_t r = warp; r < rows; r += nwarps) {
+    const int* src = reinterpret_cast<const int*>(in + r * ldin);
+    int w[WPL];
+    int s1 = 0, s2 = 0;
+#pragma unroll
+    for (int i = 0; i < WPL; ++i) {
+      const int idx = lane + 32 * i;
+      w[i] = idx < nwords ? __ldg(src + idx) : 0;
+      s1 = __dp4a(w[i], 0x01010101, s1);
+      s2 = __dp4a(w[i], w[i], s2);
+    }
+    s1 = warp_sum(s1);
+    s2 = warp_sum(s2);
+    const int mu = floordiv_pos(2 * s1 + C, 2 * C);
+    // sum (x - mu)^2 = sum x^2 - 2 mu sum x + C mu^2, exactly
+    const long long V = (long long)s2 - 2ll * mu * s1 + (long long)C * mu * mu;
+    const unsigned sd = isqrt_u32((unsigned)V);
+    const int F = sd == 0 ? 0 : (int)((1u << M_ln) / sd);
+    int* dst = reinterpret_cast<int*>(out + r * ldout);
+#pragma unroll
+    for (int i = 0; i < WPL; ++i) {
+      const int idx = lane + 32 * i;
+      if (idx < nwords) {
+        unsigned packed = 0;
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          const int c = idx * 4 + b;
+          const int x = (int)(int8_t)(w[i] >> (8 * b));
+          int v = rq((x - mu) * F, gs.m(c), gs.s(c));
+          if (beta) v += __ldg(beta + c);
+          packed |= (unsigned)(sat8(v) & 0xff) << (8 * b);
+        }
+        dst[idx] = (int)packed;
+      }
+    }
+  }
+}
+
+// Any C (multiple of 4): the row is read again from cache for the output pass.
+__global__ void __launch_bounds__(256) layernorm_i8_long_kernel(const int8_t* __restrict__ in, int64_t ldin,
+                                                                ScaleDev gs, const int32_t* __restrict__ beta,
+                                                                int M_ln, int8_t* __restrict__ out,
+                                                                int64_t ldout, int64_t rows, int C) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  const int nwords = C >> 2;
+  for (int64_t r = warp; r < rows; r += nwarps) {
+    const int* src = reinterpret_cast<const int*>(in + r * ldin);
+    int s1 = 0, s2 = 0;
+    for (int idx = lane; idx < nwords; idx += 32) {
+      const int w = __ldg(src + idx);
+      s1 = __dp4a(w, 0x01010101, s1);
+      s2 = __dp4a(w, w, s2);
+    }
+    s1 = warp_sum(s1);
+    s2 = warp_sum(s2);
+    const int mu = floordiv_pos(2 * s1 + C, 2 * C);
+    const long long V = (long long)s2 - 2ll * mu * s1 + (long long)C * mu * mu;
+    const unsigned sd = isqrt_u32((unsigned)V);
+    const int F = sd == 0 ? 0 : (int)((1u << M_ln) / sd);
+    int* dst = reinterpret_cast<int*>(out + r * ldout);
+    for (int idx = lane; idx < nwords; idx += 32) {
+      const int w = __ldg(src + idx);
+      unsigned packed = 0;
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const int c = idx * 4 + b;
+        const int x = (int)(int8_t)(w >> (8 * b));
+        int v = rq((x - mu) * F, gs.m(c), gs.s(c));
+        if (beta) v += __ldg(beta + c);
+        packed |= (unsigned)(sat8(v) & 0xff) << (8 * b);
+      }
+      dst[idx] = (int)packed;
+    }
+  }
+}
+
+// int32 input (|x| <= 2^20): 64-bit sums, two passes over the row.
+__global__ void __launch_bounds__(256) layernorm_i32_kernel(const int32_t* __restrict__ in, int64_t ldin,
+                                                            ScaleDev gs, const int32_t* __restrict__ beta,
+                                                            int M_ln, int8_t* __restrict__ out, int64_t ldout,
+                                                            int64_t rows, int C) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  for (int64_t r = warp; r < rows; r += nwarps) {
+    const int32_t* src = in + r * ldin;
+    long long s1 = 0;
+    for (int c = lane; c < C; c += 32) s1 += __ldg(src + c);
+    s1 = warp_sum_ll(s1);
+    const long long num = 2 * s1 + C, den = 2ll * C;
+    long long mu = num / den;
+    if (num - mu * den < 0) mu -= 1;
+    long long V = 0;
+    for (int c = lane; c < C; c += 32) {
+      const long long y = (long long)__ldg(src + c) - mu;
+      V += y * y;
+    }
+    V = warp_sum_ll(V);
+    const unsigned long long sd = isqrt_u64((unsigned long long)V);
+    const long long F = sd == 0 ? 0 : (long long)((1ull << M_ln) / sd);
+    for (int c = lane; c < C; c += 32) {
+      const long long y = (long long)__ldg(src + c) - mu;
+      int v = rq((int)(y * F), gs.m(c), gs.s(c));
+      if (beta) v += __ldg(beta + c);
+      out[r * ldout + c] = (int8_t)sat8(v);
+    }
+  }
+}
+
+int launch_layernorm(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, ScaleDev gs,
+                     const int32_t* beta, int M_ln, int8_t* out, int64_t ldout, int64_t rows, int64_t C) {
+  if (rows == 0) return IVIT_OK;
+  const int threads = 256, wpb = threads / 32;
+  const int64_t want = (rows + wpb - 1) / wpb;
+  const int grid = (int)(want < (int64_t)ctx->sm_count * 8 ? want : (int64_t)ctx->sm_count * 8);
+  cudaStream_t st = ctx->stream;
+  if (in_dtype == IVIT_I32) {
+    layernorm_i32_kernel<<<grid, threads, 0, st>>>((const int32_t*)in, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+    return check_launch(ctx);
+  }
+  const int8_t* x = (const int8_t*)in;
+  const int wpl = (int)((C / 4 + 31) / 32);
+  if (wpl <= 1) layernorm_i8_kernel<1><<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+  else if (wpl <= 2) layernorm_i8_kernel<2><<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+  else if (wpl <= 3) layernorm_i8_kernel<3><<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+  else if (wpl <= 4) layernorm_i8_kernel<4><<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+  else if (wpl <= 6) layernorm_i8_kernel<6><<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+  else if (wpl <= 8) layernorm_i8_kernel<8><<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+  else if (wpl <= 12) layernorm_i8_kernel<12><<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+  else layernorm_i8_long_kernel<<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+  return check_launch(ctx);
+}
+
+// ------------------------------------------------------------------ Shiftmax
+
+// Packed int8x4 word `idx` of row r.  I8: straight from memory.  I32: requantise four
+// accumulators (+ bias) to int8 first, so both entry forms run the same row algorithm.
+template <bool FROM_I32>
+struct RowLoader {
+  const void* in;
+  int64_t ldin;
+  const int32_t* bias32;
+  int64_t ldbias, bias_rows;
+  int pre_m, pre_s;
+  __device__ __forceinline__ int load(int64_t r, int idx) const {
+    if (!FROM_I32) {
+      return __ldg(reinterpret_cast<const int*>((const int8_t*)in + r * ldin) + idx);
+    } else {
+      const int4 a = __ldg(reinterpret_cast<const int4*>((const int32_t*)in + r * ldin) + idx);
+      int4 b = make_int4(0, 0, 0, 0);
+      if (bias32) b = __ldg(reinterpret_cast<const int4*>(bias32 + (r % bias_rows) * ldbias) + idx);
+      unsigned p = (unsigned)(sat8(rq(a.x + b.x, pre_m, pre_s)) & 0xff);
+      p |= (unsigned)(sat8(rq(a.y + b.y, pre_m, pre_s)) & 0xff) << 8;
+      p |= (unsigned)(sat8(rq(a.z + b.z, pre_m, pre_s)) & 0xff) << 16;
+      p |= (unsigned)(sat8(rq(a.w + b.w, pre_m, pre_s)) & 0xff) << 24;
+      return (int)p;
+    }
+  }
+};
+
+// WPL words per lane in registers (d <= 128 * WPL); WPL == 0: re-read the row for each pass.
+template <int WPL, bool FROM_I32>
+__global__ void __launch_bounds__(256) shiftmax_kernel(RowLoader<FROM_I32> ld, ivit_exp_params p,
+                                                       int8_t* __restrict__ out, int64_t ldout,
+                                                       int64_t rows, int d) {
+  __shared__ unsigned exp_tab[256];  // ShiftExp(-i), i = I_max - I in [0, 255]
+  for (int i = threadIdx.x; i < 256; i += blockDim.x) exp_tab[i] = shiftexp(-i, p.I0, p.N);
+  __syncthreads();
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  const int nwords = (d + 3) >> 2;
+  const int nwords_out = ((d + 15) >> 4) << 2;  // zero-fill up to the next multiple of 16
+  constexpr int W = WPL > 0 ? WPL : 1;
+  const int iters = WPL > 0 ? WPL : (nwords_out + 31) / 32;
+  for (int64_t r = warp; r < rows; r += nwarps) {
+    int w[W];
+    // pass 1: row max (bytes past d are replaced by -128)
+    int mx4 = (int)0x80808080;
+#pragma unroll
+    for (int i = 0; i < iters; ++i) {
+      const int idx = lane + 32 * i;
+      int v = (int)0x80808080;
+      if (idx < nwords) {
+        v = ld.load(r, idx);
+        const int valid = d - idx * 4;
+        if (valid < 4) {
+          const unsigned keep = 0xffffffffu >> (8 * (4 - valid));
+          v = (int)(((unsigned)v & keep) | (0x80808080u & ~keep));
+        }
+      }
+      if (WPL > 0) w[i] = v;
+      mx4 = (int)__vmaxs4((unsigned)mx4, (unsigned)v);
+    }
+    int mx = max(max((int)(int8_t)mx4, (int)(int8_t)(mx4 >> 8)), max((int)(int8_t)(mx4 >> 16), (int)(int8_t)(mx4 >> 24)));
+    mx = warp_max(mx);
+    // pass 2: sum of ShiftExp(I - I_max)
+    unsigned sum = 0;
+#pragma unroll
+    for (int i = 0; i < iters; ++i) {
+      const int idx = lane + 32 * i;
+      if (idx < nwords) {
+        const int v = WPL > 0 ? w[i] : ld.load(r, idx);
+#pragma unroll
+        for (int b = 0; b < 4; ++b)
+          if (idx * 4 + b < d) sum += exp_tab[mx - (int)(int8_t)(v >> (8 * b))];
+      }
+    }
+    sum = warp_sum_u(sum);
+    // Eq. (IntDiv): one reciprocal per row, M = 45, k_out = 8:
+    // (floor(2^45 / sum) * e) >> 38 == umulhi(factor, e) >> 6 since factor <= 2^31.
+    const unsigned factor = (unsigned)((1ull << 45) / (unsigned long long)sum);
+    int* dst = reinterpret_cast<int*>(out + r * ldout);
+#pragma unroll
+    for (int i = 0; i < iters; ++i) {
+      const int idx = lane + 32 * i;
+      if (idx < nwords_out) {
+        unsigned packed = 0;
+        if (idx < nwords) {
+          const int v = WPL > 0 ? w[i] : ld.load(r, idx);
+#pragma unroll
+          for (int b = 0; b < 4; ++b) {
+            if (idx * 4 + b < d) {
+              const unsigned e = exp_tab[mx - (int)(int8_t)(v >> (8 * b))];
+              const unsigned o = min(127u, __umulhi(factor, e) >> 6);
+              packed |= o << (8 * b);
+            }
+          }
+        }
+        dst[idx] = (int)packed;
+      }
+    }
+  }
+}
+
+template <bool FROM_I32>
+static void shiftmax_dispatch(RowLoader<FROM_I32> ld, ivit_exp_params p, int8_t* out, int64_t ldout,
+                              int64_t rows, int d, int grid, cudaStream_t st) {
+  const int wpl = (((d + 15) / 16) * 4 + 31) / 32;
+  if (wpl <= 2) shiftmax_kernel<2, FROM_I32><<<grid, 256, 0, st>>>(ld, p, out, ldout, rows, d);
+  else if (wpl <= 5) shiftmax_kernel<5, FROM_I32><<<grid, 256, 0, st>>>(ld, p, out, ldout, rows, d);
+  else if (wpl <= 8) shiftmax_kernel<8, FROM_I32><<<grid, 256, 0, st>>>(ld, p, out, ldout, rows, d);
+  else if (wpl <= 16) shiftmax_kernel<16, FROM_I32><<<grid, 256, 0, st>>>(ld, p, out, ldout, rows, d);
+  else shiftmax_kernel<0, FROM_I32><<<grid, 256, 0, st>>>(ld, p, out, ldout, rows, d);
+}
+
+int launch_shiftmax(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, const int32_t* bias32,
+                    int64_t ldbias, int64_t bias_rows, ScaleDev pre, ivit_exp_params p, int8_t* out,
+                    int64_t ldout, int64_t rows, int64_t d) {
+  if (rows == 0) return IVIT_OK;
+  const int64_t want = (rows + 7) / 8;
+  const int grid = (int)(want < (int64_t)ctx->sm_count * 8 ? want : (int64_t)ctx->sm_count * 8);
+  if (in_dtype == IVIT_I8) {
+    RowLoader<false> ld{in, ldin, nullptr, 0, 1, 0, 1};
+    shiftmax_dispatch<false>(ld, p, out, ldout, rows, (int)d, grid, ctx->stream);
+  } else {
+    RowLoader<true> ld{in, ldin, bias32, ldbias, bias_rows < 1 ? 1 : bias_rows, pre.mult, clamp_shift(pre.shift)};
+    shiftmax_dispatch<true>(ld, p, out, ldout, rows, (int)d, grid, ctx->stream);
+  }
+  return check_launch(ctx);
+}
+
+// ------------------------------------------------------------------ ShiftGELU
+
+// Because the input is int8 and the row statistic is I_max = max(0, I_p(max_row x)), the output
+// is a function of (max(0, row max of x), x): 128 x 256 values.  They are produced here by
+// running Algorithm 2 literally once per pair; the row kernel then only looks values up.
+__global__ void shiftgelu_table_kernel(ivit_exp_params p, int post_m, int post_s, int8_t* __restrict__ table) {
+  const int rmax = blockIdx.x;         // max(0, row max of x), 0..127
+  const int x = (int)threadIdx.x - 128;
+  int out = 0;
+  if (x <= rmax) {
+    const int Ip = x + (x >> 1) + (x >> 3) + (x >> 4);              // 1.702 x as (1.1011)b
+    const int Imax = rmax + (rmax >> 1) + (rmax >> 3) + (rmax >> 4);  // I_p is monotone in x; rmax >= 0
+    const unsigned e1 = shiftexp(-Imax, p.I0, p.N);
+    const unsigned e = shiftexp(Ip - Imax, p.I0, p.N);
+    const unsigned long long den = (unsigned long long)e + e1;
+    int div = 0;
+    if (den != 0) {
+      const unsigned long long f = (1ull << 45) / den;  // Eq. (IntDiv), M = 45
+      div = (int)((f * e) >> 38);                         // k_out = 8; f*e <= 2^45
+    }
+    out = sat8(rq(x * div, post_m, post_s));
+  }
+  table[rmax * 256 + threadIdx.x] = (int8_t)out;
+}
+
+template <int WPL>
+__global__ void __launch_bounds__(256) shiftgelu_kernel(const int8_t* __restrict__ in, int64_t ldin,
+                                                        const int8_t* __restrict__ table,
+                                                        int8_t* __restrict__ out, int64_t ldout,
+                                                        int64_t rows, int cols) {
+  __shared__ unsigned tab[8][64];  // one 256-byte table row per warp
+  const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+  const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  const int nvec = cols >> 4;  // 16-byte vectors per row
+  constexpr int W = WPL > 0 ? WPL : 1;
+  const int iters = WPL > 0 ? WPL : (nvec + 31) / 32;
+  const unsigned char* t8 = reinterpret_cast<const unsigned char*>(tab[wib]);
+  for (int64_t r = warp; r < rows; r += nwarps) {
+    const int4* src = reinterpret_cast<const int4*>(in + r * ldin);
+    int4 w[W];
+    int mx4 = (int)0x80808080;
+#pragma unroll
+    for (int i = 0; i < iters; ++i) {
+      const int idx = lane + 32 * i;
+      int4 v = make_int4((int)0x80808080, (int)0x80808080, (int)0x80808080, (int)0x80808080);
+      if (idx < nvec) v = __ldg(src + idx);
+      if (WPL > 0) w[i] = v;
+      mx4 = (int)__vmaxs4(__vmaxs4((unsigned)v.x, (unsigned)v.y), __vmaxs4(__vmaxs4((unsigned)v.z, (unsigned)v.w), (unsigned)mx4));
+    }
+    int mx = max(max((int)(int8_t)mx4, (int)(int8_t)(mx4 >> 8)), max((int)(int8_t)(mx4 >> 16), (int)(int8_t)(mx4 >> 24)));
+    mx = max(0, warp_max(mx));
+    __syncwarp();
+    const unsigned* trow = reinterpret_cast<const unsigned*>(table + mx * 256);
+    tab[wib][lane] = __ldg(trow + lane);
+    tab[wib][lane + 32] = __ldg(trow + lane + 32);
+    __syncwarp();
+    int4* dst = reinterpret_cast<int4*>(out + r * ldout);
+#pragma unroll
+    for (int i = 0; i < iters; ++i) {
+      const int idx = lane + 32 * i;
+      if (idx < nvec) {
+        const int4 v = WPL > 0 ? w[i] : __ldg(src + idx);
+        int4 o;
+        const int vin[4] = {v.x, v.y, v.z, v.w};
+        int vout[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const unsigned u = (unsigned)vin[k] ^ 0x80808080u;  // x + 128 per byte
+          unsigned pk = t8[u & 0xff];
+          pk |= (unsigned)t8[(u >> 8) & 0xff] << 8;
+          pk |= (unsigned)t8[(u >> 16) & 0xff] << 16;
+          pk |= (unsigned)t8[u >> 24] << 24;
+          vout[k] = (int)pk;
+        }
+        o = make_int4(vout[0], vout[1], vout[2], vout[3]);
+        dst[idx] = o;
+      }
+    }
+  }
+}
+
+int launch_shiftgelu(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_params p, ivit_scale post,
+                     int8_t* out, int64_t ldout, int64_t rows, int64_t cols) {
+  if (rows == 0) return IVIT_OK;
+  // find or build the lookup table of this parameter set
+  const GeluKey key{p.I0, p.N, p.M, p.k_out, post.mult, post.shift};
+  int slot = -1;
+  for (int i = 0; i < ctx->gelu_used; ++i)
+    if (ctx->gelu_keys[i] == key) { slot = i; break; }
+  if (slot < 0) {
+    if (ctx->gelu_used < kGeluTableSlots) {
+      slot = ctx->gelu_used++;
+    } else {
+      slot = ctx->gelu_next;
+      ctx->gelu_next = (ctx->gelu_next + 1) % kGeluTableSlots;
+    }
+    ctx->gelu_keys[slot] = key;
+    shiftgelu_table_kernel<<<128, 256, 0, ctx->stream>>>(p, post.mult, post.shift,
+                                                          ctx->gelu_tables + (size_t)slot * kGeluTableBytes);
+    int rc = check_launch(ctx);
+    if (rc) return rc;
+  }
+  const int8_t* table = ctx->gelu_tables + (size_t)slot * kGeluTableBytes;
+  const int64_t want = (rows + 7) / 8;
+  const int grid = (int)(want < (int64_t)ctx->sm_count * 8 ? want : (int64_t)ctx->sm_count * 8);
+  const int wpl = (int)((cols / 16 + 31) / 32);
+  cudaStream_t st = ctx->stream;
+  if (wpl <= 1) shiftgelu_kernel<1><<<grid, 256, 0, st>>>(in, ldin, table, out, ldout, rows, (int)cols);
+  else if (wpl <= 2) shiftgelu_kernel<2><<<grid, 256, 0, st>>>(in, ldin, table, out, ldout, rows, (int)cols);
+  else if (wpl <= 3) shiftgelu_kernel<3><<<grid, 256, 0, st>>>(in, ldin, table, out, ldout, rows, (int)cols);
+  else if (wpl <= 4) shiftgelu_kernel<4><<<grid, 256, 0, st>>>(in, ldin, table, out, ldout, rows, (int)cols);
+  else if (wpl <= 6) shiftgelu_kernel<6><<<grid, 256, 0, st>>>(in, ldin, table, out, ldout, rows, (int)cols);
+  else if (wpl <= 8) shiftgelu_kernel<8><<<grid, 256, 0, st>>>(in, ldin, table, out, ldout, rows, (int)cols);
+  else shiftgelu_kernel<0><<<grid, 256, 0, st>>>(in, ldin, table, out, ldout, rows, (int)cols);
+  return check_launch(ctx);
+}
+
+}  // namespace ivit

@@ -1,0 +1,75 @@
+"""GPU parity of the encoder block and the full ViT-family forward against the CPU oracle (bit-exact)."""
+import numpy as np
+import pytest
+import torch
+
+from ivit_inputs import make_config
+from ivit_inputs.gen import _Ids, make_block, make_block_input
+from oracle import api as O
+
+pytestmark = pytest.mark.gpu
+
+
+def _g():
+    import gpu_util
+    return gpu_util
+
+
+@pytest.mark.parametrize("engine", [1, 0])
+def test_config0_block_bit_exact(engine):
+    g = _g()
+    c = g.ctx()
+    c.set_gemm_engine(engine)
+    blk, X = make_config(0)
+    dblk = g.binding.DeviceBlock(blk, "cuda")
+    Y = c.block_forward(dblk, torch.from_numpy(X).cuda())
+    g.assert_equal(g.host(Y), O.block_forward(blk, X), "config 0 block")
+    assert c.poll_status() == 0
+    c.set_gemm_engine(0)
+
+
+@pytest.mark.parametrize("B,T,D,heads,H,bias", [(3, 197, 384, 6, 1536, False), (2, 577, 256, 4, 512, False),
+                                                (16, 49, 96, 3, 384, True), (2, 49, 768, 24, 3072, True),
+                                                (1, 1, 64, 1, 64, False)])
+def test_block_shapes_bit_exact(B, T, D, heads, H, bias):
+    g = _g()
+    c = g.ctx()
+    blk = make_block(_Ids(100 + B + T), 3, B, T, D, heads, H, attn_bias_batches=heads if bias else 0)
+    X = make_block_input(7, B, T, D)
+    dblk = g.binding.DeviceBlock(blk, "cuda")
+    Y = c.block_forward(dblk, torch.from_numpy(X).cuda())
+    g.assert_equal(g.host(Y), O.block_forward(blk, X), "block")
+    # attention core alone
+    rng = np.random.default_rng(1)
+    QKV = np.clip(np.rint(rng.standard_normal((B * T, 3 * D)) * 32), -128, 127).astype(np.int8)
+    Oo = c.attention(dblk, torch.from_numpy(QKV).cuda())
+    g.assert_equal(g.host(Oo), O.attention(blk, QKV), "attention")
+    assert c.poll_status() == 0
+
+
+def test_block_workspace_errors():
+    g = _g()
+    c = g.ctx()
+    blk, X = make_config(0)
+    dblk = g.binding.DeviceBlock(blk, "cuda")
+    dX = torch.from_numpy(X).cuda()
+    small = torch.empty(1024, dtype=torch.uint8, device="cuda")
+    with pytest.raises(g.binding.IvitError) as e:
+        c.block_forward(dblk, dX, workspace=small)
+    assert e.value.code == -5
+    with pytest.raises(g.binding.IvitError) as e:
+        c.block_forward(dblk, dX, Y=dX)
+    assert e.value.code == -1
+
+
+def test_vit_small_model_bit_exact():
+    """DeiT-S shapes, 2 blocks, batch 3: logits and every stage composed by the library equal the oracle."""
+    g = _g()
+    c = g.ctx()
+    model, image = make_config(1, batch=3, depth=2)
+    dm = g.binding.DeviceVit(model, "cuda")
+    logits = c.vit_forward(dm, torch.from_numpy(image).cuda())
+    want = O.vit_forward(model, image)
+    g.assert_equal(g.host(logits), want, "vit logits")
+    assert np.abs(want).max() > 100 and len(np.unique(want)) > 100
+    assert c.poll_status() == 0

@@ -1,0 +1,233 @@
+"""GPU parity, operator by operator: the CUDA kernels behind the C ABI against the CPU oracle,
+bit for bit, on seeded inputs that span several tiles and a ragged tail."""
+import numpy as np
+import pytest
+import torch
+
+from ivit_inputs import ExpParams, Scale
+from ivit_inputs.gen import dyadic, scale_channels
+from oracle import api as O
+
+pytestmark = pytest.mark.gpu
+
+
+def _g():
+    import gpu_util
+    return gpu_util
+
+
+def rand_i8(rng, shape, std=40):
+    return np.clip(np.rint(rng.standard_normal(shape) * std), -128, 127).astype(np.int8)
+
+
+@pytest.mark.parametrize("engine", [1, 0])
+@pytest.mark.parametrize("M,N,K", [(1, 16, 16), (197, 192, 192), (130, 200, 48), (393, 1152, 384), (77, 1000, 768),
+                                   (256, 256, 1536), (64, 96, 64)])
+def test_linear_parity(engine, M, N, K):
+    g = _g()
+    c = g.ctx()
+    c.set_gemm_engine(engine)
+    rng = np.random.default_rng(M * 7 + N * 3 + K)
+    A, W = rand_i8(rng, (M, K)), rand_i8(rng, (N, K))
+    bias = rng.integers(-20000, 20000, N).astype(np.int32)
+    acc_std = np.sqrt(K) * 40 * 40
+    scale = scale_channels(rng.uniform(20, 60, N) / acc_std)
+    res = rand_i8(rng, (max(1, M // 2), N))
+    rs = Scale(*dyadic(0.9))
+    dA, dW, dres = g.dev(A), g.dev(W), g.dev(res)
+    dbias = torch.from_numpy(bias).cuda()
+    ds, drs = g.binding.DevScale(scale, "cuda"), g.binding.DevScale(rs, "cuda")
+    # plain
+    got = c.linear(dA, dW, dbias, ds, out=g.dev(np.zeros((M, N), np.int8)))
+    g.assert_equal(g.host(got), O.linear(A, W, bias, scale), "linear")
+    # residual port with wrap-around rows, no bias
+    got = c.linear(dA, dW, None, ds, res=dres, res_scale=drs, out=g.dev(np.zeros((M, N), np.int8)))
+    g.assert_equal(g.host(got), O.linear(A, W, None, scale, res=res, res_scale=rs), "linear+res")
+    # int32 output (not saturated), per-tensor scale
+    pt = Scale(*dyadic(300.0 / acc_std))
+    got = c.linear(dA, dW, dbias, g.binding.DevScale(pt, "cuda"), out_dtype=g.binding.I32,
+                   out=g.dev(np.zeros((M, N), np.int32), 4))
+    g.assert_equal(g.host(got), O.linear(A, W, bias, pt, out_dtype=O.I32), "linear i32")
+    c.set_gemm_engine(0)
+    assert c.poll_status() == 0
+
+
+@pytest.mark.parametrize("engine", [1, 0])
+def test_linear_output_row_groups(engine):
+    g = _g()
+    c = g.ctx()
+    c.set_gemm_engine(engine)
+    rng = np.random.default_rng(5)
+    M, N, K, grp, stride = 196 * 3, 192, 768, 196, 197
+    A, W = rand_i8(rng, (M, K), 20), rand_i8(rng, (N, K))
+    bias = rng.integers(-20000, 20000, N).astype(np.int32)
+    scale = scale_channels(rng.uniform(10, 30, N) / (np.sqrt(K) * 20 * 40))
+    pos, ps = rand_i8(rng, (grp, N), 6), Scale(*dyadic(0.75))
+    buf = torch.full((3 * stride, N), 77, dtype=torch.int8, device="cuda")
+    c.linear(g.dev(A), g.dev(W), torch.from_numpy(bias).cuda(), g.binding.DevScale(scale, "cuda"), res=g.dev(pos),
+             res_scale=g.binding.DevScale(ps, "cuda"), res_rows=grp, out=buf[1:], out_group_rows=grp,
+             out_group_stride=stride)
+    want = np.full((3 * stride, N), 77, np.int8)
+    O.linear(A, W, bias, scale, res=pos, res_scale=ps, res_rows=grp, out=want[1:], out_group_rows=grp,
+             out_group_stride=stride)
+    g.assert_equal(g.host(buf), want, "grouped rows")
+    c.set_gemm_engine(0)
+
+
+@pytest.mark.parametrize("engine", [1, 0])
+@pytest.mark.parametrize("nb,Ma,Nb,K,transB", [(6, 197, 197, 64, True), (6, 197, 64, 197, False), (5, 49, 49, 32, True),
+                                               (5, 49, 32, 49, False), (2, 577, 577, 64, True), (2, 577, 64, 577, False),
+                                               (3, 1, 1, 16, True)])
+def test_matmul_parity(engine, nb, Ma, Nb, K, transB):
+    g = _g()
+    c = g.ctx()
+    c.set_gemm_engine(engine)
+    rng = np.random.default_rng(nb + Ma + Nb + K)
+    A = rand_i8(rng, (nb, Ma, K), 32)
+    B = rand_i8(rng, (nb, Nb, K) if transB else (nb, K, Nb), 32)
+    sc = Scale(*dyadic(30.0 / (np.sqrt(K) * 32 * 32)))
+    bias = (rng.standard_normal((2, Ma, Nb)) * 2000).astype(np.int32) if transB else None
+    dbias = None if bias is None else g.dev(bias, 4)
+    got = c.matmul(g.dev(A), g.dev(B), transB, g.binding.DevScale(sc, "cuda"), bias32=dbias)
+    g.assert_equal(g.host(got), O.matmul(A, B, transB, sc, bias32=bias), "matmul")
+    c.set_gemm_engine(0)
+
+
+@pytest.mark.parametrize("rows,d,I0", [(1, 1, 16), (3, 2, 11), (50, 49, 13), (400, 197, 11), (400, 197, 23), (130, 577, 17),
+                                       (9, 1024, 12), (5, 3000, 4), (33, 64, 20)])
+def test_shiftmax_parity(rows, d, I0):
+    g = _g()
+    c = g.ctx()
+    rng = np.random.default_rng(rows + d + I0)
+    x = rand_i8(rng, (rows, d), 32)
+    if rows > 2:
+        x[1, :] = -128           # constant row
+        x[2, :] = 127
+    p = ExpParams(I0, 15)
+    out = c.shiftmax(g.dev(x), p)
+    g.assert_equal(g.host(out), O.shiftmax(x, p), "shiftmax i8")
+    # the zero-filled pad columns
+    base = out._base if out._base is not None else out
+    full = g.host(base)
+    assert (full[:, d:((d + 15) // 16) * 16] == 0).all()
+    # int32 form: requant (+bias) first
+    acc = (rng.standard_normal((rows, d)) * 9000).astype(np.int32)
+    bias = (rng.standard_normal((7, d)) * 2000).astype(np.int32)
+    pre = Scale(*dyadic(30.0 / 8192))
+    out = c.shiftmax(g.dev(acc, 4), p, pre=g.binding.DevScale(pre, "cuda"), bias32=g.dev(bias, 4))
+    g.assert_equal(g.host(out), O.shiftmax(acc, p, pre=pre, bias32=bias), "shiftmax i32")
+
+
+def test_shiftexp_and_gelu_exhaustive_domain():
+    """All 256 int8 inputs against every possible row maximum, several I0: the whole ShiftGELU domain."""
+    g = _g()
+    c = g.ctx()
+    xs = np.arange(-128, 128)
+    for I0 in (29, 31, 33, 35, 37, 16, 64, 255):
+        p = ExpParams(I0, 23)
+        post = Scale(*dyadic(1.0 / (128 * 0.9)))
+        rows = []
+        for mx in range(-128, 128):
+            r = np.minimum(xs, mx)           # every value <= mx, max == mx
+            rows.append(np.resize(r, 256))
+        x = np.array(rows, dtype=np.int8)
+        got = c.shiftgelu(g.dev(x), p, g.binding.DevScale(post, "cuda"))
+        g.assert_equal(g.host(got), O.shiftgelu(x, p, post), f"shiftgelu domain I0={I0}")
+    # Shiftmax: every delta in [-255, 0] for many I0 (rows [127, v] and [-128 ... ] cover the table)
+    for I0 in list(range(1, 40)) + [64, 100, 181, 255]:
+        N = 15 if I0 >= 1 else 15
+        if (I0 << N) < (1 << 14):
+            continue
+        p = ExpParams(I0, N)
+        x = np.stack([np.full(256, 127), np.arange(-128, 128)], axis=1).astype(np.int8)
+        got = c.shiftmax(g.dev(x), p)
+        g.assert_equal(g.host(got), O.shiftmax(x, p), f"shiftmax domain I0={I0}")
+
+
+@pytest.mark.parametrize("rows,cols,I0", [(1, 16, 29), (200, 768, 31), (300, 1536, 33), (64, 3072, 35), (40, 4096, 37),
+                                          (7, 8192, 29), (5, 12288, 30)])
+def test_shiftgelu_parity(rows, cols, I0):
+    g = _g()
+    c = g.ctx()
+    rng = np.random.default_rng(rows + cols)
+    x = rand_i8(rng, (rows, cols), I0)
+    if rows > 3:
+        x[1] = -np.abs(x[1]) - 1          # all-negative row: max floored at 0
+        x[2] = 0
+        x[3] = np.minimum(x[3], 40)
+    p, post = ExpParams(I0, 23), Scale(*dyadic(1.0 / (128 * 0.9)))
+    dx = g.dev(x)
+    got = c.shiftgelu(dx, p, g.binding.DevScale(post, "cuda"))
+    want = O.shiftgelu(x, p, post)
+    g.assert_equal(g.host(got), want, "shiftgelu")
+    c.shiftgelu(dx, p, g.binding.DevScale(post, "cuda"), out=dx)      # in place
+    g.assert_equal(g.host(dx), want, "shiftgelu in place")
+
+
+@pytest.mark.parametrize("rows,C", [(1, 16), (197, 192), (500, 384), (300, 768), (100, 1024), (50, 96), (20, 1536),
+                                    (9, 3072), (3, 16384), (11, 4)])
+def test_layernorm_parity(rows, C):
+    g = _g()
+    c = g.ctx()
+    rng = np.random.default_rng(rows + C)
+    x = rand_i8(rng, (rows, C), 20) + rng.integers(-30, 30, (rows, 1)).astype(np.int8)
+    if rows > 2:
+        x[1] = 5                          # constant row: sd = 0 -> beta
+        x[2, : C // 2], x[2, C // 2:] = -128, 127
+    scale = scale_channels((1 + 0.1 * rng.standard_normal(C)) * 32 * np.sqrt(C) / 2.0 ** 20)
+    beta = rng.integers(-10, 10, C).astype(np.int32)
+    got = c.layernorm(g.dev(x), g.binding.DevScale(scale, "cuda"), torch.from_numpy(beta).cuda())
+    g.assert_equal(g.host(got), O.layernorm(x, scale, beta), "layernorm i8")
+    # per-tensor scale, no beta
+    pt = Scale(*dyadic(32 * np.sqrt(C) / 2.0 ** 20))
+    got = c.layernorm(g.dev(x), g.binding.DevScale(pt, "cuda"), None)
+    g.assert_equal(g.host(got), O.layernorm(x, pt, None), "layernorm per-tensor")
+    # int32 input
+    x32 = (rng.standard_normal((rows, C)) * 3000).astype(np.int32)
+    got = c.layernorm(g.dev(x32, 4), g.binding.DevScale(scale, "cuda"), torch.from_numpy(beta).cuda())
+    g.assert_equal(g.host(got), O.layernorm(x32, scale, beta), "layernorm i32")
+
+
+def test_helpers_parity():
+    g = _g()
+    c = g.ctx()
+    rng = np.random.default_rng(3)
+    img = rand_i8(rng, (3, 3, 56, 56), 20)
+    dimg = torch.from_numpy(img).cuda()
+    g.assert_equal(g.host(c.patchify(dimg, 4)), O.patchify(img, 4), "patchify")
+    g.assert_equal(g.host(c.patchify(dimg, 4, window=7)), O.patchify(img, 4, window=7), "patchify windows")
+    img16 = rand_i8(rng, (2, 3, 64, 64), 20)
+    g.assert_equal(g.host(c.patchify(torch.from_numpy(img16).cuda(), 16)), O.patchify(img16, 16), "patchify 16")
+    src = rand_i8(rng, (300, 96))
+    idx = rng.integers(0, 300, 1000).astype(np.int32)
+    g.assert_equal(g.host(c.gather_rows(g.dev(src), torch.from_numpy(idx).cuda())), O.gather_rows(src, idx), "gather")
+    sc = Scale(*dyadic(3.0 / 49))
+    x = rand_i8(rng, (49 * 5, 768))
+    g.assert_equal(g.host(c.token_mean(g.dev(x), 49, g.binding.DevScale(sc, "cuda"))), O.token_mean(x, 49, sc), "token mean")
+    dst = torch.zeros((4 * 5, 32), dtype=torch.int8, device="cuda")
+    row = rand_i8(rng, (32,))
+    c.fill_rows(torch.from_numpy(row).cuda(), dst, 5 * 32, 4)
+    want = np.zeros((20, 32), np.int8)
+    want[::5] = row
+    g.assert_equal(g.host(dst), want, "fill rows")
+
+
+def test_argument_validation_is_synchronous():
+    g = _g()
+    c = g.ctx()
+    b = g.binding
+    x = torch.zeros((4, 32), dtype=torch.int8, device="cuda")
+    sc = b.DevScale(Scale(2 ** 30, 35), "cuda")
+    with pytest.raises(b.IvitError) as e:
+        c.shiftmax(x, ExpParams(0, 15))
+    assert e.value.code == -3
+    with pytest.raises(b.IvitError) as e:
+        c.shiftgelu(x[:, :24], ExpParams(30, 23), sc)          # cols % 16
+    assert e.value.code == -4
+    with pytest.raises(b.IvitError) as e:
+        c.layernorm(x[:, 1:17], sc, None)                      # misaligned base pointer
+    assert e.value.code == -2
+    with pytest.raises(b.IvitError) as e:
+        c.linear(x, torch.zeros((32, 32), dtype=torch.int8, device="cuda"), None, b.DevScale(Scale(0, 35), "cuda"))
+    assert e.value.code == -3
+    assert c.poll_status() == 0
