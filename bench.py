@@ -1,0 +1,302 @@
+"""Benchmark of the integer-only ViT forward pass on B200 (DeiT-S shapes, batch 64, synthetic weights).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W]         # the CUDA library
+  python bench.py --impl reference [...]                      # the CPU oracle, as it stands
+
+A step is one full forward of the workload (patch embedding, 12 encoder blocks, classifier) over
+one batch of 64 synthetic images.  Prints one JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "int-only ViT images/s (DeiT-S b64)"
+WORKLOAD = "deit_small_b64"
+CONFIG_INDEX = 1
+
+
+def vit_int8_ops(p) -> float:
+    """Algorithmic int8 operations (2 per multiply-accumulate) of one forward of a ViT-family model."""
+    B, T, D, H, h = p.B, p.T, p.D, p.H, p.heads
+    M, d = B * T, p.D // p.heads
+    blk = 2 * M * D * 3 * D + 2 * (B * h * 2 * T * T * d) + 2 * M * D * D + 2 * 2 * M * D * H
+    return p.depth * blk + 2 * B * (T - 1) * (3 * p.patch * p.patch) * D + 2 * B * D * p.classes
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index, self.proc = gpu_index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        top = sorted(sm)[len(sm) // 2:]   # the busier half of the samples: the clock under load
+        return {"sm_mhz": statistics.median(top), "sm_max_mhz": max(mx), "samples": len(sm),
+                "power_w_max": max(power), "reasons": sorted(reasons)}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return d, "measured"
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "fallback"
+
+
+def time_oracle(model, image, budget_s: float = 15.0):
+    """Times the CPU oracle on a bounded sample of the workload's images; returns (images/s, n, seconds, threads)."""
+    from oracle import api as O
+    t0 = time.perf_counter()
+    O.vit_forward(model, image[:1])
+    t1 = time.perf_counter() - t0
+    n = int(max(1, min(image.shape[0], budget_s / max(t1, 1e-3))))
+    t0 = time.perf_counter()
+    O.vit_forward(model, image[:n])
+    dt = time.perf_counter() - t0
+    return n / dt, n, dt, O.num_threads()
+
+
+def run_reference(args):
+    """The CPU oracle timed as the reference arm (rank 0 only)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from ivit_inputs import make_config
+    from oracle import api as O
+    model, image = make_config(CONFIG_INDEX)
+    t0 = time.perf_counter()
+    O.vit_forward(model, image[:1])
+    t1 = time.perf_counter() - t0
+    # each step is a sample of n images, sized so that steps + warmup stay within about two minutes
+    n = int(max(1, min(image.shape[0], 120.0 / max(t1, 1e-3) / max(1, args.steps + args.warmup))))
+    for _ in range(args.warmup):
+        O.vit_forward(model, image[:n])
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        O.vit_forward(model, image[:n])
+    dt = time.perf_counter() - t0
+    value = n * args.steps / dt
+    sample = f"{n} of {image.shape[0]} images per step (images are independent)"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "images/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "images_per_step": n, "note": "CPU oracle, plain int64 loops, OpenMP over rows"},
+        "cpu_baseline": {"value": value, "unit": "images/s", "cores": O.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "images/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def run_gpu(args):
+    import numpy as np
+    import torch
+    from ivit_inputs import make_config
+    from paper_2207_01405_b200 import binding, build
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    build.build()
+    ctx = binding.Context(local_rank)
+    dev = ctx.device
+
+    # every rank serves its own batch of the same synthetic workload (weak scaling, no exchange step)
+    model, image = make_config(CONFIG_INDEX)
+    dm = binding.DeviceVit(model, dev)
+    B = model.B
+    ws = dm.host_workspace()
+    d_image = torch.from_numpy(image).to(dev)
+    d_logits = torch.empty((B, model.classes), dtype=torch.int32, device=dev)
+    h_image = torch.from_numpy(image).pin_memory()
+    h_logits = torch.empty((B, model.classes), dtype=torch.int32).pin_memory()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # > L2 (126 MB)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def step_resident():
+        ctx.vit_forward(dm, d_image, logits=d_logits, workspace=ws)
+
+    def step_e2e():
+        binding.vit_forward_host(ctx, dm, h_image, h_logits, ws)
+
+    def timed(step_fn, steps):
+        """K steps, each bracketed by its own event pair; L2 is flushed between steps outside the pairs."""
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        barrier()
+        for a, b in ev:
+            flush.zero_()
+            a.record()
+            step_fn()
+            b.record()
+        barrier()
+        return sum(a.elapsed_time(b) for a, b in ev)
+
+    for _ in range(max(args.warmup, 3)):
+        step_resident()
+    torch.cuda.synchronize()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = ctx.launch_count()
+    ms_total = timed(step_resident, args.steps)
+    launches = ctx.launch_count() - launches0
+    clocks = sampler.stop()
+
+    for _ in range(3):
+        step_e2e()
+    torch.cuda.synchronize()
+    ms_e2e = timed(step_e2e, args.steps)
+    status = ctx.poll_status()
+    if status != 0:
+        raise RuntimeError(f"device-side error {status}")
+
+    # per-kernel times of the same step, event-bracketed launch by launch (a separate pass: the
+    # event pairs serialise launches, so this pass is not the throughput number)
+    prof_steps = min(args.steps, 5)
+    ctx.profile_start()
+    for _ in range(prof_steps):
+        step_resident()
+    records = ctx.profile_stop()
+
+    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, ms_e2e = float(t[0]), float(t[1])
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_src = measured_peaks()
+    by_kind = {}
+    for kind, ms, work in records:
+        k = by_kind.setdefault(kind, {"launches": 0, "ms": 0.0, "work": 0.0})
+        k["launches"] += 1
+        k["ms"] += ms
+        k["work"] += work
+    total_kernel_ms = sum(k["ms"] for k in by_kind.values())
+    kernels = {}
+    for kind, k in sorted(by_kind.items(), key=lambda kv: -kv[1]["ms"]):
+        per_step_ms = k["ms"] / prof_steps
+        rate = k["work"] / prof_steps / (per_step_ms * 1e-3) if per_step_ms > 0 else 0.0
+        is_gemm = kind.startswith("gemm") or kind.startswith("attention")
+        kernels[kind] = {"launches_per_step": k["launches"] // prof_steps, "ms_per_step": round(per_step_ms, 4),
+                         "share": round(k["ms"] / total_kernel_ms, 4),
+                         ("TOPS" if is_gemm else "GB/s"): round(rate / (1e12 if is_gemm else 1e9), 2)}
+    dom = next(iter(kernels))
+    dk = by_kind[dom]
+    int8_peak = 2.0 * peaks["bf16_tflops_sustained"]      # int8 dense = 2 x bf16 (nominal ratio), sustained: timed inside a long step
+    if dom.startswith("gemm") or dom.startswith("attention"):
+        achieved = dk["work"] / (dk["ms"] * 1e-3) / 1e12
+        roofline = {"kernel": dom, "bound": "tensor", "achieved": round(achieved, 2), "peak": int8_peak, "unit": "TOP/s",
+                    "frac": round(achieved / int8_peak, 4), "traffic": None,
+                    "peak_source": f"2 x {peak_src} sustained bf16 cuBLAS ({peaks['bf16_tflops_sustained']} TFLOP/s)"}
+    else:
+        achieved = dk["work"] / (dk["ms"] * 1e-3) / 1e9
+        roofline = {"kernel": dom, "bound": "hbm", "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": round(achieved / peaks["hbm_gbs"], 4), "traffic": None, "peak_source": f"{peak_src} copy bandwidth"}
+
+    cpu_rate, cpu_n, cpu_s, cpu_threads = time_oracle(model, image)
+    # the timed steps really computed the forward: spot-check one image against the oracle
+    from oracle import api as O
+    ok = bool(np.array_equal(h_logits[:1].numpy(), O.vit_forward(model, image[:1])))
+
+    imgs = B * world * args.steps
+    ops = vit_int8_ops(model)
+    line = {
+        "metric": METRIC, "value": imgs / (ms_total * 1e-3), "unit": "images/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8 x int8 -> int32",
+        "data": "synthetic", "config": {"workload": WORKLOAD, "batch_per_gpu": B, "tokens": model.T, "embed": model.D,
+                                        "heads": model.heads, "mlp": model.H, "blocks": model.depth,
+                                        "l2": "256 MB buffer written between steps, outside the per-step event pairs",
+                                        "parallelism": f"dp{world} (independent batches, no collective)"},
+        "e2e": {"value": imgs / (ms_e2e * 1e-3), "unit": "images/s", "h2d_bytes_per_step": int(h_image.numel()),
+                "d2h_bytes_per_step": int(h_logits.numel() * 4), "ms_per_step": ms_e2e / args.steps},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": roofline,
+        "cpu_baseline": {"value": cpu_rate, "unit": "images/s", "cores": cpu_threads, "kind": "oracle",
+                         "sample": f"{cpu_n} of {B} images ({cpu_s:.1f} s; images are independent)"},
+        "int8_tops_whole_step": round(ops / (ms_total / args.steps * 1e-3) / 1e12, 2),
+        "kernels": kernels,
+        "parity_spot_check": ok,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ivit", choices=["ivit", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -210,6 +210,26 @@ size_t ivit_vit_workspace_bytes(const ivit_vit_params* p);
 int ivit_vit_forward(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* image, int32_t* logits,
                      void* workspace, size_t workspace_bytes);
 
+/* Same forward with HOST buffers: copies image_host (pinned or pageable) to a staging area in
+ * the workspace, runs ivit_vit_forward, and copies the logits back to logits_host, all enqueued
+ * on the context's stream (the caller synchronises the stream before reading logits_host).
+ * workspace must hold ivit_vit_host_workspace_bytes(p). */
+size_t ivit_vit_host_workspace_bytes(const ivit_vit_params* p);
+int ivit_vit_forward_host(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* image_host,
+                          int32_t* logits_host, void* workspace, size_t workspace_bytes);
+
+/* ---- per-kernel timing (measurement aid; not part of the paper's method) ----
+ * Between profile_start and profile_stop every kernel the context launches is bracketed by a pair
+ * of CUDA events on the context's stream (at most 8192 launches per session; later ones are not
+ * recorded).  profile_stop synchronises the stream and returns the number of records (or a
+ * negative error).  profile_get returns record idx: the kernel class (ivit_kernel_kind_name),
+ * its device time in milliseconds and its algorithmic work (int8 ops for GEMMs, bytes moved for
+ * the other kernels). */
+int ivit_ctx_profile_start(ivit_ctx* ctx);
+int ivit_ctx_profile_stop(ivit_ctx* ctx);
+int ivit_ctx_profile_get(ivit_ctx* ctx, int32_t idx, int32_t* kind, float* ms, double* work);
+const char* ivit_kernel_kind_name(int32_t kind);
+
 /* ---- data movement helpers (not in the paper; needed by the full models) ---- */
 
 /* img [B,C,Hi,Wi] int8 -> rows [B*(Hi/P)*(Wi/P), C*P*P], column order

@@ -22,7 +22,8 @@ EXPORTS = [
     "ivit_ctx_create", "ivit_ctx_destroy", "ivit_ctx_set_stream", "ivit_ctx_poll_status", "ivit_ctx_launch_count",
     "ivit_ctx_set_gemm_engine", "ivit_strerror", "ivit_linear", "ivit_matmul", "ivit_shiftmax", "ivit_shiftgelu",
     "ivit_layernorm", "ivit_block_workspace_bytes", "ivit_block_forward", "ivit_attention",
-    "ivit_vit_workspace_bytes", "ivit_vit_forward", "ivit_patchify", "ivit_gather_rows", "ivit_fill_rows",
+    "ivit_vit_workspace_bytes", "ivit_vit_forward", "ivit_vit_host_workspace_bytes", "ivit_vit_forward_host",
+    "ivit_ctx_profile_start", "ivit_ctx_profile_stop", "ivit_ctx_profile_get", "ivit_kernel_kind_name", "ivit_patchify", "ivit_gather_rows", "ivit_fill_rows",
     "ivit_token_mean", "ivit_dyadic_from_double", "ivit_validate_exp_params", "ivit_validate_scale",
 ]
 
@@ -97,6 +98,14 @@ def load_library():
     L.ivit_vit_workspace_bytes.argtypes = [C.POINTER(CVit)]
     L.ivit_vit_workspace_bytes.restype = C.c_size_t
     L.ivit_vit_forward.argtypes = [vp, C.POINTER(CVit), vp, vp, vp, C.c_size_t]
+    L.ivit_vit_host_workspace_bytes.argtypes = [C.POINTER(CVit)]
+    L.ivit_vit_host_workspace_bytes.restype = C.c_size_t
+    L.ivit_vit_forward_host.argtypes = [vp, C.POINTER(CVit), vp, vp, vp, C.c_size_t]
+    L.ivit_ctx_profile_start.argtypes = [vp]
+    L.ivit_ctx_profile_stop.argtypes = [vp]
+    L.ivit_ctx_profile_get.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(C.c_float), C.POINTER(C.c_double)]
+    L.ivit_kernel_kind_name.argtypes = [i32]
+    L.ivit_kernel_kind_name.restype = C.c_char_p
     L.ivit_patchify.argtypes = [vp, vp, i64, i64, i64, i64, i64, i64, vp, i64]
     L.ivit_gather_rows.argtypes = [vp, vp, i64, vp, i64, i64, vp, i64]
     L.ivit_fill_rows.argtypes = [vp, vp, i64, vp, i64, i64]
@@ -200,6 +209,21 @@ class Context:
 
     def launch_count(self) -> int:
         return int(self.lib.ivit_ctx_launch_count(self.h))
+
+    def profile_start(self):
+        _chk(self.lib.ivit_ctx_profile_start(self.h), "ivit_ctx_profile_start")
+
+    def profile_stop(self):
+        """Ends the timing session; returns a list of (kernel class, milliseconds, algorithmic work)."""
+        n = self.lib.ivit_ctx_profile_stop(self.h)
+        if n < 0:
+            raise IvitError(n, "ivit_ctx_profile_stop")
+        out = []
+        kind, ms, work = C.c_int32(), C.c_float(), C.c_double()
+        for i in range(n):
+            _chk(self.lib.ivit_ctx_profile_get(self.h, i, C.byref(kind), C.byref(ms), C.byref(work)), "ivit_ctx_profile_get")
+            out.append((self.lib.ivit_kernel_kind_name(kind.value).decode(), ms.value, work.value))
+        return out
 
     # ---- operators (device tensors in, device tensors out) ----
 
@@ -313,6 +337,12 @@ class Context:
         return logits
 
 
+def vit_forward_host(ctx: "Context", model: "DeviceVit", image_host: torch.Tensor, logits_host: torch.Tensor, workspace):
+    """ivit_vit_forward_host: host image -> host logits, copies enqueued on the context's stream."""
+    _chk(ctx.lib.ivit_vit_forward_host(ctx.h, C.byref(model.c), image_host.data_ptr(), logits_host.data_ptr(),
+                                       workspace.data_ptr(), workspace.numel()), "ivit_vit_forward_host")
+
+
 class _Uploader:
     def __init__(self, device):
         self.device = device
@@ -364,6 +394,12 @@ class DeviceBlock:
     def workspace(self) -> torch.Tensor:
         return torch.empty(self.workspace_bytes(), dtype=torch.uint8, device=self.device)
 
+    def host_workspace(self) -> torch.Tensor:
+        n = load_library().ivit_vit_host_workspace_bytes(C.byref(self.c)) if isinstance(self, DeviceVit) else 0
+        if n == 0:
+            raise ValueError("ivit_vit_host_workspace_bytes rejected the model parameters")
+        return torch.empty(int(n), dtype=torch.uint8, device=self.device)
+
 
 class DeviceVit:
     """A ViT-family model resident on the device (ivit_vit_params and everything it points at)."""
@@ -392,3 +428,9 @@ class DeviceVit:
 
     def workspace(self) -> torch.Tensor:
         return torch.empty(self.workspace_bytes(), dtype=torch.uint8, device=self.device)
+
+    def host_workspace(self) -> torch.Tensor:
+        n = load_library().ivit_vit_host_workspace_bytes(C.byref(self.c)) if isinstance(self, DeviceVit) else 0
+        if n == 0:
+            raise ValueError("ivit_vit_host_workspace_bytes rejected the model parameters")
+        return torch.empty(int(n), dtype=torch.uint8, device=self.device)

@@ -8,6 +8,9 @@
 
 namespace ivit {
 
+constexpr int kProfMax = 8192;
+enum KernelKind { KIND_GEMM_TC = 0, KIND_GEMM_SIMT, KIND_LAYERNORM, KIND_SHIFTMAX, KIND_SHIFTGELU, KIND_GELU_TABLE,
+                  KIND_ATTENTION, KIND_MOVE, KIND_COUNT };
 constexpr int kGeluTableSlots = 16;
 constexpr int kGeluTableBytes = 128 * 256;  // [max(0,row max of x)] [x + 128] -> int8 output
 
@@ -33,6 +36,12 @@ struct ivit_ctx {
   int gemm_engine;
   int sm_count;
   void* tmap_encode;  // cuTensorMapEncodeTiled, resolved at context creation
+  // per-kernel timing session (ivit_ctx_profile_*)
+  bool profiling;
+  int prof_count;
+  cudaEvent_t* prof_ev;   // 2 * kProfMax events, created on first use
+  int* prof_kind;
+  double* prof_work;
 };
 
 namespace ivit {
@@ -84,10 +93,24 @@ inline bool scale_ok(const ivit_scale& s) {
   return s.mult > 0 && s.shift >= 1 && s.shift <= 62;
 }
 
-inline int check_launch(ivit_ctx* ctx, int n = 1) {
-  ctx->launches += n;
-  return cudaGetLastError() == cudaSuccess ? IVIT_OK : IVIT_ERR_CUDA;
-}
+// Brackets one kernel launch: counts it and, inside a timing session, records an event pair.
+struct LaunchScope {
+  ivit_ctx* ctx;
+  int slot;
+  LaunchScope(ivit_ctx* c, int kind, double work) : ctx(c), slot(-1) {
+    if (c->profiling && c->prof_count < kProfMax) {
+      slot = c->prof_count++;
+      c->prof_kind[slot] = kind;
+      c->prof_work[slot] = work;
+      cudaEventRecord(c->prof_ev[2 * slot], c->stream);
+    }
+  }
+  int done() {
+    ctx->launches += 1;
+    if (slot >= 0) cudaEventRecord(ctx->prof_ev[2 * slot + 1], ctx->stream);
+    return cudaGetLastError() == cudaSuccess ? IVIT_OK : IVIT_ERR_CUDA;
+  }
+};
 
 // launchers implemented in the kernel files ---------------------------------------------
 

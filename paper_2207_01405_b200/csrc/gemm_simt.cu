@@ -110,8 +110,9 @@ int launch_gemm_simt(ivit_ctx* ctx, const GemmProblem& g) {
   const int64_t tiles_m = (g.M + TM - 1) / TM, tiles_n = (g.N + TN - 1) / TN;
   const int64_t total = batches * tiles_m * tiles_n;
   if (total > 2147483647LL) return IVIT_ERR_UNSUPPORTED;
+  LaunchScope ls(ctx, KIND_GEMM_SIMT, 2.0 * (double)batches * (double)g.M * (double)g.N * (double)g.K);
   gemm_simt_kernel<<<(unsigned)total, 256, 0, ctx->stream>>>(g, tiles_m, tiles_n);
-  return check_launch(ctx);
+  return ls.done();
 }
 
 }  // namespace ivit

@@ -71,33 +71,37 @@ int launch_patchify(ivit_ctx* ctx, const int8_t* img, int64_t B, int64_t C, int6
                     int64_t P, int64_t window, int8_t* out, int64_t ldout) {
   const int64_t total = B * C * Hi * Wi / 4;
   if (total == 0) return IVIT_OK;
+  LaunchScope ls(ctx, KIND_MOVE, 2.0 * (double)total * 4);
   patchify_kernel<<<grid_for(ctx, total, 256), 256, 0, ctx->stream>>>(img, B, (int)C, (int)Hi, (int)Wi, (int)P,
                                                                        (int)window, out, ldout, total);
-  return check_launch(ctx);
+  return ls.done();
 }
 
 int launch_gather_rows(ivit_ctx* ctx, const int8_t* src, int64_t ldsrc, const int32_t* index,
                        int64_t n_rows, int64_t width, int8_t* dst, int64_t lddst) {
   if (n_rows == 0) return IVIT_OK;
+  LaunchScope ls(ctx, KIND_MOVE, 2.0 * (double)n_rows * (double)width);
   gather_rows_kernel<<<grid_for(ctx, n_rows * (width / 16), 256), 256, 0, ctx->stream>>>(
       src, ldsrc, index, n_rows, (int)(width / 16), dst, lddst);
-  return check_launch(ctx);
+  return ls.done();
 }
 
 int launch_fill_rows(ivit_ctx* ctx, const int8_t* src_row, int64_t width, int8_t* dst,
                      int64_t group_stride, int64_t groups) {
   if (groups == 0) return IVIT_OK;
+  LaunchScope ls(ctx, KIND_MOVE, (double)groups * (double)width);
   fill_rows_kernel<<<grid_for(ctx, groups * (width / 16), 256), 256, 0, ctx->stream>>>(
       src_row, (int)(width / 16), dst, group_stride, groups);
-  return check_launch(ctx);
+  return ls.done();
 }
 
 int launch_token_mean(ivit_ctx* ctx, const int8_t* in, int64_t ldin, int64_t groups, int64_t T,
                       int64_t C, ScaleDev scale, int8_t* out, int64_t ldout) {
   if (groups == 0) return IVIT_OK;
+  LaunchScope ls(ctx, KIND_MOVE, (double)groups * (double)C * (double)(T + 1));
   token_mean_kernel<<<grid_for(ctx, groups * C, 256), 256, 0, ctx->stream>>>(in, ldin, groups, (int)T, (int)C,
                                                                              scale, out, ldout);
-  return check_launch(ctx);
+  return ls.done();
 }
 
 }  // namespace ivit

@@ -206,6 +206,12 @@ int ivit_ctx_destroy(ivit_ctx* ctx) {
   cudaSetDevice(ctx->device);
   cudaFree(ctx->gelu_tables);
   cudaFreeHost(ctx->status_host);
+  if (ctx->prof_ev) {
+    for (int i = 0; i < 2 * kProfMax; ++i) cudaEventDestroy(ctx->prof_ev[i]);
+    delete[] ctx->prof_ev;
+    delete[] ctx->prof_kind;
+    delete[] ctx->prof_work;
+  }
   delete ctx;
   return IVIT_OK;
 }
@@ -423,6 +429,77 @@ int ivit_vit_forward(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* imag
   if ((rc = launch_layernorm(ctx, X, IVIT_I8, T * D, to_dev(p->lnf_gamma), p->lnf_beta, p->blocks[0].M_ln, Z, D, B, D))) return rc;
   return launch_gemm(ctx, linear_problem(Z, D, p->Whead, D, p->bhead, p->head_scale, nullptr, 0, 1, none, logits,
                                          p->classes, IVIT_I32, 0, 0, B, p->classes, D));
+}
+
+size_t ivit_vit_host_workspace_bytes(const ivit_vit_params* p) {
+  if (check_vit(p) != IVIT_OK) return 0;
+  const size_t img = align_up((size_t)(p->B * 3 * p->img * p->img), 256);
+  const size_t lg = align_up((size_t)(p->B * p->classes) * 4, 256);
+  return vit_ws(p).total + img + lg;
+}
+
+int ivit_vit_forward_host(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* image_host,
+                          int32_t* logits_host, void* workspace, size_t workspace_bytes) {
+  if (!ctx || !image_host || !logits_host) return IVIT_ERR_INVALID_ARG;
+  int rc = check_vit(p);
+  if (rc) return rc;
+  const size_t img_bytes = (size_t)(p->B * 3 * p->img * p->img), lg_bytes = (size_t)(p->B * p->classes) * 4;
+  const size_t inner = vit_ws(p).total, img_off = inner, lg_off = inner + align_up(img_bytes, 256);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < lg_off + align_up(lg_bytes, 256))
+    return IVIT_ERR_WORKSPACE;
+  char* ws = static_cast<char*>(workspace);
+  if (cudaMemcpyAsync(ws + img_off, image_host, img_bytes, cudaMemcpyHostToDevice, ctx->stream) != cudaSuccess)
+    return IVIT_ERR_CUDA;
+  rc = ivit_vit_forward(ctx, p, reinterpret_cast<const int8_t*>(ws + img_off), reinterpret_cast<int32_t*>(ws + lg_off),
+                        workspace, inner);
+  if (rc) return rc;
+  if (cudaMemcpyAsync(logits_host, ws + lg_off, lg_bytes, cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess)
+    return IVIT_ERR_CUDA;
+  return IVIT_OK;
+}
+
+int ivit_ctx_profile_start(ivit_ctx* ctx) {
+  if (!ctx) return IVIT_ERR_INVALID_ARG;
+  if (!ctx->prof_ev) {
+    ctx->prof_ev = new (std::nothrow) cudaEvent_t[2 * kProfMax];
+    ctx->prof_kind = new (std::nothrow) int[kProfMax];
+    ctx->prof_work = new (std::nothrow) double[kProfMax];
+    if (!ctx->prof_ev || !ctx->prof_kind || !ctx->prof_work) return IVIT_ERR_CUDA;
+    for (int i = 0; i < 2 * kProfMax; ++i)
+      if (cudaEventCreate(&ctx->prof_ev[i]) != cudaSuccess) return IVIT_ERR_CUDA;
+  }
+  ctx->prof_count = 0;
+  ctx->profiling = true;
+  return IVIT_OK;
+}
+
+int ivit_ctx_profile_stop(ivit_ctx* ctx) {
+  if (!ctx || !ctx->profiling) return IVIT_ERR_INVALID_ARG;
+  ctx->profiling = false;
+  if (cudaStreamSynchronize(ctx->stream) != cudaSuccess) return IVIT_ERR_CUDA;
+  return ctx->prof_count;
+}
+
+int ivit_ctx_profile_get(ivit_ctx* ctx, int32_t idx, int32_t* kind, float* ms, double* work) {
+  if (!ctx || !kind || !ms || !work || idx < 0 || idx >= ctx->prof_count || ctx->profiling) return IVIT_ERR_INVALID_ARG;
+  if (cudaEventElapsedTime(ms, ctx->prof_ev[2 * idx], ctx->prof_ev[2 * idx + 1]) != cudaSuccess) return IVIT_ERR_CUDA;
+  *kind = ctx->prof_kind[idx];
+  *work = ctx->prof_work[idx];
+  return IVIT_OK;
+}
+
+const char* ivit_kernel_kind_name(int32_t kind) {
+  switch (kind) {
+    case KIND_GEMM_TC: return "gemm_tcgen05";
+    case KIND_GEMM_SIMT: return "gemm_dp4a";
+    case KIND_LAYERNORM: return "layernorm";
+    case KIND_SHIFTMAX: return "shiftmax";
+    case KIND_SHIFTGELU: return "shiftgelu";
+    case KIND_GELU_TABLE: return "shiftgelu_table";
+    case KIND_ATTENTION: return "attention_fused";
+    case KIND_MOVE: return "data_movement";
+    default: return "unknown";
+  }
 }
 
 int ivit_patchify(ivit_ctx* ctx, const int8_t* img, int64_t B, int64_t C, int64_t Hi, int64_t Wi,

@@ -191,9 +191,10 @@ int launch_layernorm(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, 
   const int64_t want = (rows + wpb - 1) / wpb;
   const int grid = (int)(want < (int64_t)ctx->sm_count * 8 ? want : (int64_t)ctx->sm_count * 8);
   cudaStream_t st = ctx->stream;
+  LaunchScope ls(ctx, KIND_LAYERNORM, (double)rows * (double)C * (in_dtype == IVIT_I32 ? 5.0 : 2.0));
   if (in_dtype == IVIT_I32) {
     layernorm_i32_kernel<<<grid, threads, 0, st>>>((const int32_t*)in, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-    return check_launch(ctx);
+    return ls.done();
   }
   const int8_t* x = (const int8_t*)in;
   const int wpl = (int)((C / 4 + 31) / 32);
@@ -205,7 +206,7 @@ int launch_layernorm(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, 
   else if (wpl <= 8) layernorm_i8_kernel<8><<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
   else if (wpl <= 12) layernorm_i8_kernel<12><<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
   else layernorm_i8_long_kernel<<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-  return check_launch(ctx);
+  return ls.done();
 }
 
 // ------------------------------------------------------------------ Shiftmax
@@ -327,6 +328,7 @@ int launch_shiftmax(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, c
   if (rows == 0) return IVIT_OK;
   const int64_t want = (rows + 7) / 8;
   const int grid = (int)(want < (int64_t)ctx->sm_count * 8 ? want : (int64_t)ctx->sm_count * 8);
+  LaunchScope ls(ctx, KIND_SHIFTMAX, (double)rows * (double)d * (in_dtype == IVIT_I32 ? 5.0 : 2.0));
   if (in_dtype == IVIT_I8) {
     RowLoader<false> ld{in, ldin, nullptr, 0, 1, 0, 1};
     shiftmax_dispatch<false>(ld, p, out, ldout, rows, (int)d, grid, ctx->stream);
@@ -334,7 +336,7 @@ int launch_shiftmax(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, c
     RowLoader<true> ld{in, ldin, bias32, ldbias, bias_rows < 1 ? 1 : bias_rows, pre.mult, clamp_shift(pre.shift)};
     shiftmax_dispatch<true>(ld, p, out, ldout, rows, (int)d, grid, ctx->stream);
   }
-  return check_launch(ctx);
+  return ls.done();
 }
 
 // ------------------------------------------------------------------ ShiftGELU
@@ -435,9 +437,10 @@ int launch_shiftgelu(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_par
       ctx->gelu_next = (ctx->gelu_next + 1) % kGeluTableSlots;
     }
     ctx->gelu_keys[slot] = key;
+    LaunchScope lt(ctx, KIND_GELU_TABLE, (double)kGeluTableBytes);
     shiftgelu_table_kernel<<<128, 256, 0, ctx->stream>>>(p, post.mult, post.shift,
                                                           ctx->gelu_tables + (size_t)slot * kGeluTableBytes);
-    int rc = check_launch(ctx);
+    int rc = lt.done();
     if (rc) return rc;
   }
   const int8_t* table = ctx->gelu_tables + (size_t)slot * kGeluTableBytes;
@@ -445,6 +448,7 @@ int launch_shiftgelu(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_par
   const int grid = (int)(want < (int64_t)ctx->sm_count * 8 ? want : (int64_t)ctx->sm_count * 8);
   const int wpl = (int)((cols / 16 + 31) / 32);
   cudaStream_t st = ctx->stream;
+  LaunchScope ls(ctx, KIND_SHIFTGELU, 2.0 * (double)rows * (double)cols);
   if (wpl <= 1) shiftgelu_kernel<1><<<grid, 256, 0, st>>>(in, ldin, table, out, ldout, rows, (int)cols);
   else if (wpl <= 2) shiftgelu_kernel<2><<<grid, 256, 0, st>>>(in, ldin, table, out, ldout, rows, (int)cols);
   else if (wpl <= 3) shiftgelu_kernel<3><<<grid, 256, 0, st>>>(in, ldin, table, out, ldout, rows, (int)cols);
@@ -452,7 +456,7 @@ int launch_shiftgelu(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_par
   else if (wpl <= 6) shiftgelu_kernel<6><<<grid, 256, 0, st>>>(in, ldin, table, out, ldout, rows, (int)cols);
   else if (wpl <= 8) shiftgelu_kernel<8><<<grid, 256, 0, st>>>(in, ldin, table, out, ldout, rows, (int)cols);
   else shiftgelu_kernel<0><<<grid, 256, 0, st>>>(in, ldin, table, out, ldout, rows, (int)cols);
-  return check_launch(ctx);
+  return ls.done();
 }
 
 }  // namespace ivit
