@@ -233,6 +233,17 @@ def run_gpu(args):
         k["ms"] += ms
         k["work"] += work
     total_kernel_ms = sum(k["ms"] for k in by_kind.values())
+    if args.detail:
+        shapes = {}
+        for kind, ms, work in records:
+            k = shapes.setdefault((kind, work), [0, 0.0])
+            k[0] += 1
+            k[1] += ms
+        for (kind, work), (n, ms) in sorted(shapes.items(), key=lambda kv: -kv[1][1]):
+            unit = "TOP/s" if kind.startswith(("gemm", "attention")) else "GB/s"
+            rate = work / (ms / n * 1e-3) / (1e12 if unit == "TOP/s" else 1e9)
+            print(f"  {kind:16s} work={work:14.0f} launches/step={n // prof_steps:3d} us/launch={1e3 * ms / n:8.2f} "
+                  f"{rate:9.1f} {unit}", file=sys.stderr)
     kernels = {}
     for kind, k in sorted(by_kind.items(), key=lambda kv: -kv[1]["ms"]):
         per_step_ms = k["ms"] / prof_steps
@@ -291,6 +302,7 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ivit", choices=["ivit", "reference"])
+    ap.add_argument("--detail", action="store_true", help="print per-shape kernel times to stderr")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

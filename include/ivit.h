@@ -56,8 +56,10 @@ typedef struct ivit_ctx ivit_ctx; /* opaque */
 /* Dyadic number b / 2^c of Sec. 3.2 (DN()).  Per-channel when mult_c != NULL:
  * device arrays of one (mult, shift) per output channel.  Otherwise the
  * per-tensor pair (mult, shift), passed by value.  Bounds: 0 < mult < 2^31,
- * 1 <= shift <= 62 (per-channel arrays are checked by ivit_validate_scale at
- * model-load time; kernels clamp the shift into range). */
+ * 31 <= shift <= 62, i.e. ratios below 1 (per-channel arrays are checked by
+ * ivit_validate_scale at model-load time; kernels clamp the shift into
+ * range).  With these bounds rq() of any int32 value fits 32 bits, so the
+ * saturation that follows sees the exact value. */
 typedef struct {
   const int32_t* mult_c;
   const uint8_t* shift_c;
@@ -248,11 +250,11 @@ int ivit_token_mean(ivit_ctx* ctx, const int8_t* in, int64_t ldin, int64_t group
 
 /* ---- host-only helpers (offline) ---- */
 
-/* Sec. 3.2, DN(): ratio > 0 -> mult in [2^30, 2^31), shift in [1, 62]. */
+/* Sec. 3.2, DN(): 0 < ratio < 1 -> mult in [2^30, 2^31), shift in [31, 62]. */
 int ivit_dyadic_from_double(double ratio, int32_t* mult, int32_t* shift);
 /* Checks the bounds listed at ivit_exp_params. */
 int ivit_validate_exp_params(ivit_exp_params p, int64_t row_len, int32_t is_gelu);
-/* Checks a HOST copy of a per-channel scale: 0 < mult, 1 <= shift <= 62. */
+/* Checks a HOST copy of a per-channel scale: 0 < mult, 31 <= shift <= 62. */
 int ivit_validate_scale(const int32_t* mult_host, const uint8_t* shift_host, int64_t n);
 
 #ifdef __cplusplus

@@ -60,7 +60,8 @@ __device__ __forceinline__ int rq_hi(int a, int m, int s) {
   return (int)(p >> 32) >> (s - 32);
 }
 
-__host__ __device__ __forceinline__ int clamp_shift(int s) { return s < 1 ? 1 : (s > 62 ? 62 : s); }
+// Shifts are bounded to [31, 62]: with 0 < mult < 2^31 and |a| < 2^31 the requantised value then fits 32 bits.
+__host__ __device__ __forceinline__ int clamp_shift(int s) { return s < 31 ? 31 : (s > 62 ? 62 : s); }
 
 struct ScaleDev {
   const int32_t* mult_c;
@@ -90,7 +91,7 @@ inline bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3
 
 inline bool scale_ok(const ivit_scale& s) {
   if (s.mult_c) return s.shift_c != nullptr;
-  return s.mult > 0 && s.shift >= 1 && s.shift <= 62;
+  return s.mult > 0 && s.shift >= 31 && s.shift <= 62;
 }
 
 // Brackets one kernel launch: counts it and, inside a timing session, records an event pair.

@@ -1,5 +1,556 @@
-// tcgen05 tensor-core INT8 GEMM (placeholder until the kernel lands in this file).
-#include "common.cuh"
+// INT8 x INT8 -> INT32 GEMM on the sm_100a tensor cores with the dyadic requantisation of
+// Sec. 3.2 fused into the epilogue.  Persistent and warp-specialised:
+//
+//   warp 0      TMA producer: streams the k-blocks of both operands of successive output tiles
+//               through a ring of shared-memory stages (cp.async.bulk.tensor, hardware swizzle,
+//               mbarrier transaction counts);
+//   warp 1      owns tensor memory; one thread issues tcgen05.mma.kind::i8 (M = 128, N = BN,
+//               K = 32 per instruction) into one of two accumulator buffers;
+//   warps 2..17 epilogue: read the finished accumulator with tcgen05.ld (one TMEM lane per thread),
+//               requantise, add the residual, saturate and store - while the tensor core already
+//               works on the next tile in the other buffer.
+//
+// The 128 TMEM lanes of a tile hold the "P" operand's rows, the columns the "Q" operand's rows.
+//   * Dense layers (per-channel scale / bias):  P = weight rows (output channels), Q = activation
+//     rows.  A thread then owns ONE output channel: its multiplier, shift and bias stay in registers
+//     for the whole tile (no shared-memory traffic per value), and consecutive lanes touch
+//     consecutive channels of one output row, so residual loads and output stores coalesce.
+//   * Batched MatMul (per-tensor scale): P = rows of A, Q = rows of B (K-major, Q K^T) or B is
+//     MN-major ([K, N] rows, P V; the V tile is consumed as stored, without a transpose).  A thread
+//     owns one output row and stores 32 consecutive int8 values per chunk.
+//
+// One CTA per SM walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  Every device-side wait is
+// bounded: when one runs out the CTA records IVIT_ERR_DEVICE_TIMEOUT in the context's status
+// word, drains its outstanding copies, frees its tensor memory and returns.
+#include "tc_ptx.cuh"
+
 namespace ivit {
-int launch_gemm_tc(ivit_ctx*, const GemmProblem&) { return IVIT_ERR_UNSUPPORTED; }
+
+namespace {
+
+constexpr int BM = 128;          // TMEM lanes of a tile (UMMA M, cta_group::1)
+constexpr int BK = 128;          // bytes (= int8 elements) of K per pipeline stage
+constexpr int UMMA_K = 32;       // K of one tcgen05.mma.kind::i8
+constexpr int kMaxStages = 8;
+constexpr int kEpiWarps = 16;
+constexpr int kEpiThreads = 32 * kEpiWarps;
+constexpr int kThreads = 64 + kEpiThreads;
+
+struct TcArgs {
+  GemmEpilogue epi;
+  int64_t P, Q, K;   // extents along TMEM lanes / TMEM columns / contraction
+  int64_t sCo, sCi;
+  int64_t batches_inner;
+  int64_t total_tiles;
+  int tiles_p, tiles_q;
+  int BN;            // columns of the tile (multiple of 32, <= 256)
+  int stages;
+  int tmem_cols;     // power of two >= 2 * BN (two accumulator buffers)
+  int lanes_are_channels;  // 1: Dense orientation (lane = output channel, column = output row)
+  int q_mn;          // 1: the Q operand tile is MN-major ([k, n] rows of q_row_bytes)
+  int q_row_bytes;
+  int q_stage_bytes;
+  int p_pos[3], q_pos[3];  // tensor-map dimension (1..3) that holds the row / inner-batch / outer-batch coordinate
+  int tma_out;       // Dense orientation, int8: the output tile is staged in shared memory and stored by TMA
+  int* status;
+};
+
+#ifdef IVIT_TC_TRACE
+// debugging aid (compiled out by default): per-CTA, per-tile clock64() stamps of each role
+__device__ long long g_trace[148][40][8];
+#define IVIT_TRACE(tile_it, idx) do { if ((tile_it) < 40 && blockIdx.x < 148) g_trace[blockIdx.x][tile_it][idx] = clock64(); } while (0)
+#else
+#define IVIT_TRACE(tile_it, idx) do { } while (0)
+#endif
+
+struct TileCoord {
+  int64_t batch;
+  int bo, bi, p0, q0;
+};
+
+// Tiles are ordered q-block fastest, so that CTAs running at the same time share the P operand.
+__device__ __forceinline__ TileCoord tile_coord(const TcArgs& a, int64_t t) {
+  TileCoord c;
+  const uint32_t per_batch = (uint32_t)a.tiles_p * (uint32_t)a.tiles_q;
+  c.batch = t / per_batch;
+  const uint32_t t2 = (uint32_t)(t - c.batch * per_batch);
+  c.p0 = (int)(t2 / (uint32_t)a.tiles_q) * BM;
+  c.q0 = (int)(t2 % (uint32_t)a.tiles_q) * a.BN;
+  c.bo = (int)(c.batch / a.batches_inner);
+  c.bi = (int)(c.batch - (int64_t)c.bo * a.batches_inner);
+  return c;
+}
+
+__device__ __forceinline__ uint32_t epi_all(uint32_t pred) {
+  uint32_t all;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.and.pred p, 1, %2, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(all) : "r"(pred), "n"(kEpiThreads) : "memory");
+  return all;
+}
+
+__global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmP,
+                                                              const __grid_constant__ CUtensorMap tmQ,
+                                                              const __grid_constant__ CUtensorMap tmO, TcArgs a) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  // carve: [stages x (P tile | Q tile)] [barriers] [tmem address, issued count]
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t stage_bytes = BM * BK + a.q_stage_bytes;
+  const uint32_t stage_out = base + a.stages * stage_bytes;   // [BN rows][128 channels] int8, 128B-swizzled
+  const uint32_t bars_off = a.stages * stage_bytes + (a.tma_out ? a.BN * 128 : 0);
+  const uint32_t full0 = base + bars_off, empty0 = full0 + 8 * kMaxStages;
+  const uint32_t accf0 = empty0 + 8 * kMaxStages, acce0 = accf0 + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + bars_off + 8 * (2 * kMaxStages + 4));
+  volatile int* issued_slot = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int kblocks = (int)((a.K + BK - 1) / BK);
+
+  if (threadIdx.x == 0) {
+    prefetch_tmap(&tmP);
+    prefetch_tmap(&tmQ);
+    if (a.tma_out) prefetch_tmap(&tmO);
+    for (int s = 0; s < a.stages; ++s) {
+      mbar_init(full0 + 8 * s, 1);
+      mbar_init(empty0 + 8 * s, 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(accf0 + 8 * b, 1);
+      mbar_init(acce0 + 8 * b, kEpiWarps);
+    }
+    *issued_slot = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+  }
+  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), (uint32_t)a.tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ---------------- TMA producer ----------------
+    if (lane == 0) {
+      int g = 0;  // k-blocks issued so far, over all tiles of this CTA
+      bool ok = true;
+      int pit = 0;
+      for (int64_t t = blockIdx.x; ok && t < a.total_tiles; t += gridDim.x, ++pit) {
+        const TileCoord tc = tile_coord(a, t);
+        IVIT_TRACE(pit, 0);
+        for (int kb = 0; kb < kblocks; ++kb, ++g) {
+          const int s = g % a.stages;
+          if (g >= a.stages && !mbar_wait(empty0 + 8 * s, ((g / a.stages) & 1) ^ 1, a.status)) { ok = false; break; }
+          const uint32_t sp = base + s * stage_bytes, sq = sp + BM * BK;
+          mbar_expect_tx(full0 + 8 * s, stage_bytes);
+          int cp[4], cq[4];
+          cp[0] = kb * BK; cp[a.p_pos[0]] = tc.p0; cp[a.p_pos[1]] = tc.bi; cp[a.p_pos[2]] = tc.bo;
+          cq[0] = a.q_mn ? tc.q0 : kb * BK; cq[a.q_pos[0]] = a.q_mn ? kb * BK : tc.q0;
+          cq[a.q_pos[1]] = tc.bi; cq[a.q_pos[2]] = tc.bo;
+          tma_load_4d(sp, &tmP, full0 + 8 * s, cp[0], cp[1], cp[2], cp[3]);
+          tma_load_4d(sq, &tmQ, full0 + 8 * s, cq[0], cq[1], cq[2], cq[3]);
+          *issued_slot = g + 1;
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ---------------- MMA issuer ----------------
+    if (lane == 0) {
+      // instruction descriptor: D = S32, A = B = signed 8 bit, A K-major, M = 128, N = BN, no saturation
+      const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a.q_mn << 16) |
+                             ((uint32_t)(a.BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+      // Q descriptors: K-major rows of 128 bytes (128B swizzle, 1024 bytes per 8 rows); MN-major
+      // rows of q_row_bytes (swizzle = row width, 8 rows per group)
+      const uint32_t q_layout = !a.q_mn ? 2u : (a.q_row_bytes == 128 ? 2u : (a.q_row_bytes == 64 ? 4u : 6u));
+      const uint32_t q_sbo = !a.q_mn ? 1024u : 8u * a.q_row_bytes;
+      const uint32_t q_kstep = !a.q_mn ? UMMA_K : UMMA_K * a.q_row_bytes;
+      int g = 0, it = 0;
+      bool ok = true;
+      for (int64_t t = blockIdx.x; ok && t < a.total_tiles; t += gridDim.x, ++it) {
+        const int buf = it & 1;
+        // the epilogue must have drained this buffer (its use two tiles ago)
+        if (it >= 2 && !mbar_wait(acce0 + 8 * buf, ((it >> 1) & 1) ^ 1, a.status)) { ok = false; break; }
+        tc_fence_after();
+        IVIT_TRACE(it, 1);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * a.BN);
+        for (int kb = 0; kb < kblocks; ++kb, ++g) {
+          const int s = g % a.stages;
+          if (!mbar_wait(full0 + 8 * s, (g / a.stages) & 1, a.status)) { ok = false; break; }
+          tc_fence_after();
+          if (kb == 0) IVIT_TRACE(it, 2);
+          const uint32_t sp = base + s * stage_bytes, sq = sp + BM * BK;
+          const int64_t krem = a.K - (int64_t)kb * BK;
+          const int ksteps = krem >= BK ? BK / UMMA_K : (int)((krem + UMMA_K - 1) / UMMA_K);
+          for (int k = 0; k < ksteps; ++k) {
+            const uint64_t dp = smem_desc(sp + k * UMMA_K, 16, 1024, 2);
+            const uint64_t dq = smem_desc(sq + k * q_kstep, 16, q_sbo, q_layout);
+            umma_i8(d_tmem, dp, dq, idesc, (kb | k) != 0);
+          }
+          umma_commit(empty0 + 8 * s);   // the stage may be refilled once these MMAs have read it
+        }
+        if (ok) umma_commit(accf0 + 8 * buf);  // accumulator of this tile complete
+        IVIT_TRACE(it, 3);
+      }
+      if (!ok) {
+        // drain: copies that were issued but never consumed (only after a timeout)
+        const int issued = *issued_slot;
+        for (int j = g; j < issued; ++j) mbar_wait(full0 + 8 * (j % a.stages), (j / a.stages) & 1, a.status);
+      }
+    }
+  } else {
+    // ---------------- epilogue warps; TMEM lane quarter = warp % 4, 32-column chunks dealt round-robin ----------------
+    const int et = threadIdx.x - 64;
+    const int ew = warp - 2;
+    const int qd = warp & 3;
+    const int part = ew >> 2;
+    constexpr int kParts = kEpiWarps / 4;
+    const GemmEpilogue& e = a.epi;
+    const int rs_m = e.res_scale.mult, rs_s = clamp_shift(e.res_scale.shift);
+    const long long rs_c = 1ll << (rs_s - 1);
+
+    // Dense orientation: constants of this thread's channel; fetched one tile ahead
+    int nm = 1, ns = 32, nb = 0;
+    auto fetch_channel = [&](int p0) {
+      const int c = p0 + qd * 32 + lane;
+      nm = 1; ns = 32; nb = 0;
+      if (c < a.P) {
+        nm = e.scale.m(c);
+        ns = e.scale.s(c);
+        if (e.bias) nb = __ldg(e.bias + c);
+      }
+    };
+    if (a.lanes_are_channels && (int64_t)blockIdx.x < a.total_tiles) fetch_channel(tile_coord(a, blockIdx.x).p0);
+    // MatMul orientation: one per-tensor constant set
+    const int um = e.scale.mult, us = clamp_shift(e.scale.shift);
+    const long long uc = 1ll << (us - 1);
+
+    int it = 0;
+    for (int64_t t = blockIdx.x; t < a.total_tiles; t += gridDim.x, ++it) {
+      const TileCoord tc = tile_coord(a, t);
+      const int buf = it & 1;
+      const int cm = nm, cs = ns;
+      long long cc = (long long)nb * nm + (1ll << (ns - 1));   // bias * m + 2^(s-1)
+      asm volatile("" : "+l"(cc));   // keep it one 64-bit addend of the per-value multiply-add
+      const int64_t tn = t + gridDim.x;
+      if (a.lanes_are_channels && tn < a.total_tiles) fetch_channel(tile_coord(a, tn).p0);
+
+      // all epilogue threads take the same decision, so the named barrier never sees a partial group
+      if (a.tma_out && et == 0) tma_store_wait_read();   // the staging tile is free again
+      const uint32_t got = mbar_wait(accf0 + 8 * buf, (it >> 1) & 1, a.status) ? 1u : 0u;
+      if (!epi_all(got)) break;
+      tc_fence_after();
+      if (et == 0) IVIT_TRACE(it, 4);
+      const uint32_t t_row = tmem_base + ((uint32_t)(qd * 32) << 16) + (uint32_t)(buf * a.BN);
+
+      if (a.lanes_are_channels) {
+        // lane = output channel c, TMEM column = output row
+        const int c = tc.p0 + qd * 32 + lane;
+        const bool c_ok = c < a.P;
+        const int sh_lo = min(cs, 32), sh_hi = max(cs - 32, 0);
+        for (int j0 = part * 32; j0 < a.BN; j0 += 32 * kParts) {
+          const int64_t r0 = (int64_t)tc.q0 + j0;
+          if (r0 >= a.Q) break;
+          int v[32];
+#ifdef IVIT_TC_TRACE
+          if (et == 0 && j0 == 0) IVIT_TRACE(it, 6);
+#endif
+          tmem_ld32(t_row + (uint32_t)j0, v);
+#ifdef IVIT_TC_TRACE
+          if (et == 0 && j0 == 0) IVIT_TRACE(it, 7);
+#endif
+          const int nrow = (int)min((int64_t)32, a.Q - r0);
+          // requantise: one 32x32->64 multiply-add and two shifts per value, 32 independent chains
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const long long tt = (long long)v[j] * (long long)cm + cc;
+            v[j] = (int)__funnelshift_rc((unsigned)tt, (unsigned)(tt >> 32), sh_lo) >> sh_hi;
+          }
+          // residual port: the byte of (row, channel) is a coalesced load across the lanes
+          if (e.res) {
+            int64_t rr = (int64_t)((uint64_t)r0 % (uint64_t)e.res_rows);
+#pragma unroll
+            for (int h = 0; h < 32; h += 8) {
+              int xr[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                xr[j] = (c_ok && h + j < nrow) ? (int)__ldg(e.res + rr * e.ldres + c) : 0;
+                if (++rr == e.res_rows) rr = 0;
+              }
+#pragma unroll
+              for (int j = 0; j < 8; ++j) v[h + j] += (int)(((long long)xr[j] * rs_m + rs_c) >> rs_s);
+            }
+          }
+#ifdef IVIT_TC_TRACE
+          tmem_ld_wait(v);   // no outstanding load: only ties the stamp below to the finished values
+          if (et == 0 && j0 == 0) IVIT_TRACE(it, 0);   // reuses slot 0 (producer stamp) in trace builds
+#endif
+          if (e.out_dtype == IVIT_I32) {
+            int64_t ro = r0;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (j < nrow && c_ok) reinterpret_cast<int32_t*>(e.out)[(ro + j) * e.ldo + c] = v[j];
+            continue;
+          }
+          // int8: pack four rows per word, transpose 4x4 bytes inside each group of four lanes so
+          // that a lane ends up with four consecutive channels of one row (stage by stage over all
+          // eight words, so that the shuffles overlap), then store 4 bytes per lane and word
+          const int li = lane & 3;
+          const uint32_t sel1 = (li & 1) ? 0x3715u : 0x6240u;
+          const uint32_t sel2 = (li & 2) ? 0x3276u : 0x5410u;
+          uint32_t w[8], o[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) w[k] = pack_sat8(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) o[k] = __shfl_xor_sync(0xffffffffu, w[k], 1);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) w[k] = __byte_perm(w[k], o[k], sel1);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) o[k] = __shfl_xor_sync(0xffffffffu, w[k], 2);
+#pragma unroll
+          for (int k = 0; k < 8; ++k) w[k] = __byte_perm(w[k], o[k], sel2);
+          if (a.tma_out) {
+            // staging tile [row][128 channels]; 16-byte chunk index XOR (row & 7) is the 128B swizzle
+            // of the store map.  Word k belongs to tile row j0 + li + 4k: (row & 7) alternates between
+            // two values, so two base addresses plus immediates address all eight words.
+            const int trow = j0 + li;
+            const int cb = qd * 32 + (lane & ~3);
+            uint8_t* row0 = gen_base + (stage_out - base) + trow * 128 + (cb & 15);
+            uint8_t* pe = row0 + ((((cb >> 4) ^ (trow & 7)) & 7) << 4);
+            uint8_t* po = row0 + ((((cb >> 4) ^ ((trow + 4) & 7)) & 7) << 4);
+#pragma unroll
+            for (int k = 0; k < 8; k += 2) {
+              *reinterpret_cast<uint32_t*>(pe + 512 * k) = w[k];
+              *reinterpret_cast<uint32_t*>(po + 512 * (k + 1)) = w[k + 1];
+            }
+          } else {
+            // direct stores (grouped output rows): this lane's first word is row r0 + li, then + 4 per word
+            int64_t row = r0 + li, ro = row, grem = 0;
+            if (e.group_rows > 0) {
+              grem = (int64_t)((uint64_t)row % (uint64_t)e.group_rows);
+              ro = (int64_t)((uint64_t)row / (uint64_t)e.group_rows) * e.group_stride + grem;
+            }
+            const int cbase = tc.p0 + qd * 32 + (lane & ~3);
+            const bool cg_ok = cbase < a.P;   // P % 4 == 0: a group of four channels is valid as a whole
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+              if (cg_ok && 4 * k + li < nrow)
+                *reinterpret_cast<uint32_t*>(reinterpret_cast<int8_t*>(e.out) + ro * e.ldo + cbase) = w[k];
+              ro += 4;
+              if (e.group_rows > 0) {
+                grem += 4;
+                while (grem >= e.group_rows) { grem -= e.group_rows; ro += e.group_stride - e.group_rows; }
+              }
+            }
+          }
+        }
+        if (a.tma_out) {
+          // every epilogue warp has written its part of the staging tile: one thread stores it
+          fence_async_smem();
+          asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+          if (et == 0) tma_store_4d(&tmO, stage_out, tc.p0, tc.q0, 0, 0);
+        }
+      } else {
+        // lane = output row, TMEM column = output column
+        const int64_t r = (int64_t)tc.p0 + qd * 32 + lane;
+        const bool row_ok = r < a.P;
+        const int64_t out_row = tc.bo * a.sCo + tc.bi * a.sCi + r * e.ldo;
+        const int32_t* bias_row = e.bias32 ? e.bias32 + ((tc.batch % e.bias_batches) * a.P + r) * e.ldbias : nullptr;
+        for (int j0 = part * 32; j0 < a.BN; j0 += 32 * kParts) {
+          const int c0 = tc.q0 + j0;
+          if (c0 >= a.Q) break;
+          int v[32];
+          tmem_ld32(t_row + (uint32_t)j0, v);
+          if (!row_ok) continue;
+          const int ncol = (int)min((int64_t)32, a.Q - c0);
+          if (bias_row) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (j < ncol) v[j] += __ldg(bias_row + c0 + j);
+          }
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = (int)(((long long)v[j] * um + uc) >> us);
+          int8_t* o = reinterpret_cast<int8_t*>(e.out) + out_row + c0;
+          if (ncol == 32) {
+            int4 w0, w1;
+            w0.x = (int)pack_sat8(v[0], v[1], v[2], v[3]);     w0.y = (int)pack_sat8(v[4], v[5], v[6], v[7]);
+            w0.z = (int)pack_sat8(v[8], v[9], v[10], v[11]);   w0.w = (int)pack_sat8(v[12], v[13], v[14], v[15]);
+            w1.x = (int)pack_sat8(v[16], v[17], v[18], v[19]); w1.y = (int)pack_sat8(v[20], v[21], v[22], v[23]);
+            w1.z = (int)pack_sat8(v[24], v[25], v[26], v[27]); w1.w = (int)pack_sat8(v[28], v[29], v[30], v[31]);
+            reinterpret_cast<int4*>(o)[0] = w0;
+            reinterpret_cast<int4*>(o)[1] = w1;
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (j < ncol) o[j] = (int8_t)sat8(v[j]);
+          }
+        }
+      }
+      // this warp has read everything it needs from the buffer: hand it back to the MMA warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(acce0 + 8 * buf);
+      if (et == 0) IVIT_TRACE(it, 5);
+    }
+    if (a.tma_out && et == 0) tma_store_wait_all();
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, (uint32_t)a.tmem_cols);
+  }
+}
+
+// ---- host side ------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// 4-D int8 tensor map over {inner, rows, batch_inner, batch_outer}.  The three outer dimensions are
+// ordered by ascending byte stride (a head inside a token row has a smaller stride than the row);
+// pos[0..2] receive the tensor-map dimension that holds the row, inner-batch and outer-batch
+// coordinate.  Byte strides must be multiples of 16.
+bool make_map(ivit_ctx* ctx, CUtensorMap* map, const int8_t* ptr, int64_t inner, int64_t rows, int64_t bi, int64_t bo,
+              int64_t row_stride, int64_t si, int64_t so, int box_inner, int box_rows, CUtensorMapSwizzle swz,
+              int pos[3]) {
+  if ((reinterpret_cast<uintptr_t>(ptr) & 15) || row_stride % 16) return false;
+  struct Dim { int64_t size, stride; int box, which; };
+  Dim d[3] = {{rows, row_stride, box_rows, 0}, {bi, si, 1, 1}, {bo, so, 1, 2}};
+  // size-1 dimensions never contribute to an address: give them the largest stride so they sort last
+  int64_t big = row_stride;
+  for (int i = 1; i < 3; ++i)
+    if (d[i].size > 1 && d[i].stride > big) big = d[i].stride;
+  for (int i = 1; i < 3; ++i)
+    if (d[i].size <= 1) d[i].stride = big;
+  for (int i = 0; i < 3; ++i)
+    for (int j = i + 1; j < 3; ++j)
+      if (d[j].stride < d[i].stride) { Dim t = d[i]; d[i] = d[j]; d[j] = t; }
+  cuuint64_t dims[4] = {(cuuint64_t)inner, 0, 0, 0}, strides[3];
+  cuuint32_t box[4] = {(cuuint32_t)box_inner, 1, 1, 1};
+  for (int i = 0; i < 3; ++i) {
+    if (d[i].stride % 16 || d[i].stride <= 0 || d[i].stride >= (1ll << 40)) return false;
+    dims[i + 1] = (cuuint64_t)d[i].size;
+    strides[i] = (cuuint64_t)d[i].stride;
+    box[i + 1] = (cuuint32_t)d[i].box;
+    pos[d[i].which] = i + 1;
+  }
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(ctx->tmap_encode);
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int pow2_at_least(int v) {
+  int p = 32;
+  while (p < v) p <<= 1;
+  return p;
+}
+
+constexpr size_t kSmemBudget = 227 * 1024;
+constexpr size_t kSmemFixed = 1024 + 8 * (2 * kMaxStages + 4) + 32;
+
+bool g_attr_set = false;
+
+// Tile width along the TMEM columns: the candidate with the least (waves x tile cost).
+int pick_bn(int64_t extent, int64_t tiles_other, int sm_count) {
+  if (extent <= 256) return (int)((extent + 31) / 32 * 32);
+  int best = 0;
+  double best_cost = 0;
+  for (int bn : {256, 224, 192, 160, 128}) {
+    const int64_t tiles = tiles_other * ((extent + bn - 1) / bn);
+    const double waves = (double)((tiles + sm_count - 1) / sm_count);
+    const double cost = waves * (bn + 24.0);
+    if (!best || cost < best_cost) { best = bn; best_cost = cost; }
+  }
+  return best;
+}
+
+}  // namespace
+
+int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
+  if (!ctx->tmap_encode) return IVIT_ERR_UNSUPPORTED;
+  const int64_t batches = g.batches_outer * g.batches_inner;
+  if (batches == 0 || g.M == 0 || g.N == 0) return IVIT_OK;
+  if (g.M > 2147483647LL || g.N > 2147483647LL || g.K > 65536 || batches > 2147483647LL) return IVIT_ERR_UNSUPPORTED;
+  const GemmEpilogue& e = g.epi;
+  if (g.lda % 16 || g.ldb % 16 || g.sAo % 16 || g.sAi % 16 || g.sBo % 16 || g.sBi % 16) return IVIT_ERR_UNSUPPORTED;
+
+  TcArgs a{};
+  a.epi = e;
+  a.K = g.K; a.sCo = g.sCo; a.sCi = g.sCi; a.batches_inner = g.batches_inner;
+  a.status = ctx->status_dev;
+  CUtensorMap tmP, tmQ;
+  const bool dense = g.transB && batches == 1 && !e.bias32;
+  if (dense) {
+    if (g.N % 4 || e.ldo % 4 || (reinterpret_cast<uintptr_t>(e.out) & 3)) return IVIT_ERR_UNSUPPORTED;
+    // Dense orientation: lanes = output channels (rows of W), columns = output rows (rows of A)
+    a.lanes_are_channels = 1;
+    a.P = g.N; a.Q = g.M;
+    a.tiles_p = (int)((a.P + BM - 1) / BM);
+    a.BN = pick_bn(a.Q, a.tiles_p, ctx->sm_count);
+    a.q_stage_bytes = a.BN * BK;
+    if (!make_map(ctx, &tmP, g.B, g.K, g.N, 1, 1, g.ldb, 0, 0, BK, BM, CU_TENSOR_MAP_SWIZZLE_128B, a.p_pos) ||
+        !make_map(ctx, &tmQ, g.A, g.K, g.M, 1, 1, g.lda, 0, 0, BK, a.BN, CU_TENSOR_MAP_SWIZZLE_128B, a.q_pos))
+      return IVIT_ERR_UNSUPPORTED;
+  } else {
+    // MatMul orientation: lanes = rows of A; the epilogue's 16-byte stores need aligned output rows
+    if (e.out_dtype != IVIT_I8 || e.bias || e.res || e.scale.mult_c || e.group_rows > 0) return IVIT_ERR_UNSUPPORTED;
+    if ((reinterpret_cast<uintptr_t>(e.out) & 15) || e.ldo % 16 || g.sCo % 16 || g.sCi % 16) return IVIT_ERR_UNSUPPORTED;
+    a.P = g.M; a.Q = g.N;
+    a.tiles_p = (int)((a.P + BM - 1) / BM);
+    a.q_mn = g.transB ? 0 : 1;
+    if (!make_map(ctx, &tmP, g.A, g.K, g.M, g.batches_inner, g.batches_outer, g.lda, g.sAi, g.sAo, BK, BM,
+                  CU_TENSOR_MAP_SWIZZLE_128B, a.p_pos))
+      return IVIT_ERR_UNSUPPORTED;
+    if (a.q_mn) {
+      // the whole N extent is one tile whose k rows are N bytes wide: 32, 64 or 128
+      if (g.N != 32 && g.N != 64 && g.N != 128) return IVIT_ERR_UNSUPPORTED;
+      a.BN = (int)g.N;
+      a.q_row_bytes = (int)g.N;
+      a.q_stage_bytes = BK * a.q_row_bytes;
+      const CUtensorMapSwizzle swz = a.q_row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                                     : (a.q_row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+      if (!make_map(ctx, &tmQ, g.B, g.N, g.K, g.batches_inner, g.batches_outer, g.ldb, g.sBi, g.sBo, a.q_row_bytes, BK,
+                    swz, a.q_pos))
+        return IVIT_ERR_UNSUPPORTED;
+    } else {
+      a.BN = pick_bn(a.Q, (int64_t)a.tiles_p * batches, ctx->sm_count);
+      a.q_stage_bytes = a.BN * BK;
+      if (!make_map(ctx, &tmQ, g.B, g.K, g.N, g.batches_inner, g.batches_outer, g.ldb, g.sBi, g.sBo, BK, a.BN,
+                    CU_TENSOR_MAP_SWIZZLE_128B, a.q_pos))
+        return IVIT_ERR_UNSUPPORTED;
+    }
+  }
+  CUtensorMap tmO = tmP;
+  if (dense && e.out_dtype == IVIT_I8 && e.group_rows <= 0 && !(reinterpret_cast<uintptr_t>(e.out) & 15) && e.ldo % 16 == 0) {
+    int opos[3];
+    a.tma_out = make_map(ctx, &tmO, reinterpret_cast<const int8_t*>(e.out), g.N, g.M, 1, 1, e.ldo, 0, 0, BM, a.BN,
+                         CU_TENSOR_MAP_SWIZZLE_128B, opos) ? 1 : 0;
+  }
+  const size_t stage = (size_t)BM * BK + a.q_stage_bytes;
+  const size_t out_stage = a.tma_out ? (size_t)a.BN * 128 : 0;
+  int stages = (int)((kSmemBudget - kSmemFixed - out_stage) / stage);
+  a.stages = stages > kMaxStages ? kMaxStages : stages;
+  if (a.stages < 2) return IVIT_ERR_UNSUPPORTED;
+  a.tmem_cols = pow2_at_least(2 * a.BN);
+  a.tiles_q = (int)((a.Q + a.BN - 1) / a.BN);
+  a.total_tiles = (int64_t)a.tiles_p * a.tiles_q * batches;
+
+  const size_t smem = kSmemFixed + (size_t)a.stages * stage + out_stage;
+  if (!g_attr_set) {
+    if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess)
+      return IVIT_ERR_CUDA;
+    g_attr_set = true;
+  }
+  const unsigned grid = (unsigned)(a.total_tiles < ctx->sm_count ? a.total_tiles : ctx->sm_count);
+  LaunchScope ls(ctx, KIND_GEMM_TC, 2.0 * (double)batches * (double)g.M * (double)g.N * (double)g.K);
+  gemm_tc_kernel<<<grid, kThreads, smem, ctx->stream>>>(tmP, tmQ, tmO, a);
+  return ls.done();
+}
+
 }  // namespace ivit

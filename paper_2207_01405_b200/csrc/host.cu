@@ -543,7 +543,7 @@ int ivit_dyadic_from_double(double ratio, int32_t* mult, int32_t* shift) {
   long long b = std::llround(std::ldexp(mant, 31));
   int c = 31 - e;
   if (b == (1ll << 31)) { b = 1ll << 30; c -= 1; }
-  if (c < 1 || c > 62) return IVIT_ERR_RANGE;
+  if (c < 31 || c > 62) return IVIT_ERR_RANGE;
   *mult = (int32_t)b;
   *shift = c;
   return IVIT_OK;
@@ -557,7 +557,7 @@ int ivit_validate_exp_params(ivit_exp_params p, int64_t row_len, int32_t is_gelu
 int ivit_validate_scale(const int32_t* mult_host, const uint8_t* shift_host, int64_t n) {
   if (!mult_host || !shift_host || n < 0) return IVIT_ERR_INVALID_ARG;
   for (int64_t i = 0; i < n; ++i)
-    if (mult_host[i] <= 0 || shift_host[i] < 1 || shift_host[i] > 62) return IVIT_ERR_RANGE;
+    if (mult_host[i] <= 0 || shift_host[i] < 31 || shift_host[i] > 62) return IVIT_ERR_RANGE;
   return IVIT_OK;
 }
 

@@ -52,6 +52,7 @@ def test_dyadic_from_double_host_helper(lib):
     m, s = C.c_int32(), C.c_int32()
     assert lib.ivit_dyadic_from_double(-1.0, C.byref(m), C.byref(s)) == -1
     assert lib.ivit_dyadic_from_double(1e-30, C.byref(m), C.byref(s)) == -3
+    assert lib.ivit_dyadic_from_double(1.5, C.byref(m), C.byref(s)) == -3      # ratios >= 1 are not representable
 
 
 def test_validate_exp_params_bounds(lib):
@@ -73,6 +74,7 @@ def test_validate_scale(lib):
     assert binding.validate_scale(good) == 0
     assert binding.validate_scale(Scale(np.array([0], np.int32), np.array([31], np.uint8))) == -3
     assert binding.validate_scale(Scale(np.array([5], np.int32), np.array([63], np.uint8))) == -3
+    assert binding.validate_scale(Scale(np.array([5], np.int32), np.array([30], np.uint8))) == -3
 
 
 def test_context_needs_a_gpu(lib):

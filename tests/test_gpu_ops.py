@@ -231,3 +231,22 @@ def test_argument_validation_is_synchronous():
         c.linear(x, torch.zeros((32, 32), dtype=torch.int8, device="cuda"), None, b.DevScale(Scale(0, 35), "cuda"))
     assert e.value.code == -3
     assert c.poll_status() == 0
+
+
+def test_tensor_core_engine_takes_the_model_shapes():
+    """The tcgen05 kernel (not the CUDA-core one) serves the Dense and attention shapes of the workloads."""
+    g = _g()
+    c = g.ctx()
+    c.set_gemm_engine(0)
+    rng = np.random.default_rng(0)
+    sc = g.binding.DevScale(Scale(*dyadic(1e-3)), "cuda")
+    A, W = g.dev(rand_i8(rng, (393, 384))), g.dev(rand_i8(rng, (1152, 384)))
+    Q, K = g.dev(rand_i8(rng, (6, 197, 64))), g.dev(rand_i8(rng, (6, 197, 64)))
+    P, V = g.dev(rand_i8(rng, (6, 197, 197))), g.dev(rand_i8(rng, (6, 197, 64)))
+    c.profile_start()
+    c.linear(A, W, None, sc)
+    c.matmul(Q, K, True, sc)
+    c.matmul(P, V, False, sc)
+    kinds = [k for k, _, _ in c.profile_stop()]
+    assert kinds == ["gemm_tcgen05"] * 3, kinds
+    assert c.poll_status() == 0
