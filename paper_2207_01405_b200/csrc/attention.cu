@@ -1,0 +1,281 @@
+// Fused attention core of one encoder block (Sec. 3.1 MSA equation, Sec. 3.2 and Algorithm 1):
+//   S = Q_i K_i^T (+ bias)  ->  requantise to int8  ->  Shiftmax  ->  P_i V_i  ->  requantise
+// for one (image or window, head, 128-row tile) per CTA, rows up to 256 tokens long.
+//
+// The int32 score tile lives in tensor memory, never in HBM.  A thread owns one score row (one
+// TMEM lane), so the row maximum and the row sum of Algorithm 1 are thread-local: no shuffles.
+//   pass A  tcgen05.ld the row, requantise to int8 (kept packed in registers), running max;
+//   pass B  ShiftExp by table lookup (256 entries, I_max - I in [0, 255]), row sum, and the
+//           exponentials written back over the scores in tensor memory (tcgen05.st);
+//   pass C  one reciprocal per row (Eq. (IntDiv)), then exp * reciprocal >> shift per value; the
+//           int8 probabilities are written to shared memory in the K-major 128B-swizzled layout
+//           that the second MMA consumes as its A operand.
+// V is consumed as stored ([token, d] rows, MN-major B operand).  Every wait is bounded.
+#include "tc_ptx.cuh"
+
+namespace ivit {
+
+namespace {
+
+constexpr int kAttnThreads = 160;   // warp 0: TMA + MMA issue + TMEM owner; warps 1..4: one thread per score row
+constexpr int UK = 32;              // K of one tcgen05.mma.kind::i8
+
+struct AttnArgs {
+  int T, d, heads, Npad;            // Npad = T rounded up to 32 (score columns and P.V contraction length)
+  int64_t D;                        // heads * d
+  int tiles_m;                      // ceil(T / 128)
+  int tmem_cols;
+  int qk_m, qk_s, pv_m, pv_s;
+  ivit_exp_params smax;
+  const int32_t* bias;              // [bias_batches, T, T] or nullptr
+  int64_t bias_batches;
+  int8_t* O;                        // [B*T, D]
+  int q_pos[3], k_pos[3], v_pos[3];
+  int* status;
+};
+
+__global__ void __launch_bounds__(kAttnThreads) attention_kernel(const __grid_constant__ CUtensorMap tmQ,
+                                                                 const __grid_constant__ CUtensorMap tmK,
+                                                                 const __grid_constant__ CUtensorMap tmV, AttnArgs a) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
+  // [Q 128x128B][K Npad x 128B][V Npad x d][P 128 x 128B x kblocks][exp table][barriers]
+  const uint32_t q_off = 0, k_off = 128 * 128, v_off = k_off + a.Npad * 128;
+  const uint32_t p_off = (v_off + a.Npad * a.d + 1023u) & ~1023u;
+  const int p_kblocks = (a.Npad + 127) / 128;
+  const uint32_t tab_off = p_off + p_kblocks * 128 * 128;
+  const uint32_t bar_off = tab_off + 1024;
+  unsigned* tab = reinterpret_cast<unsigned*>(gen + tab_off);
+  const uint32_t bar_load = base + bar_off, bar_s = bar_load + 8, bar_p = bar_load + 16, bar_o = bar_load + 24;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + bar_off + 32);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tile = blockIdx.x % a.tiles_m;
+  const int bh = blockIdx.x / a.tiles_m;
+  const int h = bh % a.heads, b = bh / a.heads;
+  const int m0 = tile * 128;
+
+  if (threadIdx.x == 0) {
+    prefetch_tmap(&tmQ);
+    prefetch_tmap(&tmK);
+    prefetch_tmap(&tmV);
+    mbar_init(bar_load, 1);
+    mbar_init(bar_s, 1);
+    mbar_init(bar_p, 4);
+    mbar_init(bar_o, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+  }
+  if (warp == 0) tmem_alloc(smem_u32(tmem_slot), (uint32_t)a.tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ---- loads: Q tile, all keys, all values of this (image, head) ----
+      mbar_expect_tx(bar_load, 128 * 128 + a.Npad * 128 + a.Npad * a.d);
+      int c[4];
+      c[0] = 0; c[a.q_pos[0]] = m0; c[a.q_pos[1]] = h; c[a.q_pos[2]] = b;
+      tma_load_4d(base + q_off, &tmQ, bar_load, c[0], c[1], c[2], c[3]);
+      c[0] = 0; c[a.k_pos[0]] = 0; c[a.k_pos[1]] = h; c[a.k_pos[2]] = b;
+      tma_load_4d(base + k_off, &tmK, bar_load, c[0], c[1], c[2], c[3]);
+      c[0] = 0; c[a.v_pos[0]] = 0; c[a.v_pos[1]] = h; c[a.v_pos[2]] = b;
+      tma_load_4d(base + v_off, &tmV, bar_load, c[0], c[1], c[2], c[3]);
+      bool ok = mbar_wait(bar_load, 0, a.status);
+      if (ok) {
+        tc_fence_after();
+        // ---- S = Q K^T: M = 128, N = Npad, both operands K-major rows of 128 bytes ----
+        const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(a.Npad >> 3) << 17) | (8u << 24);
+        const int ks = (a.d + UK - 1) / UK;
+        for (int k = 0; k < ks; ++k)
+          umma_i8(tmem, smem_desc(base + q_off + k * UK, 16, 1024, 2), smem_desc(base + k_off + k * UK, 16, 1024, 2),
+                  idesc, k != 0);
+        umma_commit(bar_s);
+        // ---- O = P V once the probabilities are in shared memory ----
+        ok = mbar_wait(bar_p, 0, a.status);
+      }
+      if (ok) {
+        tc_fence_after();
+        const uint32_t idesc2 = (2u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(a.d >> 3) << 17) | (8u << 24);
+        const uint32_t v_layout = a.d == 128 ? 2u : (a.d == 64 ? 4u : 6u);
+        const int ks2 = a.Npad / UK;
+        for (int k = 0; k < ks2; ++k) {
+          const uint32_t pa = base + p_off + (k >> 2) * (128 * 128) + (k & 3) * UK;
+          umma_i8(tmem, smem_desc(pa, 16, 1024, 2), smem_desc(base + v_off + k * UK * a.d, 16, 8 * a.d, v_layout),
+                  idesc2, k != 0);
+        }
+        umma_commit(bar_o);
+      }
+    }
+  } else {
+    // ---- softmax / epilogue threads: TMEM lane quarter = warp % 4, thread = score row ----
+    const int st = threadIdx.x - 32;   // 0..127
+    for (int i = st; i < 256; i += 128) tab[i] = shiftexp(-i, a.smax.I0, a.smax.N);
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+    const int qd = warp & 3;
+    const int r = m0 + qd * 32 + lane;            // token (row) inside this image / window
+    const bool row_ok = r < a.T;
+    const uint32_t t_row = tmem + ((uint32_t)(qd * 32) << 16);
+    const int nch = a.Npad / 32;
+    const int64_t batch = (int64_t)b * a.heads + h;
+    const int32_t* brow = a.bias ? a.bias + ((batch % a.bias_batches) * a.T + (row_ok ? r : 0)) * (int64_t)a.T : nullptr;
+    const long long qk_c = 1ll << (a.qk_s - 1);
+
+    uint32_t xs[64];   // int8 scores of the row, packed four per word (Npad <= 256)
+    int mx = -128;
+    const bool got_s = mbar_wait(bar_s, 0, a.status);
+    if (got_s) {
+      tc_fence_after();
+      // pass A: requantise the scores to int8 (Sec. 3.2), running maximum
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        if (c < nch) {
+          int v[32];
+          tmem_ld32(t_row + c * 32, v);
+          if (brow) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (c * 32 + j < a.T) v[j] += __ldg(brow + c * 32 + j);
+          }
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = (int)(((long long)v[j] * a.qk_m + qk_c) >> a.qk_s);
+          uint32_t m4 = 0x80808080u;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            uint32_t w = pack_sat8(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+            const int valid = a.T - (c * 32 + 4 * k);   // columns of this word inside the row
+            if (valid < 4) {
+              const uint32_t keep = valid <= 0 ? 0u : (0xffffffffu >> (8 * (4 - valid)));
+              w = (w & keep) | (0x80808080u & ~keep);    // columns past T never win the maximum
+            }
+            xs[c * 8 + k] = w;
+            m4 = __vmaxs4(m4, w);
+          }
+          mx = max(mx, max(max((int)(int8_t)m4, (int)(int8_t)(m4 >> 8)), max((int)(int8_t)(m4 >> 16), (int)(int8_t)(m4 >> 24))));
+        }
+      }
+      // pass B: ShiftExp(I - I_max) by table, row sum, exponentials back into tensor memory
+      unsigned sum = 0;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        if (c < nch) {
+          int ev[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int x = (int)(int8_t)(xs[c * 8 + (j >> 2)] >> (8 * (j & 3)));
+            const unsigned e = (c * 32 + j < a.T) ? tab[mx - x] : 0u;
+            sum += e;
+            ev[j] = (int)e;
+          }
+          tmem_st32(t_row + c * 32, ev);
+        }
+      }
+      tmem_st_wait();
+      // pass C: Eq. (IntDiv) with M = 45, k_out = 8: (floor(2^45 / sum) * e) >> 38 = umulhi(factor, e) >> 6
+      const unsigned factor = (unsigned)((1ull << 45) / (unsigned long long)(sum ? sum : 1u));
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        if (c < nch) {
+          int ev[32];
+          tmem_ld32(t_row + c * 32, ev);
+          uint32_t w[8];
+#pragma unroll
+          for (int k = 0; k < 8; ++k) {
+            uint32_t o0 = min(127u, __umulhi(factor, (unsigned)ev[4 * k]) >> 6);
+            uint32_t o1 = min(127u, __umulhi(factor, (unsigned)ev[4 * k + 1]) >> 6);
+            uint32_t o2 = min(127u, __umulhi(factor, (unsigned)ev[4 * k + 2]) >> 6);
+            uint32_t o3 = min(127u, __umulhi(factor, (unsigned)ev[4 * k + 3]) >> 6);
+            w[k] = o0 | (o1 << 8) | (o2 << 16) | (o3 << 24);
+          }
+          // A operand of P V: row = tile row, k-block = 128 columns, 16-byte chunks XOR (row & 7)
+          const int trow = qd * 32 + lane;
+          uint8_t* prow = gen + p_off + (c >> 2) * (128 * 128) + trow * 128;
+          const int ch0 = (c & 3) * 2;
+          *reinterpret_cast<uint4*>(prow + (((ch0) ^ (trow & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(prow + (((ch0 + 1) ^ (trow & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+        }
+      }
+      fence_async_smem();
+    }
+    tc_fence_before();
+    __syncwarp();
+    if (got_s && lane == 0) mbar_arrive(bar_p);
+    // ---- output: O = sat8(rq(P V; pv_scale)), heads concatenated along the feature dimension ----
+    if (got_s && mbar_wait(bar_o, 0, a.status)) {
+      tc_fence_after();
+      const long long pv_c = 1ll << (a.pv_s - 1);
+      int8_t* orow = a.O + ((int64_t)b * a.T + r) * a.D + (int64_t)h * a.d;
+      for (int c = 0; c < a.d / 32; ++c) {
+        int v[32];
+        tmem_ld32(t_row + c * 32, v);
+        if (row_ok) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = (int)(((long long)v[j] * a.pv_m + pv_c) >> a.pv_s);
+          int4 w0, w1;
+          w0.x = (int)pack_sat8(v[0], v[1], v[2], v[3]);     w0.y = (int)pack_sat8(v[4], v[5], v[6], v[7]);
+          w0.z = (int)pack_sat8(v[8], v[9], v[10], v[11]);   w0.w = (int)pack_sat8(v[12], v[13], v[14], v[15]);
+          w1.x = (int)pack_sat8(v[16], v[17], v[18], v[19]); w1.y = (int)pack_sat8(v[20], v[21], v[22], v[23]);
+          w1.z = (int)pack_sat8(v[24], v[25], v[26], v[27]); w1.w = (int)pack_sat8(v[28], v[29], v[30], v[31]);
+          reinterpret_cast<int4*>(orow + c * 32)[0] = w0;
+          reinterpret_cast<int4*>(orow + c * 32)[1] = w1;
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after();
+    tmem_dealloc(tmem, (uint32_t)a.tmem_cols);
+  }
+}
+
+bool g_attn_attr = false;
+
+}  // namespace
+
+// Returns IVIT_ERR_UNSUPPORTED when the shape is outside the fused kernel (T > 256, d not 32/64/128,
+// misaligned tensors); the caller then composes the attention from MatMul and Shiftmax kernels.
+int launch_attention_fused(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* QKV, int8_t* O) {
+  if (!ctx->tmap_encode) return IVIT_ERR_UNSUPPORTED;
+  const int64_t B = p->B, T = p->T, D = p->D, h = p->heads, d = D / h;
+  if (T > 256 || (d != 32 && d != 64 && d != 128) || B * h > 2147483647LL / 2) return IVIT_ERR_UNSUPPORTED;
+  if ((reinterpret_cast<uintptr_t>(QKV) & 15) || (reinterpret_cast<uintptr_t>(O) & 15)) return IVIT_ERR_UNSUPPORTED;
+  if (B == 0) return IVIT_OK;
+  AttnArgs a{};
+  a.T = (int)T; a.d = (int)d; a.heads = (int)h; a.D = D;
+  a.Npad = (int)((T + 31) / 32 * 32);
+  a.tiles_m = (int)((T + 127) / 128);
+  a.tmem_cols = 32;
+  while (a.tmem_cols < a.Npad) a.tmem_cols <<= 1;
+  a.qk_m = p->qk_scale.mult; a.qk_s = clamp_shift(p->qk_scale.shift);
+  a.pv_m = p->pv_scale.mult; a.pv_s = clamp_shift(p->pv_scale.shift);
+  a.smax = p->smax;
+  a.bias = p->attn_bias; a.bias_batches = p->attn_bias ? p->attn_bias_batches : 1;
+  a.O = O;
+  a.status = ctx->status_dev;
+  const int64_t ldq = 3 * D;
+  CUtensorMap tmQ, tmK, tmV;
+  const CUtensorMapSwizzle vsw = d == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : (d == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+  if (!make_tensor_map(ctx, &tmQ, QKV, d, T, h, B, ldq, d, T * ldq, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B, a.q_pos) ||
+      !make_tensor_map(ctx, &tmK, QKV + D, d, T, h, B, ldq, d, T * ldq, 128, a.Npad, CU_TENSOR_MAP_SWIZZLE_128B, a.k_pos) ||
+      !make_tensor_map(ctx, &tmV, QKV + 2 * D, d, T, h, B, ldq, d, T * ldq, (int)d, a.Npad, vsw, a.v_pos))
+    return IVIT_ERR_UNSUPPORTED;
+  const uint32_t v_off = 128 * 128 + a.Npad * 128;
+  const uint32_t p_off = (v_off + a.Npad * a.d + 1023u) & ~1023u;
+  const size_t smem = 1024 + p_off + (size_t)((a.Npad + 127) / 128) * 128 * 128 + 1024 + 64;
+  if (!g_attn_attr) {
+    if (cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+      return IVIT_ERR_CUDA;
+    g_attn_attr = true;
+  }
+  const int64_t grid = B * h * a.tiles_m;
+  LaunchScope ls(ctx, KIND_ATTENTION, 4.0 * (double)(B * h) * (double)T * (double)T * (double)d);
+  attention_kernel<<<(unsigned)grid, kAttnThreads, smem, ctx->stream>>>(tmQ, tmK, tmV, a);
+  return ls.done();
+}
+
+}  // namespace ivit

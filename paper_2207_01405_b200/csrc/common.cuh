@@ -143,6 +143,8 @@ int launch_gemm_simt(ivit_ctx* ctx, const GemmProblem& g);
 // Returns IVIT_ERR_UNSUPPORTED when the shape does not qualify for the tensor-core kernel.
 int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g);
 int launch_gemm(ivit_ctx* ctx, const GemmProblem& g);
+// Fused Q K^T -> requant -> Shiftmax -> P V -> requant; IVIT_ERR_UNSUPPORTED when the shape does not qualify.
+int launch_attention_fused(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* QKV, int8_t* O);
 
 int launch_layernorm(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, ScaleDev gs,
                      const int32_t* beta, int M_ln, int8_t* out, int64_t ldout, int64_t rows, int64_t C);

@@ -26,6 +26,45 @@
 
 namespace ivit {
 
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// 4-D int8 tensor map over {inner, rows, batch_inner, batch_outer}.  The three outer dimensions are
+// ordered by ascending byte stride (a head inside a token row has a smaller stride than the row);
+// pos[0..2] receive the tensor-map dimension that holds the row, inner-batch and outer-batch
+// coordinate.  Byte strides must be multiples of 16.
+bool make_tensor_map(ivit_ctx* ctx, CUtensorMap* map, const int8_t* ptr, int64_t inner, int64_t rows, int64_t bi, int64_t bo,
+              int64_t row_stride, int64_t si, int64_t so, int box_inner, int box_rows, CUtensorMapSwizzle swz,
+              int pos[3]) {
+  if ((reinterpret_cast<uintptr_t>(ptr) & 15) || row_stride % 16) return false;
+  struct Dim { int64_t size, stride; int box, which; };
+  Dim d[3] = {{rows, row_stride, box_rows, 0}, {bi, si, 1, 1}, {bo, so, 1, 2}};
+  // size-1 dimensions never contribute to an address: give them the largest stride so they sort last
+  int64_t big = row_stride;
+  for (int i = 1; i < 3; ++i)
+    if (d[i].size > 1 && d[i].stride > big) big = d[i].stride;
+  for (int i = 1; i < 3; ++i)
+    if (d[i].size <= 1) d[i].stride = big;
+  for (int i = 0; i < 3; ++i)
+    for (int j = i + 1; j < 3; ++j)
+      if (d[j].stride < d[i].stride) { Dim t = d[i]; d[i] = d[j]; d[j] = t; }
+  cuuint64_t dims[4] = {(cuuint64_t)inner, 0, 0, 0}, strides[3];
+  cuuint32_t box[4] = {(cuuint32_t)box_inner, 1, 1, 1};
+  for (int i = 0; i < 3; ++i) {
+    if (d[i].stride % 16 || d[i].stride <= 0 || d[i].stride >= (1ll << 40)) return false;
+    dims[i + 1] = (cuuint64_t)d[i].size;
+    strides[i] = (cuuint64_t)d[i].stride;
+    box[i + 1] = (cuuint32_t)d[i].box;
+    pos[d[i].which] = i + 1;
+  }
+  const cuuint32_t estr[4] = {1, 1, 1, 1};
+  EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(ctx->tmap_encode);
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 namespace {
 
 constexpr int BM = 128;          // TMEM lanes of a tile (UMMA M, cta_group::1)
@@ -406,45 +445,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
 
 // ---- host side ------------------------------------------------------------------------------
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-// 4-D int8 tensor map over {inner, rows, batch_inner, batch_outer}.  The three outer dimensions are
-// ordered by ascending byte stride (a head inside a token row has a smaller stride than the row);
-// pos[0..2] receive the tensor-map dimension that holds the row, inner-batch and outer-batch
-// coordinate.  Byte strides must be multiples of 16.
-bool make_map(ivit_ctx* ctx, CUtensorMap* map, const int8_t* ptr, int64_t inner, int64_t rows, int64_t bi, int64_t bo,
-              int64_t row_stride, int64_t si, int64_t so, int box_inner, int box_rows, CUtensorMapSwizzle swz,
-              int pos[3]) {
-  if ((reinterpret_cast<uintptr_t>(ptr) & 15) || row_stride % 16) return false;
-  struct Dim { int64_t size, stride; int box, which; };
-  Dim d[3] = {{rows, row_stride, box_rows, 0}, {bi, si, 1, 1}, {bo, so, 1, 2}};
-  // size-1 dimensions never contribute to an address: give them the largest stride so they sort last
-  int64_t big = row_stride;
-  for (int i = 1; i < 3; ++i)
-    if (d[i].size > 1 && d[i].stride > big) big = d[i].stride;
-  for (int i = 1; i < 3; ++i)
-    if (d[i].size <= 1) d[i].stride = big;
-  for (int i = 0; i < 3; ++i)
-    for (int j = i + 1; j < 3; ++j)
-      if (d[j].stride < d[i].stride) { Dim t = d[i]; d[i] = d[j]; d[j] = t; }
-  cuuint64_t dims[4] = {(cuuint64_t)inner, 0, 0, 0}, strides[3];
-  cuuint32_t box[4] = {(cuuint32_t)box_inner, 1, 1, 1};
-  for (int i = 0; i < 3; ++i) {
-    if (d[i].stride % 16 || d[i].stride <= 0 || d[i].stride >= (1ll << 40)) return false;
-    dims[i + 1] = (cuuint64_t)d[i].size;
-    strides[i] = (cuuint64_t)d[i].stride;
-    box[i + 1] = (cuuint32_t)d[i].box;
-    pos[d[i].which] = i + 1;
-  }
-  const cuuint32_t estr[4] = {1, 1, 1, 1};
-  EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(ctx->tmap_encode);
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(ptr), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 int pow2_at_least(int v) {
   int p = 32;
   while (p < v) p <<= 1;
@@ -494,8 +494,8 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
     a.tiles_p = (int)((a.P + BM - 1) / BM);
     a.BN = pick_bn(a.Q, a.tiles_p, ctx->sm_count);
     a.q_stage_bytes = a.BN * BK;
-    if (!make_map(ctx, &tmP, g.B, g.K, g.N, 1, 1, g.ldb, 0, 0, BK, BM, CU_TENSOR_MAP_SWIZZLE_128B, a.p_pos) ||
-        !make_map(ctx, &tmQ, g.A, g.K, g.M, 1, 1, g.lda, 0, 0, BK, a.BN, CU_TENSOR_MAP_SWIZZLE_128B, a.q_pos))
+    if (!make_tensor_map(ctx, &tmP, g.B, g.K, g.N, 1, 1, g.ldb, 0, 0, BK, BM, CU_TENSOR_MAP_SWIZZLE_128B, a.p_pos) ||
+        !make_tensor_map(ctx, &tmQ, g.A, g.K, g.M, 1, 1, g.lda, 0, 0, BK, a.BN, CU_TENSOR_MAP_SWIZZLE_128B, a.q_pos))
       return IVIT_ERR_UNSUPPORTED;
   } else {
     // MatMul orientation: lanes = rows of A; the epilogue's 16-byte stores need aligned output rows
@@ -504,7 +504,7 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
     a.P = g.M; a.Q = g.N;
     a.tiles_p = (int)((a.P + BM - 1) / BM);
     a.q_mn = g.transB ? 0 : 1;
-    if (!make_map(ctx, &tmP, g.A, g.K, g.M, g.batches_inner, g.batches_outer, g.lda, g.sAi, g.sAo, BK, BM,
+    if (!make_tensor_map(ctx, &tmP, g.A, g.K, g.M, g.batches_inner, g.batches_outer, g.lda, g.sAi, g.sAo, BK, BM,
                   CU_TENSOR_MAP_SWIZZLE_128B, a.p_pos))
       return IVIT_ERR_UNSUPPORTED;
     if (a.q_mn) {
@@ -515,13 +515,13 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
       a.q_stage_bytes = BK * a.q_row_bytes;
       const CUtensorMapSwizzle swz = a.q_row_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
                                      : (a.q_row_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
-      if (!make_map(ctx, &tmQ, g.B, g.N, g.K, g.batches_inner, g.batches_outer, g.ldb, g.sBi, g.sBo, a.q_row_bytes, BK,
+      if (!make_tensor_map(ctx, &tmQ, g.B, g.N, g.K, g.batches_inner, g.batches_outer, g.ldb, g.sBi, g.sBo, a.q_row_bytes, BK,
                     swz, a.q_pos))
         return IVIT_ERR_UNSUPPORTED;
     } else {
       a.BN = pick_bn(a.Q, (int64_t)a.tiles_p * batches, ctx->sm_count);
       a.q_stage_bytes = a.BN * BK;
-      if (!make_map(ctx, &tmQ, g.B, g.K, g.N, g.batches_inner, g.batches_outer, g.ldb, g.sBi, g.sBo, BK, a.BN,
+      if (!make_tensor_map(ctx, &tmQ, g.B, g.K, g.N, g.batches_inner, g.batches_outer, g.ldb, g.sBi, g.sBo, BK, a.BN,
                     CU_TENSOR_MAP_SWIZZLE_128B, a.q_pos))
         return IVIT_ERR_UNSUPPORTED;
     }
@@ -529,7 +529,7 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
   CUtensorMap tmO = tmP;
   if (dense && e.out_dtype == IVIT_I8 && e.group_rows <= 0 && !(reinterpret_cast<uintptr_t>(e.out) & 15) && e.ldo % 16 == 0) {
     int opos[3];
-    a.tma_out = make_map(ctx, &tmO, reinterpret_cast<const int8_t*>(e.out), g.N, g.M, 1, 1, e.ldo, 0, 0, BM, a.BN,
+    a.tma_out = make_tensor_map(ctx, &tmO, reinterpret_cast<const int8_t*>(e.out), g.N, g.M, 1, 1, e.ldo, 0, 0, BM, a.BN,
                          CU_TENSOR_MAP_SWIZZLE_128B, opos) ? 1 : 0;
   }
   const size_t stage = (size_t)BM * BK + a.q_stage_bytes;

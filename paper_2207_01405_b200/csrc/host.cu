@@ -86,6 +86,10 @@ GemmProblem linear_problem(const int8_t* A, int64_t lda, const int8_t* W, int64_
 }
 
 int attention_impl(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* QKV, int8_t* O, char* ws, const BlockWs& w) {
+  if (ctx->gemm_engine == 0) {
+    const int rc = launch_attention_fused(ctx, p, QKV, O);
+    if (rc != IVIT_ERR_UNSUPPORTED) return rc;
+  }
   const int64_t B = p->B, T = p->T, D = p->D, h = p->heads, d = D / h, ldq = 3 * D, ldS = w.ldS;
   int8_t* S = reinterpret_cast<int8_t*>(ws + w.S);
   int8_t* P = reinterpret_cast<int8_t*>(ws + w.P);

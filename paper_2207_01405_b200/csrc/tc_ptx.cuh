@@ -11,6 +11,12 @@ namespace ivit {
 
 constexpr uint32_t kSpinLimit = 1u << 20;
 
+// 4-D int8 tensor map over {inner, rows, batch_inner, batch_outer} (defined with the GEMM); pos[0..2]
+// receive the tensor-map dimension (1..3) holding the row, inner-batch and outer-batch coordinate.
+bool make_tensor_map(ivit_ctx* ctx, CUtensorMap* map, const int8_t* ptr, int64_t inner, int64_t rows, int64_t bi,
+                     int64_t bo, int64_t row_stride, int64_t si, int64_t so, int box_inner, int box_rows,
+                     CUtensorMapSwizzle swz, int pos[3]);
+
 // ---- PTX wrappers -------------------------------------------------------------------------
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }

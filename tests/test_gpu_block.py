@@ -73,3 +73,20 @@ def test_vit_small_model_bit_exact():
     g.assert_equal(g.host(logits), want, "vit logits")
     assert np.abs(want).max() > 100 and len(np.unique(want)) > 100
     assert c.poll_status() == 0
+
+
+def test_fused_attention_kernel_serves_short_rows():
+    """Rows up to 256 tokens go through the fused tensor-core attention kernel; longer rows are composed."""
+    g = _g()
+    c = g.ctx()
+    rng = np.random.default_rng(2)
+    for (B, T, D, heads, fused) in [(2, 197, 384, 6, True), (4, 49, 96, 3, True), (1, 256, 128, 2, True), (1, 300, 128, 2, False)]:
+        blk = make_block(_Ids(50 + T), 1, B, T, D, heads, 4 * D, attn_bias_batches=heads if T == 49 else 0)
+        dblk = g.binding.DeviceBlock(blk, "cuda")
+        QKV = np.clip(np.rint(rng.standard_normal((B * T, 3 * D)) * 32), -128, 127).astype(np.int8)
+        c.profile_start()
+        Oo = c.attention(dblk, torch.from_numpy(QKV).cuda())
+        kinds = [k for k, _, _ in c.profile_stop()]
+        assert (kinds == ["attention_fused"]) == fused, (T, kinds)
+        g.assert_equal(g.host(Oo), O.attention(blk, QKV), f"attention T={T}")
+    assert c.poll_status() == 0
