@@ -91,6 +91,7 @@ struct TcArgs {
   int q_stage_bytes;
   int p_pos[3], q_pos[3];  // tensor-map dimension (1..3) that holds the row / inner-batch / outer-batch coordinate
   int tma_out;       // Dense orientation, int8: the output tile is staged in shared memory and stored by TMA
+  int tma_res;       // ... and the residual tile of the same shape is fetched by TMA into shared memory
   int* status;
 };
 
@@ -133,17 +134,19 @@ __device__ __forceinline__ uint32_t epi_all(uint32_t pred) {
 
 __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmP,
                                                               const __grid_constant__ CUtensorMap tmQ,
-                                                              const __grid_constant__ CUtensorMap tmO, TcArgs a) {
+                                                              const __grid_constant__ CUtensorMap tmO,
+                                                              const __grid_constant__ CUtensorMap tmR, TcArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   // carve: [stages x (P tile | Q tile)] [barriers] [tmem address, issued count]
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t stage_bytes = BM * BK + a.q_stage_bytes;
   const uint32_t stage_out = base + a.stages * stage_bytes;   // [BN rows][128 channels] int8, 128B-swizzled
-  const uint32_t bars_off = a.stages * stage_bytes + (a.tma_out ? a.BN * 128 : 0);
+  const uint32_t stage_res = stage_out + (a.tma_out ? a.BN * 128 : 0);   // residual tile, same layout
+  const uint32_t bars_off = a.stages * stage_bytes + (a.tma_out ? a.BN * 128 : 0) + (a.tma_res ? a.BN * 128 : 0);
   const uint32_t full0 = base + bars_off, empty0 = full0 + 8 * kMaxStages;
-  const uint32_t accf0 = empty0 + 8 * kMaxStages, acce0 = accf0 + 16;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + bars_off + 8 * (2 * kMaxStages + 4));
+  const uint32_t accf0 = empty0 + 8 * kMaxStages, acce0 = accf0 + 16, resf = acce0 + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + bars_off + 8 * (2 * kMaxStages + 5));
   volatile int* issued_slot = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -153,6 +156,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     prefetch_tmap(&tmP);
     prefetch_tmap(&tmQ);
     if (a.tma_out) prefetch_tmap(&tmO);
+    if (a.tma_res) prefetch_tmap(&tmR);
     for (int s = 0; s < a.stages; ++s) {
       mbar_init(full0 + 8 * s, 1);
       mbar_init(empty0 + 8 * s, 1);
@@ -161,6 +165,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       mbar_init(accf0 + 8 * b, 1);
       mbar_init(acce0 + 8 * b, kEpiWarps);
     }
+    mbar_init(resf, 1);
     *issued_slot = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -266,6 +271,13 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     const int um = e.scale.mult, us = clamp_shift(e.scale.shift);
     const long long uc = 1ll << (us - 1);
 
+    int res_issued = 0, res_waited = 0;   // residual tiles requested / consumed (thread et == 0 issues them)
+    if (a.tma_res && et == 0 && (int64_t)blockIdx.x < a.total_tiles) {
+      const TileCoord t0 = tile_coord(a, blockIdx.x);
+      mbar_expect_tx(resf, (uint32_t)a.BN * 128u);
+      tma_load_4d(stage_res, &tmR, resf, t0.p0, t0.q0, 0, 0);
+      ++res_issued;
+    }
     int it = 0;
     for (int64_t t = blockIdx.x; t < a.total_tiles; t += gridDim.x, ++it) {
       const TileCoord tc = tile_coord(a, t);
@@ -278,7 +290,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
 
       // all epilogue threads take the same decision, so the named barrier never sees a partial group
       if (a.tma_out && et == 0) tma_store_wait_read();   // the staging tile is free again
-      const uint32_t got = mbar_wait(accf0 + 8 * buf, (it >> 1) & 1, a.status) ? 1u : 0u;
+      uint32_t got = mbar_wait(accf0 + 8 * buf, (it >> 1) & 1, a.status) ? 1u : 0u;
+      if (a.tma_res && got) {
+        got = mbar_wait(resf, it & 1, a.status) ? 1u : 0u;
+        if (got) ++res_waited;
+      }
       if (!epi_all(got)) break;
       tc_fence_after();
       if (et == 0) IVIT_TRACE(it, 4);
@@ -308,7 +324,19 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
             v[j] = (int)__funnelshift_rc((unsigned)tt, (unsigned)(tt >> 32), sh_lo) >> sh_hi;
           }
           // residual port: the byte of (row, channel) is a coalesced load across the lanes
-          if (e.res) {
+          if (a.tma_res) {
+            // residual tile in shared memory: [row][128 channels], 16-byte chunks XOR (row & 7)
+            const int cb = qd * 32 + lane;
+            const uint8_t* rt = gen_base + (stage_res - base) + j0 * 128 + (cb & 15);
+            int off[8];
+#pragma unroll
+            for (int x = 0; x < 8; ++x) off[x] = ((cb >> 4) ^ x) << 4;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              const int xr = (int)*reinterpret_cast<const int8_t*>(rt + j * 128 + off[j & 7]);
+              v[j] += (int)(((long long)xr * rs_m + rs_c) >> rs_s);
+            }
+          } else if (e.res) {
             int64_t rr = (int64_t)((uint64_t)r0 % (uint64_t)e.res_rows);
 #pragma unroll
             for (int h = 0; h < 32; h += 8) {
@@ -389,7 +417,16 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
           // every epilogue warp has written its part of the staging tile: one thread stores it
           fence_async_smem();
           asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
-          if (et == 0) tma_store_4d(&tmO, stage_out, tc.p0, tc.q0, 0, 0);
+          if (et == 0) {
+            tma_store_4d(&tmO, stage_out, tc.p0, tc.q0, 0, 0);
+            if (a.tma_res && tn < a.total_tiles) {
+              // every warp is past its reads of the residual tile: fetch the next tile's
+              const TileCoord tq = tile_coord(a, tn);
+              mbar_expect_tx(resf, (uint32_t)a.BN * 128u);
+              tma_load_4d(stage_res, &tmR, resf, tq.p0, tq.q0, 0, 0);
+              ++res_issued;
+            }
+          }
         }
       } else {
         // lane = output row, TMEM column = output column
@@ -434,6 +471,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       if (et == 0) IVIT_TRACE(it, 5);
     }
     if (a.tma_out && et == 0) tma_store_wait_all();
+    // only after a timeout: a residual tile may still be in flight into shared memory
+    if (et == 0 && res_issued > res_waited) mbar_wait(resf, res_waited & 1, a.status);
   }
   tc_fence_before();
   __syncthreads();
@@ -452,7 +491,7 @@ int pow2_at_least(int v) {
 }
 
 constexpr size_t kSmemBudget = 227 * 1024;
-constexpr size_t kSmemFixed = 1024 + 8 * (2 * kMaxStages + 4) + 32;
+constexpr size_t kSmemFixed = 1024 + 8 * (2 * kMaxStages + 5) + 32;
 
 bool g_attr_set = false;
 
@@ -532,8 +571,14 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
     a.tma_out = make_tensor_map(ctx, &tmO, reinterpret_cast<const int8_t*>(e.out), g.N, g.M, 1, 1, e.ldo, 0, 0, BM, a.BN,
                          CU_TENSOR_MAP_SWIZZLE_128B, opos) ? 1 : 0;
   }
+  CUtensorMap tmR = tmP;
+  if (a.tma_out && e.res && e.res_rows >= g.M && !(reinterpret_cast<uintptr_t>(e.res) & 15) && e.ldres % 16 == 0) {
+    int rpos[3];
+    a.tma_res = make_tensor_map(ctx, &tmR, e.res, g.N, g.M, 1, 1, e.ldres, 0, 0, BM, a.BN, CU_TENSOR_MAP_SWIZZLE_128B,
+                                rpos) ? 1 : 0;
+  }
   const size_t stage = (size_t)BM * BK + a.q_stage_bytes;
-  const size_t out_stage = a.tma_out ? (size_t)a.BN * 128 : 0;
+  const size_t out_stage = (a.tma_out ? (size_t)a.BN * 128 : 0) + (a.tma_res ? (size_t)a.BN * 128 : 0);
   int stages = (int)((kSmemBudget - kSmemFixed - out_stage) / stage);
   a.stages = stages > kMaxStages ? kMaxStages : stages;
   if (a.stages < 2) return IVIT_ERR_UNSUPPORTED;
@@ -549,7 +594,7 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
   }
   const unsigned grid = (unsigned)(a.total_tiles < ctx->sm_count ? a.total_tiles : ctx->sm_count);
   LaunchScope ls(ctx, KIND_GEMM_TC, 2.0 * (double)batches * (double)g.M * (double)g.N * (double)g.K);
-  gemm_tc_kernel<<<grid, kThreads, smem, ctx->stream>>>(tmP, tmQ, tmO, a);
+  gemm_tc_kernel<<<grid, kThreads, smem, ctx->stream>>>(tmP, tmQ, tmO, tmR, a);
   return ls.done();
 }
 
