@@ -151,7 +151,7 @@ int ivit_shiftgelu(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_param
  *   F = sd ? floor(2^M_ln / sd) : 0;
  *   out[c] = sat8( rq(y[c] * F; gamma_scale[c]) + beta[c] )
  * gamma_scale per-channel or per-tensor; beta int32 [C] or NULL.
- * in_dtype IVIT_I8, or IVIT_I32 with |x| <= 2^20.  8 <= M_ln <= 30.
+ * in_dtype IVIT_I8, or IVIT_I32 with |x| <= 2^20.  8 <= M_ln <= 29 (so that y * F fits 32 bits).
  * C % 4 == 0, C <= 16384. */
 int ivit_layernorm(ivit_ctx* ctx, const void* in, int32_t in_dtype, int64_t ldin,
                    ivit_scale gamma_scale, const int32_t* beta, int32_t M_ln, int8_t* out,

@@ -2,8 +2,9 @@
 //   S = Q_i K_i^T (+ bias)  ->  requantise to int8  ->  Shiftmax  ->  P_i V_i  ->  requantise
 // for one (image or window, head, 128-row tile) per CTA, rows up to 256 tokens long.
 //
-// The int32 score tile lives in tensor memory, never in HBM.  A thread owns one score row (one
-// TMEM lane), so the row maximum and the row sum of Algorithm 1 are thread-local: no shuffles.
+// The int32 score tile lives in tensor memory, never in HBM.  Two threads share one score row (one
+// TMEM lane; they take alternate 32-column chunks), so the row maximum and the row sum of
+// Algorithm 1 need one exchange of two words through shared memory each: no shuffles.
 //   pass A  tcgen05.ld the row, requantise to int8 (kept packed in registers), running max;
 //   pass B  ShiftExp by table lookup (256 entries, I_max - I in [0, 255]), row sum, and the
 //           exponentials written back over the scores in tensor memory (tcgen05.st);
@@ -17,8 +18,16 @@ namespace ivit {
 
 namespace {
 
-constexpr int kAttnThreads = 160;   // warp 0: TMA + MMA issue + TMEM owner; warps 1..4: one thread per score row
+constexpr int kAttnThreads = 288;   // warp 0: TMA + MMA issue + TMEM owner; warps 1..8: two threads per score row
 constexpr int UK = 32;              // K of one tcgen05.mma.kind::i8
+
+#ifdef IVIT_ATTN_TRACE
+// debugging aid (compiled out by default): clock64() stamps of the phases of the first CTAs
+__device__ long long g_attn_trace[64][12];
+#define ATRACE(i) do { if (blockIdx.x < 64) g_attn_trace[blockIdx.x][i] = clock64(); } while (0)
+#else
+#define ATRACE(i) do { } while (0)
+#endif
 
 struct AttnArgs {
   int T, d, heads, Npad;            // Npad = T rounded up to 32 (score columns and P.V contraction length)
@@ -45,7 +54,8 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const __grid_co
   const uint32_t p_off = (v_off + a.Npad * a.d + 1023u) & ~1023u;
   const int p_kblocks = (a.Npad + 127) / 128;
   const uint32_t tab_off = p_off + p_kblocks * 128 * 128;
-  const uint32_t bar_off = tab_off + 1024;
+  const uint32_t part_off = tab_off + 1024;            // [2 halves][128 rows] partial max, then partial sum
+  const uint32_t bar_off = part_off + 2 * 128 * 4 * 2;
   unsigned* tab = reinterpret_cast<unsigned*>(gen + tab_off);
   const uint32_t bar_load = base + bar_off, bar_s = bar_load + 8, bar_p = bar_load + 16, bar_o = bar_load + 24;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + bar_off + 32);
@@ -57,12 +67,13 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const __grid_co
   const int m0 = tile * 128;
 
   if (threadIdx.x == 0) {
+    ATRACE(0);
     prefetch_tmap(&tmQ);
     prefetch_tmap(&tmK);
     prefetch_tmap(&tmV);
     mbar_init(bar_load, 1);
     mbar_init(bar_s, 1);
-    mbar_init(bar_p, 4);
+    mbar_init(bar_p, 8);
     mbar_init(bar_o, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -75,6 +86,7 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const __grid_co
 
   if (warp == 0) {
     if (lane == 0) {
+      ATRACE(1);
       // ---- loads: Q tile, all keys, all values of this (image, head) ----
       mbar_expect_tx(bar_load, 128 * 128 + a.Npad * 128 + a.Npad * a.d);
       int c[4];
@@ -85,6 +97,7 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const __grid_co
       c[0] = 0; c[a.v_pos[0]] = 0; c[a.v_pos[1]] = h; c[a.v_pos[2]] = b;
       tma_load_4d(base + v_off, &tmV, bar_load, c[0], c[1], c[2], c[3]);
       bool ok = mbar_wait(bar_load, 0, a.status);
+      ATRACE(2);
       if (ok) {
         tc_fence_after();
         // ---- S = Q K^T: M = 128, N = Npad, both operands K-major rows of 128 bytes ----
@@ -96,6 +109,7 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const __grid_co
         umma_commit(bar_s);
         // ---- O = P V once the probabilities are in shared memory ----
         ok = mbar_wait(bar_p, 0, a.status);
+        ATRACE(7);
       }
       if (ok) {
         tc_fence_after();
@@ -111,27 +125,34 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const __grid_co
       }
     }
   } else {
-    // ---- softmax / epilogue threads: TMEM lane quarter = warp % 4, thread = score row ----
-    const int st = threadIdx.x - 32;   // 0..127
-    for (int i = st; i < 256; i += 128) tab[i] = shiftexp(-i, a.smax.I0, a.smax.N);
-    asm volatile("bar.sync 1, 128;" ::: "memory");
+    // ---- softmax / epilogue threads: TMEM lane quarter = warp % 4; the two warps of a quarter
+    //      take the even / odd 32-column chunks of the same 32 rows ----
+    const int st = threadIdx.x - 32;   // 0..255
+    tab[st] = shiftexp(-st, a.smax.I0, a.smax.N);
     const int qd = warp & 3;
-    const int r = m0 + qd * 32 + lane;            // token (row) inside this image / window
+    const int half = (warp - 1) >> 2;
+    const int trow = qd * 32 + lane;              // row inside the tile
+    const int r = m0 + trow;                      // token (row) inside this image / window
     const bool row_ok = r < a.T;
+    const bool warp_ok = m0 + qd * 32 < a.T;      // warps whose 32 rows all lie past T only keep the barriers
     const uint32_t t_row = tmem + ((uint32_t)(qd * 32) << 16);
     const int nch = a.Npad / 32;
     const int64_t batch = (int64_t)b * a.heads + h;
     const int32_t* brow = a.bias ? a.bias + ((batch % a.bias_batches) * a.T + (row_ok ? r : 0)) * (int64_t)a.T : nullptr;
     const long long qk_c = 1ll << (a.qk_s - 1);
+    int* part_max = reinterpret_cast<int*>(gen + part_off);
+    unsigned* part_sum = reinterpret_cast<unsigned*>(gen + part_off + 2 * 128 * 4);
 
-    uint32_t xs[64];   // int8 scores of the row, packed four per word (Npad <= 256)
+    uint32_t xs[32];   // int8 scores of this thread's chunks, packed four per word
     int mx = -128;
     const bool got_s = mbar_wait(bar_s, 0, a.status);
-    if (got_s) {
-      tc_fence_after();
+    if (got_s) tc_fence_after();
+    if (st == 0) ATRACE(3);
+    if (got_s && warp_ok) {
       // pass A: requantise the scores to int8 (Sec. 3.2), running maximum
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
+      for (int cc = 0; cc < 4; ++cc) {
+        const int c = 2 * cc + half;
         if (c < nch) {
           int v[32];
           tmem_ld32(t_row + c * 32, v);
@@ -140,58 +161,84 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const __grid_co
             for (int j = 0; j < 32; ++j)
               if (c * 32 + j < a.T) v[j] += __ldg(brow + c * 32 + j);
           }
+          if (a.qk_s >= 32) {   // the usual case: high word of the 64-bit multiply-add, shifted by s - 32
+            const int sh = a.qk_s - 32;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) v[j] = (int)(((long long)v[j] * a.qk_m + qk_c) >> a.qk_s);
+            for (int j = 0; j < 32; ++j) v[j] = (int)(((long long)v[j] * a.qk_m + qk_c) >> 32) >> sh;
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = (int)(((long long)v[j] * a.qk_m + qk_c) >> a.qk_s);
+          }
           uint32_t m4 = 0x80808080u;
 #pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            uint32_t w = pack_sat8(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
-            const int valid = a.T - (c * 32 + 4 * k);   // columns of this word inside the row
-            if (valid < 4) {
-              const uint32_t keep = valid <= 0 ? 0u : (0xffffffffu >> (8 * (4 - valid)));
-              w = (w & keep) | (0x80808080u & ~keep);    // columns past T never win the maximum
+          for (int k = 0; k < 8; ++k) xs[cc * 8 + k] = pack_sat8(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+          if (c == nch - 1) {   // only the last chunk can hold columns past T: they never win the maximum
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+              const int valid = a.T - (c * 32 + 4 * k);
+              if (valid < 4) {
+                const uint32_t keep = valid <= 0 ? 0u : (0xffffffffu >> (8 * (4 - valid)));
+                xs[cc * 8 + k] = (xs[cc * 8 + k] & keep) | (0x80808080u & ~keep);
+              }
             }
-            xs[c * 8 + k] = w;
-            m4 = __vmaxs4(m4, w);
           }
+#pragma unroll
+          for (int k = 0; k < 8; ++k) m4 = __vmaxs4(m4, xs[cc * 8 + k]);
           mx = max(mx, max(max((int)(int8_t)m4, (int)(int8_t)(m4 >> 8)), max((int)(int8_t)(m4 >> 16), (int)(int8_t)(m4 >> 24))));
         }
       }
+      part_max[half * 128 + trow] = mx;
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (st == 0) ATRACE(4);
+    unsigned sum = 0;
+    if (got_s && warp_ok) {
+      mx = max(part_max[trow], part_max[128 + trow]);
       // pass B: ShiftExp(I - I_max) by table, row sum, exponentials back into tensor memory
-      unsigned sum = 0;
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
+      for (int cc = 0; cc < 4; ++cc) {
+        const int c = 2 * cc + half;
         if (c < nch) {
           int ev[32];
+          const uint32_t mx4 = (uint32_t)(mx & 0xff) * 0x01010101u;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const int x = (int)(int8_t)(xs[c * 8 + (j >> 2)] >> (8 * (j & 3)));
-            const unsigned e = (c * 32 + j < a.T) ? tab[mx - x] : 0u;
-            sum += e;
-            ev[j] = (int)e;
+          for (int k = 0; k < 8; ++k) {
+            const uint32_t d4 = __vsub4(mx4, xs[cc * 8 + k]);   // I_max - I per byte, in [0, 255]
+#pragma unroll
+            for (int b = 0; b < 4; ++b)
+              ev[4 * k + b] = (int)tab[__byte_perm(d4, 0, 0x4440 + b)];
           }
+          if (c == nch - 1) {   // columns past T contribute nothing
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (c * 32 + j >= a.T) ev[j] = 0;
+          }
+#pragma unroll
+          for (int j = 0; j < 32; ++j) sum += (unsigned)ev[j];
           tmem_st32(t_row + c * 32, ev);
         }
       }
       tmem_st_wait();
+      part_sum[half * 128 + trow] = sum;
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    if (st == 0) ATRACE(5);
+    if (got_s && warp_ok) {
+      sum = part_sum[trow] + part_sum[128 + trow];
       // pass C: Eq. (IntDiv) with M = 45, k_out = 8: (floor(2^45 / sum) * e) >> 38 = umulhi(factor, e) >> 6
       const unsigned factor = (unsigned)((1ull << 45) / (unsigned long long)(sum ? sum : 1u));
 #pragma unroll
-      for (int c = 0; c < 8; ++c) {
+      for (int cc = 0; cc < 4; ++cc) {
+        const int c = 2 * cc + half;
         if (c < nch) {
           int ev[32];
           tmem_ld32(t_row + c * 32, ev);
           uint32_t w[8];
 #pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            uint32_t o0 = min(127u, __umulhi(factor, (unsigned)ev[4 * k]) >> 6);
-            uint32_t o1 = min(127u, __umulhi(factor, (unsigned)ev[4 * k + 1]) >> 6);
-            uint32_t o2 = min(127u, __umulhi(factor, (unsigned)ev[4 * k + 2]) >> 6);
-            uint32_t o3 = min(127u, __umulhi(factor, (unsigned)ev[4 * k + 3]) >> 6);
-            w[k] = o0 | (o1 << 8) | (o2 << 16) | (o3 << 24);
-          }
+          for (int k = 0; k < 8; ++k)   // values are <= 128: the saturating pack clamps the one possible 128 to 127
+            w[k] = pack_sat8((int)(__umulhi(factor, (unsigned)ev[4 * k]) >> 6), (int)(__umulhi(factor, (unsigned)ev[4 * k + 1]) >> 6),
+                             (int)(__umulhi(factor, (unsigned)ev[4 * k + 2]) >> 6), (int)(__umulhi(factor, (unsigned)ev[4 * k + 3]) >> 6));
           // A operand of P V: row = tile row, k-block = 128 columns, 16-byte chunks XOR (row & 7)
-          const int trow = qd * 32 + lane;
           uint8_t* prow = gen + p_off + (c >> 2) * (128 * 128) + trow * 128;
           const int ch0 = (c & 3) * 2;
           *reinterpret_cast<uint4*>(prow + (((ch0) ^ (trow & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -203,12 +250,15 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const __grid_co
     tc_fence_before();
     __syncwarp();
     if (got_s && lane == 0) mbar_arrive(bar_p);
+    if (st == 0) ATRACE(6);
     // ---- output: O = sat8(rq(P V; pv_scale)), heads concatenated along the feature dimension ----
     if (got_s && mbar_wait(bar_o, 0, a.status)) {
       tc_fence_after();
+      if (st == 0) ATRACE(8);
       const long long pv_c = 1ll << (a.pv_s - 1);
       int8_t* orow = a.O + ((int64_t)b * a.T + r) * a.D + (int64_t)h * a.d;
-      for (int c = 0; c < a.d / 32; ++c) {
+      for (int c = half; c < a.d / 32; c += 2) {
+        if (!warp_ok) break;
         int v[32];
         tmem_ld32(t_row + c * 32, v);
         if (row_ok) {
@@ -227,6 +277,7 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const __grid_co
   }
   tc_fence_before();
   __syncthreads();
+  if (threadIdx.x == 0) ATRACE(9);
   if (warp == 0) {
     tc_fence_after();
     tmem_dealloc(tmem, (uint32_t)a.tmem_cols);
@@ -266,7 +317,7 @@ int launch_attention_fused(ivit_ctx* ctx, const ivit_block_params* p, const int8
     return IVIT_ERR_UNSUPPORTED;
   const uint32_t v_off = 128 * 128 + a.Npad * 128;
   const uint32_t p_off = (v_off + a.Npad * a.d + 1023u) & ~1023u;
-  const size_t smem = 1024 + p_off + (size_t)((a.Npad + 127) / 128) * 128 * 128 + 1024 + 64;
+  const size_t smem = 1024 + p_off + (size_t)((a.Npad + 127) / 128) * 128 * 128 + 1024 + 2048 + 64;
   if (!g_attn_attr) {
     if (cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
       return IVIT_ERR_CUDA;

@@ -54,7 +54,7 @@ int check_block(const ivit_block_params* p) {
   const int64_t d = p->D / p->heads;
   if (d % 16 || p->D % 16 || p->H % 16) return IVIT_ERR_UNSUPPORTED;
   if (!p->Wqkv || !p->Wo || !p->W1 || !p->W2) return IVIT_ERR_INVALID_ARG;
-  if (p->M_ln < 8 || p->M_ln > 30) return IVIT_ERR_RANGE;
+  if (p->M_ln < 8 || p->M_ln > 29) return IVIT_ERR_RANGE;
   const ivit_scale* sc[] = {&p->ln1_gamma, &p->qkv_scale, &p->qk_scale, &p->pv_scale, &p->o_scale, &p->res1_scale,
                             &p->ln2_gamma, &p->fc1_scale, &p->gelu_post, &p->fc2_scale, &p->res2_scale};
   for (const ivit_scale* s : sc)
@@ -329,7 +329,7 @@ int ivit_layernorm(ivit_ctx* ctx, const void* in, int32_t in_dtype, int64_t ldin
   if (!ctx || !in || !out || rows < 0 || C < 1) return IVIT_ERR_INVALID_ARG;
   if (in_dtype != IVIT_I8 && in_dtype != IVIT_I32) return IVIT_ERR_INVALID_ARG;
   if (C % 4 || C > 16384) return IVIT_ERR_UNSUPPORTED;
-  if (M_ln < 8 || M_ln > 30) return IVIT_ERR_RANGE;
+  if (M_ln < 8 || M_ln > 29) return IVIT_ERR_RANGE;
   if (ldin < C || ldout < C) return IVIT_ERR_INVALID_ARG;
   if (!aligned16(in) || !aligned16(out) || ldout % 16 || ldin % (in_dtype == IVIT_I8 ? 16 : 4)) return IVIT_ERR_ALIGNMENT;
   if (!scale_ok(gamma_scale)) return IVIT_ERR_RANGE;

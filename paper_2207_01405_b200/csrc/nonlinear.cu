@@ -111,6 +111,96 @@ __global__ void __launch_bounds__(256) layernorm_i8_kernel(const int8_t* __restr
   }
 }
 
+// Batched form: a warp owns ROWS consecutive rows.  The rows' sums are reduced together, the
+// per-row scalars (mean, integer square root, reciprocal) are then computed by ROWS different lanes
+// at once instead of redundantly by all 32, and the per-channel constants of the lane's channels
+// are loaded once for all ROWS rows: v = ((x*F - mu*F) * m + 2^(s-1)) >> s + beta.
+template <int WPL, int ROWS>
+__global__ void __launch_bounds__(256) layernorm_i8_batched_kernel(const int8_t* __restrict__ in, int64_t ldin,
+                                                                   ScaleDev gs, const int32_t* __restrict__ beta,
+                                                                   int M_ln, int8_t* __restrict__ out, int64_t ldout,
+                                                                   int64_t rows, int C) {
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  const int nwords = C >> 2;
+  // constants of this lane's channels (word i of the lane covers channels 4*(lane+32i) .. +3):
+  // v = (yF * m + 2^(s-1)) >> s + beta, the shift split into min(s,32) and s - 32
+  int pm[WPL][4], ps[WPL][4], pb[WPL][4];
+  bool all_hi = true;   // every shift >= 32: the value is the high product word shifted by s - 32
+#pragma unroll
+  for (int i = 0; i < WPL; ++i) {
+    const int idx = lane + 32 * i;
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      const int c = idx * 4 + b;
+      pm[i][b] = idx < nwords ? gs.m(c) : 1;
+      ps[i][b] = idx < nwords ? gs.s(c) : 32;
+      pb[i][b] = (idx < nwords && beta) ? __ldg(beta + c) : 0;
+      all_hi = all_hi && ps[i][b] >= 32;
+    }
+  }
+  all_hi = __all_sync(0xffffffffu, all_hi);
+  for (int64_t r0 = warp * ROWS; r0 < rows; r0 += nwarps * ROWS) {
+    int w[ROWS][WPL];
+    int my_s1 = 0, my_s2 = 0;
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) {
+      const bool ok = r0 + r < rows;
+      const int* src = reinterpret_cast<const int*>(in + (r0 + r) * ldin);
+      int s1 = 0, s2 = 0;
+#pragma unroll
+      for (int i = 0; i < WPL; ++i) {
+        const int idx = lane + 32 * i;
+        w[r][i] = (ok && idx < nwords) ? __ldg(src + idx) : 0;
+        s1 = __dp4a(w[r][i], 0x01010101, s1);
+        s2 = __dp4a(w[r][i], w[r][i], s2);
+      }
+      s1 = warp_sum(s1);
+      s2 = warp_sum(s2);
+      if (lane == r) { my_s1 = s1; my_s2 = s2; }
+    }
+    // lane r (< ROWS) holds the sums of row r0 + r: mean (round half up), sum of squared
+    // deviations = sum x^2 - 2 mu sum x + C mu^2, integer square root, reciprocal
+    const int mu = floordiv_pos(2 * my_s1 + C, 2 * C);
+    const long long V = (long long)my_s2 - 2ll * mu * my_s1 + (long long)C * mu * mu;
+    const unsigned sd = isqrt_u32((unsigned)V);
+    const int F = sd == 0 ? 0 : (int)((1u << M_ln) / sd);
+    const int muF = (int)((unsigned)mu * (unsigned)F);
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) {
+      const int Fr = __shfl_sync(0xffffffffu, F, r);
+      const int muFr = __shfl_sync(0xffffffffu, muF, r);
+      if (r0 + r < rows) {
+        int* dst = reinterpret_cast<int*>(out + (r0 + r) * ldout);
+#pragma unroll
+        for (int i = 0; i < WPL; ++i) {
+          const int idx = lane + 32 * i;
+          if (idx < nwords) {
+            int v[4];
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+              const int x = (int)(int8_t)(w[r][i] >> (8 * b));
+              // (x - mu) * F, formed modulo 2^32 (the difference always fits: |y F| <= 2^(M_ln+1))
+              const int yF = (int)((unsigned)x * (unsigned)Fr - (unsigned)muFr);
+              if (all_hi) {
+                const long long t = (long long)yF * pm[i][b] + (1ll << (ps[i][b] - 1));
+                v[b] = ((int)(t >> 32) >> (ps[i][b] - 32)) + pb[i][b];
+              } else {
+                v[b] = rq(yF, pm[i][b], ps[i][b]) + pb[i][b];
+              }
+            }
+            unsigned t, d;
+            asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(t) : "r"(v[3]), "r"(v[2]), "r"(0));
+            asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(v[1]), "r"(v[0]), "r"(t));
+            dst[idx] = (int)d;
+          }
+        }
+      }
+    }
+  }
+}
+
 // Any C (multiple of 4): the row is read again from cache for the output pass.
 __global__ void __launch_bounds__(256) layernorm_i8_long_kernel(const int8_t* __restrict__ in, int64_t ldin,
                                                                 ScaleDev gs, const int32_t* __restrict__ beta,
@@ -198,11 +288,19 @@ int launch_layernorm(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, 
   }
   const int8_t* x = (const int8_t*)in;
   const int wpl = (int)((C / 4 + 31) / 32);
-  if (wpl <= 1) layernorm_i8_kernel<1><<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-  else if (wpl <= 2) layernorm_i8_kernel<2><<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-  else if (wpl <= 3) layernorm_i8_kernel<3><<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-  else if (wpl <= 4) layernorm_i8_kernel<4><<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-  else if (wpl <= 6) layernorm_i8_kernel<6><<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+  if (wpl <= 4) {
+    // batched kernel: 4 rows per warp, small blocks so that one wave covers the rows
+    const int rpw = 4, tb = 128;
+    const int64_t warps = (rows + rpw - 1) / rpw;
+    const int64_t wantb = (warps + tb / 32 - 1) / (tb / 32);
+    const int gridb = (int)(wantb < (int64_t)ctx->sm_count * 16 ? wantb : (int64_t)ctx->sm_count * 16);
+    if (wpl <= 1) layernorm_i8_batched_kernel<1, 4><<<gridb, tb, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+    else if (wpl <= 2) layernorm_i8_batched_kernel<2, 4><<<gridb, tb, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+    else if (wpl <= 3) layernorm_i8_batched_kernel<3, 4><<<gridb, tb, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+    else layernorm_i8_batched_kernel<4, 4><<<gridb, tb, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+    return ls.done();
+  }
+  if (wpl <= 6) layernorm_i8_kernel<6><<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
   else if (wpl <= 8) layernorm_i8_kernel<8><<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
   else if (wpl <= 12) layernorm_i8_kernel<12><<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
   else layernorm_i8_long_kernel<<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
