@@ -92,6 +92,8 @@ struct TcArgs {
   int p_pos[3], q_pos[3];  // tensor-map dimension (1..3) that holds the row / inner-batch / outer-batch coordinate
   int tma_out;       // Dense orientation, int8: the output tile is staged in shared memory and stored by TMA
   int tma_res;       // ... and the residual tile of the same shape is fetched by TMA into shared memory
+  int q_resident;    // Dense orientation, short K: all k-blocks of the Q (activation row) tile stay in shared
+                     // memory while the CTA walks the channel blocks; only weight tiles stream through the ring
   int* status;
 };
 
@@ -108,18 +110,41 @@ struct TileCoord {
   int bo, bi, p0, q0;
 };
 
-// Tiles are ordered q-block fastest, so that CTAs running at the same time share the P operand.
+// Tiles are ordered p-block fastest and every CTA owns a contiguous range of them, so that the tiles a
+// CTA works on in a row share their Q operand (the activation rows of a Dense layer).
 __device__ __forceinline__ TileCoord tile_coord(const TcArgs& a, int64_t t) {
   TileCoord c;
   const uint32_t per_batch = (uint32_t)a.tiles_p * (uint32_t)a.tiles_q;
   c.batch = t / per_batch;
   const uint32_t t2 = (uint32_t)(t - c.batch * per_batch);
-  c.p0 = (int)(t2 / (uint32_t)a.tiles_q) * BM;
-  c.q0 = (int)(t2 % (uint32_t)a.tiles_q) * a.BN;
+  c.q0 = (int)(t2 / (uint32_t)a.tiles_p) * a.BN;
+  c.p0 = (int)(t2 % (uint32_t)a.tiles_p) * BM;
   c.bo = (int)(c.batch / a.batches_inner);
   c.bi = (int)(c.batch - (int64_t)c.bo * a.batches_inner);
   return c;
 }
+
+// Walks a contiguous range of tiles without divisions: p-block fastest, then q-block, then batch.
+struct TileIter {
+  int p, q, bi, bo;       // block indices
+  long long batch;
+  __device__ __forceinline__ void init(const TcArgs& a, int64_t t) {
+    const TileCoord c = tile_coord(a, t);
+    p = c.p0 / BM; q = c.q0 / a.BN; bi = c.bi; bo = c.bo; batch = c.batch;
+  }
+  __device__ __forceinline__ void next(const TcArgs& a) {
+    if (++p == a.tiles_p) {
+      p = 0;
+      if (++q == a.tiles_q) {
+        q = 0;
+        ++batch;
+        if (++bi == (int)a.batches_inner) { bi = 0; ++bo; }
+      }
+    }
+  }
+  __device__ __forceinline__ int p0() const { return p * BM; }
+  __device__ __forceinline__ int q0(const TcArgs& a) const { return q * a.BN; }
+};
 
 __device__ __forceinline__ uint32_t epi_all(uint32_t pred) {
   uint32_t all;
@@ -140,17 +165,22 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
   // carve: [stages x (P tile | Q tile)] [barriers] [tmem address, issued count]
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t stage_bytes = BM * BK + a.q_stage_bytes;
-  const uint32_t stage_out = base + a.stages * stage_bytes;   // [BN rows][128 channels] int8, 128B-swizzled
+  const uint32_t stage_bytes = BM * BK + (a.q_resident ? 0 : a.q_stage_bytes);
+  const int kblocks = (int)((a.K + BK - 1) / BK);
+  const uint32_t qres_bytes = a.q_resident ? kblocks * a.q_stage_bytes : 0;
+  const uint32_t qres = base + a.stages * stage_bytes;         // resident Q tile: kblocks x [BN rows x 128 B]
+  const uint32_t stage_out = qres + qres_bytes;                // [BN rows][128 channels] int8, 128B-swizzled
   const uint32_t stage_res = stage_out + (a.tma_out ? a.BN * 128 : 0);   // residual tile, same layout
-  const uint32_t bars_off = a.stages * stage_bytes + (a.tma_out ? a.BN * 128 : 0) + (a.tma_res ? a.BN * 128 : 0);
+  const uint32_t bars_off = a.stages * stage_bytes + qres_bytes + (a.tma_out ? a.BN * 128 : 0) + (a.tma_res ? a.BN * 128 : 0);
   const uint32_t full0 = base + bars_off, empty0 = full0 + 8 * kMaxStages;
-  const uint32_t accf0 = empty0 + 8 * kMaxStages, acce0 = accf0 + 16, resf = acce0 + 16;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + bars_off + 8 * (2 * kMaxStages + 5));
+  const uint32_t accf0 = empty0 + 8 * kMaxStages, acce0 = accf0 + 16, resf = acce0 + 16, qresf = resf + 8, qrese = resf + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + bars_off + 8 * (2 * kMaxStages + 7));
   volatile int* issued_slot = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int kblocks = (int)((a.K + BK - 1) / BK);
+  // this CTA's contiguous range of tiles
+  const int64_t t_begin = a.total_tiles * blockIdx.x / gridDim.x, t_end = a.total_tiles * (blockIdx.x + 1) / gridDim.x;
+  volatile int* qres_issued = issued_slot + 1;
 
   if (threadIdx.x == 0) {
     prefetch_tmap(&tmP);
@@ -166,6 +196,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       mbar_init(acce0 + 8 * b, kEpiWarps);
     }
     mbar_init(resf, 1);
+    mbar_init(qresf, 1);
+    mbar_init(qrese, 1);
+    *qres_issued = 0;
     *issued_slot = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -179,24 +212,41 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
   if (warp == 0) {
     // ---------------- TMA producer ----------------
     if (lane == 0) {
-      int g = 0;  // k-blocks issued so far, over all tiles of this CTA
+      int issued = 0;            // k-blocks issued so far, over all tiles of this CTA
+      int s = 0, wrap = 0;       // ring slot of the next k-block and how often the ring has wrapped
       bool ok = true;
-      int pit = 0;
-      for (int64_t t = blockIdx.x; ok && t < a.total_tiles; t += gridDim.x, ++pit) {
-        const TileCoord tc = tile_coord(a, t);
+      int pit = 0, qi = 0, cur_q = -1;
+      TileIter ti;
+      ti.init(a, t_begin);
+      // which tensor-map coordinate (1..3) carries the row / inner batch / outer batch index
+      const int pr = a.p_pos[0], pbi = a.p_pos[1], qr = a.q_pos[0], qbi = a.q_pos[1];
+      for (int64_t t = t_begin; ok && t < t_end; ++t, ++pit, ti.next(a)) {
+        const int p0 = ti.p0(), q0 = ti.q0(a);
         IVIT_TRACE(pit, 0);
-        for (int kb = 0; kb < kblocks; ++kb, ++g) {
-          const int s = g % a.stages;
-          if (g >= a.stages && !mbar_wait(empty0 + 8 * s, ((g / a.stages) & 1) ^ 1, a.status)) { ok = false; break; }
+        const int pc1 = pr == 1 ? p0 : (pbi == 1 ? ti.bi : ti.bo), pc2 = pr == 2 ? p0 : (pbi == 2 ? ti.bi : ti.bo),
+                  pc3 = pr == 3 ? p0 : (pbi == 3 ? ti.bi : ti.bo);
+        if (a.q_resident && q0 != cur_q) {
+          // new activation row block: refill the resident tile once every MMA on the old one is done
+          if (qi > 0 && !mbar_wait(qrese, (qi - 1) & 1, a.status)) { ok = false; break; }
+          mbar_expect_tx(qresf, qres_bytes);
+          for (int kb = 0; kb < kblocks; ++kb)
+            tma_load_4d(qres + kb * a.q_stage_bytes, &tmQ, qresf, kb * BK, qr == 1 ? q0 : 0, qr == 2 ? q0 : 0, qr == 3 ? q0 : 0);
+          cur_q = q0;
+          *qres_issued = ++qi;
+        }
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (wrap > 0 && !mbar_wait(empty0 + 8 * s, (wrap & 1) ^ 1, a.status)) { ok = false; break; }
           const uint32_t sp = base + s * stage_bytes, sq = sp + BM * BK;
           mbar_expect_tx(full0 + 8 * s, stage_bytes);
-          int cp[4], cq[4];
-          cp[0] = kb * BK; cp[a.p_pos[0]] = tc.p0; cp[a.p_pos[1]] = tc.bi; cp[a.p_pos[2]] = tc.bo;
-          cq[0] = a.q_mn ? tc.q0 : kb * BK; cq[a.q_pos[0]] = a.q_mn ? kb * BK : tc.q0;
-          cq[a.q_pos[1]] = tc.bi; cq[a.q_pos[2]] = tc.bo;
-          tma_load_4d(sp, &tmP, full0 + 8 * s, cp[0], cp[1], cp[2], cp[3]);
-          tma_load_4d(sq, &tmQ, full0 + 8 * s, cq[0], cq[1], cq[2], cq[3]);
-          *issued_slot = g + 1;
+          tma_load_4d(sp, &tmP, full0 + 8 * s, kb * BK, pc1, pc2, pc3);
+          if (!a.q_resident) {
+            const int qrow = a.q_mn ? kb * BK : q0;     // MN-major: rows of the map are k, the inner index is n
+            const int qc0 = a.q_mn ? q0 : kb * BK;
+            tma_load_4d(sq, &tmQ, full0 + 8 * s, qc0, qr == 1 ? qrow : (qbi == 1 ? ti.bi : ti.bo),
+                        qr == 2 ? qrow : (qbi == 2 ? ti.bi : ti.bo), qr == 3 ? qrow : (qbi == 3 ? ti.bi : ti.bo));
+          }
+          *issued_slot = ++issued;
+          if (++s == a.stages) { s = 0; ++wrap; }
         }
       }
     }
@@ -206,42 +256,69 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       // instruction descriptor: D = S32, A = B = signed 8 bit, A K-major, M = 128, N = BN, no saturation
       const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a.q_mn << 16) |
                              ((uint32_t)(a.BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-      // Q descriptors: K-major rows of 128 bytes (128B swizzle, 1024 bytes per 8 rows); MN-major
-      // rows of q_row_bytes (swizzle = row width, 8 rows per group)
-      const uint32_t q_layout = !a.q_mn ? 2u : (a.q_row_bytes == 128 ? 2u : (a.q_row_bytes == 64 ? 4u : 6u));
-      const uint32_t q_sbo = !a.q_mn ? 1024u : 8u * a.q_row_bytes;
-      const uint32_t q_kstep = !a.q_mn ? UMMA_K : UMMA_K * a.q_row_bytes;
-      int g = 0, it = 0;
+      // P descriptors: K-major rows of 128 bytes (128B swizzle, 1024 bytes per 8 rows).  Q: the same,
+      // or MN-major rows of q_row_bytes (swizzle = row width, 8 rows per group).  Along K a descriptor
+      // advances by 32 bytes (K-major) or 32 rows (MN-major): an add on the low word.
+      const uint32_t p_hi = desc_hi(1024, 2);
+      const uint32_t q_hi = !a.q_mn ? desc_hi(1024, 2)
+                                    : desc_hi(8u * a.q_row_bytes, a.q_row_bytes == 128 ? 2u : (a.q_row_bytes == 64 ? 4u : 6u));
+      const uint32_t q_kstep16 = (!a.q_mn ? UMMA_K : UMMA_K * a.q_row_bytes) >> 4;
+      const int k_tail = (int)(a.K - (int64_t)(kblocks - 1) * BK);            // bytes of K in the last k-block
+      const int tail_steps = k_tail >= BK ? BK / UMMA_K : (k_tail + UMMA_K - 1) / UMMA_K;
+      int consumed = 0, s = 0, wrap = 0, it = 0;
       bool ok = true;
-      for (int64_t t = blockIdx.x; ok && t < a.total_tiles; t += gridDim.x, ++it) {
+      int qi = 0, cur_q = -1;
+      TileIter ti;
+      ti.init(a, t_begin);
+      for (int64_t t = t_begin; ok && t < t_end; ++t, ++it) {
         const int buf = it & 1;
+        bool last_of_q = false;
+        if (a.q_resident) {
+          const int q0 = ti.q0(a);
+          if (q0 != cur_q) {
+            if (!mbar_wait(qresf, qi & 1, a.status)) { ok = false; break; }
+            cur_q = q0;
+            ++qi;
+          }
+          ti.next(a);
+          last_of_q = t + 1 >= t_end || ti.q0(a) != cur_q;
+        }
         // the epilogue must have drained this buffer (its use two tiles ago)
         if (it >= 2 && !mbar_wait(acce0 + 8 * buf, ((it >> 1) & 1) ^ 1, a.status)) { ok = false; break; }
         tc_fence_after();
         IVIT_TRACE(it, 1);
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * a.BN);
-        for (int kb = 0; kb < kblocks; ++kb, ++g) {
-          const int s = g % a.stages;
-          if (!mbar_wait(full0 + 8 * s, (g / a.stages) & 1, a.status)) { ok = false; break; }
+        for (int kb = 0; kb < kblocks; ++kb) {
+#ifndef IVIT_DBG_NOWAITFULL
+          if (!mbar_wait(full0 + 8 * s, wrap & 1, a.status)) { ok = false; break; }
+#endif
           tc_fence_after();
           if (kb == 0) IVIT_TRACE(it, 2);
-          const uint32_t sp = base + s * stage_bytes, sq = sp + BM * BK;
-          const int64_t krem = a.K - (int64_t)kb * BK;
-          const int ksteps = krem >= BK ? BK / UMMA_K : (int)((krem + UMMA_K - 1) / UMMA_K);
+          const uint32_t sp = base + s * stage_bytes, sq = a.q_resident ? qres + kb * a.q_stage_bytes : sp + BM * BK;
+          uint32_t p_lo = desc_lo(sp, 16), q_lo = desc_lo(sq, 16);
+          const int ksteps = kb == kblocks - 1 ? tail_steps : BK / UMMA_K;
           for (int k = 0; k < ksteps; ++k) {
-            const uint64_t dp = smem_desc(sp + k * UMMA_K, 16, 1024, 2);
-            const uint64_t dq = smem_desc(sq + k * q_kstep, 16, q_sbo, q_layout);
-            umma_i8(d_tmem, dp, dq, idesc, (kb | k) != 0);
+            umma_i8_lohi(d_tmem, p_lo, p_hi, q_lo, q_hi, idesc, (kb | k) != 0);
+            p_lo += UMMA_K >> 4;
+            q_lo += q_kstep16;
           }
           umma_commit(empty0 + 8 * s);   // the stage may be refilled once these MMAs have read it
+          ++consumed;
+          if (++s == a.stages) { s = 0; ++wrap; }
         }
         if (ok) umma_commit(accf0 + 8 * buf);  // accumulator of this tile complete
+        if (ok && last_of_q) umma_commit(qrese);   // the resident tile may be replaced once these MMAs are done
         IVIT_TRACE(it, 3);
       }
       if (!ok) {
         // drain: copies that were issued but never consumed (only after a timeout)
         const int issued = *issued_slot;
-        for (int j = g; j < issued; ++j) mbar_wait(full0 + 8 * (j % a.stages), (j / a.stages) & 1, a.status);
+        for (int j = consumed; j < issued; ++j) {
+          mbar_wait(full0 + 8 * s, wrap & 1, a.status);
+          if (++s == a.stages) { s = 0; ++wrap; }
+        }
+        const int qissued = *qres_issued;
+        for (int j = qi; j < qissued; ++j) mbar_wait(qresf, j & 1, a.status);
       }
     }
   } else {
@@ -266,27 +343,31 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         if (e.bias) nb = __ldg(e.bias + c);
       }
     };
-    if (a.lanes_are_channels && (int64_t)blockIdx.x < a.total_tiles) fetch_channel(tile_coord(a, blockIdx.x).p0);
+    if (a.lanes_are_channels && t_begin < t_end) fetch_channel(tile_coord(a, t_begin).p0);
     // MatMul orientation: one per-tensor constant set
     const int um = e.scale.mult, us = clamp_shift(e.scale.shift);
     const long long uc = 1ll << (us - 1);
 
     int res_issued = 0, res_waited = 0;   // residual tiles requested / consumed (thread et == 0 issues them)
-    if (a.tma_res && et == 0 && (int64_t)blockIdx.x < a.total_tiles) {
-      const TileCoord t0 = tile_coord(a, blockIdx.x);
+    if (a.tma_res && et == 0 && t_begin < t_end) {
+      const TileCoord t0 = tile_coord(a, t_begin);
       mbar_expect_tx(resf, (uint32_t)a.BN * 128u);
       tma_load_4d(stage_res, &tmR, resf, t0.p0, t0.q0, 0, 0);
       ++res_issued;
     }
     int it = 0;
-    for (int64_t t = blockIdx.x; t < a.total_tiles; t += gridDim.x, ++it) {
-      const TileCoord tc = tile_coord(a, t);
+    TileIter ti;
+    ti.init(a, t_begin);
+    for (int64_t t = t_begin; t < t_end; ++t, ++it) {
+      TileCoord tc;
+      tc.batch = ti.batch; tc.bo = ti.bo; tc.bi = ti.bi; tc.p0 = ti.p0(); tc.q0 = ti.q0(a);
+      ti.next(a);   // ti now describes the next tile
       const int buf = it & 1;
       const int cm = nm, cs = ns;
       long long cc = (long long)nb * nm + (1ll << (ns - 1));   // bias * m + 2^(s-1)
       asm volatile("" : "+l"(cc));   // keep it one 64-bit addend of the per-value multiply-add
-      const int64_t tn = t + gridDim.x;
-      if (a.lanes_are_channels && tn < a.total_tiles) fetch_channel(tile_coord(a, tn).p0);
+      const int64_t tn = t + 1;
+      if (a.lanes_are_channels && tn < t_end) fetch_channel(ti.p0());
 
       // all epilogue threads take the same decision, so the named barrier never sees a partial group
       if (a.tma_out && et == 0) tma_store_wait_read();   // the staging tile is free again
@@ -308,6 +389,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         for (int j0 = part * 32; j0 < a.BN; j0 += 32 * kParts) {
           const int64_t r0 = (int64_t)tc.q0 + j0;
           if (r0 >= a.Q) break;
+#ifdef IVIT_DBG_NOEPI
+          break;
+#endif
           int v[32];
 #ifdef IVIT_TC_TRACE
           if (et == 0 && j0 == 0) IVIT_TRACE(it, 6);
@@ -317,6 +401,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
           if (et == 0 && j0 == 0) IVIT_TRACE(it, 7);
 #endif
           const int nrow = (int)min((int64_t)32, a.Q - r0);
+#ifdef IVIT_DBG_EPI_LDONLY
+          asm volatile("" :: "r"(v[0]), "r"(v[31]));
+          continue;
+#endif
           // requantise: one 32x32->64 multiply-add and two shifts per value, 32 independent chains
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
@@ -378,6 +466,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
           for (int k = 0; k < 8; ++k) o[k] = __shfl_xor_sync(0xffffffffu, w[k], 2);
 #pragma unroll
           for (int k = 0; k < 8; ++k) w[k] = __byte_perm(w[k], o[k], sel2);
+#ifdef IVIT_DBG_EPI_NOSTS
+          asm volatile("" :: "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]));
+          continue;
+#endif
           if (a.tma_out) {
             // staging tile [row][128 channels]; 16-byte chunk index XOR (row & 7) is the 128B swizzle
             // of the store map.  Word k belongs to tile row j0 + li + 4k: (row & 7) alternates between
@@ -419,11 +511,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
           asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
           if (et == 0) {
             tma_store_4d(&tmO, stage_out, tc.p0, tc.q0, 0, 0);
-            if (a.tma_res && tn < a.total_tiles) {
+            if (a.tma_res && tn < t_end) {
               // every warp is past its reads of the residual tile: fetch the next tile's
-              const TileCoord tq = tile_coord(a, tn);
               mbar_expect_tx(resf, (uint32_t)a.BN * 128u);
-              tma_load_4d(stage_res, &tmR, resf, tq.p0, tq.q0, 0, 0);
+              tma_load_4d(stage_res, &tmR, resf, ti.p0(), ti.q0(a), 0, 0);
               ++res_issued;
             }
           }
@@ -491,7 +582,7 @@ int pow2_at_least(int v) {
 }
 
 constexpr size_t kSmemBudget = 227 * 1024;
-constexpr size_t kSmemFixed = 1024 + 8 * (2 * kMaxStages + 5) + 32;
+constexpr size_t kSmemFixed = 1024 + 8 * (2 * kMaxStages + 7) + 32;
 
 bool g_attr_set = false;
 
@@ -577,16 +668,21 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
     a.tma_res = make_tensor_map(ctx, &tmR, e.res, g.N, g.M, 1, 1, e.ldres, 0, 0, BM, a.BN, CU_TENSOR_MAP_SWIZZLE_128B,
                                 rpos) ? 1 : 0;
   }
-  const size_t stage = (size_t)BM * BK + a.q_stage_bytes;
   const size_t out_stage = (a.tma_out ? (size_t)a.BN * 128 : 0) + (a.tma_res ? (size_t)a.BN * 128 : 0);
-  int stages = (int)((kSmemBudget - kSmemFixed - out_stage) / stage);
+  // short K: keep the activation tile resident if that still leaves four weight stages
+  const size_t kblocks = (size_t)((g.K + BK - 1) / BK);
+  const size_t qres_bytes = kblocks * a.q_stage_bytes;
+  a.q_resident = (dense && kSmemFixed + out_stage + qres_bytes + 4 * (size_t)BM * BK <= kSmemBudget) ? 1 : 0;
+  const size_t stage = (size_t)BM * BK + (a.q_resident ? 0 : a.q_stage_bytes);
+  const size_t fixed = out_stage + (a.q_resident ? qres_bytes : 0);
+  int stages = (int)((kSmemBudget - kSmemFixed - fixed) / stage);
   a.stages = stages > kMaxStages ? kMaxStages : stages;
   if (a.stages < 2) return IVIT_ERR_UNSUPPORTED;
   a.tmem_cols = pow2_at_least(2 * a.BN);
   a.tiles_q = (int)((a.Q + a.BN - 1) / a.BN);
   a.total_tiles = (int64_t)a.tiles_p * a.tiles_q * batches;
 
-  const size_t smem = kSmemFixed + (size_t)a.stages * stage + out_stage;
+  const size_t smem = kSmemFixed + (size_t)a.stages * stage + fixed;
   if (!g_attr_set) {
     if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess)
       return IVIT_ERR_CUDA;

@@ -289,15 +289,16 @@ int launch_layernorm(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, 
   const int8_t* x = (const int8_t*)in;
   const int wpl = (int)((C / 4 + 31) / 32);
   if (wpl <= 4) {
-    // batched kernel: 4 rows per warp, small blocks so that one wave covers the rows
-    const int rpw = 4, tb = 128;
+    // batched kernel: 8 rows per warp (4 for the wider rows) amortise the per-row scalar work and the
+    // per-channel constants
+    const int rpw = wpl <= 3 ? 8 : 4;
     const int64_t warps = (rows + rpw - 1) / rpw;
-    const int64_t wantb = (warps + tb / 32 - 1) / (tb / 32);
-    const int gridb = (int)(wantb < (int64_t)ctx->sm_count * 16 ? wantb : (int64_t)ctx->sm_count * 16);
-    if (wpl <= 1) layernorm_i8_batched_kernel<1, 4><<<gridb, tb, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-    else if (wpl <= 2) layernorm_i8_batched_kernel<2, 4><<<gridb, tb, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-    else if (wpl <= 3) layernorm_i8_batched_kernel<3, 4><<<gridb, tb, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-    else layernorm_i8_batched_kernel<4, 4><<<gridb, tb, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+    const int64_t wantb = (warps + wpb - 1) / wpb;
+    const int gridb = (int)(wantb < (int64_t)ctx->sm_count * 8 ? wantb : (int64_t)ctx->sm_count * 8);
+    if (wpl <= 1) layernorm_i8_batched_kernel<1, 8><<<gridb, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+    else if (wpl <= 2) layernorm_i8_batched_kernel<2, 8><<<gridb, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+    else if (wpl <= 3) layernorm_i8_batched_kernel<3, 8><<<gridb, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+    else layernorm_i8_batched_kernel<4, 4><<<gridb, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
     return ls.done();
   }
   if (wpl <= 6) layernorm_i8_kernel<6><<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
