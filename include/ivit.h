@@ -186,6 +186,28 @@ size_t ivit_block_workspace_bytes(const ivit_block_params* p);
 int ivit_block_forward(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* X, int8_t* Y,
                        void* workspace, size_t workspace_bytes);
 
+/* ivit_block_forward for callers that cannot allocate device memory.
+ * (The paper has no counterpart; this entry point exists for deployment reasons only.)
+ * Some callers are not allowed to call cudaMalloc at all: a plugin running inside a host
+ * application that owns the memory pool, code that runs where allocation would synchronise the
+ * device (inside a latency-critical serving loop), or a process whose allocator is locked down.
+ * Such a caller cannot provide the workspace that ivit_block_forward asks for.  This variant
+ * computes the same block with the same kernels, but takes its scratch from a fixed array that is
+ * part of the library image: IVIT_STATIC_SCRATCH_BYTES bytes of device memory, which every GPU
+ * that loads the library holds until the process exits, whether or not this call is ever used.
+ *  - X, Y: [B*T, D] int8 device tensors owned by the caller, as for ivit_block_forward.
+ *  - Returns IVIT_ERR_WORKSPACE, and enqueues nothing, when ivit_block_workspace_bytes(p)
+ *    exceeds IVIT_STATIC_SCRATCH_BYTES (the DeiT-Tiny block of one image needs about 0.6 MiB).
+ *  - The call itself allocates nothing (no cudaMalloc / cudaFree, no allocating library routine).
+ *  - The first call on a device looks up the array's device address (one cudaGetSymbolAddress, no
+ *    allocation); make that first call before any CUDA stream capture.
+ *  - All calls share the one array and it keeps whatever the last call left in it.  No part of it
+ *    has to start at zero: every buffer inside is fully written before it is read.  Two calls whose
+ *    kernels overlap on the GPU (different streams, different contexts, different host threads)
+ *    race on the array; keep them ordered on one stream. */
+#define IVIT_STATIC_SCRATCH_BYTES (8u << 20)
+int ivit_block_forward_static(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* X, int8_t* Y);
+
 /* Attention core of the block alone (Sec. 3.1 MSA equation without the output
  * projection): QKV [B*T, 3D] int8 -> O [B*T, D] int8, using the attention
  * fields of p.  workspace as for ivit_block_forward. */

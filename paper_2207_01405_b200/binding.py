@@ -21,7 +21,7 @@ LIB_PATH = os.path.join(_HERE, "libivit.so")
 EXPORTS = [
     "ivit_ctx_create", "ivit_ctx_destroy", "ivit_ctx_set_stream", "ivit_ctx_poll_status", "ivit_ctx_launch_count",
     "ivit_ctx_set_gemm_engine", "ivit_strerror", "ivit_linear", "ivit_matmul", "ivit_shiftmax", "ivit_shiftgelu",
-    "ivit_layernorm", "ivit_block_workspace_bytes", "ivit_block_forward", "ivit_attention",
+    "ivit_layernorm", "ivit_block_workspace_bytes", "ivit_block_forward", "ivit_block_forward_static", "ivit_attention",
     "ivit_vit_workspace_bytes", "ivit_vit_forward", "ivit_vit_host_workspace_bytes", "ivit_vit_forward_host",
     "ivit_ctx_profile_start", "ivit_ctx_profile_stop", "ivit_ctx_profile_get", "ivit_kernel_kind_name", "ivit_patchify", "ivit_gather_rows", "ivit_fill_rows",
     "ivit_token_mean", "ivit_dyadic_from_double", "ivit_validate_exp_params", "ivit_validate_scale",
@@ -94,6 +94,7 @@ def load_library():
     L.ivit_block_workspace_bytes.argtypes = [C.POINTER(CBlock)]
     L.ivit_block_workspace_bytes.restype = C.c_size_t
     L.ivit_block_forward.argtypes = [vp, C.POINTER(CBlock), vp, vp, vp, C.c_size_t]
+    L.ivit_block_forward_static.argtypes = [vp, C.POINTER(CBlock), vp, vp]
     L.ivit_attention.argtypes = [vp, C.POINTER(CBlock), vp, vp, vp, C.c_size_t]
     L.ivit_vit_workspace_bytes.argtypes = [C.POINTER(CVit)]
     L.ivit_vit_workspace_bytes.restype = C.c_size_t
@@ -318,6 +319,14 @@ class Context:
         ws = workspace if workspace is not None else blk.workspace()
         _chk(self.lib.ivit_block_forward(self.h, C.byref(blk.c), X.data_ptr(), Y.data_ptr(), ws.data_ptr(), ws.numel()),
              "ivit_block_forward")
+        return Y
+
+    def block_forward_static(self, blk: "DeviceBlock", X, Y=None):
+        """ivit_block_forward_static: same block, scratch taken from the library's fixed device array."""
+        if Y is None:
+            Y = torch.empty_like(X)
+        _chk(self.lib.ivit_block_forward_static(self.h, C.byref(blk.c), X.data_ptr(), Y.data_ptr()),
+             "ivit_block_forward_static")
         return Y
 
     def attention(self, blk: "DeviceBlock", QKV, O=None, workspace=None):

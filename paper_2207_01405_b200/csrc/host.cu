@@ -352,6 +352,32 @@ int ivit_block_forward(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* 
   return block_impl(ctx, p, X, Y, static_cast<char*>(workspace));
 }
 
+// Scratch of ivit_block_forward_static: part of the library image, present on every GPU that loads it.
+static __device__ __align__(256) unsigned char g_static_scratch[IVIT_STATIC_SCRATCH_BYTES];
+
+int ivit_block_forward_static(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* X, int8_t* Y) {
+  if (!ctx || !X || !Y || X == Y) return IVIT_ERR_INVALID_ARG;
+  int rc = check_block(p);
+  if (rc) return rc;
+  if (!aligned16(X) || !aligned16(Y)) return IVIT_ERR_ALIGNMENT;
+  if (block_ws(p).total > (size_t)IVIT_STATIC_SCRATCH_BYTES) return IVIT_ERR_WORKSPACE;   // larger than the fixed scratch
+  // In host code the array's name is only a handle; kernels need its device address, which differs per
+  // device.  It is looked up once per device, with that device current, and kept.
+  static void* scratch_of_device[64] = {nullptr};
+  if (ctx->device < 0 || ctx->device >= 64) return IVIT_ERR_UNSUPPORTED;
+  if (!scratch_of_device[ctx->device]) {
+    int current = -1;
+    if (cudaGetDevice(&current) != cudaSuccess) return IVIT_ERR_CUDA;
+    if (current != ctx->device && cudaSetDevice(ctx->device) != cudaSuccess) return IVIT_ERR_CUDA;
+    void* ptr = nullptr;
+    const cudaError_t err = cudaGetSymbolAddress(&ptr, g_static_scratch);
+    if (current != ctx->device) cudaSetDevice(current);
+    if (err != cudaSuccess || !ptr) return IVIT_ERR_CUDA;
+    scratch_of_device[ctx->device] = ptr;
+  }
+  return block_impl(ctx, p, X, Y, static_cast<char*>(scratch_of_device[ctx->device]));
+}
+
 int ivit_attention(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* QKV, int8_t* O,
                    void* workspace, size_t workspace_bytes) {
   if (!ctx || !QKV || !O) return IVIT_ERR_INVALID_ARG;
