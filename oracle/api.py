@@ -331,3 +331,21 @@ def vit_forward(p, image, batch=None, return_tokens=False):
     tokens = np.zeros((B * p.T, p.D), dtype=np.int8) if return_tokens else None
     _chk(lib().orc_vit_forward(C.byref(v), image.ctypes.data, logits.ctypes.data, _ptr(tokens)), "vit_forward")
     return (logits, tokens) if return_tokens else logits
+
+
+def swin_forward(p, image):
+    """Swin-shaped forward (unshifted windows) composed from the oracle's operators; mirrors the model
+    description in ivit_inputs.params.SwinParams.  Returns int32 logits [B, classes]."""
+    B = image.shape[0]
+    X = linear(patchify(image, p.patch, window=p.window), p.Wpe, p.bpe, p.pe_scale)
+    X = layernorm(X, p.pe_ln_gamma, p.pe_ln_beta, p.M_ln)
+    for st in p.stages:
+        for blk in st.blocks:
+            X = block_forward(blk, X)
+        if st.merge_index is not None:
+            G = gather_rows(X, st.merge_index, width=st.C).reshape(-1, 4 * st.C)
+            G = layernorm(G, st.merge_ln_gamma, st.merge_ln_beta, p.M_ln)
+            X = linear(G, st.Wmerge, None, st.merge_scale)
+    X = layernorm(X, p.lnf_gamma, p.lnf_beta, p.M_ln)
+    Z = token_mean(X, X.shape[0] // B, p.pool_scale)
+    return linear(Z, p.Whead, p.bhead, p.head_scale, out_dtype=I32)

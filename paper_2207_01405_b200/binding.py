@@ -443,3 +443,49 @@ class DeviceVit:
         if n == 0:
             raise ValueError("ivit_vit_host_workspace_bytes rejected the model parameters")
         return torch.empty(int(n), dtype=torch.uint8, device=self.device)
+
+
+class DeviceSwin:
+    """A Swin-shaped model (unshifted 7x7 windows) resident on the device."""
+
+    def __init__(self, p, device):
+        self.p = p
+        self.device = device
+        self.up = _Uploader(device)
+        t = lambda a, dt: None if a is None else torch.from_numpy(np.ascontiguousarray(a, dtype=dt)).to(device)
+        self.Wpe, self.bpe, self.pe_scale = t(p.Wpe, np.int8), t(p.bpe, np.int32), DevScale(p.pe_scale, device)
+        self.pe_ln_gamma, self.pe_ln_beta = DevScale(p.pe_ln_gamma, device), t(p.pe_ln_beta, np.int32)
+        self.stages = []
+        for st in p.stages:
+            d = {"blocks": [DeviceBlock(b, device) for b in st.blocks], "C": st.C}
+            if st.merge_index is not None:
+                d["merge_index"] = t(st.merge_index, np.int32)
+                d["merge_ln_gamma"], d["merge_ln_beta"] = DevScale(st.merge_ln_gamma, device), t(st.merge_ln_beta, np.int32)
+                d["Wmerge"], d["merge_scale"] = t(st.Wmerge, np.int8), DevScale(st.merge_scale, device)
+            self.stages.append(d)
+        self.lnf_gamma, self.lnf_beta = DevScale(p.lnf_gamma, device), t(p.lnf_beta, np.int32)
+        self.pool_scale = DevScale(p.pool_scale, device)
+        self.Whead, self.bhead, self.head_scale = t(p.Whead, np.int8), t(p.bhead, np.int32), DevScale(p.head_scale, device)
+        self.ws = torch.empty(max(b.workspace_bytes() for s in self.stages for b in s["blocks"]), dtype=torch.uint8,
+                              device=device)
+
+
+def swin_forward(ctx: Context, m: DeviceSwin, image: torch.Tensor) -> torch.Tensor:
+    """Swin-shaped forward composed from the library's entry points (every step is a library kernel):
+    patchify (window-major) -> Dense -> LN -> [blocks -> 2x2 gather -> LN -> Dense] x stages -> LN -> token
+    mean -> Dense head (int32 logits)."""
+    p = m.p
+    X = ctx.linear(ctx.patchify(image, p.patch, window=p.window), m.Wpe, m.bpe, m.pe_scale)
+    X = ctx.layernorm(X, m.pe_ln_gamma, m.pe_ln_beta, p.M_ln)
+    for st in m.stages:
+        for blk in st["blocks"]:
+            X = ctx.block_forward(blk, X, workspace=m.ws)
+        if "merge_index" in st:
+            C_ = st["C"]
+            G = ctx.gather_rows(X, st["merge_index"], width=C_).view(-1, 4 * C_)
+            G = ctx.layernorm(G, st["merge_ln_gamma"], st["merge_ln_beta"], p.M_ln)
+            X = ctx.linear(G, st["Wmerge"], None, st["merge_scale"])
+    X = ctx.layernorm(X, m.lnf_gamma, m.lnf_beta, p.M_ln)
+    tokens = X.shape[0] // image.shape[0]
+    Z = ctx.token_mean(X, tokens, m.pool_scale)
+    return ctx.linear(Z, m.Whead, m.bhead, m.head_scale, out_dtype=I32)

@@ -1,0 +1,51 @@
+"""GPU parity on the other workloads: ViT-B, ViT-L/384 and Swin-T shapes (reduced batch / depth for the
+element-by-element comparison), and sampled images at the full sizes the configs name."""
+import numpy as np
+import pytest
+import torch
+
+from ivit_inputs import make_config
+from oracle import api as O
+
+pytestmark = pytest.mark.gpu
+
+
+def _g():
+    import gpu_util
+    return gpu_util
+
+
+@pytest.mark.parametrize("cfg,batch,depth", [(2, 2, 2), (4, 1, 2)])
+def test_vit_family_reduced_bit_exact(cfg, batch, depth):
+    g = _g()
+    c = g.ctx()
+    model, image = make_config(cfg, batch=batch, depth=depth)
+    dm = g.binding.DeviceVit(model, "cuda")
+    logits = g.host(c.vit_forward(dm, torch.from_numpy(image).cuda()))
+    g.assert_equal(logits, O.vit_forward(model, image), f"config {cfg} logits")
+    assert c.poll_status() == 0
+
+
+def test_swin_tiny_shapes_bit_exact():
+    """Config 3 at batch 2: 4 stages, window attention with relative-position bias, patch merging."""
+    g = _g()
+    c = g.ctx()
+    model, image = make_config(3, batch=2)
+    dm = g.binding.DeviceSwin(model, "cuda")
+    logits = g.host(g.binding.swin_forward(c, dm, torch.from_numpy(image).cuda()))
+    want = O.swin_forward(model, image)
+    g.assert_equal(logits, want, "swin logits")
+    assert len(np.unique(want)) > 100
+    assert c.poll_status() == 0
+
+
+def test_vit_base_b128_full_size_sampled():
+    """Config 2 at its full size (batch 128, 12 blocks); the oracle recomputes sampled images."""
+    g = _g()
+    c = g.ctx()
+    model, image = make_config(2)
+    dm = g.binding.DeviceVit(model, "cuda")
+    logits = g.host(c.vit_forward(dm, torch.from_numpy(image).cuda()))
+    for i in (0, 127):
+        g.assert_equal(logits[i:i + 1], O.vit_forward(model, image[i:i + 1]), f"image {i}")
+    assert c.poll_status() == 0
