@@ -24,7 +24,10 @@ constexpr int UK = 32;              // K of one tcgen05.mma.kind::i8
 #ifdef IVIT_ATTN_TRACE
 // debugging aid (compiled out by default): clock64() stamps of the phases of the first CTAs
 __device__ long long g_attn_trace[64][12];
-#define ATRACE(i) do { if (blockIdx.x < 64) g_attn_trace[blockIdx.x][i] = clock64(); } while (0)
+__device__ unsigned long long g_attn_span[1024][3];   // per CTA: global ns at start, at end, SM id
+#define ATRACE(i) do { if (blockIdx.x < 64) g_attn_trace[blockIdx.x][i] = clock64(); \
+  if ((i) == 0 || (i) == 9) { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); unsigned sm; asm volatile("mov.u32 %0, %%smid;" : "=r"(sm)); \
+    if (blockIdx.x < 1024) { g_attn_span[blockIdx.x][(i) == 0 ? 0 : 1] = t; g_attn_span[blockIdx.x][2] = sm; } } } while (0)
 #else
 #define ATRACE(i) do { } while (0)
 #endif
@@ -169,24 +172,24 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const __grid_co
 #pragma unroll
             for (int j = 0; j < 32; ++j) v[j] = (int)(((long long)v[j] * a.qk_m + qk_c) >> a.qk_s);
           }
-          uint32_t m4 = 0x80808080u;
+          // columns past T (only in the last chunk) never win the maximum and look up a valid table entry
+          if (c == nch - 1) {
 #pragma unroll
-          for (int k = 0; k < 8; ++k) xs[cc * 8 + k] = pack_sat8(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
-          if (c == nch - 1) {   // only the last chunk can hold columns past T: they never win the maximum
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-              const int valid = a.T - (c * 32 + 4 * k);
-              if (valid < 4) {
-                const uint32_t keep = valid <= 0 ? 0u : (0xffffffffu >> (8 * (4 - valid)));
-                xs[cc * 8 + k] = (xs[cc * 8 + k] & keep) | (0x80808080u & ~keep);
-              }
-            }
+            for (int j = 0; j < 32; ++j)
+              if (c * 32 + j >= a.T) v[j] = -128;
           }
+          // running maximum on the unsaturated values (saturation is monotone: it is applied to the result)
+          int m = v[0];
 #pragma unroll
-          for (int k = 0; k < 8; ++k) m4 = __vmaxs4(m4, xs[cc * 8 + k]);
-          mx = max(mx, max(max((int)(int8_t)m4, (int)(int8_t)(m4 >> 8)), max((int)(int8_t)(m4 >> 16), (int)(int8_t)(m4 >> 24))));
+          for (int j = 1; j < 32; j += 2) m = max(m, max(v[j], v[(j + 1) & 31]));
+          mx = max(mx, m);
+          // scores are kept as biased bytes (x + 128, i.e. x ^ 0x80) so that pass B can index with them
+#pragma unroll
+          for (int k = 0; k < 8; ++k)
+            xs[cc * 8 + k] = pack_sat8(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]) ^ 0x80808080u;
         }
       }
+      mx = max(-128, min(127, mx));
       part_max[half * 128 + trow] = mx;
     }
     asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -200,13 +203,14 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const __grid_co
         const int c = 2 * cc + half;
         if (c < nch) {
           int ev[32];
-          const uint32_t mx4 = (uint32_t)(mx & 0xff) * 0x01010101u;
+          // entry (I_max - I) of the table = word at tab + 4*(I_max + 128) - 4*(I + 128)
+          const uint8_t* tmx = reinterpret_cast<const uint8_t*>(tab) + 4 * (mx + 128);
 #pragma unroll
           for (int k = 0; k < 8; ++k) {
-            const uint32_t d4 = __vsub4(mx4, xs[cc * 8 + k]);   // I_max - I per byte, in [0, 255]
+            const uint32_t w = xs[cc * 8 + k];
 #pragma unroll
             for (int b = 0; b < 4; ++b)
-              ev[4 * k + b] = (int)tab[__byte_perm(d4, 0, 0x4440 + b)];
+              ev[4 * k + b] = (int)*reinterpret_cast<const unsigned*>(tmx - 4 * (int)__byte_perm(w, 0, 0x4440 + b));
           }
           if (c == nch - 1) {   // columns past T contribute nothing
 #pragma unroll

@@ -9,7 +9,8 @@
 
 namespace ivit {
 
-constexpr uint32_t kSpinLimit = 1u << 20;
+constexpr uint32_t kSpinLimit = 1u << 20;     // polls before a wait gives up
+constexpr uint32_t kSuspendHintNs = 2000;      // suspend-time hint of one poll
 
 // 4-D int8 tensor map over {inner, rows, batch_inner, batch_outer} (defined with the GEMM); pos[0..2]
 // receive the tensor-map dimension (1..3) holding the row, inner-batch and outer-batch coordinate.
@@ -27,13 +28,15 @@ __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
 __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// One poll: the thread may be suspended by the hardware for up to kSuspendHintNs while the phase is
+// incomplete (it resumes at once when the phase completes), so a waiting warp issues few instructions.
 __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+      : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendHintNs) : "memory");
   return ok != 0;
 }
 // Bounded wait: false (and the timeout recorded) when the phase did not complete in time.
