@@ -86,6 +86,8 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const __grid_co
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
+  pdl_trigger();
+  pdl_wait();   // the QKV tensor comes from the previous kernel
 
   if (warp == 0) {
     if (lane == 0) {
@@ -329,7 +331,7 @@ int launch_attention_fused(ivit_ctx* ctx, const ivit_block_params* p, const int8
   }
   const int64_t grid = B * h * a.tiles_m;
   LaunchScope ls(ctx, KIND_ATTENTION, 4.0 * (double)(B * h) * (double)T * (double)T * (double)d);
-  attention_kernel<<<(unsigned)grid, kAttnThreads, smem, ctx->stream>>>(tmQ, tmK, tmV, a);
+  launch_k(attention_kernel, dim3((unsigned)grid), dim3(kAttnThreads), smem, ctx->stream, tmQ, tmK, tmV, a);
   return ls.done();
 }
 

@@ -113,6 +113,30 @@ struct LaunchScope {
   }
 };
 
+// ---- programmatic dependent launch ---------------------------------------------------------
+// Every kernel of the library is launched with programmatic stream serialization: the next kernel
+// of the stream may be scheduled (and run its set-up) while this one drains.  A kernel therefore
+// calls pdl_wait() before it reads or writes anything another kernel may touch, and pdl_trigger()
+// to let its successor be scheduled early.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                            Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // launchers implemented in the kernel files ---------------------------------------------
 
 struct GemmEpilogue {

@@ -8,6 +8,8 @@ namespace ivit {
 constexpr int TM = 64, TN = 64, TKW = 8;  // tile: 64 x 64 outputs, 8 words (32 int8) of K per step
 
 __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmProblem g, int64_t tiles_m, int64_t tiles_n) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ int As[TM][TKW + 1];
   __shared__ int Bs[TN][TKW + 1];
   const int tid = threadIdx.x;
@@ -111,7 +113,7 @@ int launch_gemm_simt(ivit_ctx* ctx, const GemmProblem& g) {
   const int64_t total = batches * tiles_m * tiles_n;
   if (total > 2147483647LL) return IVIT_ERR_UNSUPPORTED;
   LaunchScope ls(ctx, KIND_GEMM_SIMT, 2.0 * (double)batches * (double)g.M * (double)g.N * (double)g.K);
-  gemm_simt_kernel<<<(unsigned)total, 256, 0, ctx->stream>>>(g, tiles_m, tiles_n);
+  launch_k(gemm_simt_kernel, dim3((unsigned)total), dim3(256), 0, ctx->stream, g, tiles_m, tiles_n);
   return ls.done();
 }
 

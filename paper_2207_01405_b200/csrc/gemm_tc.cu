@@ -71,7 +71,7 @@ constexpr int BM = 128;          // TMEM lanes of a tile (UMMA M, cta_group::1)
 constexpr int BK = 128;          // bytes (= int8 elements) of K per pipeline stage
 constexpr int UMMA_K = 32;       // K of one tcgen05.mma.kind::i8
 constexpr int kMaxStages = 8;
-constexpr int kEpiWarps = 16;
+constexpr int kEpiWarps = 8;
 constexpr int kEpiThreads = 32 * kEpiWarps;
 constexpr int kThreads = 64 + kEpiThreads;
 
@@ -208,6 +208,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // set-up done (barriers, tensor memory, descriptor prefetch): let the next kernel be scheduled, then wait
+  // for the previous kernel's results before touching global memory
+  pdl_trigger();
+  pdl_wait();
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
@@ -690,7 +694,7 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
   }
   const unsigned grid = (unsigned)(a.total_tiles < ctx->sm_count ? a.total_tiles : ctx->sm_count);
   LaunchScope ls(ctx, KIND_GEMM_TC, 2.0 * (double)batches * (double)g.M * (double)g.N * (double)g.K);
-  gemm_tc_kernel<<<grid, kThreads, smem, ctx->stream>>>(tmP, tmQ, tmO, tmR, a);
+  launch_k(gemm_tc_kernel, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
   return ls.done();
 }
 

@@ -7,6 +7,8 @@ namespace ivit {
 // One thread per 4 output bytes (px .. px+3 of one patch row); P % 4 == 0.
 __global__ void patchify_kernel(const int8_t* __restrict__ img, int64_t B, int C, int Hi, int Wi, int P,
                                 int window, int8_t* __restrict__ out, int64_t ldout, int64_t total_words) {
+  pdl_trigger();
+  pdl_wait();
   const int gh = Hi / P, gw = Wi / P;
   const int kw = C * P * P / 4;
   for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total_words;
@@ -30,6 +32,8 @@ __global__ void patchify_kernel(const int8_t* __restrict__ img, int64_t B, int C
 
 __global__ void gather_rows_kernel(const int8_t* __restrict__ src, int64_t ldsrc, const int32_t* __restrict__ index,
                                    int64_t n_rows, int vec_per_row, int8_t* __restrict__ dst, int64_t lddst) {
+  pdl_trigger();
+  pdl_wait();
   const int64_t total = n_rows * vec_per_row;
   for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
     const int64_t r = t / vec_per_row;
@@ -41,6 +45,8 @@ __global__ void gather_rows_kernel(const int8_t* __restrict__ src, int64_t ldsrc
 
 __global__ void fill_rows_kernel(const int8_t* __restrict__ src_row, int vec_per_row, int8_t* __restrict__ dst,
                                  int64_t group_stride, int64_t groups) {
+  pdl_trigger();
+  pdl_wait();
   const int64_t total = groups * vec_per_row;
   for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
     const int64_t g = t / vec_per_row;
@@ -51,6 +57,8 @@ __global__ void fill_rows_kernel(const int8_t* __restrict__ src_row, int vec_per
 
 __global__ void token_mean_kernel(const int8_t* __restrict__ in, int64_t ldin, int64_t groups, int T, int C,
                                   ScaleDev scale, int8_t* __restrict__ out, int64_t ldout) {
+  pdl_trigger();
+  pdl_wait();
   const int64_t total = groups * C;
   for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
     const int64_t g = t / C;
@@ -72,7 +80,7 @@ int launch_patchify(ivit_ctx* ctx, const int8_t* img, int64_t B, int64_t C, int6
   const int64_t total = B * C * Hi * Wi / 4;
   if (total == 0) return IVIT_OK;
   LaunchScope ls(ctx, KIND_MOVE, 2.0 * (double)total * 4);
-  patchify_kernel<<<grid_for(ctx, total, 256), 256, 0, ctx->stream>>>(img, B, (int)C, (int)Hi, (int)Wi, (int)P,
+  launch_k(patchify_kernel, dim3(grid_for(ctx, total, 256)), dim3(256), 0, ctx->stream, img, B, (int)C, (int)Hi, (int)Wi, (int)P,
                                                                        (int)window, out, ldout, total);
   return ls.done();
 }
@@ -81,7 +89,7 @@ int launch_gather_rows(ivit_ctx* ctx, const int8_t* src, int64_t ldsrc, const in
                        int64_t n_rows, int64_t width, int8_t* dst, int64_t lddst) {
   if (n_rows == 0) return IVIT_OK;
   LaunchScope ls(ctx, KIND_MOVE, 2.0 * (double)n_rows * (double)width);
-  gather_rows_kernel<<<grid_for(ctx, n_rows * (width / 16), 256), 256, 0, ctx->stream>>>(
+  launch_k(gather_rows_kernel, dim3(grid_for(ctx, n_rows * (width / 16), 256)), dim3(256), 0, ctx->stream, 
       src, ldsrc, index, n_rows, (int)(width / 16), dst, lddst);
   return ls.done();
 }
@@ -90,7 +98,7 @@ int launch_fill_rows(ivit_ctx* ctx, const int8_t* src_row, int64_t width, int8_t
                      int64_t group_stride, int64_t groups) {
   if (groups == 0) return IVIT_OK;
   LaunchScope ls(ctx, KIND_MOVE, (double)groups * (double)width);
-  fill_rows_kernel<<<grid_for(ctx, groups * (width / 16), 256), 256, 0, ctx->stream>>>(
+  launch_k(fill_rows_kernel, dim3(grid_for(ctx, groups * (width / 16), 256)), dim3(256), 0, ctx->stream, 
       src_row, (int)(width / 16), dst, group_stride, groups);
   return ls.done();
 }
@@ -99,7 +107,7 @@ int launch_token_mean(ivit_ctx* ctx, const int8_t* in, int64_t ldin, int64_t gro
                       int64_t C, ScaleDev scale, int8_t* out, int64_t ldout) {
   if (groups == 0) return IVIT_OK;
   LaunchScope ls(ctx, KIND_MOVE, (double)groups * (double)C * (double)(T + 1));
-  token_mean_kernel<<<grid_for(ctx, groups * C, 256), 256, 0, ctx->stream>>>(in, ldin, groups, (int)T, (int)C,
+  launch_k(token_mean_kernel, dim3(grid_for(ctx, groups * C, 256)), dim3(256), 0, ctx->stream, in, ldin, groups, (int)T, (int)C,
                                                                              scale, out, ldout);
   return ls.done();
 }

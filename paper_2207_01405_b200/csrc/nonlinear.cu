@@ -69,6 +69,8 @@ __global__ void __launch_bounds__(256) layernorm_i8_kernel(const int8_t* __restr
                                                            ScaleDev gs, const int32_t* __restrict__ beta,
                                                            int M_ln, int8_t* __restrict__ out, int64_t ldout,
                                                            int64_t rows, int C) {
+  pdl_trigger();
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
@@ -120,6 +122,8 @@ __global__ void __launch_bounds__(256) layernorm_i8_batched_kernel(const int8_t*
                                                                    ScaleDev gs, const int32_t* __restrict__ beta,
                                                                    int M_ln, int8_t* __restrict__ out, int64_t ldout,
                                                                    int64_t rows, int C) {
+  pdl_trigger();
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
@@ -206,6 +210,8 @@ __global__ void __launch_bounds__(256) layernorm_i8_long_kernel(const int8_t* __
                                                                 ScaleDev gs, const int32_t* __restrict__ beta,
                                                                 int M_ln, int8_t* __restrict__ out,
                                                                 int64_t ldout, int64_t rows, int C) {
+  pdl_trigger();
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
@@ -246,6 +252,8 @@ __global__ void __launch_bounds__(256) layernorm_i32_kernel(const int32_t* __res
                                                             ScaleDev gs, const int32_t* __restrict__ beta,
                                                             int M_ln, int8_t* __restrict__ out, int64_t ldout,
                                                             int64_t rows, int C) {
+  pdl_trigger();
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
@@ -283,7 +291,7 @@ int launch_layernorm(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, 
   cudaStream_t st = ctx->stream;
   LaunchScope ls(ctx, KIND_LAYERNORM, (double)rows * (double)C * (in_dtype == IVIT_I32 ? 5.0 : 2.0));
   if (in_dtype == IVIT_I32) {
-    layernorm_i32_kernel<<<grid, threads, 0, st>>>((const int32_t*)in, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+    launch_k(layernorm_i32_kernel, dim3(grid), dim3(threads), 0, st, (const int32_t*)in, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
     return ls.done();
   }
   const int8_t* x = (const int8_t*)in;
@@ -295,16 +303,16 @@ int launch_layernorm(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, 
     const int64_t warps = (rows + rpw - 1) / rpw;
     const int64_t wantb = (warps + wpb - 1) / wpb;
     const int gridb = (int)(wantb < (int64_t)ctx->sm_count * 8 ? wantb : (int64_t)ctx->sm_count * 8);
-    if (wpl <= 1) layernorm_i8_batched_kernel<1, 8><<<gridb, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-    else if (wpl <= 2) layernorm_i8_batched_kernel<2, 8><<<gridb, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-    else if (wpl <= 3) layernorm_i8_batched_kernel<3, 8><<<gridb, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-    else layernorm_i8_batched_kernel<4, 4><<<gridb, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+    if (wpl <= 1) launch_k(layernorm_i8_batched_kernel<1, 8>, dim3(gridb), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+    else if (wpl <= 2) launch_k(layernorm_i8_batched_kernel<2, 8>, dim3(gridb), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+    else if (wpl <= 3) launch_k(layernorm_i8_batched_kernel<3, 8>, dim3(gridb), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+    else launch_k(layernorm_i8_batched_kernel<4, 4>, dim3(gridb), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
     return ls.done();
   }
-  if (wpl <= 6) layernorm_i8_kernel<6><<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-  else if (wpl <= 8) layernorm_i8_kernel<8><<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-  else if (wpl <= 12) layernorm_i8_kernel<12><<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-  else layernorm_i8_long_kernel<<<grid, threads, 0, st>>>(x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+  if (wpl <= 6) launch_k(layernorm_i8_kernel<6>, dim3(grid), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+  else if (wpl <= 8) launch_k(layernorm_i8_kernel<8>, dim3(grid), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+  else if (wpl <= 12) launch_k(layernorm_i8_kernel<12>, dim3(grid), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+  else launch_k(layernorm_i8_long_kernel, dim3(grid), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
   return ls.done();
 }
 
@@ -340,6 +348,8 @@ template <int WPL, bool FROM_I32>
 __global__ void __launch_bounds__(256) shiftmax_kernel(RowLoader<FROM_I32> ld, ivit_exp_params p,
                                                        int8_t* __restrict__ out, int64_t ldout,
                                                        int64_t rows, int d) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ unsigned exp_tab[256];  // ShiftExp(-i), i = I_max - I in [0, 255]
   for (int i = threadIdx.x; i < 256; i += blockDim.x) exp_tab[i] = shiftexp(-i, p.I0, p.N);
   __syncthreads();
@@ -414,11 +424,11 @@ template <bool FROM_I32>
 static void shiftmax_dispatch(RowLoader<FROM_I32> ld, ivit_exp_params p, int8_t* out, int64_t ldout,
                               int64_t rows, int d, int grid, cudaStream_t st) {
   const int wpl = (((d + 15) / 16) * 4 + 31) / 32;
-  if (wpl <= 2) shiftmax_kernel<2, FROM_I32><<<grid, 256, 0, st>>>(ld, p, out, ldout, rows, d);
-  else if (wpl <= 5) shiftmax_kernel<5, FROM_I32><<<grid, 256, 0, st>>>(ld, p, out, ldout, rows, d);
-  else if (wpl <= 8) shiftmax_kernel<8, FROM_I32><<<grid, 256, 0, st>>>(ld, p, out, ldout, rows, d);
-  else if (wpl <= 16) shiftmax_kernel<16, FROM_I32><<<grid, 256, 0, st>>>(ld, p, out, ldout, rows, d);
-  else shiftmax_kernel<0, FROM_I32><<<grid, 256, 0, st>>>(ld, p, out, ldout, rows, d);
+  if (wpl <= 2) launch_k(shiftmax_kernel<2, FROM_I32>, dim3(grid), dim3(256), 0, st, ld, p, out, ldout, rows, d);
+  else if (wpl <= 5) launch_k(shiftmax_kernel<5, FROM_I32>, dim3(grid), dim3(256), 0, st, ld, p, out, ldout, rows, d);
+  else if (wpl <= 8) launch_k(shiftmax_kernel<8, FROM_I32>, dim3(grid), dim3(256), 0, st, ld, p, out, ldout, rows, d);
+  else if (wpl <= 16) launch_k(shiftmax_kernel<16, FROM_I32>, dim3(grid), dim3(256), 0, st, ld, p, out, ldout, rows, d);
+  else launch_k(shiftmax_kernel<0, FROM_I32>, dim3(grid), dim3(256), 0, st, ld, p, out, ldout, rows, d);
 }
 
 int launch_shiftmax(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, const int32_t* bias32,
@@ -444,6 +454,8 @@ int launch_shiftmax(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, c
 // is a function of (max(0, row max of x), x): 128 x 256 values.  They are produced here by
 // running Algorithm 2 literally once per pair; the row kernel then only looks values up.
 __global__ void shiftgelu_table_kernel(ivit_exp_params p, int post_m, int post_s, int8_t* __restrict__ table) {
+  pdl_trigger();
+  pdl_wait();
   const int rmax = blockIdx.x;         // max(0, row max of x), 0..127
   const int x = (int)threadIdx.x - 128;
   int out = 0;
@@ -468,6 +480,8 @@ __global__ void __launch_bounds__(256) shiftgelu_kernel(const int8_t* __restrict
                                                         const int8_t* __restrict__ table,
                                                         int8_t* __restrict__ out, int64_t ldout,
                                                         int64_t rows, int cols) {
+  pdl_trigger();
+  pdl_wait();
   __shared__ unsigned tab[8][64];  // one 256-byte table row per warp
   const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
   const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -537,7 +551,7 @@ int launch_shiftgelu(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_par
     }
     ctx->gelu_keys[slot] = key;
     LaunchScope lt(ctx, KIND_GELU_TABLE, (double)kGeluTableBytes);
-    shiftgelu_table_kernel<<<128, 256, 0, ctx->stream>>>(p, post.mult, post.shift,
+    launch_k(shiftgelu_table_kernel, dim3(128), dim3(256), 0, ctx->stream, p, post.mult, post.shift,
                                                           ctx->gelu_tables + (size_t)slot * kGeluTableBytes);
     int rc = lt.done();
     if (rc) return rc;
@@ -548,13 +562,13 @@ int launch_shiftgelu(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_par
   const int wpl = (int)((cols / 16 + 31) / 32);
   cudaStream_t st = ctx->stream;
   LaunchScope ls(ctx, KIND_SHIFTGELU, 2.0 * (double)rows * (double)cols);
-  if (wpl <= 1) shiftgelu_kernel<1><<<grid, 256, 0, st>>>(in, ldin, table, out, ldout, rows, (int)cols);
-  else if (wpl <= 2) shiftgelu_kernel<2><<<grid, 256, 0, st>>>(in, ldin, table, out, ldout, rows, (int)cols);
-  else if (wpl <= 3) shiftgelu_kernel<3><<<grid, 256, 0, st>>>(in, ldin, table, out, ldout, rows, (int)cols);
-  else if (wpl <= 4) shiftgelu_kernel<4><<<grid, 256, 0, st>>>(in, ldin, table, out, ldout, rows, (int)cols);
-  else if (wpl <= 6) shiftgelu_kernel<6><<<grid, 256, 0, st>>>(in, ldin, table, out, ldout, rows, (int)cols);
-  else if (wpl <= 8) shiftgelu_kernel<8><<<grid, 256, 0, st>>>(in, ldin, table, out, ldout, rows, (int)cols);
-  else shiftgelu_kernel<0><<<grid, 256, 0, st>>>(in, ldin, table, out, ldout, rows, (int)cols);
+  if (wpl <= 1) launch_k(shiftgelu_kernel<1>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols);
+  else if (wpl <= 2) launch_k(shiftgelu_kernel<2>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols);
+  else if (wpl <= 3) launch_k(shiftgelu_kernel<3>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols);
+  else if (wpl <= 4) launch_k(shiftgelu_kernel<4>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols);
+  else if (wpl <= 6) launch_k(shiftgelu_kernel<6>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols);
+  else if (wpl <= 8) launch_k(shiftgelu_kernel<8>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols);
+  else launch_k(shiftgelu_kernel<0>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols);
   return ls.done();
 }
 
