@@ -71,9 +71,13 @@ constexpr int BM = 128;          // TMEM lanes of a tile (UMMA M, cta_group::1)
 constexpr int BK = 128;          // bytes (= int8 elements) of K per pipeline stage
 constexpr int UMMA_K = 32;       // K of one tcgen05.mma.kind::i8
 constexpr int kMaxStages = 8;
-constexpr int kEpiWarps = 8;
+#ifndef IVIT_EPI_WARPS
+#define IVIT_EPI_WARPS 16
+#endif
+constexpr int kEpiWarps = IVIT_EPI_WARPS;
 constexpr int kEpiThreads = 32 * kEpiWarps;
-constexpr int kThreads = 64 + kEpiThreads;
+constexpr int kFirstEpiWarp = 2;   // warp 0: TMA loads, warp 1: MMA
+constexpr int kThreads = 32 * kFirstEpiWarp + kEpiThreads;
 
 struct TcArgs {
   GemmEpilogue epi;
@@ -101,7 +105,10 @@ struct TcArgs {
 // debugging aid (compiled out by default): per-CTA, per-tile clock64() stamps of each role
 __device__ long long g_trace[148][40][8];
 #define IVIT_TRACE(tile_it, idx) do { if ((tile_it) < 40 && blockIdx.x < 148) g_trace[blockIdx.x][tile_it][idx] = clock64(); } while (0)
+__device__ long long g_trace2[148][4][16];
+#define IVIT_TRACE2(cond, ckk, idx) do { const int i_ = (idx); if ((cond) && i_ < 16) g_trace2[blockIdx.x][ckk][i_] = clock64(); } while (0)
 #else
+#define IVIT_TRACE2(cond, ckk, idx) do { } while (0)
 #define IVIT_TRACE(tile_it, idx) do { } while (0)
 #endif
 
@@ -146,22 +153,19 @@ struct TileIter {
   __device__ __forceinline__ int q0(const TcArgs& a) const { return q * a.BN; }
 };
 
-__device__ __forceinline__ uint32_t epi_all(uint32_t pred) {
-  uint32_t all;
-  asm volatile(
-      "{\n\t.reg .pred p, q;\n\t"
-      "setp.ne.u32 q, %1, 0;\n\t"
-      "bar.red.and.pred p, 1, %2, q;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(all) : "r"(pred), "n"(kEpiThreads) : "memory");
-  return all;
-}
-
+// MODE fixes the run-time choices of the epilogue at compile time for the shapes of an encoder block, so that
+// the per-chunk code carries no branches on kernel arguments: 0 = everything decided at run time (any
+// orientation, output type and residual port), 1 = Dense orientation, int8 output staged for TMA stores, no
+// residual, 2 = the same with the residual tile fetched by TMA.
+template <int MODE>
 __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmP,
                                                               const __grid_constant__ CUtensorMap tmQ,
                                                               const __grid_constant__ CUtensorMap tmO,
                                                               const __grid_constant__ CUtensorMap tmR, TcArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
+#ifdef IVIT_TC_TRACE
+  if (threadIdx.x == 0) { IVIT_TRACE(39, 0); long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); g_trace[blockIdx.x][39][4] = g; }
+#endif
   // carve: [stages x (P tile | Q tile)] [barriers] [tmem address, issued count]
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
@@ -173,8 +177,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
   const uint32_t stage_res = stage_out + (a.tma_out ? a.BN * 128 : 0);   // residual tile, same layout
   const uint32_t bars_off = a.stages * stage_bytes + qres_bytes + (a.tma_out ? a.BN * 128 : 0) + (a.tma_res ? a.BN * 128 : 0);
   const uint32_t full0 = base + bars_off, empty0 = full0 + 8 * kMaxStages;
-  const uint32_t accf0 = empty0 + 8 * kMaxStages, acce0 = accf0 + 16, resf = acce0 + 16, qresf = resf + 8, qrese = resf + 16;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + bars_off + 8 * (2 * kMaxStages + 7));
+  const uint32_t accf0 = empty0 + 8 * kMaxStages, acce0 = accf0 + 16, resf = acce0 + 16, sfull = resf + 128, sfree = sfull + 128, qresf = sfree + 128, qrese = qresf + 8;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + bars_off + 8 * (2 * kMaxStages + 54));
   volatile int* issued_slot = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -195,7 +199,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       mbar_init(accf0 + 8 * b, 1);
       mbar_init(acce0 + 8 * b, kEpiWarps);
     }
-    mbar_init(resf, 1);
+    for (int b = 0; b < 16; ++b) {   // staging slots: 4 per epilogue part
+      mbar_init(resf + 8 * b, 1);
+      *reinterpret_cast<uint32_t*>(gen_base + (sfull - base) + 8 * b) = 0;   // arrivals of a part's warps at a slot
+      mbar_init(sfree + 8 * b, 1);
+    }
     mbar_init(qresf, 1);
     mbar_init(qrese, 1);
     *qres_issued = 0;
@@ -210,12 +218,22 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
   const uint32_t tmem_base = *tmem_slot;
   // set-up done (barriers, tensor memory, descriptor prefetch): let the next kernel be scheduled, then wait
   // for the previous kernel's results before touching global memory
+#ifdef IVIT_TC_TRACE
+  if (threadIdx.x == 0) IVIT_TRACE(39, 1);
+#endif
   pdl_trigger();
   pdl_wait();
+#ifdef IVIT_TC_TRACE
+  if (threadIdx.x == 0) IVIT_TRACE(39, 2);
+#endif
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
+#ifdef IVIT_DBG_NOMMA
+    if (false) {
+#else
     if (lane == 0) {
+#endif
       int issued = 0;            // k-blocks issued so far, over all tiles of this CTA
       int s = 0, wrap = 0;       // ring slot of the next k-block and how often the ring has wrapped
       bool ok = true;
@@ -277,7 +295,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       for (int64_t t = t_begin; ok && t < t_end; ++t, ++it) {
         const int buf = it & 1;
         bool last_of_q = false;
+#ifdef IVIT_DBG_NOMMA
+        if (false) {
+#else
         if (a.q_resident) {
+#endif
           const int q0 = ti.q0(a);
           if (q0 != cur_q) {
             if (!mbar_wait(qresf, qi & 1, a.status)) { ok = false; break; }
@@ -293,9 +315,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         IVIT_TRACE(it, 1);
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * a.BN);
         for (int kb = 0; kb < kblocks; ++kb) {
-#ifndef IVIT_DBG_NOWAITFULL
-          if (!mbar_wait(full0 + 8 * s, wrap & 1, a.status)) { ok = false; break; }
+#ifdef IVIT_DBG_NOMMA
+          continue;
 #endif
+          if (!mbar_wait(full0 + 8 * s, wrap & 1, a.status)) { ok = false; break; }
           tc_fence_after();
           if (kb == 0) IVIT_TRACE(it, 2);
           const uint32_t sp = base + s * stage_bytes, sq = a.q_resident ? qres + kb * a.q_stage_bytes : sp + BM * BK;
@@ -327,14 +350,22 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     }
   } else {
     // ---------------- epilogue warps; TMEM lane quarter = warp % 4, 32-column chunks dealt round-robin ----------------
-    const int et = threadIdx.x - 64;
-    const int ew = warp - 2;
+    // The groups of four warps ("parts") work independently.  A wait that times out is recorded and the
+    // warp carries on without further waits (its results are then meaningless and the status word says so).
+    const int et = threadIdx.x - 32 * kFirstEpiWarp;
+    const int ew = warp - kFirstEpiWarp;
     const int qd = warp & 3;
     const int part = ew >> 2;
     constexpr int kParts = kEpiWarps / 4;
     const GemmEpilogue& e = a.epi;
+    const bool dense = MODE ? true : a.lanes_are_channels != 0;
+    const bool tma_out = MODE ? true : a.tma_out != 0;
+    const bool tma_res = MODE ? MODE == 2 : a.tma_res != 0;
+    const bool ldg_res = MODE ? false : (e.res != nullptr && !a.tma_res);
+    const bool out_i32 = MODE ? false : e.out_dtype == IVIT_I32;
     const int rs_m = e.res_scale.mult, rs_s = clamp_shift(e.res_scale.shift);
     const long long rs_c = 1ll << (rs_s - 1);
+    bool ok = true;
 
     // Dense orientation: constants of this thread's channel; fetched one tile ahead
     int nm = 1, ns = 32, nb = 0;
@@ -347,146 +378,176 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         if (e.bias) nb = __ldg(e.bias + c);
       }
     };
-    if (a.lanes_are_channels && t_begin < t_end) fetch_channel(tile_coord(a, t_begin).p0);
+    if (dense && t_begin < t_end) fetch_channel(tile_coord(a, t_begin).p0);
     // MatMul orientation: one per-tensor constant set
     const int um = e.scale.mult, us = clamp_shift(e.scale.shift);
     const long long uc = 1ll << (us - 1);
 
-    int res_issued = 0, res_waited = 0;   // residual tiles requested / consumed (thread et == 0 issues them)
-    if (a.tma_res && et == 0 && t_begin < t_end) {
-      const TileCoord t0 = tile_coord(a, t_begin);
-      mbar_expect_tx(resf, (uint32_t)a.BN * 128u);
-      tma_load_4d(stage_res, &tmR, resf, t0.p0, t0.q0, 0, 0);
-      ++res_issued;
+    // Staged output (and residual input) of the Dense orientation: each part owns nslots slots of
+    // [32 rows][128 channels] bytes and uses them in turn, one per chunk.  The warp of a part that arrives
+    // last at a filled slot stores it by TMA and fetches the residual bytes of the chunk that will use the slot
+    // next (nslots chunks ahead); one chunk later the same thread sees the store's read of the slot complete
+    // and hands the slot back through its "free" barrier.
+    const int nchunks = a.BN >> 5;
+    const int nslots = tma_out ? (nchunks - part + kParts - 1) / kParts : 0;
+    int slots_before = 0;
+    for (int q = 0; q < part; ++q) slots_before += (nchunks - q + kParts - 1) / kParts;
+    const uint32_t part_off = (uint32_t)slots_before * 4096u;
+    const uint32_t my_out = stage_out + part_off, my_res = stage_res + part_off;
+    const uint32_t my_resf = resf + 8u * (uint32_t)(part * 4), my_scnt = sfull + 8u * (uint32_t)(part * 4),
+                   my_sfree = sfree + 8u * (uint32_t)(part * 4);
+    int slot = 0;                  // slot of the chunk in hand
+    uint32_t sround = 0;           // how often that slot has been used
+    int pend_prev = -1, pend_cur = -1;   // lane 0: slots of the stores it issued one chunk ago / in this chunk
+    // every warp follows the part's chunk sequence nslots chunks ahead (the residual bytes to fetch next)
+    TileIter pf_ti;
+    int64_t pf_t = t_begin;
+    int pf_ck = part;
+    auto pf_settle = [&]() {
+      while (pf_t < t_end) {
+        const int64_t left = a.Q - pf_ti.q0(a);
+        const int nck = (int)((left < a.BN ? left : a.BN) + 31) >> 5;
+        if (pf_ck < nck) break;
+        pf_ti.next(a);
+        ++pf_t;
+        pf_ck = part;
+      }
+    };
+    auto pf_advance = [&]() {
+      pf_ck += kParts;
+      pf_settle();
+    };
+    auto pf_fetch = [&](int sl) {
+      mbar_expect_tx(my_resf + 8u * sl, 4096u);
+      tma_load_4d(my_res + 4096u * sl, &tmR, my_resf + 8u * sl, pf_ti.p0(), pf_ti.q0(a) + 32 * pf_ck, 0, 0);
+    };
+    if (tma_res && t_begin < t_end) {
+      pf_ti.init(a, t_begin);
+      pf_settle();
+      for (int sl = 0; sl < nslots && pf_t < t_end; ++sl) {
+        if (qd == 0 && lane == 0) pf_fetch(sl);
+        pf_advance();
+      }
     }
+
     int it = 0;
     TileIter ti;
     ti.init(a, t_begin);
     for (int64_t t = t_begin; t < t_end; ++t, ++it) {
       TileCoord tc;
+      if (et == 0) IVIT_TRACE(it, 6);
       tc.batch = ti.batch; tc.bo = ti.bo; tc.bi = ti.bi; tc.p0 = ti.p0(); tc.q0 = ti.q0(a);
       ti.next(a);   // ti now describes the next tile
       const int buf = it & 1;
       const int cm = nm, cs = ns;
-      long long cc = (long long)nb * nm + (1ll << (ns - 1));   // bias * m + 2^(s-1)
-      asm volatile("" : "+l"(cc));   // keep it one 64-bit addend of the per-value multiply-add
-      const int64_t tn = t + 1;
-      if (a.lanes_are_channels && tn < t_end) fetch_channel(ti.p0());
+      const long long cc = (long long)nb * nm + (1ll << (ns - 1));   // bias * m + 2^(s-1)
+      const bool hi_ok = __all_sync(0xffffffffu, cs >= 32);    // the usual case: the shift is past the low word
+      // ... and when the rounding constant is past it too and acc + bias cannot leave 32 bits (|acc| <= 2^30
+      // since K <= 65536), only the high word of (acc + bias) * m is needed
+      const int cbias = nb;
+      const bool hi_only = __all_sync(0xffffffffu, cs >= 33 && nb > -(1 << 30) && nb < (1 << 30));
+      const int rnd_hi = cs >= 33 ? 1 << (cs - 33) : 0;
+      if (dense && t + 1 < t_end) fetch_channel(ti.p0());
 
-      // all epilogue threads take the same decision, so the named barrier never sees a partial group
-      if (a.tma_out && et == 0) tma_store_wait_read();   // the staging tile is free again
-      uint32_t got = mbar_wait(accf0 + 8 * buf, (it >> 1) & 1, a.status) ? 1u : 0u;
-      if (a.tma_res && got) {
-        got = mbar_wait(resf, it & 1, a.status) ? 1u : 0u;
-        if (got) ++res_waited;
-      }
-      if (!epi_all(got)) break;
+      if (et == 0) IVIT_TRACE(it, 7);
+      if (ok) ok = mbar_wait(accf0 + 8 * buf, (it >> 1) & 1, a.status);
       tc_fence_after();
       if (et == 0) IVIT_TRACE(it, 4);
       const uint32_t t_row = tmem_base + ((uint32_t)(qd * 32) << 16) + (uint32_t)(buf * a.BN);
+      const int64_t cols_left = a.Q - tc.q0;
+      const int nck = (int)((cols_left < a.BN ? cols_left : a.BN) + 31) >> 5;   // chunks that hold output
 
-      if (a.lanes_are_channels) {
+      if (dense) {
         // lane = output channel c, TMEM column = output row
         const int c = tc.p0 + qd * 32 + lane;
         const bool c_ok = c < a.P;
         const int sh_lo = min(cs, 32), sh_hi = max(cs - 32, 0);
-        for (int j0 = part * 32; j0 < a.BN; j0 += 32 * kParts) {
+        const int li = lane & 3;
+        const uint32_t sel1 = (li & 1) ? 0x3715u : 0x6240u;
+        const uint32_t sel2 = (li & 2) ? 0x3276u : 0x5410u;
+        const int cb = qd * 32 + lane;          // channel within the tile
+
+        // One chunk = 32 output rows x this warp's 32 channels, worked through in two halves of 16 rows to keep
+        // the register footprint small: the SM holds four epilogue warps per scheduler, and it is their number
+        // that hides the latencies of the shuffles, the shared-memory traffic and the barrier operations.
+        auto half = [&](int ck, int h, uint8_t* pe, uint8_t* po) {
+          const int j0 = ck * 32 + h * 16;
           const int64_t r0 = (int64_t)tc.q0 + j0;
-          if (r0 >= a.Q) break;
-#ifdef IVIT_DBG_NOEPI
-          break;
-#endif
-          int v[32];
-#ifdef IVIT_TC_TRACE
-          if (et == 0 && j0 == 0) IVIT_TRACE(it, 6);
-#endif
-          tmem_ld32(t_row + (uint32_t)j0, v);
-#ifdef IVIT_TC_TRACE
-          if (et == 0 && j0 == 0) IVIT_TRACE(it, 7);
-#endif
-          const int nrow = (int)min((int64_t)32, a.Q - r0);
-#ifdef IVIT_DBG_EPI_LDONLY
-          asm volatile("" :: "r"(v[0]), "r"(v[31]));
-          continue;
-#endif
-          // requantise: one 32x32->64 multiply-add and two shifts per value, 32 independent chains
+          const int nrow = (int)min((int64_t)16, a.Q - r0);
+          int v[16];
+          tmem_ld16(t_row + (uint32_t)j0, v);
+          if (hi_only) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const long long tt = (long long)v[j] * (long long)cm + cc;
-            v[j] = (int)__funnelshift_rc((unsigned)tt, (unsigned)(tt >> 32), sh_lo) >> sh_hi;
+            for (int j = 0; j < 16; ++j) v[j] = mad_hi(v[j] + cbias, cm, rnd_hi) >> sh_hi;
+          } else if (hi_ok) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] = mad_wide_hi(v[j], cm, cc) >> sh_hi;
+          } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+              const long long tt = mad_wide(v[j], cm, cc);
+              v[j] = (int)__funnelshift_rc((unsigned)tt, (unsigned)(tt >> 32), sh_lo) >> sh_hi;
+            }
           }
-          // residual port: the byte of (row, channel) is a coalesced load across the lanes
-          if (a.tma_res) {
-            // residual tile in shared memory: [row][128 channels], 16-byte chunks XOR (row & 7)
-            const int cb = qd * 32 + lane;
-            const uint8_t* rt = gen_base + (stage_res - base) + j0 * 128 + (cb & 15);
+          // residual port
+          if (tma_res) {
+            // residual bytes of this chunk in shared memory: [row][128 channels], 16-byte pieces XOR (row & 7)
+            const uint8_t* rt = gen_base + (my_res - base) + slot * 4096 + h * 2048 + (cb & 15);
             int off[8];
 #pragma unroll
             for (int x = 0; x < 8; ++x) off[x] = ((cb >> 4) ^ x) << 4;
+            if (rs_s >= 32) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j) {
-              const int xr = (int)*reinterpret_cast<const int8_t*>(rt + j * 128 + off[j & 7]);
-              v[j] += (int)(((long long)xr * rs_m + rs_c) >> rs_s);
+              for (int j = 0; j < 16; ++j) {
+                const int xr = (int)*reinterpret_cast<const int8_t*>(rt + j * 128 + off[j & 7]);
+                v[j] += mad_wide_hi(xr, rs_m, rs_c) >> (rs_s - 32);
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) {
+                const int xr = (int)*reinterpret_cast<const int8_t*>(rt + j * 128 + off[j & 7]);
+                v[j] += (int)(mad_wide(xr, rs_m, rs_c) >> rs_s);
+              }
             }
-          } else if (e.res) {
+          } else if (ldg_res) {
             int64_t rr = (int64_t)((uint64_t)r0 % (uint64_t)e.res_rows);
 #pragma unroll
-            for (int h = 0; h < 32; h += 8) {
+            for (int g = 0; g < 16; g += 8) {
               int xr[8];
 #pragma unroll
               for (int j = 0; j < 8; ++j) {
-                xr[j] = (c_ok && h + j < nrow) ? (int)__ldg(e.res + rr * e.ldres + c) : 0;
+                xr[j] = (c_ok && g + j < nrow) ? (int)__ldg(e.res + rr * e.ldres + c) : 0;
                 if (++rr == e.res_rows) rr = 0;
               }
 #pragma unroll
-              for (int j = 0; j < 8; ++j) v[h + j] += (int)(((long long)xr[j] * rs_m + rs_c) >> rs_s);
+              for (int j = 0; j < 8; ++j) v[g + j] += (int)(mad_wide(xr[j], rs_m, rs_c) >> rs_s);
             }
           }
-#ifdef IVIT_TC_TRACE
-          tmem_ld_wait(v);   // no outstanding load: only ties the stamp below to the finished values
-          if (et == 0 && j0 == 0) IVIT_TRACE(it, 0);   // reuses slot 0 (producer stamp) in trace builds
-#endif
-          if (e.out_dtype == IVIT_I32) {
-            int64_t ro = r0;
+          if (out_i32) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (j < nrow && c_ok) reinterpret_cast<int32_t*>(e.out)[(ro + j) * e.ldo + c] = v[j];
-            continue;
+            for (int j = 0; j < 16; ++j)
+              if (j < nrow && c_ok) reinterpret_cast<int32_t*>(e.out)[(r0 + j) * e.ldo + c] = v[j];
+            return;
           }
-          // int8: pack four rows per word, transpose 4x4 bytes inside each group of four lanes so
-          // that a lane ends up with four consecutive channels of one row (stage by stage over all
-          // eight words, so that the shuffles overlap), then store 4 bytes per lane and word
-          const int li = lane & 3;
-          const uint32_t sel1 = (li & 1) ? 0x3715u : 0x6240u;
-          const uint32_t sel2 = (li & 2) ? 0x3276u : 0x5410u;
-          uint32_t w[8], o[8];
+          // int8: pack four rows per word, transpose 4x4 bytes inside each group of four lanes so that a lane
+          // ends up with four consecutive channels of one row, then store 4 bytes per lane and word
+          uint32_t w[4], o[4];
 #pragma unroll
-          for (int k = 0; k < 8; ++k) w[k] = pack_sat8(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
+          for (int k = 0; k < 4; ++k) w[k] = pack_sat8(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]);
 #pragma unroll
-          for (int k = 0; k < 8; ++k) o[k] = __shfl_xor_sync(0xffffffffu, w[k], 1);
+          for (int k = 0; k < 4; ++k) o[k] = __shfl_xor_sync(0xffffffffu, w[k], 1);
 #pragma unroll
-          for (int k = 0; k < 8; ++k) w[k] = __byte_perm(w[k], o[k], sel1);
+          for (int k = 0; k < 4; ++k) w[k] = __byte_perm(w[k], o[k], sel1);
 #pragma unroll
-          for (int k = 0; k < 8; ++k) o[k] = __shfl_xor_sync(0xffffffffu, w[k], 2);
+          for (int k = 0; k < 4; ++k) o[k] = __shfl_xor_sync(0xffffffffu, w[k], 2);
 #pragma unroll
-          for (int k = 0; k < 8; ++k) w[k] = __byte_perm(w[k], o[k], sel2);
-#ifdef IVIT_DBG_EPI_NOSTS
-          asm volatile("" :: "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]));
-          continue;
-#endif
-          if (a.tma_out) {
-            // staging tile [row][128 channels]; 16-byte chunk index XOR (row & 7) is the 128B swizzle
-            // of the store map.  Word k belongs to tile row j0 + li + 4k: (row & 7) alternates between
-            // two values, so two base addresses plus immediates address all eight words.
-            const int trow = j0 + li;
-            const int cb = qd * 32 + (lane & ~3);
-            uint8_t* row0 = gen_base + (stage_out - base) + trow * 128 + (cb & 15);
-            uint8_t* pe = row0 + ((((cb >> 4) ^ (trow & 7)) & 7) << 4);
-            uint8_t* po = row0 + ((((cb >> 4) ^ ((trow + 4) & 7)) & 7) << 4);
+          for (int k = 0; k < 4; ++k) w[k] = __byte_perm(w[k], o[k], sel2);
+          if (tma_out) {
+            // word k belongs to slot row 16h + li + 4k
 #pragma unroll
-            for (int k = 0; k < 8; k += 2) {
-              *reinterpret_cast<uint32_t*>(pe + 512 * k) = w[k];
-              *reinterpret_cast<uint32_t*>(po + 512 * (k + 1)) = w[k + 1];
+            for (int k = 0; k < 4; k += 2) {
+              *reinterpret_cast<uint32_t*>(pe + 2048 * h + 512 * k) = w[k];
+              *reinterpret_cast<uint32_t*>(po + 2048 * h + 512 * (k + 1)) = w[k + 1];
             }
           } else {
             // direct stores (grouped output rows): this lane's first word is row r0 + li, then + 4 per word
@@ -498,7 +559,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
             const int cbase = tc.p0 + qd * 32 + (lane & ~3);
             const bool cg_ok = cbase < a.P;   // P % 4 == 0: a group of four channels is valid as a whole
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
+            for (int k = 0; k < 4; ++k) {
               if (cg_ok && 4 * k + li < nrow)
                 *reinterpret_cast<uint32_t*>(reinterpret_cast<int8_t*>(e.out) + ro * e.ldo + cbase) = w[k];
               ro += 4;
@@ -508,19 +569,51 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
               }
             }
           }
-        }
-        if (a.tma_out) {
-          // every epilogue warp has written its part of the staging tile: one thread stores it
-          fence_async_smem();
-          asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
-          if (et == 0) {
-            tma_store_4d(&tmO, stage_out, tc.p0, tc.q0, 0, 0);
-            if (a.tma_res && tn < t_end) {
-              // every warp is past its reads of the residual tile: fetch the next tile's
-              mbar_expect_tx(resf, (uint32_t)a.BN * 128u);
-              tma_load_4d(stage_res, &tmR, resf, ti.p0(), ti.q0(a), 0, 0);
-              ++res_issued;
+        };
+
+        for (int ck = part; ck < nck; ck += kParts) {
+          uint8_t *pe = nullptr, *po = nullptr;
+          if (tma_out) {
+            if (nslots == 1 && lane == 0 && pend_prev >= 0) {
+              // a single slot: the store issued in the previous chunk must have read it before anyone goes on
+              tma_store_wait_read();
+              mbar_arrive(my_sfree + 8u * pend_prev);
+              pend_prev = -1;
             }
+            // the slot's previous store must have read it; its residual bytes must have arrived
+            if (sround > 0 && ok) ok = mbar_wait(my_sfree + 8u * slot, (sround - 1u) & 1u, a.status);
+            if (tma_res && ok) ok = mbar_wait(my_resf + 8u * slot, sround & 1u, a.status);
+            // slot layout [row][128 channels]; 16-byte piece index XOR (row & 7) is the 128B swizzle of the
+            // store map.  A lane's words belong to slot rows li + 4k: (row & 7) alternates between two values,
+            // so two base addresses plus immediates address all of them.
+            const int cg = qd * 32 + (lane & ~3);
+            uint8_t* row0 = gen_base + (my_out - base) + slot * 4096 + li * 128 + (cg & 15);
+            pe = row0 + ((((cg >> 4) ^ li) & 7) << 4);
+            po = row0 + ((((cg >> 4) ^ (li + 4)) & 7) << 4);
+          }
+          half(ck, 0, pe, po);
+          half(ck, 1, pe, po);
+          if (tma_out) {
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+              // fourth arrival: every warp's bytes are in the slot and visible to the copy engine
+              if ((smem_add_acq_rel(my_scnt + 8u * slot, 1u) & 3u) == 3u) {
+                tma_store_4d(&tmO, my_out + 4096u * slot, tc.p0, tc.q0 + 32 * ck, 0, 0);
+                // ... and every warp is past its reads of the slot's residual bytes
+                if (tma_res && pf_t < t_end) pf_fetch(slot);
+                pend_cur = slot;
+              }
+              if (pend_prev >= 0) {
+                // the store issued one chunk ago has had a chunk's time to read its slot
+                tma_store_wait_read1_or_all(pend_cur >= 0);
+                mbar_arrive(my_sfree + 8u * pend_prev);
+              }
+              pend_prev = pend_cur;
+              pend_cur = -1;
+            }
+            pf_advance();
+            if (++slot == nslots) { slot = 0; ++sround; }
           }
         }
       } else {
@@ -529,9 +622,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         const bool row_ok = r < a.P;
         const int64_t out_row = tc.bo * a.sCo + tc.bi * a.sCi + r * e.ldo;
         const int32_t* bias_row = e.bias32 ? e.bias32 + ((tc.batch % e.bias_batches) * a.P + r) * e.ldbias : nullptr;
-        for (int j0 = part * 32; j0 < a.BN; j0 += 32 * kParts) {
+        for (int ck = part; ck < nck; ck += kParts) {
+          const int j0 = ck * 32;
           const int c0 = tc.q0 + j0;
-          if (c0 >= a.Q) break;
           int v[32];
           tmem_ld32(t_row + (uint32_t)j0, v);
           if (!row_ok) continue;
@@ -559,15 +652,20 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
           }
         }
       }
+      if (et == 0) IVIT_TRACE(it, 0);
       // this warp has read everything it needs from the buffer: hand it back to the MMA warp
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(acce0 + 8 * buf);
       if (et == 0) IVIT_TRACE(it, 5);
     }
-    if (a.tma_out && et == 0) tma_store_wait_all();
-    // only after a timeout: a residual tile may still be in flight into shared memory
-    if (et == 0 && res_issued > res_waited) mbar_wait(resf, res_waited & 1, a.status);
+    if (tma_out && lane == 0) {
+      tma_store_wait_all();
+      if (pend_prev >= 0) mbar_arrive(my_sfree + 8u * pend_prev);
+    }
+    // only after a timeout: residual bytes fetched for chunks that were never worked on may be in flight
+    if (tma_res && !ok && qd == 0 && lane == 0)
+      for (int sl = 0; sl < nslots; ++sl) mbar_wait(my_resf + 8u * sl, ((uint32_t)(sl < slot) + sround) & 1u, a.status);
   }
   tc_fence_before();
   __syncthreads();
@@ -575,6 +673,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     tc_fence_after();
     tmem_dealloc(tmem_base, (uint32_t)a.tmem_cols);
   }
+#ifdef IVIT_TC_TRACE
+  if (threadIdx.x == 0) { IVIT_TRACE(39, 3); long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); g_trace[blockIdx.x][39][5] = g; }
+#endif
 }
 
 // ---- host side ------------------------------------------------------------------------------
@@ -586,7 +687,7 @@ int pow2_at_least(int v) {
 }
 
 constexpr size_t kSmemBudget = 227 * 1024;
-constexpr size_t kSmemFixed = 1024 + 8 * (2 * kMaxStages + 7) + 32;
+constexpr size_t kSmemFixed = 1024 + 8 * (2 * kMaxStages + 54) + 32;
 
 bool g_attr_set = false;
 
@@ -663,13 +764,13 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
   CUtensorMap tmO = tmP;
   if (dense && e.out_dtype == IVIT_I8 && e.group_rows <= 0 && !(reinterpret_cast<uintptr_t>(e.out) & 15) && e.ldo % 16 == 0) {
     int opos[3];
-    a.tma_out = make_tensor_map(ctx, &tmO, reinterpret_cast<const int8_t*>(e.out), g.N, g.M, 1, 1, e.ldo, 0, 0, BM, a.BN,
+    a.tma_out = make_tensor_map(ctx, &tmO, reinterpret_cast<const int8_t*>(e.out), g.N, g.M, 1, 1, e.ldo, 0, 0, BM, 32,
                          CU_TENSOR_MAP_SWIZZLE_128B, opos) ? 1 : 0;
   }
   CUtensorMap tmR = tmP;
   if (a.tma_out && e.res && e.res_rows >= g.M && !(reinterpret_cast<uintptr_t>(e.res) & 15) && e.ldres % 16 == 0) {
     int rpos[3];
-    a.tma_res = make_tensor_map(ctx, &tmR, e.res, g.N, g.M, 1, 1, e.ldres, 0, 0, BM, a.BN, CU_TENSOR_MAP_SWIZZLE_128B,
+    a.tma_res = make_tensor_map(ctx, &tmR, e.res, g.N, g.M, 1, 1, e.ldres, 0, 0, BM, 32, CU_TENSOR_MAP_SWIZZLE_128B,
                                 rpos) ? 1 : 0;
   }
   const size_t out_stage = (a.tma_out ? (size_t)a.BN * 128 : 0) + (a.tma_res ? (size_t)a.BN * 128 : 0);
@@ -688,13 +789,19 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
 
   const size_t smem = kSmemFixed + (size_t)a.stages * stage + fixed;
   if (!g_attr_set) {
-    if (cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess)
+    if (cudaFuncSetAttribute(gemm_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess)
       return IVIT_ERR_CUDA;
     g_attr_set = true;
   }
   const unsigned grid = (unsigned)(a.total_tiles < ctx->sm_count ? a.total_tiles : ctx->sm_count);
   LaunchScope ls(ctx, KIND_GEMM_TC, 2.0 * (double)batches * (double)g.M * (double)g.N * (double)g.K);
-  launch_k(gemm_tc_kernel, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
+  // the encoder block's Dense layers take the specialised instantiations
+  const int mode = (a.lanes_are_channels && a.tma_out && (!e.res || a.tma_res)) ? (a.tma_res ? 2 : 1) : 0;
+  if (mode == 2) launch_k(gemm_tc_kernel<2>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
+  else if (mode == 1) launch_k(gemm_tc_kernel<1>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
+  else launch_k(gemm_tc_kernel<0>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
   return ls.done();
 }
 

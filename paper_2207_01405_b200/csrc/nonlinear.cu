@@ -160,8 +160,8 @@ __global__ void __launch_bounds__(256) layernorm_i8_batched_kernel(const int8_t*
         s1 = __dp4a(w[r][i], 0x01010101, s1);
         s2 = __dp4a(w[r][i], w[r][i], s2);
       }
-      s1 = warp_sum(s1);
-      s2 = warp_sum(s2);
+      s1 = __reduce_add_sync(0xffffffffu, s1);   // one redux.sync per sum instead of a shuffle tree
+      s2 = __reduce_add_sync(0xffffffffu, s2);
       if (lane == r) { my_s1 = s1; my_s2 = s2; }
     }
     // lane r (< ROWS) holds the sums of row r0 + r: mean (round half up), sum of squared
@@ -297,16 +297,16 @@ int launch_layernorm(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, 
   const int8_t* x = (const int8_t*)in;
   const int wpl = (int)((C / 4 + 31) / 32);
   if (wpl <= 4) {
-    // batched kernel: 8 rows per warp (4 for the wider rows) amortise the per-row scalar work and the
-    // per-channel constants
-    const int rpw = wpl <= 3 ? 8 : 4;
+    // batched kernel: 4 rows per warp amortise the per-row scalar work and the per-channel constants;
+    // 128-thread blocks keep enough warps in flight on every SM
+    const int rpw = 4, tb = 128;
     const int64_t warps = (rows + rpw - 1) / rpw;
-    const int64_t wantb = (warps + wpb - 1) / wpb;
-    const int gridb = (int)(wantb < (int64_t)ctx->sm_count * 8 ? wantb : (int64_t)ctx->sm_count * 8);
-    if (wpl <= 1) launch_k(layernorm_i8_batched_kernel<1, 8>, dim3(gridb), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-    else if (wpl <= 2) launch_k(layernorm_i8_batched_kernel<2, 8>, dim3(gridb), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-    else if (wpl <= 3) launch_k(layernorm_i8_batched_kernel<3, 8>, dim3(gridb), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-    else launch_k(layernorm_i8_batched_kernel<4, 4>, dim3(gridb), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+    const int64_t wantb = (warps + tb / 32 - 1) / (tb / 32);
+    const int gridb = (int)(wantb < (int64_t)ctx->sm_count * 16 ? wantb : (int64_t)ctx->sm_count * 16);
+    if (wpl <= 1) launch_k(layernorm_i8_batched_kernel<1, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+    else if (wpl <= 2) launch_k(layernorm_i8_batched_kernel<2, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+    else if (wpl <= 3) launch_k(layernorm_i8_batched_kernel<3, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+    else launch_k(layernorm_i8_batched_kernel<4, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
     return ls.done();
   }
   if (wpl <= 6) launch_k(layernorm_i8_kernel<6>, dim3(grid), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);

@@ -39,6 +39,16 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity), "r"(kSuspendHintNs) : "memory");
   return ok != 0;
 }
+// One non-blocking test of the phase.
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
 // Bounded wait: false (and the timeout recorded) when the phase did not complete in time.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* status) {
   for (uint32_t i = 0; i < kSpinLimit; ++i)
@@ -62,6 +72,20 @@ __device__ __forceinline__ void tma_store_4d(const CUtensorMap* map, uint32_t sr
 }
 // Blocks until the shared-memory source of every committed store has been read.
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// ... of every committed store but the latest.
+__device__ __forceinline__ void tma_store_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+// ... of every committed store of this thread, or of all but the one committed last.
+__device__ __forceinline__ void tma_store_wait_read1_or_all(bool keep_last) {
+  if (keep_last) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+  else asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+// Adds to a 32-bit word in shared memory; releases this thread's earlier writes and acquires those of the
+// threads whose additions it observes.  Returns the old value.
+__device__ __forceinline__ uint32_t smem_add_acq_rel(uint32_t addr, uint32_t v) {
+  uint32_t old;
+  asm volatile("atom.acq_rel.cta.shared::cta.add.u32 %0, [%1], %2;" : "=r"(old) : "r"(addr), "r"(v) : "memory");
+  return old;
+}
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
@@ -132,6 +156,27 @@ __device__ __forceinline__ void tmem_ld_wait(int (&v)[32]) {
                  "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])
                :: "memory");
 }
+// The same for 16 consecutive columns (load and wait in one).
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr) : "memory");
+}
+// The same for 8 consecutive columns.
+__device__ __forceinline__ void tmem_ld8_issue(uint32_t taddr, int (&v)[8]) {
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+               : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait8(int (&v)[8]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7])
+               :: "memory");
+}
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, int (&v)[32]) {
   tmem_ld32_issue(taddr, v);
   tmem_ld_wait(v);
@@ -171,6 +216,26 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
 }
 
 // saturating pack of four int32 into int8x4 (x0 in the lowest byte)
+// High word of a * m + c: one multiply-add with a 64-bit addend.
+__device__ __forceinline__ int mad_wide_hi(int a, int m, long long c) {
+  int hi;
+  asm("{\n\t.reg .s64 t;\n\t.reg .b32 lo;\n\tmad.wide.s32 t, %1, %2, %3;\n\tmov.b64 {lo, %0}, t;\n\t}"
+      : "=r"(hi) : "r"(a), "r"(m), "l"(c));
+  return hi;
+}
+// High word of a * m, plus c.
+__device__ __forceinline__ int mad_hi(int a, int m, int c) {
+  int d;
+  asm("mad.hi.s32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(m), "r"(c));
+  return d;
+}
+// a * m + c as one multiply-add with a 64-bit addend.
+__device__ __forceinline__ long long mad_wide(int a, int m, long long c) {
+  long long t;
+  asm("mad.wide.s32 %0, %1, %2, %3;" : "=l"(t) : "r"(a), "r"(m), "l"(c));
+  return t;
+}
+
 __device__ __forceinline__ uint32_t pack_sat8(int x0, int x1, int x2, int x3) {
   uint32_t t, d;
   asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(t) : "r"(x3), "r"(x2), "r"(0));
