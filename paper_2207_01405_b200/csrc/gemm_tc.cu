@@ -173,45 +173,56 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
   const int kblocks = (int)((a.K + BK - 1) / BK);
   const uint32_t qres_bytes = a.q_resident ? kblocks * a.q_stage_bytes : 0;
   const uint32_t qres = base + a.stages * stage_bytes;         // resident Q tile: kblocks x [BN rows x 128 B]
-  const uint32_t stage_out = qres + qres_bytes;                // [BN rows][128 channels] int8, 128B-swizzled
-  const uint32_t stage_res = stage_out + (a.tma_out ? a.BN * 128 : 0);   // residual tile, same layout
-  const uint32_t bars_off = a.stages * stage_bytes + qres_bytes + (a.tma_out ? a.BN * 128 : 0) + (a.tma_res ? a.BN * 128 : 0);
+  const uint32_t stage_out = qres + qres_bytes;                // output slots: 2 x [32 rows][32 channels] int8 per epilogue warp
+  const uint32_t stage_res = stage_out + (a.tma_out ? kEpiWarps * 2048 : 0);   // residual slots, same layout
+  const uint32_t bars_off = a.stages * stage_bytes + qres_bytes + (a.tma_out ? kEpiWarps * 2048 : 0) + (a.tma_res ? kEpiWarps * 2048 : 0);
   const uint32_t full0 = base + bars_off, empty0 = full0 + 8 * kMaxStages;
-  const uint32_t accf0 = empty0 + 8 * kMaxStages, acce0 = accf0 + 16, resf = acce0 + 16, sfull = resf + 128, sfree = sfull + 128, qresf = sfree + 128, qrese = qresf + 8;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + bars_off + 8 * (2 * kMaxStages + 54));
+  const uint32_t accf0 = empty0 + 8 * kMaxStages, acce0 = accf0 + 16, resf = acce0 + 16, qrese = resf + 16 * kEpiWarps;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + bars_off + 8 * (2 * kMaxStages + 5 + 2 * kEpiWarps));
   volatile int* issued_slot = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // this CTA's contiguous range of tiles
   const int64_t t_begin = a.total_tiles * blockIdx.x / gridDim.x, t_end = a.total_tiles * (blockIdx.x + 1) / gridDim.x;
-  volatile int* qres_issued = issued_slot + 1;
 
-  if (threadIdx.x == 0) {
-    prefetch_tmap(&tmP);
-    prefetch_tmap(&tmQ);
-    if (a.tma_out) prefetch_tmap(&tmO);
-    if (a.tma_res) prefetch_tmap(&tmR);
-    for (int s = 0; s < a.stages; ++s) {
-      mbar_init(full0 + 8 * s, 1);
-      mbar_init(empty0 + 8 * s, 1);
+  // set-up, spread over the epilogue threads: one barrier (or descriptor prefetch) each
+  {
+    const int i = (int)threadIdx.x - 64;
+    if (i >= 0 && i < kMaxStages) {
+      mbar_init(full0 + 8 * i, 1);
+    } else if (i < 2 * kMaxStages) {
+      mbar_init(empty0 + 8 * (i - kMaxStages), 1);
+    } else if (i < 2 * kMaxStages + 2) {
+      mbar_init(accf0 + 8 * (i - 2 * kMaxStages), 1);
+    } else if (i < 2 * kMaxStages + 4) {
+      mbar_init(acce0 + 8 * (i - 2 * kMaxStages - 2), kEpiWarps);
+    } else if (i < 2 * kMaxStages + 4 + 2 * kEpiWarps) {
+      mbar_init(resf + 8 * (i - 2 * kMaxStages - 4), 1);   // residual slots: 2 per epilogue warp
+    } else if (i == 2 * kMaxStages + 4 + 2 * kEpiWarps) {
+      mbar_init(qrese, 1);
+      *issued_slot = 0;
+    } else if (i == 2 * kMaxStages + 5 + 2 * kEpiWarps) {
+      prefetch_tmap(&tmP);
+    } else if (i == 2 * kMaxStages + 6 + 2 * kEpiWarps) {
+      prefetch_tmap(&tmQ);
+    } else if (i == 2 * kMaxStages + 7 + 2 * kEpiWarps) {
+      if (a.tma_out) prefetch_tmap(&tmO);
+    } else if (i == 2 * kMaxStages + 8 + 2 * kEpiWarps) {
+      if (a.tma_res) prefetch_tmap(&tmR);
     }
-    for (int b = 0; b < 2; ++b) {
-      mbar_init(accf0 + 8 * b, 1);
-      mbar_init(acce0 + 8 * b, kEpiWarps);
+    if (i >= 0 && i < 2 * kMaxStages + 5 + 2 * kEpiWarps) {
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      fence_async_smem();
     }
-    for (int b = 0; b < 16; ++b) {   // staging slots: 4 per epilogue part
-      mbar_init(resf + 8 * b, 1);
-      *reinterpret_cast<uint32_t*>(gen_base + (sfull - base) + 8 * b) = 0;   // arrivals of a part's warps at a slot
-      mbar_init(sfree + 8 * b, 1);
-    }
-    mbar_init(qresf, 1);
-    mbar_init(qrese, 1);
-    *qres_issued = 0;
-    *issued_slot = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    fence_async_smem();
   }
+#ifdef IVIT_TC_TRACE
+  if (threadIdx.x == 64) IVIT_TRACE(38, 0);
+  if (threadIdx.x == 32) IVIT_TRACE(38, 1);
+#endif
   if (warp == 1) tmem_alloc(smem_u32(tmem_slot), (uint32_t)a.tmem_cols);
+#ifdef IVIT_TC_TRACE
+  if (threadIdx.x == 32) IVIT_TRACE(38, 2);
+#endif
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
@@ -247,19 +258,22 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         IVIT_TRACE(pit, 0);
         const int pc1 = pr == 1 ? p0 : (pbi == 1 ? ti.bi : ti.bo), pc2 = pr == 2 ? p0 : (pbi == 2 ? ti.bi : ti.bo),
                   pc3 = pr == 3 ? p0 : (pbi == 3 ? ti.bi : ti.bo);
+        bool bring_q = false;
         if (a.q_resident && q0 != cur_q) {
-          // new activation row block: refill the resident tile once every MMA on the old one is done
+          // new activation row block: its k-blocks come in beside this tile's weight k-blocks, once every MMA
+          // on the old block is done
           if (qi > 0 && !mbar_wait(qrese, (qi - 1) & 1, a.status)) { ok = false; break; }
-          mbar_expect_tx(qresf, qres_bytes);
-          for (int kb = 0; kb < kblocks; ++kb)
-            tma_load_4d(qres + kb * a.q_stage_bytes, &tmQ, qresf, kb * BK, qr == 1 ? q0 : 0, qr == 2 ? q0 : 0, qr == 3 ? q0 : 0);
+          bring_q = true;
           cur_q = q0;
-          *qres_issued = ++qi;
+          ++qi;
         }
         for (int kb = 0; kb < kblocks; ++kb) {
           if (wrap > 0 && !mbar_wait(empty0 + 8 * s, (wrap & 1) ^ 1, a.status)) { ok = false; break; }
           const uint32_t sp = base + s * stage_bytes, sq = sp + BM * BK;
-          mbar_expect_tx(full0 + 8 * s, stage_bytes);
+          mbar_expect_tx(full0 + 8 * s, stage_bytes + (bring_q ? a.q_stage_bytes : 0));
+          if (bring_q)
+            tma_load_4d(qres + kb * a.q_stage_bytes, &tmQ, full0 + 8 * s, kb * BK, qr == 1 ? q0 : 0, qr == 2 ? q0 : 0,
+                        qr == 3 ? q0 : 0);
           tma_load_4d(sp, &tmP, full0 + 8 * s, kb * BK, pc1, pc2, pc3);
           if (!a.q_resident) {
             const int qrow = a.q_mn ? kb * BK : q0;     // MN-major: rows of the map are k, the inner index is n
@@ -289,7 +303,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       const int tail_steps = k_tail >= BK ? BK / UMMA_K : (k_tail + UMMA_K - 1) / UMMA_K;
       int consumed = 0, s = 0, wrap = 0, it = 0;
       bool ok = true;
-      int qi = 0, cur_q = -1;
+      int cur_q = -1;
       TileIter ti;
       ti.init(a, t_begin);
       for (int64_t t = t_begin; ok && t < t_end; ++t, ++it) {
@@ -300,12 +314,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
 #else
         if (a.q_resident) {
 #endif
-          const int q0 = ti.q0(a);
-          if (q0 != cur_q) {
-            if (!mbar_wait(qresf, qi & 1, a.status)) { ok = false; break; }
-            cur_q = q0;
-            ++qi;
-          }
+          // a new activation row block arrives k-block by k-block on the stage barriers of this tile
+          cur_q = ti.q0(a);
           ti.next(a);
           last_of_q = t + 1 >= t_end || ti.q0(a) != cur_q;
         }
@@ -344,8 +354,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
           mbar_wait(full0 + 8 * s, wrap & 1, a.status);
           if (++s == a.stages) { s = 0; ++wrap; }
         }
-        const int qissued = *qres_issued;
-        for (int j = qi; j < qissued; ++j) mbar_wait(qresf, j & 1, a.status);
       }
     }
   } else {
@@ -383,26 +391,20 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     const int um = e.scale.mult, us = clamp_shift(e.scale.shift);
     const long long uc = 1ll << (us - 1);
 
-    // Staged output (and residual input) of the Dense orientation: each part owns nslots slots of
-    // [32 rows][128 channels] bytes and uses them in turn, one per chunk.  The warp of a part that arrives
-    // last at a filled slot stores it by TMA and fetches the residual bytes of the chunk that will use the slot
-    // next (nslots chunks ahead); one chunk later the same thread sees the store's read of the slot complete
-    // and hands the slot back through its "free" barrier.
-    const int nchunks = a.BN >> 5;
-    const int nslots = tma_out ? (nchunks - part + kParts - 1) / kParts : 0;
-    int slots_before = 0;
-    for (int q = 0; q < part; ++q) slots_before += (nchunks - q + kParts - 1) / kParts;
-    const uint32_t part_off = (uint32_t)slots_before * 4096u;
-    const uint32_t my_out = stage_out + part_off, my_res = stage_res + part_off;
-    const uint32_t my_resf = resf + 8u * (uint32_t)(part * 4), my_scnt = sfull + 8u * (uint32_t)(part * 4),
-                   my_sfree = sfree + 8u * (uint32_t)(part * 4);
-    int slot = 0;                  // slot of the chunk in hand
-    uint32_t sround = 0;           // how often that slot has been used
-    int pend_prev = -1, pend_cur = -1;   // lane 0: slots of the stores it issued one chunk ago / in this chunk
-    // every warp follows the part's chunk sequence nslots chunks ahead (the residual bytes to fetch next)
+    // Staged output (and residual input) of the Dense orientation: every warp owns two slots of
+    // [32 rows][32 channels] bytes for each direction and needs no other warp to move them.  Its lane 0 stores a
+    // filled output slot by TMA (a box of 32 channels x 32 rows) and fetches the residual bytes two chunks
+    // ahead of the arithmetic into the slot whose bytes have just been used.
+    const uint32_t my_out = stage_out + (uint32_t)ew * 2048u, my_res = stage_res + (uint32_t)ew * 2048u;
+    const uint32_t my_resf = resf + 16u * (uint32_t)ew;
+    const int c_first = qd * 32;        // first channel of this warp inside the tile
+    uint32_t g = 0;                     // chunks this warp has worked on
+    uint32_t rpar = 0, rpend = 0;       // per residual slot (bit 0 / 1): parity of its next arrival; a fetch in flight
+    // the warp's chunk sequence two chunks ahead: tile by tile, chunks part, part + kParts, ...
     TileIter pf_ti;
     int64_t pf_t = t_begin;
     int pf_ck = part;
+    uint32_t pf_g = 0;
     auto pf_settle = [&]() {
       while (pf_t < t_end) {
         const int64_t left = a.Q - pf_ti.q0(a);
@@ -413,21 +415,28 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         pf_ck = part;
       }
     };
-    auto pf_advance = [&]() {
-      pf_ck += kParts;
-      pf_settle();
-    };
-    auto pf_fetch = [&](int sl) {
-      mbar_expect_tx(my_resf + 8u * sl, 4096u);
-      tma_load_4d(my_res + 4096u * sl, &tmR, my_resf + 8u * sl, pf_ti.p0(), pf_ti.q0(a) + 32 * pf_ck, 0, 0);
+    // residual bytes of the next chunk of the look-ahead into slot pf_g & 1 (a box wholly past the last channel
+    // is not fetched: the arithmetic does not wait for it either)
+    auto pf_fetch = [&]() {
+      if (pf_t < t_end) {
+        if (pf_ti.p0() + c_first < a.P) {
+          const uint32_t sl = pf_g & 1u;
+          if (lane == 0) {
+            mbar_expect_tx(my_resf + 8u * sl, 1024u);
+            tma_load_4d(my_res + 1024u * sl, &tmR, my_resf + 8u * sl, pf_ti.p0() + c_first, pf_ti.q0(a) + 32 * pf_ck, 0, 0);
+          }
+          rpend |= 1u << sl;
+        }
+        ++pf_g;
+        pf_ck += kParts;
+        pf_settle();
+      }
     };
     if (tma_res && t_begin < t_end) {
       pf_ti.init(a, t_begin);
       pf_settle();
-      for (int sl = 0; sl < nslots && pf_t < t_end; ++sl) {
-        if (qd == 0 && lane == 0) pf_fetch(sl);
-        pf_advance();
-      }
+      pf_fetch();
+      pf_fetch();
     }
 
     int it = 0;
@@ -470,12 +479,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         // One chunk = 32 output rows x this warp's 32 channels, worked through in two halves of 16 rows to keep
         // the register footprint small: the SM holds four epilogue warps per scheduler, and it is their number
         // that hides the latencies of the shuffles, the shared-memory traffic and the barrier operations.
-        auto half = [&](int ck, int h, uint8_t* pe, uint8_t* po) {
+        auto half = [&](int (&v)[16], int ck, int h, uint8_t* pe) {
           const int j0 = ck * 32 + h * 16;
           const int64_t r0 = (int64_t)tc.q0 + j0;
           const int nrow = (int)min((int64_t)16, a.Q - r0);
-          int v[16];
-          tmem_ld16(t_row + (uint32_t)j0, v);
           if (hi_only) {
 #pragma unroll
             for (int j = 0; j < 16; ++j) v[j] = mad_hi(v[j] + cbias, cm, rnd_hi) >> sh_hi;
@@ -491,21 +498,18 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
           }
           // residual port
           if (tma_res) {
-            // residual bytes of this chunk in shared memory: [row][128 channels], 16-byte pieces XOR (row & 7)
-            const uint8_t* rt = gen_base + (my_res - base) + slot * 4096 + h * 2048 + (cb & 15);
-            int off[8];
-#pragma unroll
-            for (int x = 0; x < 8; ++x) off[x] = ((cb >> 4) ^ x) << 4;
+            // residual bytes of this chunk in shared memory: [row][32 channels]
+            const uint8_t* rt = gen_base + (my_res - base) + (g & 1u) * 1024 + h * 512 + lane;
             if (rs_s >= 32) {
 #pragma unroll
               for (int j = 0; j < 16; ++j) {
-                const int xr = (int)*reinterpret_cast<const int8_t*>(rt + j * 128 + off[j & 7]);
+                const int xr = (int)*reinterpret_cast<const int8_t*>(rt + j * 32);
                 v[j] += mad_wide_hi(xr, rs_m, rs_c) >> (rs_s - 32);
               }
             } else {
 #pragma unroll
               for (int j = 0; j < 16; ++j) {
-                const int xr = (int)*reinterpret_cast<const int8_t*>(rt + j * 128 + off[j & 7]);
+                const int xr = (int)*reinterpret_cast<const int8_t*>(rt + j * 32);
                 v[j] += (int)(mad_wide(xr, rs_m, rs_c) >> rs_s);
               }
             }
@@ -543,12 +547,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
 #pragma unroll
           for (int k = 0; k < 4; ++k) w[k] = __byte_perm(w[k], o[k], sel2);
           if (tma_out) {
-            // word k belongs to slot row 16h + li + 4k
+            // word k belongs to slot row 16h + li + 4k: rows of 32 bytes, one bank per lane
 #pragma unroll
-            for (int k = 0; k < 4; k += 2) {
-              *reinterpret_cast<uint32_t*>(pe + 2048 * h + 512 * k) = w[k];
-              *reinterpret_cast<uint32_t*>(po + 2048 * h + 512 * (k + 1)) = w[k + 1];
-            }
+            for (int k = 0; k < 4; ++k) *reinterpret_cast<uint32_t*>(pe + 512 * h + 128 * k) = w[k];
           } else {
             // direct stores (grouped output rows): this lane's first word is row r0 + li, then + 4 per word
             int64_t row = r0 + li, ro = row, grem = 0;
@@ -571,49 +572,33 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
           }
         };
 
+        const bool c_any = tc.p0 + c_first < a.P;   // else the warp's box lies wholly past the last channel
         for (int ck = part; ck < nck; ck += kParts) {
-          uint8_t *pe = nullptr, *po = nullptr;
+          uint8_t* pe = nullptr;
           if (tma_out) {
-            if (nslots == 1 && lane == 0 && pend_prev >= 0) {
-              // a single slot: the store issued in the previous chunk must have read it before anyone goes on
-              tma_store_wait_read();
-              mbar_arrive(my_sfree + 8u * pend_prev);
-              pend_prev = -1;
+            const uint32_t sl = g & 1u;
+            // the store that used this slot two chunks ago must have read it; the residual bytes must be here
+            if (lane == 0) tma_store_wait_read1();
+            if (tma_res && c_any) {
+              if (ok) ok = mbar_wait(my_resf + 8u * sl, (rpar >> sl) & 1u, a.status);
+              if (ok) { rpar ^= 1u << sl; rpend &= ~(1u << sl); }
             }
-            // the slot's previous store must have read it; its residual bytes must have arrived
-            if (sround > 0 && ok) ok = mbar_wait(my_sfree + 8u * slot, (sround - 1u) & 1u, a.status);
-            if (tma_res && ok) ok = mbar_wait(my_resf + 8u * slot, sround & 1u, a.status);
-            // slot layout [row][128 channels]; 16-byte piece index XOR (row & 7) is the 128B swizzle of the
-            // store map.  A lane's words belong to slot rows li + 4k: (row & 7) alternates between two values,
-            // so two base addresses plus immediates address all of them.
-            const int cg = qd * 32 + (lane & ~3);
-            uint8_t* row0 = gen_base + (my_out - base) + slot * 4096 + li * 128 + (cg & 15);
-            pe = row0 + ((((cg >> 4) ^ li) & 7) << 4);
-            po = row0 + ((((cg >> 4) ^ (li + 4)) & 7) << 4);
+            __syncwarp();
+            // after the transposes a lane holds 4 consecutive channels (lane >> 2) of slot row li + 4k
+            pe = gen_base + (my_out - base) + sl * 1024 + li * 32 + (lane >> 2) * 4;
           }
-          half(ck, 0, pe, po);
-          half(ck, 1, pe, po);
+          int v[16];
+          tmem_ld16(t_row + (uint32_t)(32 * ck), v);
+          half(v, ck, 0, pe);
+          tmem_ld16(t_row + (uint32_t)(32 * ck + 16), v);
+          half(v, ck, 1, pe);
           if (tma_out) {
             fence_async_smem();
             __syncwarp();
-            if (lane == 0) {
-              // fourth arrival: every warp's bytes are in the slot and visible to the copy engine
-              if ((smem_add_acq_rel(my_scnt + 8u * slot, 1u) & 3u) == 3u) {
-                tma_store_4d(&tmO, my_out + 4096u * slot, tc.p0, tc.q0 + 32 * ck, 0, 0);
-                // ... and every warp is past its reads of the slot's residual bytes
-                if (tma_res && pf_t < t_end) pf_fetch(slot);
-                pend_cur = slot;
-              }
-              if (pend_prev >= 0) {
-                // the store issued one chunk ago has had a chunk's time to read its slot
-                tma_store_wait_read1_or_all(pend_cur >= 0);
-                mbar_arrive(my_sfree + 8u * pend_prev);
-              }
-              pend_prev = pend_cur;
-              pend_cur = -1;
-            }
-            pf_advance();
-            if (++slot == nslots) { slot = 0; ++sround; }
+            if (lane == 0 && c_any) tma_store_4d(&tmO, my_out + 1024u * (g & 1u), tc.p0 + c_first, tc.q0 + 32 * ck, 0, 0);
+            // every lane is past its reads of this slot's residual bytes: fetch those of two chunks on
+            if (tma_res) pf_fetch();
+            ++g;
           }
         }
       } else {
@@ -659,13 +644,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       if (lane == 0) mbar_arrive(acce0 + 8 * buf);
       if (et == 0) IVIT_TRACE(it, 5);
     }
-    if (tma_out && lane == 0) {
-      tma_store_wait_all();
-      if (pend_prev >= 0) mbar_arrive(my_sfree + 8u * pend_prev);
-    }
+    if (tma_out && lane == 0) tma_store_wait_all();
     // only after a timeout: residual bytes fetched for chunks that were never worked on may be in flight
-    if (tma_res && !ok && qd == 0 && lane == 0)
-      for (int sl = 0; sl < nslots; ++sl) mbar_wait(my_resf + 8u * sl, ((uint32_t)(sl < slot) + sround) & 1u, a.status);
+    if (tma_res && !ok && lane == 0)
+      for (uint32_t sl = 0; sl < 2; ++sl)
+        if ((rpend >> sl) & 1u) mbar_wait(my_resf + 8u * sl, (rpar >> sl) & 1u, a.status);
   }
   tc_fence_before();
   __syncthreads();
@@ -687,7 +670,7 @@ int pow2_at_least(int v) {
 }
 
 constexpr size_t kSmemBudget = 227 * 1024;
-constexpr size_t kSmemFixed = 1024 + 8 * (2 * kMaxStages + 54) + 32;
+constexpr size_t kSmemFixed = 1024 + 8 * (2 * kMaxStages + 5 + 2 * kEpiWarps) + 32;
 
 bool g_attr_set = false;
 
@@ -764,16 +747,16 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
   CUtensorMap tmO = tmP;
   if (dense && e.out_dtype == IVIT_I8 && e.group_rows <= 0 && !(reinterpret_cast<uintptr_t>(e.out) & 15) && e.ldo % 16 == 0) {
     int opos[3];
-    a.tma_out = make_tensor_map(ctx, &tmO, reinterpret_cast<const int8_t*>(e.out), g.N, g.M, 1, 1, e.ldo, 0, 0, BM, 32,
-                         CU_TENSOR_MAP_SWIZZLE_128B, opos) ? 1 : 0;
+    a.tma_out = make_tensor_map(ctx, &tmO, reinterpret_cast<const int8_t*>(e.out), g.N, g.M, 1, 1, e.ldo, 0, 0, 32, 32,
+                         CU_TENSOR_MAP_SWIZZLE_NONE, opos) ? 1 : 0;
   }
   CUtensorMap tmR = tmP;
   if (a.tma_out && e.res && e.res_rows >= g.M && !(reinterpret_cast<uintptr_t>(e.res) & 15) && e.ldres % 16 == 0) {
     int rpos[3];
-    a.tma_res = make_tensor_map(ctx, &tmR, e.res, g.N, g.M, 1, 1, e.ldres, 0, 0, BM, 32, CU_TENSOR_MAP_SWIZZLE_128B,
+    a.tma_res = make_tensor_map(ctx, &tmR, e.res, g.N, g.M, 1, 1, e.ldres, 0, 0, 32, 32, CU_TENSOR_MAP_SWIZZLE_NONE,
                                 rpos) ? 1 : 0;
   }
-  const size_t out_stage = (a.tma_out ? (size_t)a.BN * 128 : 0) + (a.tma_res ? (size_t)a.BN * 128 : 0);
+  const size_t out_stage = (a.tma_out ? (size_t)kEpiWarps * 2048 : 0) + (a.tma_res ? (size_t)kEpiWarps * 2048 : 0);
   // short K: keep the activation tile resident if that still leaves four weight stages
   const size_t kblocks = (size_t)((g.K + BK - 1) / BK);
   const size_t qres_bytes = kblocks * a.q_stage_bytes;

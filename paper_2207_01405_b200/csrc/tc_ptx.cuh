@@ -79,13 +79,14 @@ __device__ __forceinline__ void tma_store_wait_read1_or_all(bool keep_last) {
   if (keep_last) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
   else asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
 }
-// Adds to a 32-bit word in shared memory; releases this thread's earlier writes and acquires those of the
-// threads whose additions it observes.  Returns the old value.
-__device__ __forceinline__ uint32_t smem_add_acq_rel(uint32_t addr, uint32_t v) {
+// Adds to a 32-bit word in shared memory and returns the old value; releases this thread's earlier writes.
+// A thread that acts on the additions of others it has observed follows up with fence_acquire_cta().
+__device__ __forceinline__ uint32_t smem_add_release(uint32_t addr, uint32_t v) {
   uint32_t old;
-  asm volatile("atom.acq_rel.cta.shared::cta.add.u32 %0, [%1], %2;" : "=r"(old) : "r"(addr), "r"(v) : "memory");
+  asm volatile("atom.release.cta.shared::cta.add.u32 %0, [%1], %2;" : "=r"(old) : "r"(addr), "r"(v) : "memory");
   return old;
 }
+__device__ __forceinline__ void fence_acquire_cta() { asm volatile("fence.acq_rel.cta;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
@@ -156,15 +157,24 @@ __device__ __forceinline__ void tmem_ld_wait(int (&v)[32]) {
                  "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31])
                :: "memory");
 }
-// The same for 16 consecutive columns (load and wait in one).
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int (&v)[16]) {
+// The same for 16 consecutive columns.
+__device__ __forceinline__ void tmem_ld16_issue(uint32_t taddr, int (&v)[16]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x16.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n\t"
-      "tcgen05.wait::ld.sync.aligned;"
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
       : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
         "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
       : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait16(int (&v)[16]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
+                 "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15])
+               :: "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int (&v)[16]) {
+  tmem_ld16_issue(taddr, v);
+  tmem_ld_wait16(v);
 }
 // The same for 8 consecutive columns.
 __device__ __forceinline__ void tmem_ld8_issue(uint32_t taddr, int (&v)[8]) {
