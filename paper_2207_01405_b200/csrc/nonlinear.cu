@@ -117,21 +117,22 @@ __global__ void __launch_bounds__(256) layernorm_i8_kernel(const int8_t* __restr
 // per-row scalars (mean, integer square root, reciprocal) are then computed by ROWS different lanes
 // at once instead of redundantly by all 32, and the per-channel constants of the lane's channels
 // are loaded once for all ROWS rows: v = ((x*F - mu*F) * m + 2^(s-1)) >> s + beta.
+// mean_magic = floor(2^32 / (2C)) + 1 turns the mean's division into a multiplication (exact for the
+// numerators of int8 rows, which stay below 2^18).
 template <int WPL, int ROWS>
-__global__ void __launch_bounds__(256) layernorm_i8_batched_kernel(const int8_t* __restrict__ in, int64_t ldin,
-                                                                   ScaleDev gs, const int32_t* __restrict__ beta,
-                                                                   int M_ln, int8_t* __restrict__ out, int64_t ldout,
-                                                                   int64_t rows, int C) {
+__global__ void __launch_bounds__(128, 6) layernorm_i8_batched_kernel(const int8_t* __restrict__ in, int64_t ldin,
+                                                                      ScaleDev gs, const int32_t* __restrict__ beta,
+                                                                      int M_ln, int8_t* __restrict__ out, int64_t ldout,
+                                                                      int64_t rows, int C, unsigned mean_magic) {
   pdl_trigger();
   pdl_wait();
   const int lane = threadIdx.x & 31;
   const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
   const int nwords = C >> 2;
-  // constants of this lane's channels (word i of the lane covers channels 4*(lane+32i) .. +3):
-  // v = (yF * m + 2^(s-1)) >> s + beta, the shift split into min(s,32) and s - 32
+  // constants of this lane's channels (word i of the lane covers channels 4*(lane+32i) .. +3)
   int pm[WPL][4], ps[WPL][4], pb[WPL][4];
-  bool all_hi = true;   // every shift >= 32: the value is the high product word shifted by s - 32
+  bool all_hi = true;   // every shift >= 33: only the high word of the product is needed (see below)
 #pragma unroll
   for (int i = 0; i < WPL; ++i) {
     const int idx = lane + 32 * i;
@@ -139,12 +140,19 @@ __global__ void __launch_bounds__(256) layernorm_i8_batched_kernel(const int8_t*
     for (int b = 0; b < 4; ++b) {
       const int c = idx * 4 + b;
       pm[i][b] = idx < nwords ? gs.m(c) : 1;
-      ps[i][b] = idx < nwords ? gs.s(c) : 32;
+      ps[i][b] = idx < nwords ? gs.s(c) : 40;
       pb[i][b] = (idx < nwords && beta) ? __ldg(beta + c) : 0;
-      all_hi = all_hi && ps[i][b] >= 32;
+      all_hi = all_hi && ps[i][b] >= 33;
     }
   }
   all_hi = __all_sync(0xffffffffu, all_hi);
+  if (all_hi) {
+    // keep s - 32 instead of s
+#pragma unroll
+    for (int i = 0; i < WPL; ++i)
+#pragma unroll
+      for (int b = 0; b < 4; ++b) ps[i][b] -= 32;
+  }
   for (int64_t r0 = warp * ROWS; r0 < rows; r0 += nwarps * ROWS) {
     int w[ROWS][WPL];
     int my_s1 = 0, my_s2 = 0;
@@ -152,22 +160,29 @@ __global__ void __launch_bounds__(256) layernorm_i8_batched_kernel(const int8_t*
     for (int r = 0; r < ROWS; ++r) {
       const bool ok = r0 + r < rows;
       const int* src = reinterpret_cast<const int*>(in + (r0 + r) * ldin);
-      int s1 = 0, s2 = 0;
 #pragma unroll
       for (int i = 0; i < WPL; ++i) {
         const int idx = lane + 32 * i;
         w[r][i] = (ok && idx < nwords) ? __ldg(src + idx) : 0;
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < ROWS; ++r) {
+      int s1 = 0, s2 = 0;
+#pragma unroll
+      for (int i = 0; i < WPL; ++i) {
         s1 = __dp4a(w[r][i], 0x01010101, s1);
         s2 = __dp4a(w[r][i], w[r][i], s2);
       }
-      s1 = __reduce_add_sync(0xffffffffu, s1);   // one redux.sync per sum instead of a shuffle tree
+      s1 = __reduce_add_sync(0xffffffffu, s1);
       s2 = __reduce_add_sync(0xffffffffu, s2);
       if (lane == r) { my_s1 = s1; my_s2 = s2; }
     }
-    // lane r (< ROWS) holds the sums of row r0 + r: mean (round half up), sum of squared
-    // deviations = sum x^2 - 2 mu sum x + C mu^2, integer square root, reciprocal
-    const int mu = floordiv_pos(2 * my_s1 + C, 2 * C);
-    const long long V = (long long)my_s2 - 2ll * mu * my_s1 + (long long)C * mu * mu;
+    // lane r (< ROWS) holds the sums of row r0 + r: mean (round half up) = floor((2 S1 + C) / 2C), taken on the
+    // numerator shifted by 256 C to make it positive; sum of squared deviations = sum x^2 - 2 mu sum x + C mu^2
+    // (every term below 2^25 for int8 rows of up to 512 channels); integer square root; reciprocal
+    const int mu = (int)__umulhi((unsigned)(2 * my_s1 + 257 * C), mean_magic) - 128;
+    const int V = my_s2 - 2 * mu * my_s1 + C * mu * mu;
     const unsigned sd = isqrt_u32((unsigned)V);
     const int F = sd == 0 ? 0 : (int)((1u << M_ln) / sd);
     const int muF = (int)((unsigned)mu * (unsigned)F);
@@ -184,12 +199,15 @@ __global__ void __launch_bounds__(256) layernorm_i8_batched_kernel(const int8_t*
             int v[4];
 #pragma unroll
             for (int b = 0; b < 4; ++b) {
-              const int x = (int)(int8_t)(w[r][i] >> (8 * b));
+              // byte b, sign-extended by one byte permute
+              int x;
+              asm("prmt.b32 %0, %1, %1, %2;" : "=r"(x) : "r"(w[r][i]), "r"(0x8880 + 0x1111 * b));
               // (x - mu) * F, formed modulo 2^32 (the difference always fits: |y F| <= 2^(M_ln+1))
               const int yF = (int)((unsigned)x * (unsigned)Fr - (unsigned)muFr);
               if (all_hi) {
-                const long long t = (long long)yF * pm[i][b] + (1ll << (ps[i][b] - 1));
-                v[b] = ((int)(t >> 32) >> (ps[i][b] - 32)) + pb[i][b];
+                // s >= 33: the rounding constant 2^(s-1) is a multiple of 2^32, so
+                // (yF m + 2^(s-1)) >> s = (hi32(yF m) + 2^(s-33)) >> (s - 32)
+                v[b] = ((__mulhi(yF, pm[i][b]) + (1 << (ps[i][b] - 1))) >> ps[i][b]) + pb[i][b];
               } else {
                 v[b] = rq(yF, pm[i][b], ps[i][b]) + pb[i][b];
               }
@@ -298,15 +316,16 @@ int launch_layernorm(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, 
   const int wpl = (int)((C / 4 + 31) / 32);
   if (wpl <= 4) {
     // batched kernel: 4 rows per warp amortise the per-row scalar work and the per-channel constants;
-    // 128-thread blocks keep enough warps in flight on every SM
+    // 128-thread blocks, six of them resident per SM
     const int rpw = 4, tb = 128;
     const int64_t warps = (rows + rpw - 1) / rpw;
     const int64_t wantb = (warps + tb / 32 - 1) / (tb / 32);
-    const int gridb = (int)(wantb < (int64_t)ctx->sm_count * 16 ? wantb : (int64_t)ctx->sm_count * 16);
-    if (wpl <= 1) launch_k(layernorm_i8_batched_kernel<1, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-    else if (wpl <= 2) launch_k(layernorm_i8_batched_kernel<2, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-    else if (wpl <= 3) launch_k(layernorm_i8_batched_kernel<3, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-    else launch_k(layernorm_i8_batched_kernel<4, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+    const int gridb = (int)(wantb < (int64_t)ctx->sm_count * 12 ? wantb : (int64_t)ctx->sm_count * 12);
+    const unsigned magic = (unsigned)(0x100000000ull / (unsigned long long)(2 * C)) + 1u;
+    if (wpl <= 1) launch_k(layernorm_i8_batched_kernel<1, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic);
+    else if (wpl <= 2) launch_k(layernorm_i8_batched_kernel<2, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic);
+    else if (wpl <= 3) launch_k(layernorm_i8_batched_kernel<3, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic);
+    else launch_k(layernorm_i8_batched_kernel<4, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic);
     return ls.done();
   }
   if (wpl <= 6) launch_k(layernorm_i8_kernel<6>, dim3(grid), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
