@@ -36,6 +36,8 @@ struct AttnArgs {
   int T, d, heads, Npad;            // Npad = T rounded up to 32 (score columns and P.V contraction length)
   int64_t D;                        // heads * d
   int tiles_m;                      // ceil(T / 128)
+  int bh;                           // images (or windows) x heads
+  int items;                        // bh * tiles_m
   int tmem_cols;
   int qk_m, qk_s, pv_m, pv_s;
   ivit_exp_params smax;
@@ -43,41 +45,51 @@ struct AttnArgs {
   int64_t bias_batches;
   int8_t* O;                        // [B*T, D]
   int q_pos[3], k_pos[3], v_pos[3];
+  unsigned* sched;                  // [0] next work item, [1] CTAs that have finished; both zero between launches
   int* status;
 };
 
-__global__ void __launch_bounds__(kAttnThreads) attention_kernel(const __grid_constant__ CUtensorMap tmQ,
+constexpr uint32_t kItemWaitRounds = 16;   // the item barrier outlasts every bounded wait of the control thread
+
+// Persistent CTAs (two per SM) draw work items = (image or window, head, 128-row tile) from a counter, the
+// full 128-row tiles first.  One control thread issues the TMA loads and the MMAs; the loads of the next item
+// are issued as soon as the MMAs that read the shared-memory operands of the current one have completed, so
+// they overlap the Shiftmax passes.  Barriers are used once per item: the parity of a wait is the item count.
+__global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid_constant__ CUtensorMap tmQ,
                                                                  const __grid_constant__ CUtensorMap tmK,
                                                                  const __grid_constant__ CUtensorMap tmV, AttnArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
-  // [Q 128x128B][K Npad x 128B][V Npad x d][P 128 x 128B x kblocks][exp table][barriers]
+  // [Q 128x128B][K Npad x 128B][V Npad x d][P 128 x 128B x kblocks][exp table][row partials][item ring][barriers]
   const uint32_t q_off = 0, k_off = 128 * 128, v_off = k_off + a.Npad * 128;
   const uint32_t p_off = (v_off + a.Npad * a.d + 1023u) & ~1023u;
   const int p_kblocks = (a.Npad + 127) / 128;
   const uint32_t tab_off = p_off + p_kblocks * 128 * 128;
   const uint32_t part_off = tab_off + 1024;            // [2 halves][128 rows] partial max, then partial sum
-  const uint32_t bar_off = part_off + 2 * 128 * 4 * 2;
+  const uint32_t item_off = part_off + 2 * 128 * 4 * 2;   // [2] work item of even / odd iterations (-1: no more work)
+  const uint32_t bar_off = item_off + 16;
   unsigned* tab = reinterpret_cast<unsigned*>(gen + tab_off);
-  const uint32_t bar_load = base + bar_off, bar_s = bar_load + 8, bar_p = bar_load + 16, bar_o = bar_load + 24;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + bar_off + 32);
+  volatile int* item_ring = reinterpret_cast<volatile int*>(gen + item_off);
+  // Q and K landed | V landed | scores ready | probabilities written | output ready | output read | item published
+  const uint32_t bar_qk = base + bar_off, bar_v = bar_qk + 8, bar_s = bar_qk + 16, bar_p = bar_qk + 24,
+                 bar_o = bar_qk + 32, bar_e = bar_qk + 40, bar_item = bar_qk + 48;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen + bar_off + 64);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tile = blockIdx.x % a.tiles_m;
-  const int bh = blockIdx.x / a.tiles_m;
-  const int h = bh % a.heads, b = bh / a.heads;
-  const int m0 = tile * 128;
 
   if (threadIdx.x == 0) {
     ATRACE(0);
     prefetch_tmap(&tmQ);
     prefetch_tmap(&tmK);
     prefetch_tmap(&tmV);
-    mbar_init(bar_load, 1);
+    mbar_init(bar_qk, 1);
+    mbar_init(bar_v, 1);
     mbar_init(bar_s, 1);
     mbar_init(bar_p, 8);
     mbar_init(bar_o, 1);
+    mbar_init(bar_e, 8);
+    mbar_init(bar_item, 1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
@@ -89,45 +101,91 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const __grid_co
   pdl_trigger();
   pdl_wait();   // the QKV tensor comes from the previous kernel
 
+  // item -> (tile, image/window * heads + head): all first tiles before all second tiles
   if (warp == 0) {
     if (lane == 0) {
       ATRACE(1);
-      // ---- loads: Q tile, all keys, all values of this (image, head) ----
-      mbar_expect_tx(bar_load, 128 * 128 + a.Npad * 128 + a.Npad * a.d);
-      int c[4];
-      c[0] = 0; c[a.q_pos[0]] = m0; c[a.q_pos[1]] = h; c[a.q_pos[2]] = b;
-      tma_load_4d(base + q_off, &tmQ, bar_load, c[0], c[1], c[2], c[3]);
-      c[0] = 0; c[a.k_pos[0]] = 0; c[a.k_pos[1]] = h; c[a.k_pos[2]] = b;
-      tma_load_4d(base + k_off, &tmK, bar_load, c[0], c[1], c[2], c[3]);
-      c[0] = 0; c[a.v_pos[0]] = 0; c[a.v_pos[1]] = h; c[a.v_pos[2]] = b;
-      tma_load_4d(base + v_off, &tmV, bar_load, c[0], c[1], c[2], c[3]);
-      bool ok = mbar_wait(bar_load, 0, a.status);
-      ATRACE(2);
-      if (ok) {
+      auto load_qk = [&](int item) {
+        const int tile = item / a.bh, bhid = item - tile * a.bh;
+        const int h = bhid % a.heads, b = bhid / a.heads;
+        mbar_expect_tx(bar_qk, 128 * 128 + a.Npad * 128);
+        int c[4];
+        c[0] = 0; c[a.q_pos[0]] = tile * 128; c[a.q_pos[1]] = h; c[a.q_pos[2]] = b;
+        tma_load_4d(base + q_off, &tmQ, bar_qk, c[0], c[1], c[2], c[3]);
+        c[0] = 0; c[a.k_pos[0]] = 0; c[a.k_pos[1]] = h; c[a.k_pos[2]] = b;
+        tma_load_4d(base + k_off, &tmK, bar_qk, c[0], c[1], c[2], c[3]);
+      };
+      auto load_v = [&](int item) {
+        const int tile = item / a.bh, bhid = item - tile * a.bh;
+        const int h = bhid % a.heads, b = bhid / a.heads;
+        mbar_expect_tx(bar_v, a.Npad * a.d);
+        int c[4];
+        c[0] = 0; c[a.v_pos[0]] = 0; c[a.v_pos[1]] = h; c[a.v_pos[2]] = b;
+        tma_load_4d(base + v_off, &tmV, bar_v, c[0], c[1], c[2], c[3]);
+      };
+      auto draw = [&]() {
+        const unsigned t = atomicAdd(a.sched, 1u);
+        return t < (unsigned)a.items ? (int)t : -1;
+      };
+      auto publish = [&](uint32_t n, int item) {
+        item_ring[n & 1u] = item;
+        mbar_arrive(bar_item);   // release: the item is visible to whoever sees this phase complete
+      };
+      // S = Q K^T: M = 128, N = Npad, both operands K-major rows of 128 bytes.  O = P V: V as stored (MN-major).
+      const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(a.Npad >> 3) << 17) | (8u << 24);
+      const uint32_t idesc2 = (2u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(a.d >> 3) << 17) | (8u << 24);
+      const uint32_t v_layout = a.d == 128 ? 2u : (a.d == 64 ? 4u : 6u);
+      const int ks = (a.d + UK - 1) / UK, ks2 = a.Npad / UK;
+
+      int item = draw();
+      bool qk_flying = false, v_flying = false;   // loads issued and not yet waited for (their barrier phase = item count)
+      if (item >= 0) { load_qk(item); load_v(item); qk_flying = v_flying = true; }
+      bool ok = true;
+      uint32_t n = 0, qk_par = 0, v_par = 0;
+      for (; item >= 0; ++n) {
+        const uint32_t par = n & 1u;
+        publish(n, item);
+        ok = mbar_wait(bar_qk, par, a.status);
+        qk_flying = !ok;
+        // the output of the previous item must have left tensor memory
+        if (ok && n > 0) ok = mbar_wait(bar_e, par ^ 1u, a.status);
+        if (!ok) break;
+        ATRACE(2);
         tc_fence_after();
-        // ---- S = Q K^T: M = 128, N = Npad, both operands K-major rows of 128 bytes ----
-        const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(a.Npad >> 3) << 17) | (8u << 24);
-        const int ks = (a.d + UK - 1) / UK;
         for (int k = 0; k < ks; ++k)
           umma_i8(tmem, smem_desc(base + q_off + k * UK, 16, 1024, 2), smem_desc(base + k_off + k * UK, 16, 1024, 2),
                   idesc, k != 0);
         umma_commit(bar_s);
-        // ---- O = P V once the probabilities are in shared memory ----
-        ok = mbar_wait(bar_p, 0, a.status);
+        const int next = draw();
+        // Q and K may be overwritten once the score MMAs have read them
+        ok = mbar_wait(bar_s, par, a.status);
+        if (!ok) break;
+        if (next >= 0) { load_qk(next); qk_flying = true; qk_par = par ^ 1u; }
+        // O = P V once the probabilities are in shared memory and V has landed
+        ok = mbar_wait(bar_p, par, a.status);
+        if (ok) { ok = mbar_wait(bar_v, par, a.status); v_flying = !ok; }
+        if (!ok) break;
         ATRACE(7);
-      }
-      if (ok) {
         tc_fence_after();
-        const uint32_t idesc2 = (2u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(a.d >> 3) << 17) | (8u << 24);
-        const uint32_t v_layout = a.d == 128 ? 2u : (a.d == 64 ? 4u : 6u);
-        const int ks2 = a.Npad / UK;
         for (int k = 0; k < ks2; ++k) {
           const uint32_t pa = base + p_off + (k >> 2) * (128 * 128) + (k & 3) * UK;
           umma_i8(tmem, smem_desc(pa, 16, 1024, 2), smem_desc(base + v_off + k * UK * a.d, 16, 8 * a.d, v_layout),
                   idesc2, k != 0);
         }
         umma_commit(bar_o);
+        // V may be overwritten once these MMAs have read it
+        ok = mbar_wait(bar_o, par, a.status);
+        if (!ok) break;
+        if (next >= 0) { load_v(next); v_flying = true; v_par = par ^ 1u; }
+        item = next;
       }
+      // end of work (or a wait that timed out): tell the other warps; nothing may be in flight at exit
+#ifdef IVIT_ATTN_TRACE
+      if (blockIdx.x < 64) g_attn_trace[blockIdx.x][10] = n;
+#endif
+      publish(ok ? n : n + 1, -1);
+      if (qk_flying) mbar_wait(bar_qk, qk_par, a.status);
+      if (v_flying) mbar_wait(bar_v, v_par, a.status);
     }
   } else {
     // ---- softmax / epilogue threads: TMEM lane quarter = warp % 4; the two warps of a quarter
@@ -137,153 +195,186 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(const __grid_co
     const int qd = warp & 3;
     const int half = (warp - 1) >> 2;
     const int trow = qd * 32 + lane;              // row inside the tile
-    const int r = m0 + trow;                      // token (row) inside this image / window
-    const bool row_ok = r < a.T;
-    const bool warp_ok = m0 + qd * 32 < a.T;      // warps whose 32 rows all lie past T only keep the barriers
     const uint32_t t_row = tmem + ((uint32_t)(qd * 32) << 16);
     const int nch = a.Npad / 32;
-    const int64_t batch = (int64_t)b * a.heads + h;
-    const int32_t* brow = a.bias ? a.bias + ((batch % a.bias_batches) * a.T + (row_ok ? r : 0)) * (int64_t)a.T : nullptr;
+    const bool qk_hi = a.qk_s >= 33;              // rounding constant and shift both past the low product word
     const long long qk_c = 1ll << (a.qk_s - 1);
+    const int qk_rnd = qk_hi ? 1 << (a.qk_s - 33) : 0, qk_sh = a.qk_s - 32;
     int* part_max = reinterpret_cast<int*>(gen + part_off);
     unsigned* part_sum = reinterpret_cast<unsigned*>(gen + part_off + 2 * 128 * 4);
+    asm volatile("bar.sync 1, 256;" ::: "memory");   // the table is complete
 
-    uint32_t xs[32];   // int8 scores of this thread's chunks, packed four per word
-    int mx = -128;
-    const bool got_s = mbar_wait(bar_s, 0, a.status);
-    if (got_s) tc_fence_after();
-    if (st == 0) ATRACE(3);
-    if (got_s && warp_ok) {
-      // pass A: requantise the scores to int8 (Sec. 3.2), running maximum
+    bool alive = true;   // false after a wait that timed out: no more waits, no more work, only the barriers
+    for (uint32_t n = 0;; ++n) {
+      const uint32_t par = n & 1u;
+      // All 256 threads leave the loop together: the decision is taken on a value that every thread reads
+      // after the same barrier phase.
+      bool got_item = false;
+      if (alive) {
+        for (uint32_t w = 0; w < kItemWaitRounds && !got_item; ++w) got_item = mbar_wait(bar_item, par, a.status);
+      }
+      const int item = got_item ? item_ring[par] : -1;
+      if (item < 0) break;
+      const int tile = item / a.bh, bhid = item - tile * a.bh;
+      const int h = bhid % a.heads, b = bhid / a.heads;
+      const int m0 = tile * 128;
+      const int r = m0 + trow;                      // token (row) inside this image / window
+      const bool row_ok = r < a.T;
+      const bool warp_ok = m0 + qd * 32 < a.T;      // warps whose 32 rows all lie past T only keep the barriers
+      const int32_t* brow = a.bias ? a.bias + (((int64_t)bhid % a.bias_batches) * a.T + (row_ok ? r : 0)) * (int64_t)a.T : nullptr;
+
+      uint32_t xs[32];   // int8 scores of this thread's chunks, packed four per word
+      int mx = -128;
+      bool got_s = mbar_wait(bar_s, par, a.status);
+      alive = alive && got_s;
+      if (got_s) tc_fence_after();
+      if (st == 0) ATRACE(3);
+      if (got_s && warp_ok) {
+        // pass A: requantise the scores to int8 (Sec. 3.2), running maximum
 #pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
-        const int c = 2 * cc + half;
-        if (c < nch) {
+        for (int cc = 0; cc < 4; ++cc) {
+          const int c = 2 * cc + half;
+          if (c < nch) {
+            int v[32];
+            tmem_ld32(t_row + c * 32, v);
+            if (brow) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (c * 32 + j < a.T) v[j] += __ldg(brow + c * 32 + j);
+            }
+            if (qk_hi) {          // the usual case: high product word plus 2^(s-33), shifted by s - 32
+#pragma unroll
+              for (int j = 0; j < 32; ++j) v[j] = mad_hi(v[j], a.qk_m, qk_rnd) >> qk_sh;
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) v[j] = (int)(((long long)v[j] * a.qk_m + qk_c) >> a.qk_s);
+            }
+            // columns past T (only in the last chunk) never win the maximum and look up a valid table entry
+            if (c == nch - 1) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (c * 32 + j >= a.T) v[j] = -128;
+            }
+            // running maximum on the unsaturated values (saturation is monotone: it is applied to the result)
+            int m = v[0];
+#pragma unroll
+            for (int j = 1; j < 32; j += 2) m = max(m, max(v[j], v[(j + 1) & 31]));
+            mx = max(mx, m);
+            // scores are kept as biased bytes (x + 128, i.e. x ^ 0x80) so that pass B can index with them
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+              xs[cc * 8 + k] = pack_sat8(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]) ^ 0x80808080u;
+          }
+        }
+        mx = max(-128, min(127, mx));
+        part_max[half * 128 + trow] = mx;
+      }
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (st == 0) ATRACE(4);
+      unsigned sum = 0;
+      if (got_s && warp_ok) {
+        mx = max(part_max[trow], part_max[128 + trow]);
+        // pass B: ShiftExp(I - I_max) by table, row sum, exponentials back into tensor memory
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          const int c = 2 * cc + half;
+          if (c < nch) {
+            int ev[32];
+            // entry (I_max - I) of the table = word at tab + 4*(I_max + 128) - 4*(I + 128)
+            const uint8_t* tmx = reinterpret_cast<const uint8_t*>(tab) + 4 * (mx + 128);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+              const uint32_t w = xs[cc * 8 + k];
+#pragma unroll
+              for (int bb = 0; bb < 4; ++bb)
+                ev[4 * k + bb] = (int)*reinterpret_cast<const unsigned*>(tmx - 4 * (int)__byte_perm(w, 0, 0x4440 + bb));
+            }
+            if (c == nch - 1) {   // columns past T contribute nothing
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (c * 32 + j >= a.T) ev[j] = 0;
+            }
+#pragma unroll
+            for (int j = 0; j < 32; ++j) sum += (unsigned)ev[j];
+            tmem_st32(t_row + c * 32, ev);
+          }
+        }
+        tmem_st_wait();
+        part_sum[half * 128 + trow] = sum;
+      }
+      asm volatile("bar.sync 1, 256;" ::: "memory");
+      if (st == 0) ATRACE(5);
+      if (got_s && warp_ok) {
+        sum = part_sum[trow] + part_sum[128 + trow];
+        // pass C: Eq. (IntDiv) with M = 45, k_out = 8: (floor(2^45 / sum) * e) >> 38 = umulhi(factor, e) >> 6
+        const unsigned factor = (unsigned)((1ull << 45) / (unsigned long long)(sum ? sum : 1u));
+#pragma unroll
+        for (int cc = 0; cc < 4; ++cc) {
+          const int c = 2 * cc + half;
+          if (c < nch) {
+            int ev[32];
+            tmem_ld32(t_row + c * 32, ev);
+            uint32_t w[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k)   // values are <= 128: the saturating pack clamps the one possible 128 to 127
+              w[k] = pack_sat8((int)(__umulhi(factor, (unsigned)ev[4 * k]) >> 6), (int)(__umulhi(factor, (unsigned)ev[4 * k + 1]) >> 6),
+                               (int)(__umulhi(factor, (unsigned)ev[4 * k + 2]) >> 6), (int)(__umulhi(factor, (unsigned)ev[4 * k + 3]) >> 6));
+            // A operand of P V: row = tile row, k-block = 128 columns, 16-byte chunks XOR (row & 7)
+            uint8_t* prow = gen + p_off + (c >> 2) * (128 * 128) + trow * 128;
+            const int ch0 = (c & 3) * 2;
+            *reinterpret_cast<uint4*>(prow + (((ch0) ^ (trow & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4*>(prow + (((ch0 + 1) ^ (trow & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+          }
+        }
+        fence_async_smem();
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_p);
+      if (st == 0) ATRACE(6);
+      // ---- output: O = sat8(rq(P V; pv_scale)), heads concatenated along the feature dimension ----
+      const bool got_o = alive && mbar_wait(bar_o, par, a.status);
+      alive = alive && got_o;
+      if (got_o) {
+        tc_fence_after();
+        if (st == 0) ATRACE(8);
+        const long long pv_c = 1ll << (a.pv_s - 1);
+        int8_t* orow = a.O + ((int64_t)b * a.T + r) * a.D + (int64_t)h * a.d;
+        for (int c = half; c < a.d / 32; c += 2) {
+          if (!warp_ok) break;
           int v[32];
           tmem_ld32(t_row + c * 32, v);
-          if (brow) {
+          if (row_ok) {
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (c * 32 + j < a.T) v[j] += __ldg(brow + c * 32 + j);
+            for (int j = 0; j < 32; ++j) v[j] = (int)(((long long)v[j] * a.pv_m + pv_c) >> a.pv_s);
+            int4 w0, w1;
+            w0.x = (int)pack_sat8(v[0], v[1], v[2], v[3]);     w0.y = (int)pack_sat8(v[4], v[5], v[6], v[7]);
+            w0.z = (int)pack_sat8(v[8], v[9], v[10], v[11]);   w0.w = (int)pack_sat8(v[12], v[13], v[14], v[15]);
+            w1.x = (int)pack_sat8(v[16], v[17], v[18], v[19]); w1.y = (int)pack_sat8(v[20], v[21], v[22], v[23]);
+            w1.z = (int)pack_sat8(v[24], v[25], v[26], v[27]); w1.w = (int)pack_sat8(v[28], v[29], v[30], v[31]);
+            reinterpret_cast<int4*>(orow + c * 32)[0] = w0;
+            reinterpret_cast<int4*>(orow + c * 32)[1] = w1;
           }
-          if (a.qk_s >= 32) {   // the usual case: high word of the 64-bit multiply-add, shifted by s - 32
-            const int sh = a.qk_s - 32;
-#pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = (int)(((long long)v[j] * a.qk_m + qk_c) >> 32) >> sh;
-          } else {
-#pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = (int)(((long long)v[j] * a.qk_m + qk_c) >> a.qk_s);
-          }
-          // columns past T (only in the last chunk) never win the maximum and look up a valid table entry
-          if (c == nch - 1) {
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (c * 32 + j >= a.T) v[j] = -128;
-          }
-          // running maximum on the unsaturated values (saturation is monotone: it is applied to the result)
-          int m = v[0];
-#pragma unroll
-          for (int j = 1; j < 32; j += 2) m = max(m, max(v[j], v[(j + 1) & 31]));
-          mx = max(mx, m);
-          // scores are kept as biased bytes (x + 128, i.e. x ^ 0x80) so that pass B can index with them
-#pragma unroll
-          for (int k = 0; k < 8; ++k)
-            xs[cc * 8 + k] = pack_sat8(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]) ^ 0x80808080u;
         }
       }
-      mx = max(-128, min(127, mx));
-      part_max[half * 128 + trow] = mx;
-    }
-    asm volatile("bar.sync 1, 256;" ::: "memory");
-    if (st == 0) ATRACE(4);
-    unsigned sum = 0;
-    if (got_s && warp_ok) {
-      mx = max(part_max[trow], part_max[128 + trow]);
-      // pass B: ShiftExp(I - I_max) by table, row sum, exponentials back into tensor memory
-#pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
-        const int c = 2 * cc + half;
-        if (c < nch) {
-          int ev[32];
-          // entry (I_max - I) of the table = word at tab + 4*(I_max + 128) - 4*(I + 128)
-          const uint8_t* tmx = reinterpret_cast<const uint8_t*>(tab) + 4 * (mx + 128);
-#pragma unroll
-          for (int k = 0; k < 8; ++k) {
-            const uint32_t w = xs[cc * 8 + k];
-#pragma unroll
-            for (int b = 0; b < 4; ++b)
-              ev[4 * k + b] = (int)*reinterpret_cast<const unsigned*>(tmx - 4 * (int)__byte_perm(w, 0, 0x4440 + b));
-          }
-          if (c == nch - 1) {   // columns past T contribute nothing
-#pragma unroll
-            for (int j = 0; j < 32; ++j)
-              if (c * 32 + j >= a.T) ev[j] = 0;
-          }
-#pragma unroll
-          for (int j = 0; j < 32; ++j) sum += (unsigned)ev[j];
-          tmem_st32(t_row + c * 32, ev);
-        }
-      }
-      tmem_st_wait();
-      part_sum[half * 128 + trow] = sum;
-    }
-    asm volatile("bar.sync 1, 256;" ::: "memory");
-    if (st == 0) ATRACE(5);
-    if (got_s && warp_ok) {
-      sum = part_sum[trow] + part_sum[128 + trow];
-      // pass C: Eq. (IntDiv) with M = 45, k_out = 8: (floor(2^45 / sum) * e) >> 38 = umulhi(factor, e) >> 6
-      const unsigned factor = (unsigned)((1ull << 45) / (unsigned long long)(sum ? sum : 1u));
-#pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
-        const int c = 2 * cc + half;
-        if (c < nch) {
-          int ev[32];
-          tmem_ld32(t_row + c * 32, ev);
-          uint32_t w[8];
-#pragma unroll
-          for (int k = 0; k < 8; ++k)   // values are <= 128: the saturating pack clamps the one possible 128 to 127
-            w[k] = pack_sat8((int)(__umulhi(factor, (unsigned)ev[4 * k]) >> 6), (int)(__umulhi(factor, (unsigned)ev[4 * k + 1]) >> 6),
-                             (int)(__umulhi(factor, (unsigned)ev[4 * k + 2]) >> 6), (int)(__umulhi(factor, (unsigned)ev[4 * k + 3]) >> 6));
-          // A operand of P V: row = tile row, k-block = 128 columns, 16-byte chunks XOR (row & 7)
-          uint8_t* prow = gen + p_off + (c >> 2) * (128 * 128) + trow * 128;
-          const int ch0 = (c & 3) * 2;
-          *reinterpret_cast<uint4*>(prow + (((ch0) ^ (trow & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-          *reinterpret_cast<uint4*>(prow + (((ch0 + 1) ^ (trow & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
-        }
-      }
-      fence_async_smem();
-    }
-    tc_fence_before();
-    __syncwarp();
-    if (got_s && lane == 0) mbar_arrive(bar_p);
-    if (st == 0) ATRACE(6);
-    // ---- output: O = sat8(rq(P V; pv_scale)), heads concatenated along the feature dimension ----
-    if (got_s && mbar_wait(bar_o, 0, a.status)) {
-      tc_fence_after();
-      if (st == 0) ATRACE(8);
-      const long long pv_c = 1ll << (a.pv_s - 1);
-      int8_t* orow = a.O + ((int64_t)b * a.T + r) * a.D + (int64_t)h * a.d;
-      for (int c = half; c < a.d / 32; c += 2) {
-        if (!warp_ok) break;
-        int v[32];
-        tmem_ld32(t_row + c * 32, v);
-        if (row_ok) {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) v[j] = (int)(((long long)v[j] * a.pv_m + pv_c) >> a.pv_s);
-          int4 w0, w1;
-          w0.x = (int)pack_sat8(v[0], v[1], v[2], v[3]);     w0.y = (int)pack_sat8(v[4], v[5], v[6], v[7]);
-          w0.z = (int)pack_sat8(v[8], v[9], v[10], v[11]);   w0.w = (int)pack_sat8(v[12], v[13], v[14], v[15]);
-          w1.x = (int)pack_sat8(v[16], v[17], v[18], v[19]); w1.y = (int)pack_sat8(v[20], v[21], v[22], v[23]);
-          w1.z = (int)pack_sat8(v[24], v[25], v[26], v[27]); w1.w = (int)pack_sat8(v[28], v[29], v[30], v[31]);
-          reinterpret_cast<int4*>(orow + c * 32)[0] = w0;
-          reinterpret_cast<int4*>(orow + c * 32)[1] = w1;
-        }
-      }
+      // tensor memory may take the next item's scores
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_e);
     }
   }
   tc_fence_before();
   __syncthreads();
-  if (threadIdx.x == 0) ATRACE(9);
+  if (threadIdx.x == 0) {
+    ATRACE(9);
+    // the last CTA to finish leaves the counters at zero for the next launch
+    __threadfence();
+    if (atomicAdd(a.sched + 1, 1u) == gridDim.x - 1) {
+      a.sched[0] = 0;
+      a.sched[1] = 0;
+      __threadfence();
+    }
+  }
   if (warp == 0) {
     tc_fence_after();
     tmem_dealloc(tmem, (uint32_t)a.tmem_cols);
@@ -299,7 +390,7 @@ bool g_attn_attr = false;
 int launch_attention_fused(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* QKV, int8_t* O) {
   if (!ctx->tmap_encode) return IVIT_ERR_UNSUPPORTED;
   const int64_t B = p->B, T = p->T, D = p->D, h = p->heads, d = D / h;
-  if (T > 256 || (d != 32 && d != 64 && d != 128) || B * h > 2147483647LL / 2) return IVIT_ERR_UNSUPPORTED;
+  if (T > 256 || (d != 32 && d != 64 && d != 128) || B * h > 2147483647LL / 4) return IVIT_ERR_UNSUPPORTED;
   if ((reinterpret_cast<uintptr_t>(QKV) & 15) || (reinterpret_cast<uintptr_t>(O) & 15)) return IVIT_ERR_UNSUPPORTED;
   if (B == 0) return IVIT_OK;
   AttnArgs a{};
@@ -323,13 +414,17 @@ int launch_attention_fused(ivit_ctx* ctx, const ivit_block_params* p, const int8
     return IVIT_ERR_UNSUPPORTED;
   const uint32_t v_off = 128 * 128 + a.Npad * 128;
   const uint32_t p_off = (v_off + a.Npad * a.d + 1023u) & ~1023u;
-  const size_t smem = 1024 + p_off + (size_t)((a.Npad + 127) / 128) * 128 * 128 + 1024 + 2048 + 64;
+  const size_t smem = 1024 + p_off + (size_t)((a.Npad + 127) / 128) * 128 * 128 + 1024 + 2048 + 16 + 64 + 16;
   if (!g_attn_attr) {
     if (cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
       return IVIT_ERR_CUDA;
     g_attn_attr = true;
   }
-  const int64_t grid = B * h * a.tiles_m;
+  a.bh = (int)(B * h);
+  a.items = (int)(B * h * a.tiles_m);
+  a.sched = ctx->sched_dev;
+  const int64_t slots = 2 * (int64_t)ctx->sm_count;
+  const int64_t grid = a.items < slots ? a.items : slots;
   LaunchScope ls(ctx, KIND_ATTENTION, 4.0 * (double)(B * h) * (double)T * (double)T * (double)d);
   launch_k(attention_kernel, dim3((unsigned)grid), dim3(kAttnThreads), smem, ctx->stream, tmQ, tmK, tmV, a);
   return ls.done();

@@ -190,7 +190,8 @@ int ivit_ctx_create(ivit_ctx** out, int device, void* cuda_stream) {
   if (cudaHostAlloc((void**)&c->status_host, sizeof(int), cudaHostAllocMapped) != cudaSuccess) { delete c; return IVIT_ERR_CUDA; }
   *c->status_host = 0;
   if (cudaHostGetDevicePointer((void**)&c->status_dev, c->status_host, 0) != cudaSuccess ||
-      cudaMalloc((void**)&c->gelu_tables, (size_t)kGeluTableSlots * kGeluTableBytes) != cudaSuccess) {
+      cudaMalloc((void**)&c->gelu_tables, (size_t)kGeluTableSlots * kGeluTableBytes + 64) != cudaSuccess ||
+      cudaMemset(c->gelu_tables + (size_t)kGeluTableSlots * kGeluTableBytes, 0, 64) != cudaSuccess) {
     cudaFreeHost(c->status_host);
     delete c;
     return IVIT_ERR_CUDA;
@@ -201,6 +202,7 @@ int ivit_ctx_create(ivit_ctx** out, int device, void* cuda_stream) {
       qres != cudaDriverEntryPointSuccess)
     fn = nullptr;
   c->tmap_encode = fn;
+  c->sched_dev = reinterpret_cast<unsigned*>(c->gelu_tables + (size_t)kGeluTableSlots * kGeluTableBytes);
   *out = c;
   return IVIT_OK;
 }
