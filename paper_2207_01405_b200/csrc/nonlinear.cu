@@ -123,7 +123,7 @@ template <int WPL, int ROWS>
 __global__ void __launch_bounds__(128, 6) layernorm_i8_batched_kernel(const int8_t* __restrict__ in, int64_t ldin,
                                                                       ScaleDev gs, const int32_t* __restrict__ beta,
                                                                       int M_ln, int8_t* __restrict__ out, int64_t ldout,
-                                                                      int64_t rows, int C, unsigned mean_magic) {
+                                                                      int64_t rows, int C, unsigned mean_magic, int vec) {
   pdl_trigger();
   pdl_wait();
   const int lane = threadIdx.x & 31;
@@ -132,26 +132,50 @@ __global__ void __launch_bounds__(128, 6) layernorm_i8_batched_kernel(const int8
   const int nwords = C >> 2;
   // constants of this lane's channels (word i of the lane covers channels 4*(lane+32i) .. +3)
   int pm[WPL][4], ps[WPL][4], pb[WPL][4];
-  bool all_hi = true;   // every shift >= 33: only the high word of the product is needed (see below)
+  // Fast form, taken when it is exact for every channel of the warp: with s >= 33 the rounding constant
+  // 2^(s-1) is a multiple of 2^32, so (yF m + 2^(s-1)) >> s = (hi32(yF m) + 2^(s-33)) >> (s - 32), and beta
+  // joins the constant as beta 2^(s-32) when that stays far from 32 bits (|hi32| < 2^21 here).
+  bool fast = true;
 #pragma unroll
   for (int i = 0; i < WPL; ++i) {
     const int idx = lane + 32 * i;
+    if (vec) {
+      // per-channel arrays aligned for one 16-byte (4-byte for the shifts) load per word of four channels
+      int4 m4 = make_int4(1, 1, 1, 1), b4 = make_int4(0, 0, 0, 0);
+      uchar4 s4 = make_uchar4(40, 40, 40, 40);
+      if (idx < nwords) {
+        m4 = __ldg(reinterpret_cast<const int4*>(gs.mult_c) + idx);
+        s4 = __ldg(reinterpret_cast<const uchar4*>(gs.shift_c) + idx);
+        if (beta) b4 = __ldg(reinterpret_cast<const int4*>(beta) + idx);
+      }
+      pm[i][0] = m4.x; pm[i][1] = m4.y; pm[i][2] = m4.z; pm[i][3] = m4.w;
+      ps[i][0] = clamp_shift(s4.x); ps[i][1] = clamp_shift(s4.y); ps[i][2] = clamp_shift(s4.z); ps[i][3] = clamp_shift(s4.w);
+      pb[i][0] = b4.x; pb[i][1] = b4.y; pb[i][2] = b4.z; pb[i][3] = b4.w;
+    } else {
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const int c = idx * 4 + b;
+        pm[i][b] = idx < nwords ? gs.m(c) : 1;
+        ps[i][b] = idx < nwords ? gs.s(c) : 40;
+        pb[i][b] = (idx < nwords && beta) ? __ldg(beta + c) : 0;
+      }
+    }
 #pragma unroll
     for (int b = 0; b < 4; ++b) {
-      const int c = idx * 4 + b;
-      pm[i][b] = idx < nwords ? gs.m(c) : 1;
-      ps[i][b] = idx < nwords ? gs.s(c) : 40;
-      pb[i][b] = (idx < nwords && beta) ? __ldg(beta + c) : 0;
-      all_hi = all_hi && ps[i][b] >= 33;
+      const int sh = ps[i][b] - 32;
+      fast = fast && sh >= 1 && pb[i][b] > -(1 << (29 - sh)) && pb[i][b] < (1 << (29 - sh));
     }
   }
-  all_hi = __all_sync(0xffffffffu, all_hi);
-  if (all_hi) {
-    // keep s - 32 instead of s
+  fast = __all_sync(0xffffffffu, fast);
+  if (fast) {
+    // keep s - 32 and the combined constant instead of s and beta
 #pragma unroll
     for (int i = 0; i < WPL; ++i)
 #pragma unroll
-      for (int b = 0; b < 4; ++b) ps[i][b] -= 32;
+      for (int b = 0; b < 4; ++b) {
+        ps[i][b] -= 32;
+        pb[i][b] = (1 << (ps[i][b] - 1)) + pb[i][b] * (1 << ps[i][b]);
+      }
   }
   for (int64_t r0 = warp * ROWS; r0 < rows; r0 += nwarps * ROWS) {
     int w[ROWS][WPL];
@@ -204,10 +228,8 @@ __global__ void __launch_bounds__(128, 6) layernorm_i8_batched_kernel(const int8
               asm("prmt.b32 %0, %1, %1, %2;" : "=r"(x) : "r"(w[r][i]), "r"(0x8880 + 0x1111 * b));
               // (x - mu) * F, formed modulo 2^32 (the difference always fits: |y F| <= 2^(M_ln+1))
               const int yF = (int)((unsigned)x * (unsigned)Fr - (unsigned)muFr);
-              if (all_hi) {
-                // s >= 33: the rounding constant 2^(s-1) is a multiple of 2^32, so
-                // (yF m + 2^(s-1)) >> s = (hi32(yF m) + 2^(s-33)) >> (s - 32)
-                v[b] = ((__mulhi(yF, pm[i][b]) + (1 << (ps[i][b] - 1))) >> ps[i][b]) + pb[i][b];
+              if (fast) {
+                v[b] = (__mulhi(yF, pm[i][b]) + pb[i][b]) >> ps[i][b];
               } else {
                 v[b] = rq(yF, pm[i][b], ps[i][b]) + pb[i][b];
               }
@@ -322,10 +344,12 @@ int launch_layernorm(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, 
     const int64_t wantb = (warps + tb / 32 - 1) / (tb / 32);
     const int gridb = (int)(wantb < (int64_t)ctx->sm_count * 12 ? wantb : (int64_t)ctx->sm_count * 12);
     const unsigned magic = (unsigned)(0x100000000ull / (unsigned long long)(2 * C)) + 1u;
-    if (wpl <= 1) launch_k(layernorm_i8_batched_kernel<1, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic);
-    else if (wpl <= 2) launch_k(layernorm_i8_batched_kernel<2, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic);
-    else if (wpl <= 3) launch_k(layernorm_i8_batched_kernel<3, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic);
-    else launch_k(layernorm_i8_batched_kernel<4, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic);
+    const int vec = gs.mult_c && gs.shift_c && !(reinterpret_cast<uintptr_t>(gs.mult_c) & 15) && !(reinterpret_cast<uintptr_t>(gs.shift_c) & 3) &&
+                    !(reinterpret_cast<uintptr_t>(beta) & 15);
+    if (wpl <= 1) launch_k(layernorm_i8_batched_kernel<1, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
+    else if (wpl <= 2) launch_k(layernorm_i8_batched_kernel<2, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
+    else if (wpl <= 3) launch_k(layernorm_i8_batched_kernel<3, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
+    else launch_k(layernorm_i8_batched_kernel<4, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
     return ls.done();
   }
   if (wpl <= 6) launch_k(layernorm_i8_kernel<6>, dim3(grid), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
