@@ -52,6 +52,47 @@ def test_linear_parity(engine, M, N, K):
     assert c.poll_status() == 0
 
 
+@pytest.mark.parametrize("M,N,K", [(130, 200, 48), (197, 384, 1536), (393, 1000, 384), (33, 36, 96), (700, 384, 384)])
+def test_linear_residual_full_rows(M, N, K):
+    """Residual with one row per output row (the encoder block's form): the residual tile is staged by TMA."""
+    g = _g()
+    c = g.ctx()
+    rng = np.random.default_rng(M * 11 + N * 5 + K)
+    A, W = rand_i8(rng, (M, K)), rand_i8(rng, (N, K))
+    bias = rng.integers(-20000, 20000, N).astype(np.int32)
+    acc_std = np.sqrt(K) * 40 * 40
+    scale = scale_channels(rng.uniform(20, 60, N) / acc_std)
+    res = rand_i8(rng, (M, N))
+    for ratio in (0.9, 0.3, 0.004):   # residual shifts of 31, 32 and 38
+        rs = Scale(*dyadic(ratio))
+        got = c.linear(g.dev(A), g.dev(W), torch.from_numpy(bias).cuda(), g.binding.DevScale(scale, "cuda"), res=g.dev(res),
+                       res_scale=g.binding.DevScale(rs, "cuda"), out=g.dev(np.zeros((M, N), np.int8)))
+        g.assert_equal(g.host(got), O.linear(A, W, bias, scale, res=res, res_scale=rs), f"linear+res {ratio}")
+    assert c.poll_status() == 0
+
+
+@pytest.mark.parametrize("M,N,K", [(130, 200, 16), (260, 128, 32)])
+def test_linear_low_shifts(M, N, K):
+    """Per-channel shifts of 31 and 32 next to larger ones: the requantisation leaves its high-word form."""
+    g = _g()
+    c = g.ctx()
+    rng = np.random.default_rng(M + N + K)
+    A, W = rand_i8(rng, (M, K), std=3), rand_i8(rng, (N, K), std=3)
+    bias = rng.integers(-50, 50, N).astype(np.int32)
+    for lo, hi in ((0.55, 0.95), (0.26, 0.49), (0.26, 0.95), (0.001, 0.95)):
+        scale = scale_channels(rng.uniform(lo, hi, N))
+        got = c.linear(g.dev(A), g.dev(W), torch.from_numpy(bias).cuda(), g.binding.DevScale(scale, "cuda"),
+                       out=g.dev(np.zeros((M, N), np.int8)))
+        g.assert_equal(g.host(got), O.linear(A, W, bias, scale), f"linear shifts {lo}-{hi}")
+    # a bias too large for the 32-bit sum with the accumulator
+    big = rng.integers(-(2 ** 31) + 1, 2 ** 31 - 1, N).astype(np.int32)
+    scale = scale_channels(rng.uniform(1e-9, 3e-9, N))
+    got = c.linear(g.dev(A), g.dev(W), torch.from_numpy(big).cuda(), g.binding.DevScale(scale, "cuda"),
+                   out=g.dev(np.zeros((M, N), np.int8)))
+    g.assert_equal(g.host(got), O.linear(A, W, big, scale), "linear big bias")
+    assert c.poll_status() == 0
+
+
 @pytest.mark.parametrize("engine", [1, 0])
 def test_linear_output_row_groups(engine):
     g = _g()
