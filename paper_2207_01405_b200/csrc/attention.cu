@@ -223,18 +223,18 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
       const bool warp_ok = m0 + qd * 32 < a.T;      // warps whose 32 rows all lie past T only keep the barriers
       const int32_t* brow = a.bias ? a.bias + (((int64_t)bhid % a.bias_batches) * a.T + (row_ok ? r : 0)) * (int64_t)a.T : nullptr;
 
-      uint32_t xs[32];   // int8 scores of this thread's chunks, packed four per word
       int mx = -128;
       bool got_s = mbar_wait(bar_s, par, a.status);
       alive = alive && got_s;
       if (got_s) tc_fence_after();
       if (st == 0) ATRACE(3);
       if (got_s && warp_ok) {
-        // pass A: requantise the scores to int8 (Sec. 3.2), running maximum
-#pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-          const int c = 2 * cc + half;
-          if (c < nch) {
+        // pass A: requantise the scores to int8 (Sec. 3.2), running maximum.  The chunk loops are rolled (the
+        // kernel's code stays within the instruction cache); what a later pass needs of a chunk waits in the
+        // chunk's own tensor-memory columns.
+#pragma unroll 1
+        for (int c = half; c < nch; c += 2) {
+          {
             int v[32];
             tmem_ld32(t_row + c * 32, v);
             if (brow) {
@@ -260,12 +260,16 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
 #pragma unroll
             for (int j = 1; j < 32; j += 2) m = max(m, max(v[j], v[(j + 1) & 31]));
             mx = max(mx, m);
-            // scores are kept as biased bytes (x + 128, i.e. x ^ 0x80) so that pass B can index with them
+            // scores are kept as biased bytes (x + 128, i.e. x ^ 0x80) so that pass B can index with them:
+            // four per word in the first eight columns of the chunk
+            uint32_t xs[8];
 #pragma unroll
             for (int k = 0; k < 8; ++k)
-              xs[cc * 8 + k] = pack_sat8(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]) ^ 0x80808080u;
+              xs[k] = pack_sat8(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]) ^ 0x80808080u;
+            tmem_st8(t_row + c * 32, xs);
           }
         }
+        tmem_st_wait();
         mx = max(-128, min(127, mx));
         part_max[half * 128 + trow] = mx;
       }
@@ -275,16 +279,17 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
       if (got_s && warp_ok) {
         mx = max(part_max[trow], part_max[128 + trow]);
         // pass B: ShiftExp(I - I_max) by table, row sum, exponentials back into tensor memory
-#pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-          const int c = 2 * cc + half;
-          if (c < nch) {
+#pragma unroll 1
+        for (int c = half; c < nch; c += 2) {
+          {
             int ev[32];
+            uint32_t xs[8];
+            tmem_ld8(t_row + c * 32, xs);
             // entry (I_max - I) of the table = word at tab + 4*(I_max + 128) - 4*(I + 128)
             const uint8_t* tmx = reinterpret_cast<const uint8_t*>(tab) + 4 * (mx + 128);
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
-              const uint32_t w = xs[cc * 8 + k];
+              const uint32_t w = xs[k];
 #pragma unroll
               for (int bb = 0; bb < 4; ++bb)
                 ev[4 * k + bb] = (int)*reinterpret_cast<const unsigned*>(tmx - 4 * (int)__byte_perm(w, 0, 0x4440 + bb));
@@ -308,10 +313,9 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
         sum = part_sum[trow] + part_sum[128 + trow];
         // pass C: Eq. (IntDiv) with M = 45, k_out = 8: (floor(2^45 / sum) * e) >> 38 = umulhi(factor, e) >> 6
         const unsigned factor = (unsigned)((1ull << 45) / (unsigned long long)(sum ? sum : 1u));
-#pragma unroll
-        for (int cc = 0; cc < 4; ++cc) {
-          const int c = 2 * cc + half;
-          if (c < nch) {
+#pragma unroll 1
+        for (int c = half; c < nch; c += 2) {
+          {
             int ev[32];
             tmem_ld32(t_row + c * 32, ev);
             uint32_t w[8];
