@@ -9,6 +9,7 @@ one batch of 64 synthetic images.  Prints one JSON line (rank 0).
 from __future__ import annotations
 
 import argparse
+import datetime
 import json
 import os
 import statistics
@@ -22,6 +23,10 @@ if ROOT not in sys.path:
 
 METRIC = "int-only ViT images/s (DeiT-S b64)"
 WORKLOAD = "deit_small_b64"
+# dram__bytes_read.sum + dram__bytes_write.sum per GEMM launch of this workload, averaged over the four Dense
+# layers of an encoder block in one ncu capture (profiles/gemm_tc_kernel_deit_small_b64.md): well below the
+# 10 to 34 MB of operands and results per launch, because the activations stay in L2.
+GEMM_DRAM_BYTES_PER_LAUNCH = 11.4e6
 CONFIG_INDEX = 1
 
 
@@ -34,9 +39,9 @@ def vit_int8_ops(p) -> float:
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clock and throttle reasons with nvidia-smi; stop() keeps the samples taken inside the timed region."""
 
-    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    Q = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
          "clocks_event_reasons.sw_power_cap")
 
@@ -46,12 +51,13 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.Q}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
 
-    def stop(self) -> dict:
+    def stop(self, t_begin: float, t_end: float) -> dict:
+        """t_begin, t_end: time.time() at the two ends of the timed region."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -64,13 +70,16 @@ class ClockSampler:
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in out.strip().splitlines():
             f = [x.strip() for x in line.split(",")]
-            if len(f) < 7:
+            if len(f) < 8:
                 continue
             try:
-                sm.append(float(f[0])); mx.append(float(f[1])); power.append(float(f[2]))
+                ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                if ts < t_begin - 0.02 or ts > t_end + 0.02:
+                    continue
+                sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
             except ValueError:
                 continue
-            for n, v in zip(names, f[3:7]):
+            for n, v in zip(names, f[4:8]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
         if not sm:
@@ -203,16 +212,18 @@ def run_gpu(args):
         barrier()
         return sum(a.elapsed_time(b) for a, b in ev)
 
+    sampler = ClockSampler(local_rank)
+    sampler.start()   # before the warm-up: the first sample takes a while to come
     for _ in range(max(args.warmup, 3)):
         step_resident()
     torch.cuda.synchronize()
 
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     launches0 = ctx.launch_count()
+    t_begin = time.time()
     ms_total = timed(step_resident, args.steps)
+    t_end = time.time()
     launches = ctx.launch_count() - launches0
-    clocks = sampler.stop()
+    clocks = sampler.stop(t_begin, t_end)
 
     for _ in range(3):
         step_e2e()
@@ -269,7 +280,10 @@ def run_gpu(args):
     if dom.startswith("gemm") or dom.startswith("attention"):
         achieved = dk["work"] / (dk["ms"] * 1e-3) / 1e12
         roofline = {"kernel": dom, "bound": "tensor", "achieved": round(achieved, 2), "peak": int8_peak, "unit": "TOP/s",
-                    "frac": round(achieved / int8_peak, 4), "traffic": None,
+                    "frac": round(achieved / int8_peak, 4), "traffic": GEMM_DRAM_BYTES_PER_LAUNCH,
+                    # the event pair around every launch costs a few microseconds and stops the overlap of one kernel's
+                    # set-up with its predecessor's tail; the same work over (un-bracketed step time x this kernel's share)
+                    "achieved_in_step": round(dk["work"] / prof_steps / (ms_total / args.steps * 1e-3 * dk["ms"] / total_kernel_ms) / 1e12, 2),
                     "peak_source": f"2 x {peak_src} sustained bf16 cuBLAS ({peaks['bf16_tflops_sustained']} TFLOP/s)"}
     else:
         achieved = dk["work"] / (dk["ms"] * 1e-3) / 1e9
@@ -309,8 +323,8 @@ def run_gpu(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ivit", choices=["ivit", "reference"])
     ap.add_argument("--detail", action="store_true", help="print per-shape kernel times to stderr")
     args = ap.parse_args()
