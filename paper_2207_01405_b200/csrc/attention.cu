@@ -45,7 +45,8 @@ struct AttnArgs {
   int64_t bias_batches;
   int8_t* O;                        // [B*T, D]
   int q_pos[3], k_pos[3], v_pos[3];
-  unsigned* sched;                  // [0] next work item, [1] CTAs that have finished; both zero between launches
+  unsigned* sched;                  // this launch's counters: [0] next work item, [1] CTAs that have finished
+  unsigned* sched_other;            // the counters of the next launch
   int* status;
 };
 
@@ -100,6 +101,12 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
   const uint32_t tmem = *tmem_slot;
   pdl_trigger();
   pdl_wait();   // the QKV tensor comes from the previous kernel
+  // Launches alternate between two pairs of counters.  A launch leaves its own pair at zero when its last CTA
+  // finishes, and also zeroes the other pair here, so that a launch that was cut short cannot poison the next.
+  if (blockIdx.x == 0 && threadIdx.x == 32) {
+    a.sched_other[0] = 0;
+    a.sched_other[1] = 0;
+  }
 
   // item -> (tile, image/window * heads + head): all first tiles before all second tiles
   if (warp == 0) {
@@ -426,7 +433,9 @@ int launch_attention_fused(ivit_ctx* ctx, const ivit_block_params* p, const int8
   }
   a.bh = (int)(B * h);
   a.items = (int)(B * h * a.tiles_m);
-  a.sched = ctx->sched_dev;
+  a.sched = ctx->sched_dev + 2 * ctx->attn_gen;
+  a.sched_other = ctx->sched_dev + 2 * (ctx->attn_gen ^ 1);
+  ctx->attn_gen ^= 1;
   const int64_t slots = 2 * (int64_t)ctx->sm_count;
   const int64_t grid = a.items < slots ? a.items : slots;
   LaunchScope ls(ctx, KIND_ATTENTION, 4.0 * (double)(B * h) * (double)T * (double)T * (double)d);

@@ -29,7 +29,8 @@ struct ivit_ctx {
   int* status_host;  // mapped pinned memory: kernels write the first device-side error here
   int* status_dev;   // device view of the same word
   int8_t* gelu_tables;  // kGeluTableSlots tables on the device
-  unsigned* sched_dev;  // two work counters of the attention kernel (behind the tables), zero between launches
+  unsigned* sched_dev;  // two pairs of work counters of the attention kernel (behind the tables), used alternately
+  int attn_gen;         // pair of the next launch
   ivit::GeluKey gelu_keys[ivit::kGeluTableSlots];
   int gelu_used;
   int gelu_next;
