@@ -203,7 +203,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
     const int half = (warp - 1) >> 2;
     const int trow = qd * 32 + lane;              // row inside the tile
     const uint32_t t_row = tmem + ((uint32_t)(qd * 32) << 16);
-    const int nch = a.Npad / 32;
+    const int nch = a.Npad / 16;
     const bool qk_hi = a.qk_s >= 33;              // rounding constant and shift both past the low product word
     const long long qk_c = 1ll << (a.qk_s - 1);
     const int qk_rnd = qk_hi ? 1 << (a.qk_s - 33) : 0, qk_sh = a.qk_s - 32;
@@ -236,45 +236,44 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
       if (got_s) tc_fence_after();
       if (st == 0) ATRACE(3);
       if (got_s && warp_ok) {
-        // pass A: requantise the scores to int8 (Sec. 3.2), running maximum.  The chunk loops are rolled (the
-        // kernel's code stays within the instruction cache); what a later pass needs of a chunk waits in the
-        // chunk's own tensor-memory columns.
+        // pass A: requantise the scores to int8 (Sec. 3.2), running maximum.  The two threads of a row take
+        // alternate 16-column chunks (Npad / 16 is even: equal shares).  The chunk loops are rolled (the kernel's
+        // code stays within the instruction cache); what a later pass needs of a chunk waits in the chunk's own
+        // tensor-memory columns.
 #pragma unroll 1
         for (int c = half; c < nch; c += 2) {
-          {
-            int v[32];
-            tmem_ld32(t_row + c * 32, v);
-            if (brow) {
+          int v[16];
+          tmem_ld16(t_row + c * 16, v);
+          if (brow) {
 #pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (c * 32 + j < a.T) v[j] += __ldg(brow + c * 32 + j);
-            }
-            if (qk_hi) {          // the usual case: high product word plus 2^(s-33), shifted by s - 32
-#pragma unroll
-              for (int j = 0; j < 32; ++j) v[j] = mad_hi(v[j], a.qk_m, qk_rnd) >> qk_sh;
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; ++j) v[j] = (int)(((long long)v[j] * a.qk_m + qk_c) >> a.qk_s);
-            }
-            // columns past T (only in the last chunk) never win the maximum and look up a valid table entry
-            if (c == nch - 1) {
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (c * 32 + j >= a.T) v[j] = -128;
-            }
-            // running maximum on the unsaturated values (saturation is monotone: it is applied to the result)
-            int m = v[0];
-#pragma unroll
-            for (int j = 1; j < 32; j += 2) m = max(m, max(v[j], v[(j + 1) & 31]));
-            mx = max(mx, m);
-            // scores are kept as biased bytes (x + 128, i.e. x ^ 0x80) so that pass B can index with them:
-            // four per word in the first eight columns of the chunk
-            uint32_t xs[8];
-#pragma unroll
-            for (int k = 0; k < 8; ++k)
-              xs[k] = pack_sat8(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]) ^ 0x80808080u;
-            tmem_st8(t_row + c * 32, xs);
+            for (int j = 0; j < 16; ++j)
+              if (c * 16 + j < a.T) v[j] += __ldg(brow + c * 16 + j);
           }
+          if (qk_hi) {          // the usual case: high product word plus 2^(s-33), shifted by s - 32
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] = mad_hi(v[j], a.qk_m, qk_rnd) >> qk_sh;
+          } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] = (int)(((long long)v[j] * a.qk_m + qk_c) >> a.qk_s);
+          }
+          // columns past T (only in the last two chunks) never win the maximum and look up a valid table entry
+          if (c >= nch - 2) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+              if (c * 16 + j >= a.T) v[j] = -128;
+          }
+          // running maximum on the unsaturated values (saturation is monotone: it is applied to the result)
+          int m = v[0];
+#pragma unroll
+          for (int j = 1; j < 16; j += 2) m = max(m, max(v[j], v[(j + 1) & 15]));
+          mx = max(mx, m);
+          // scores are kept as biased bytes (x + 128, i.e. x ^ 0x80) so that pass B can index with them:
+          // four per word in the first four columns of the chunk
+          uint32_t xs[4];
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            xs[k] = pack_sat8(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]) ^ 0x80808080u;
+          tmem_st4(t_row + c * 16, xs);
         }
         tmem_st_wait();
         mx = max(-128, min(127, mx));
@@ -286,30 +285,28 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
       if (got_s && warp_ok) {
         mx = max(part_max[trow], part_max[128 + trow]);
         // pass B: ShiftExp(I - I_max) by table, row sum, exponentials back into tensor memory
+        // entry (I_max - I) of the table = word at tab + 4*(I_max + 128) - 4*(I + 128)
+        const uint8_t* tmx = reinterpret_cast<const uint8_t*>(tab) + 4 * (mx + 128);
 #pragma unroll 1
         for (int c = half; c < nch; c += 2) {
-          {
-            int ev[32];
-            uint32_t xs[8];
-            tmem_ld8(t_row + c * 32, xs);
-            // entry (I_max - I) of the table = word at tab + 4*(I_max + 128) - 4*(I + 128)
-            const uint8_t* tmx = reinterpret_cast<const uint8_t*>(tab) + 4 * (mx + 128);
+          int ev[16];
+          uint32_t xs[4];
+          tmem_ld4(t_row + c * 16, xs);
 #pragma unroll
-            for (int k = 0; k < 8; ++k) {
-              const uint32_t w = xs[k];
+          for (int k = 0; k < 4; ++k) {
+            const uint32_t w = xs[k];
 #pragma unroll
-              for (int bb = 0; bb < 4; ++bb)
-                ev[4 * k + bb] = (int)*reinterpret_cast<const unsigned*>(tmx - 4 * (int)__byte_perm(w, 0, 0x4440 + bb));
-            }
-            if (c == nch - 1) {   // columns past T contribute nothing
-#pragma unroll
-              for (int j = 0; j < 32; ++j)
-                if (c * 32 + j >= a.T) ev[j] = 0;
-            }
-#pragma unroll
-            for (int j = 0; j < 32; ++j) sum += (unsigned)ev[j];
-            tmem_st32(t_row + c * 32, ev);
+            for (int bb = 0; bb < 4; ++bb)
+              ev[4 * k + bb] = (int)*reinterpret_cast<const unsigned*>(tmx - 4 * (int)__byte_perm(w, 0, 0x4440 + bb));
           }
+          if (c >= nch - 2) {   // columns past T contribute nothing
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+              if (c * 16 + j >= a.T) ev[j] = 0;
+          }
+#pragma unroll
+          for (int j = 0; j < 16; ++j) sum += (unsigned)ev[j];
+          tmem_st16(t_row + c * 16, ev);
         }
         tmem_st_wait();
         part_sum[half * 128 + trow] = sum;
@@ -322,20 +319,16 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
         const unsigned factor = (unsigned)((1ull << 45) / (unsigned long long)(sum ? sum : 1u));
 #pragma unroll 1
         for (int c = half; c < nch; c += 2) {
-          {
-            int ev[32];
-            tmem_ld32(t_row + c * 32, ev);
-            uint32_t w[8];
+          int ev[16];
+          tmem_ld16(t_row + c * 16, ev);
+          uint32_t w[4];
 #pragma unroll
-            for (int k = 0; k < 8; ++k)   // values are <= 128: the saturating pack clamps the one possible 128 to 127
-              w[k] = pack_sat8((int)(__umulhi(factor, (unsigned)ev[4 * k]) >> 6), (int)(__umulhi(factor, (unsigned)ev[4 * k + 1]) >> 6),
-                               (int)(__umulhi(factor, (unsigned)ev[4 * k + 2]) >> 6), (int)(__umulhi(factor, (unsigned)ev[4 * k + 3]) >> 6));
-            // A operand of P V: row = tile row, k-block = 128 columns, 16-byte chunks XOR (row & 7)
-            uint8_t* prow = gen + p_off + (c >> 2) * (128 * 128) + trow * 128;
-            const int ch0 = (c & 3) * 2;
-            *reinterpret_cast<uint4*>(prow + (((ch0) ^ (trow & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
-            *reinterpret_cast<uint4*>(prow + (((ch0 + 1) ^ (trow & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
-          }
+          for (int k = 0; k < 4; ++k)   // values are <= 128: the saturating pack clamps the one possible 128 to 127
+            w[k] = pack_sat8((int)(__umulhi(factor, (unsigned)ev[4 * k]) >> 6), (int)(__umulhi(factor, (unsigned)ev[4 * k + 1]) >> 6),
+                             (int)(__umulhi(factor, (unsigned)ev[4 * k + 2]) >> 6), (int)(__umulhi(factor, (unsigned)ev[4 * k + 3]) >> 6));
+          // A operand of P V: row = tile row, k-block = 128 columns, 16-byte pieces XOR (row & 7)
+          uint8_t* prow = gen + p_off + (c >> 3) * (128 * 128) + trow * 128;
+          *reinterpret_cast<uint4*>(prow + ((((c & 7)) ^ (trow & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
         }
         fence_async_smem();
       }
