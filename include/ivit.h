@@ -234,10 +234,15 @@ size_t ivit_vit_workspace_bytes(const ivit_vit_params* p);
 int ivit_vit_forward(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* image, int32_t* logits,
                      void* workspace, size_t workspace_bytes);
 
-/* Same forward with HOST buffers: copies image_host (pinned or pageable) to a staging area in
- * the workspace, runs ivit_vit_forward, and copies the logits back to logits_host, all enqueued
- * on the context's stream (the caller synchronises the stream before reading logits_host).
- * workspace must hold ivit_vit_host_workspace_bytes(p). */
+/* Same forward with HOST buffers: copies image_host to a staging area in the workspace, runs
+ * ivit_vit_forward, and copies the logits back to logits_host.  The call only enqueues work and
+ * returns: the caller synchronises the context's stream before reading logits_host, and both host
+ * buffers must stay valid (and the image unchanged) until then.  The input copy runs on a stream
+ * of the context's own into one of two staging buffers used alternately, so the copy of one call
+ * overlaps the compute of the call before it when calls are enqueued back to back (pinned host
+ * memory is needed for that overlap; pageable memory works but copies synchronously).  The first
+ * call on a context creates that stream and its events.  All calls on one context must use the
+ * same workspace.  workspace must hold ivit_vit_host_workspace_bytes(p). */
 size_t ivit_vit_host_workspace_bytes(const ivit_vit_params* p);
 int ivit_vit_forward_host(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* image_host,
                           int32_t* logits_host, void* workspace, size_t workspace_bytes);

@@ -38,6 +38,10 @@ struct ivit_ctx {
   int gemm_engine;
   int sm_count;
   void* tmap_encode;  // cuTensorMapEncodeTiled, resolved at context creation
+  // ivit_vit_forward_host: input copies run on their own stream into two staging buffers (created on first use)
+  cudaStream_t copy_stream;
+  cudaEvent_t img_ready[2], img_free[2];
+  uint64_t host_calls;
   // per-kernel timing session (ivit_ctx_profile_*)
   bool profiling;
   int prof_count;

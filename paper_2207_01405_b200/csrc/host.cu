@@ -212,6 +212,14 @@ int ivit_ctx_destroy(ivit_ctx* ctx) {
   cudaSetDevice(ctx->device);
   cudaFree(ctx->gelu_tables);
   cudaFreeHost(ctx->status_host);
+  if (ctx->copy_stream) {
+    cudaStreamSynchronize(ctx->copy_stream);
+    for (int i = 0; i < 2; ++i) {
+      cudaEventDestroy(ctx->img_ready[i]);
+      cudaEventDestroy(ctx->img_free[i]);
+    }
+    cudaStreamDestroy(ctx->copy_stream);
+  }
   if (ctx->prof_ev) {
     for (int i = 0; i < 2 * kProfMax; ++i) cudaEventDestroy(ctx->prof_ev[i]);
     delete[] ctx->prof_ev;
@@ -467,7 +475,7 @@ size_t ivit_vit_host_workspace_bytes(const ivit_vit_params* p) {
   if (check_vit(p) != IVIT_OK) return 0;
   const size_t img = align_up((size_t)(p->B * 3 * p->img * p->img), 256);
   const size_t lg = align_up((size_t)(p->B * p->classes) * 4, 256);
-  return vit_ws(p).total + img + lg;
+  return vit_ws(p).total + 2 * img + lg;
 }
 
 int ivit_vit_forward_host(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* image_host,
@@ -476,14 +484,36 @@ int ivit_vit_forward_host(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t*
   int rc = check_vit(p);
   if (rc) return rc;
   const size_t img_bytes = (size_t)(p->B * 3 * p->img * p->img), lg_bytes = (size_t)(p->B * p->classes) * 4;
-  const size_t inner = vit_ws(p).total, img_off = inner, lg_off = inner + align_up(img_bytes, 256);
+  const size_t img_slot = align_up(img_bytes, 256);
+  const size_t inner = vit_ws(p).total, img_off = inner, lg_off = inner + 2 * img_slot;
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < lg_off + align_up(lg_bytes, 256))
     return IVIT_ERR_WORKSPACE;
+  if (!ctx->copy_stream) {
+    // first use: a stream of its own for the input copies, and the events that order it with the compute stream
+    if (cudaSetDevice(ctx->device) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess)
+      return IVIT_ERR_CUDA;
+    for (int i = 0; i < 2; ++i)
+      if (cudaEventCreateWithFlags(&ctx->img_ready[i], cudaEventDisableTiming) != cudaSuccess ||
+          cudaEventCreateWithFlags(&ctx->img_free[i], cudaEventDisableTiming) != cudaSuccess)
+        return IVIT_ERR_CUDA;
+    ctx->host_calls = 0;
+  }
+  // Two staging buffers used alternately: the copy of this call's image runs on the copy stream while the
+  // compute stream still works on the previous call; it only waits for the call before that to have finished
+  // with the buffer.
+  const int slot = (int)(ctx->host_calls & 1);
   char* ws = static_cast<char*>(workspace);
-  if (cudaMemcpyAsync(ws + img_off, image_host, img_bytes, cudaMemcpyHostToDevice, ctx->stream) != cudaSuccess)
+  char* img_dev = ws + img_off + (size_t)slot * img_slot;
+  if (ctx->host_calls >= 2 && cudaStreamWaitEvent(ctx->copy_stream, ctx->img_free[slot], 0) != cudaSuccess) return IVIT_ERR_CUDA;
+  if (cudaMemcpyAsync(img_dev, image_host, img_bytes, cudaMemcpyHostToDevice, ctx->copy_stream) != cudaSuccess ||
+      cudaEventRecord(ctx->img_ready[slot], ctx->copy_stream) != cudaSuccess ||
+      cudaStreamWaitEvent(ctx->stream, ctx->img_ready[slot], 0) != cudaSuccess)
     return IVIT_ERR_CUDA;
-  rc = ivit_vit_forward(ctx, p, reinterpret_cast<const int8_t*>(ws + img_off), reinterpret_cast<int32_t*>(ws + lg_off),
-                        workspace, inner);
+  ++ctx->host_calls;
+  rc = ivit_vit_forward(ctx, p, reinterpret_cast<const int8_t*>(img_dev), reinterpret_cast<int32_t*>(ws + lg_off), workspace, inner);
+  // recorded even after an error: a later copy into this buffer waits for it
+  if (cudaEventRecord(ctx->img_free[slot], ctx->stream) != cudaSuccess) return IVIT_ERR_CUDA;
   if (rc) return rc;
   if (cudaMemcpyAsync(logits_host, ws + lg_off, lg_bytes, cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess)
     return IVIT_ERR_CUDA;

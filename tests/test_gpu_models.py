@@ -49,3 +49,24 @@ def test_vit_base_b128_full_size_sampled():
     for i in (0, 127):
         g.assert_equal(logits[i:i + 1], O.vit_forward(model, image[i:i + 1]), f"image {i}")
     assert c.poll_status() == 0
+
+
+def test_host_forward_back_to_back_calls():
+    """ivit_vit_forward_host enqueued four times without a synchronisation in between: the input copy of a call
+    overlaps the compute of the call before it (two staging buffers), and every call must still see its own image."""
+    import gpu_util as g
+    c = g.ctx()
+    model, image = make_config(1, batch=4, depth=2)
+    dm = g.binding.DeviceVit(model, "cuda")
+    ws = dm.host_workspace()
+    rng = np.random.default_rng(5)
+    images = [image] + [np.clip(image.astype(np.int32) + rng.integers(-40, 40, image.shape), -128, 127).astype(np.int8)
+                        for _ in range(3)]
+    h_img = [torch.from_numpy(x).pin_memory() for x in images]
+    h_out = [torch.empty((4, model.classes), dtype=torch.int32).pin_memory() for _ in images]
+    for x, y in zip(h_img, h_out):
+        g.binding.vit_forward_host(c, dm, x, y, ws)
+    torch.cuda.synchronize()
+    for k, (x, y) in enumerate(zip(images, h_out)):
+        g.assert_equal(y.numpy(), O.vit_forward(model, x), f"call {k}")
+    assert c.poll_status() == 0
