@@ -56,6 +56,14 @@ __device__ __forceinline__ unsigned long long isqrt_u64(unsigned long long n) {
   return x;
 }
 
+// Four int32 values saturated to int8 and packed, x0 in the low byte.
+__device__ __forceinline__ unsigned pack_sat8_u(int x0, int x1, int x2, int x3) {
+  unsigned t, d;
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(t) : "r"(x3), "r"(x2), "r"(0));
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(x1), "r"(x0), "r"(t));
+  return d;
+}
+
 __device__ __forceinline__ int floordiv_pos(int a, int b) {  // b > 0
   int q = a / b;
   return (a - q * b < 0) ? q - 1 : q;
@@ -387,7 +395,10 @@ struct RowLoader {
 };
 
 // WPL words per lane in registers (d <= 128 * WPL); WPL == 0: re-read the row for each pass.
-template <int WPL, bool FROM_I32>
+// Bytes are handled as biased values u = x + 128 (x ^ 0x80), so that one byte permute yields the table index:
+// ShiftExp(x - max) = tab[max - x] = tab[(max + 128) - u].  Positions past d hold u = 0 (x = -128); they never
+// win the maximum and their table entries are taken out of the sum again.
+template <int WPL, int ROWS, bool FROM_I32>
 __global__ void __launch_bounds__(256) shiftmax_kernel(RowLoader<FROM_I32> ld, ivit_exp_params p,
                                                        int8_t* __restrict__ out, int64_t ldout,
                                                        int64_t rows, int d) {
@@ -401,63 +412,84 @@ __global__ void __launch_bounds__(256) shiftmax_kernel(RowLoader<FROM_I32> ld, i
   const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
   const int nwords = (d + 3) >> 2;
   const int nwords_out = ((d + 15) >> 4) << 2;  // zero-fill up to the next multiple of 16
+  const int npad = nwords * 4 - d;              // bytes past d in the last word
   constexpr int W = WPL > 0 ? WPL : 1;
+  constexpr int R = WPL > 0 ? ROWS : 1;         // rows a warp works on together (their reciprocals in parallel lanes)
   const int iters = WPL > 0 ? WPL : (nwords_out + 31) / 32;
-  for (int64_t r = warp; r < rows; r += nwarps) {
-    int w[W];
-    // pass 1: row max (bytes past d are replaced by -128)
-    int mx4 = (int)0x80808080;
+  // biased word idx of row r: bytes past d (and whole words past the row) read as 0
+  auto load_biased = [&](int64_t r, int idx) -> unsigned {
+    if (idx >= nwords) return 0u;
+    unsigned v = (unsigned)ld.load(r, idx) ^ 0x80808080u;
+    if (idx == nwords - 1 && npad) v &= 0xffffffffu >> (8 * npad);
+    return v;
+  };
+  for (int64_t r0 = warp * R; r0 < rows; r0 += nwarps * R) {
+    unsigned e[R][W][4];
+    unsigned my_sum = 1, my_mxu = 0;
 #pragma unroll
-    for (int i = 0; i < iters; ++i) {
-      const int idx = lane + 32 * i;
-      int v = (int)0x80808080;
-      if (idx < nwords) {
-        v = ld.load(r, idx);
-        const int valid = d - idx * 4;
-        if (valid < 4) {
-          const unsigned keep = 0xffffffffu >> (8 * (4 - valid));
-          v = (int)(((unsigned)v & keep) | (0x80808080u & ~keep));
-        }
+    for (int q = 0; q < R; ++q) {
+      const int64_t r = r0 + q < rows ? r0 + q : rows - 1;   // a row past the end repeats the last one (not stored)
+      unsigned w[W];
+      // pass 1: row max
+      unsigned mxu = 0;
+#pragma unroll
+      for (int i = 0; i < iters; ++i) {
+        const unsigned v = load_biased(r, lane + 32 * i);
+        if (WPL > 0) w[i] = v;
+        mxu = max(max(mxu, __byte_perm(v, 0, 0x4440)), max(__byte_perm(v, 0, 0x4441), max(__byte_perm(v, 0, 0x4442), v >> 24)));
       }
-      if (WPL > 0) w[i] = v;
-      mx4 = (int)__vmaxs4((unsigned)mx4, (unsigned)v);
-    }
-    int mx = max(max((int)(int8_t)mx4, (int)(int8_t)(mx4 >> 8)), max((int)(int8_t)(mx4 >> 16), (int)(int8_t)(mx4 >> 24)));
-    mx = warp_max(mx);
-    // pass 2: sum of ShiftExp(I - I_max)
-    unsigned sum = 0;
+      mxu = __reduce_max_sync(0xffffffffu, mxu);   // biased maximum = I_max + 128
+      // pass 2: sum of ShiftExp(I - I_max): entry (I_max + 128) - u
+      const uint8_t* tmx = reinterpret_cast<const uint8_t*>(exp_tab) + 4 * mxu;
+      unsigned sum = 0;
 #pragma unroll
-    for (int i = 0; i < iters; ++i) {
-      const int idx = lane + 32 * i;
-      if (idx < nwords) {
-        const int v = WPL > 0 ? w[i] : ld.load(r, idx);
-#pragma unroll
-        for (int b = 0; b < 4; ++b)
-          if (idx * 4 + b < d) sum += exp_tab[mx - (int)(int8_t)(v >> (8 * b))];
+      for (int i = 0; i < iters; ++i) {
+        const unsigned v = WPL > 0 ? w[i] : load_biased(r, lane + 32 * i);
+        unsigned e0 = *reinterpret_cast<const unsigned*>(tmx - 4 * (int)__byte_perm(v, 0, 0x4440));
+        unsigned e1 = *reinterpret_cast<const unsigned*>(tmx - 4 * (int)__byte_perm(v, 0, 0x4441));
+        unsigned e2 = *reinterpret_cast<const unsigned*>(tmx - 4 * (int)__byte_perm(v, 0, 0x4442));
+        unsigned e3 = *reinterpret_cast<const unsigned*>(tmx - 4 * (int)(v >> 24));
+        if (WPL > 0) { e[q][i][0] = e0; e[q][i][1] = e1; e[q][i][2] = e2; e[q][i][3] = e3; }
+        sum += (e0 + e1) + (e2 + e3);
       }
+      sum = __reduce_add_sync(0xffffffffu, sum);
+      // every position past d of the 32 * iters words counted exp_tab[I_max + 128]: take them out
+      sum -= (unsigned)(32 * iters * 4 - d) * exp_tab[mxu];
+      if (lane == q) { my_sum = sum; my_mxu = mxu; }
     }
-    sum = warp_sum_u(sum);
-    // Eq. (IntDiv): one reciprocal per row, M = 45, k_out = 8:
+    // Eq. (IntDiv): one reciprocal per row (lane q for row q), M = 45, k_out = 8:
     // (floor(2^45 / sum) * e) >> 38 == umulhi(factor, e) >> 6 since factor <= 2^31.
-    const unsigned factor = (unsigned)((1ull << 45) / (unsigned long long)sum);
-    int* dst = reinterpret_cast<int*>(out + r * ldout);
+    const unsigned my_factor = (unsigned)((1ull << 45) / (unsigned long long)my_sum);
 #pragma unroll
-    for (int i = 0; i < iters; ++i) {
-      const int idx = lane + 32 * i;
-      if (idx < nwords_out) {
-        unsigned packed = 0;
-        if (idx < nwords) {
-          const int v = WPL > 0 ? w[i] : ld.load(r, idx);
+    for (int q = 0; q < R; ++q) {
+      const unsigned factor = __shfl_sync(0xffffffffu, my_factor, q);
+      const unsigned mxu = __shfl_sync(0xffffffffu, my_mxu, q);
+      const int64_t r = r0 + q;
+      if (r >= rows) break;
+      const uint8_t* tmx = reinterpret_cast<const uint8_t*>(exp_tab) + 4 * mxu;
+      int* dst = reinterpret_cast<int*>(out + r * ldout);
 #pragma unroll
-          for (int b = 0; b < 4; ++b) {
-            if (idx * 4 + b < d) {
-              const unsigned e = exp_tab[mx - (int)(int8_t)(v >> (8 * b))];
-              const unsigned o = min(127u, __umulhi(factor, e) >> 6);
-              packed |= o << (8 * b);
-            }
+      for (int i = 0; i < iters; ++i) {
+        const int idx = lane + 32 * i;
+        if (idx < nwords_out) {
+          unsigned e0, e1, e2, e3;
+          if (WPL > 0) {
+            e0 = e[q][i][0]; e1 = e[q][i][1]; e2 = e[q][i][2]; e3 = e[q][i][3];
+          } else {
+            const unsigned v = load_biased(r, idx);
+            e0 = *reinterpret_cast<const unsigned*>(tmx - 4 * (int)__byte_perm(v, 0, 0x4440));
+            e1 = *reinterpret_cast<const unsigned*>(tmx - 4 * (int)__byte_perm(v, 0, 0x4441));
+            e2 = *reinterpret_cast<const unsigned*>(tmx - 4 * (int)__byte_perm(v, 0, 0x4442));
+            e3 = *reinterpret_cast<const unsigned*>(tmx - 4 * (int)(v >> 24));
           }
+          // values are <= 128: the saturating pack clamps the one possible 128 to 127
+          unsigned packed = pack_sat8_u((int)(__umulhi(factor, e0) >> 6), (int)(__umulhi(factor, e1) >> 6),
+                                        (int)(__umulhi(factor, e2) >> 6), (int)(__umulhi(factor, e3) >> 6));
+          // positions past d are written as zero
+          if (idx >= nwords) packed = 0;
+          else if (idx == nwords - 1 && npad) packed &= 0xffffffffu >> (8 * npad);
+          dst[idx] = (int)packed;
         }
-        dst[idx] = (int)packed;
       }
     }
   }
@@ -467,11 +499,11 @@ template <bool FROM_I32>
 static void shiftmax_dispatch(RowLoader<FROM_I32> ld, ivit_exp_params p, int8_t* out, int64_t ldout,
                               int64_t rows, int d, int grid, cudaStream_t st) {
   const int wpl = (((d + 15) / 16) * 4 + 31) / 32;
-  if (wpl <= 2) launch_k(shiftmax_kernel<2, FROM_I32>, dim3(grid), dim3(256), 0, st, ld, p, out, ldout, rows, d);
-  else if (wpl <= 5) launch_k(shiftmax_kernel<5, FROM_I32>, dim3(grid), dim3(256), 0, st, ld, p, out, ldout, rows, d);
-  else if (wpl <= 8) launch_k(shiftmax_kernel<8, FROM_I32>, dim3(grid), dim3(256), 0, st, ld, p, out, ldout, rows, d);
-  else if (wpl <= 16) launch_k(shiftmax_kernel<16, FROM_I32>, dim3(grid), dim3(256), 0, st, ld, p, out, ldout, rows, d);
-  else launch_k(shiftmax_kernel<0, FROM_I32>, dim3(grid), dim3(256), 0, st, ld, p, out, ldout, rows, d);
+  if (wpl <= 2) launch_k(shiftmax_kernel<2, 4, FROM_I32>, dim3(grid), dim3(256), 0, st, ld, p, out, ldout, rows, d);
+  else if (wpl <= 5) launch_k(shiftmax_kernel<5, 2, FROM_I32>, dim3(grid), dim3(256), 0, st, ld, p, out, ldout, rows, d);
+  else if (wpl <= 8) launch_k(shiftmax_kernel<8, 1, FROM_I32>, dim3(grid), dim3(256), 0, st, ld, p, out, ldout, rows, d);
+  else if (wpl <= 16) launch_k(shiftmax_kernel<16, 1, FROM_I32>, dim3(grid), dim3(256), 0, st, ld, p, out, ldout, rows, d);
+  else launch_k(shiftmax_kernel<0, 1, FROM_I32>, dim3(grid), dim3(256), 0, st, ld, p, out, ldout, rows, d);
 }
 
 int launch_shiftmax(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, const int32_t* bias32,
