@@ -126,27 +126,22 @@ __global__ void __launch_bounds__(256) layernorm_i8_kernel(const int8_t* __restr
 // at once instead of redundantly by all 32, and the per-channel constants of the lane's channels
 // are loaded once for all ROWS rows: v = ((x*F - mu*F) * m + 2^(s-1)) >> s + beta.
 // mean_magic = floor(2^32 / (2C)) + 1 turns the mean's division into a multiplication (exact for the
-// numerators of int8 rows, which stay below 2^18).
-template <int WPL, int ROWS>
-__global__ void __launch_bounds__(128, 6) layernorm_i8_batched_kernel(const int8_t* __restrict__ in, int64_t ldin,
+// numerators of int8 rows of up to 1024 channels, which stay below 2^19).
+// SMEMC: the per-channel constants live in shared memory (rows too wide for registers), set up once per block.
+template <int WPL, int ROWS, bool SMEMC>
+__global__ void __launch_bounds__(128, SMEMC ? 4 : 6) layernorm_i8_batched_kernel(const int8_t* __restrict__ in, int64_t ldin,
                                                                       ScaleDev gs, const int32_t* __restrict__ beta,
                                                                       int M_ln, int8_t* __restrict__ out, int64_t ldout,
                                                                       int64_t rows, int C, unsigned mean_magic, int vec) {
+  extern __shared__ int4 ln_consts[];   // SMEMC: [3][C / 4] multipliers, shifts, addends (or betas)
   pdl_trigger();
   pdl_wait();
   const int lane = threadIdx.x & 31;
   const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
   const int nwords = C >> 2;
-  // constants of this lane's channels (word i of the lane covers channels 4*(lane+32i) .. +3)
-  int pm[WPL][4], ps[WPL][4], pb[WPL][4];
-  // Fast form, taken when it is exact for every channel of the warp: with s >= 33 the rounding constant
-  // 2^(s-1) is a multiple of 2^32, so (yF m + 2^(s-1)) >> s = (hi32(yF m) + 2^(s-33)) >> (s - 32), and beta
-  // joins the constant as beta 2^(s-32) when that stays far from 32 bits (|hi32| < 2^21 here).
-  bool fast = true;
-#pragma unroll
-  for (int i = 0; i < WPL; ++i) {
-    const int idx = lane + 32 * i;
+  // constants of four channels (one word of the row)
+  auto load_consts = [&](int idx, int (&m)[4], int (&sft)[4], int (&b)[4]) {
     if (vec) {
       // per-channel arrays aligned for one 16-byte (4-byte for the shifts) load per word of four channels
       int4 m4 = make_int4(1, 1, 1, 1), b4 = make_int4(0, 0, 0, 0);
@@ -156,34 +151,67 @@ __global__ void __launch_bounds__(128, 6) layernorm_i8_batched_kernel(const int8
         s4 = __ldg(reinterpret_cast<const uchar4*>(gs.shift_c) + idx);
         if (beta) b4 = __ldg(reinterpret_cast<const int4*>(beta) + idx);
       }
-      pm[i][0] = m4.x; pm[i][1] = m4.y; pm[i][2] = m4.z; pm[i][3] = m4.w;
-      ps[i][0] = clamp_shift(s4.x); ps[i][1] = clamp_shift(s4.y); ps[i][2] = clamp_shift(s4.z); ps[i][3] = clamp_shift(s4.w);
-      pb[i][0] = b4.x; pb[i][1] = b4.y; pb[i][2] = b4.z; pb[i][3] = b4.w;
+      m[0] = m4.x; m[1] = m4.y; m[2] = m4.z; m[3] = m4.w;
+      sft[0] = clamp_shift(s4.x); sft[1] = clamp_shift(s4.y); sft[2] = clamp_shift(s4.z); sft[3] = clamp_shift(s4.w);
+      b[0] = b4.x; b[1] = b4.y; b[2] = b4.z; b[3] = b4.w;
     } else {
 #pragma unroll
-      for (int b = 0; b < 4; ++b) {
-        const int c = idx * 4 + b;
-        pm[i][b] = idx < nwords ? gs.m(c) : 1;
-        ps[i][b] = idx < nwords ? gs.s(c) : 40;
-        pb[i][b] = (idx < nwords && beta) ? __ldg(beta + c) : 0;
+      for (int k = 0; k < 4; ++k) {
+        const int c = idx * 4 + k;
+        m[k] = idx < nwords ? gs.m(c) : 1;
+        sft[k] = idx < nwords ? gs.s(c) : 40;
+        b[k] = (idx < nwords && beta) ? __ldg(beta + c) : 0;
       }
     }
+  };
+  // Fast form, taken when it is exact for every channel: with s >= 33 the rounding constant 2^(s-1) is a
+  // multiple of 2^32, so (yF m + 2^(s-1)) >> s = (hi32(yF m) + 2^(s-33)) >> (s - 32), and beta joins the
+  // constant as beta 2^(s-32) when that stays far from 32 bits (|hi32| < 2^21 here).
+  auto fast_ok = [](const int (&sft)[4], const int (&b)[4]) {
+    bool f = true;
 #pragma unroll
-    for (int b = 0; b < 4; ++b) {
-      const int sh = ps[i][b] - 32;
-      fast = fast && sh >= 1 && pb[i][b] > -(1 << (29 - sh)) && pb[i][b] < (1 << (29 - sh));
+    for (int k = 0; k < 4; ++k) {
+      const int sh = sft[k] - 32;
+      f = f && sh >= 1 && b[k] > -(1 << (29 - sh)) && b[k] < (1 << (29 - sh));
     }
-  }
-  fast = __all_sync(0xffffffffu, fast);
-  if (fast) {
-    // keep s - 32 and the combined constant instead of s and beta
+    return f;
+  };
+  // the fast form keeps s - 32 and the combined constant instead of s and beta
+  auto to_fast = [](int (&sft)[4], int (&b)[4]) {
 #pragma unroll
-    for (int i = 0; i < WPL; ++i)
+    for (int k = 0; k < 4; ++k) {
+      sft[k] -= 32;
+      b[k] = (1 << (sft[k] - 1)) + b[k] * (1 << sft[k]);
+    }
+  };
+  constexpr int WR = SMEMC ? 1 : WPL;
+  int pm[WR][4], ps[WR][4], pb[WR][4];   // registers: the constants of this lane's channels
+  bool fast = true;
+  if (SMEMC) {
+    for (int idx = threadIdx.x; idx < nwords; idx += blockDim.x) {
+      load_consts(idx, pm[0], ps[0], pb[0]);
+      fast = fast && fast_ok(ps[0], pb[0]);
+    }
+    fast = __syncthreads_and(fast) != 0;
+    for (int idx = threadIdx.x; idx < nwords; idx += blockDim.x) {
+      load_consts(idx, pm[0], ps[0], pb[0]);
+      if (fast) to_fast(ps[0], pb[0]);
+      ln_consts[idx] = make_int4(pm[0][0], pm[0][1], pm[0][2], pm[0][3]);
+      ln_consts[nwords + idx] = make_int4(ps[0][0], ps[0][1], ps[0][2], ps[0][3]);
+      ln_consts[2 * nwords + idx] = make_int4(pb[0][0], pb[0][1], pb[0][2], pb[0][3]);
+    }
+    __syncthreads();
+  } else {
 #pragma unroll
-      for (int b = 0; b < 4; ++b) {
-        ps[i][b] -= 32;
-        pb[i][b] = (1 << (ps[i][b] - 1)) + pb[i][b] * (1 << ps[i][b]);
-      }
+    for (int i = 0; i < WR; ++i) {
+      load_consts(lane + 32 * i, pm[i], ps[i], pb[i]);
+      fast = fast && fast_ok(ps[i], pb[i]);
+    }
+    fast = __all_sync(0xffffffffu, fast);
+    if (fast) {
+#pragma unroll
+      for (int i = 0; i < WR; ++i) to_fast(ps[i], pb[i]);
+    }
   }
   for (int64_t r0 = warp * ROWS; r0 < rows; r0 += nwarps * ROWS) {
     int w[ROWS][WPL];
@@ -212,7 +240,7 @@ __global__ void __launch_bounds__(128, 6) layernorm_i8_batched_kernel(const int8
     }
     // lane r (< ROWS) holds the sums of row r0 + r: mean (round half up) = floor((2 S1 + C) / 2C), taken on the
     // numerator shifted by 256 C to make it positive; sum of squared deviations = sum x^2 - 2 mu sum x + C mu^2
-    // (every term below 2^25 for int8 rows of up to 512 channels); integer square root; reciprocal
+    // (every term below 2^26 for int8 rows of up to 1024 channels); integer square root; reciprocal
     const int mu = (int)__umulhi((unsigned)(2 * my_s1 + 257 * C), mean_magic) - 128;
     const int V = my_s2 - 2 * mu * my_s1 + C * mu * mu;
     const unsigned sd = isqrt_u32((unsigned)V);
@@ -228,6 +256,16 @@ __global__ void __launch_bounds__(128, 6) layernorm_i8_batched_kernel(const int8
         for (int i = 0; i < WPL; ++i) {
           const int idx = lane + 32 * i;
           if (idx < nwords) {
+            int cm[4], cs[4], cb[4];
+            if (SMEMC) {
+              const int4 m4 = ln_consts[idx], s4 = ln_consts[nwords + idx], b4 = ln_consts[2 * nwords + idx];
+              cm[0] = m4.x; cm[1] = m4.y; cm[2] = m4.z; cm[3] = m4.w;
+              cs[0] = s4.x; cs[1] = s4.y; cs[2] = s4.z; cs[3] = s4.w;
+              cb[0] = b4.x; cb[1] = b4.y; cb[2] = b4.z; cb[3] = b4.w;
+            } else {
+#pragma unroll
+              for (int b = 0; b < 4; ++b) { cm[b] = pm[SMEMC ? 0 : i][b]; cs[b] = ps[SMEMC ? 0 : i][b]; cb[b] = pb[SMEMC ? 0 : i][b]; }
+            }
             int v[4];
 #pragma unroll
             for (int b = 0; b < 4; ++b) {
@@ -237,9 +275,9 @@ __global__ void __launch_bounds__(128, 6) layernorm_i8_batched_kernel(const int8
               // (x - mu) * F, formed modulo 2^32 (the difference always fits: |y F| <= 2^(M_ln+1))
               const int yF = (int)((unsigned)x * (unsigned)Fr - (unsigned)muFr);
               if (fast) {
-                v[b] = (__mulhi(yF, pm[i][b]) + pb[i][b]) >> ps[i][b];
+                v[b] = (__mulhi(yF, cm[b]) + cb[b]) >> cs[b];
               } else {
-                v[b] = rq(yF, pm[i][b], ps[i][b]) + pb[i][b];
+                v[b] = rq(yF, cm[b], cs[b]) + cb[b];
               }
             }
             unsigned t, d;
@@ -344,20 +382,23 @@ int launch_layernorm(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, 
   }
   const int8_t* x = (const int8_t*)in;
   const int wpl = (int)((C / 4 + 31) / 32);
-  if (wpl <= 4) {
-    // batched kernel: 4 rows per warp amortise the per-row scalar work and the per-channel constants;
-    // 128-thread blocks, six of them resident per SM
-    const int rpw = 4, tb = 128;
+  if (wpl <= 8) {
+    // batched kernel: 16 to 2 rows per warp, fewer for wider rows, amortise the per-row scalar work and the
+    // per-channel constants (in registers up to 512 channels, in shared memory up to 1024); 128-thread blocks
+    const int rpw = wpl <= 1 ? 16 : (wpl <= 2 ? 8 : (wpl <= 4 ? 4 : 2)), tb = 128;
     const int64_t warps = (rows + rpw - 1) / rpw;
     const int64_t wantb = (warps + tb / 32 - 1) / (tb / 32);
     const int gridb = (int)(wantb < (int64_t)ctx->sm_count * 12 ? wantb : (int64_t)ctx->sm_count * 12);
     const unsigned magic = (unsigned)(0x100000000ull / (unsigned long long)(2 * C)) + 1u;
     const int vec = gs.mult_c && gs.shift_c && !(reinterpret_cast<uintptr_t>(gs.mult_c) & 15) && !(reinterpret_cast<uintptr_t>(gs.shift_c) & 3) &&
                     !(reinterpret_cast<uintptr_t>(beta) & 15);
-    if (wpl <= 1) launch_k(layernorm_i8_batched_kernel<1, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
-    else if (wpl <= 2) launch_k(layernorm_i8_batched_kernel<2, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
-    else if (wpl <= 3) launch_k(layernorm_i8_batched_kernel<3, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
-    else launch_k(layernorm_i8_batched_kernel<4, 4>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
+    const size_t cbytes = (size_t)(C / 4) * 3 * sizeof(int4);
+    if (wpl <= 1) launch_k(layernorm_i8_batched_kernel<1, 16, false>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
+    else if (wpl <= 2) launch_k(layernorm_i8_batched_kernel<2, 8, false>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
+    else if (wpl <= 3) launch_k(layernorm_i8_batched_kernel<3, 4, false>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
+    else if (wpl <= 4) launch_k(layernorm_i8_batched_kernel<4, 4, false>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
+    else if (wpl <= 6) launch_k(layernorm_i8_batched_kernel<6, 2, true>, dim3(gridb), dim3(tb), cbytes, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
+    else launch_k(layernorm_i8_batched_kernel<8, 2, true>, dim3(gridb), dim3(tb), cbytes, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
     return ls.done();
   }
   if (wpl <= 6) launch_k(layernorm_i8_kernel<6>, dim3(grid), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);

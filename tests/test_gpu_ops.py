@@ -205,7 +205,7 @@ def test_shiftgelu_parity(rows, cols, I0):
     g.assert_equal(g.host(dx), want, "shiftgelu in place")
 
 
-@pytest.mark.parametrize("rows,C", [(1, 16), (197, 192), (500, 384), (300, 768), (100, 1024), (50, 96), (20, 1536),
+@pytest.mark.parametrize("rows,C", [(1, 16), (197, 192), (500, 384), (301, 768), (100, 1024), (5, 520), (50, 96), (67, 128), (20, 1536),
                                     (9, 3072), (3, 16384), (11, 4)])
 def test_layernorm_parity(rows, C):
     g = _g()
