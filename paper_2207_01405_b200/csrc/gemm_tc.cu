@@ -619,8 +619,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
             for (int j = 0; j < 32; ++j)
               if (j < ncol) v[j] += __ldg(bias_row + c0 + j);
           }
+          if (us >= 33) {   // the usual case: high product word plus 2^(s-33), shifted by s - 32
+            const int u_rnd = 1 << (us - 33), u_sh = us - 32;
 #pragma unroll
-          for (int j = 0; j < 32; ++j) v[j] = (int)(((long long)v[j] * um + uc) >> us);
+            for (int j = 0; j < 32; ++j) v[j] = mad_hi(v[j], um, u_rnd) >> u_sh;
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) v[j] = (int)(((long long)v[j] * um + uc) >> us);
+          }
           int8_t* o = reinterpret_cast<int8_t*>(e.out) + out_row + c0;
           if (ncol == 32) {
             int4 w0, w1;
