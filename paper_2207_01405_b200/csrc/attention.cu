@@ -21,16 +21,6 @@ namespace {
 constexpr int kAttnThreads = 288;   // warp 0: TMA + MMA issue + TMEM owner; warps 1..8: two threads per score row
 constexpr int UK = 32;              // K of one tcgen05.mma.kind::i8
 
-#ifdef IVIT_ATTN_TRACE
-// debugging aid (compiled out by default): clock64() stamps of the phases of the first CTAs
-__device__ long long g_attn_trace[64][12];
-__device__ unsigned long long g_attn_span[1024][3];   // per CTA: global ns at start, at end, SM id
-#define ATRACE(i) do { if (blockIdx.x < 64) g_attn_trace[blockIdx.x][i] = clock64(); \
-  if ((i) == 0 || (i) == 9) { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); unsigned sm; asm volatile("mov.u32 %0, %%smid;" : "=r"(sm)); \
-    if (blockIdx.x < 1024) { g_attn_span[blockIdx.x][(i) == 0 ? 0 : 1] = t; g_attn_span[blockIdx.x][2] = sm; } } } while (0)
-#else
-#define ATRACE(i) do { } while (0)
-#endif
 
 struct AttnArgs {
   int T, d, heads, Npad;            // Npad = T rounded up to 32 (score columns and P.V contraction length)
@@ -80,7 +70,6 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   if (threadIdx.x == 0) {
-    ATRACE(0);
     prefetch_tmap(&tmQ);
     prefetch_tmap(&tmK);
     prefetch_tmap(&tmV);
@@ -111,7 +100,6 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
   // item -> (tile, image/window * heads + head): all first tiles before all second tiles
   if (warp == 0) {
     if (lane == 0) {
-      ATRACE(1);
       auto load_qk = [&](int item) {
         const int tile = item / a.bh, bhid = item - tile * a.bh;
         const int h = bhid % a.heads, b = bhid / a.heads;
@@ -157,7 +145,6 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
         // the output of the previous item must have left tensor memory
         if (ok && n > 0) ok = mbar_wait(bar_e, par ^ 1u, a.status);
         if (!ok) break;
-        ATRACE(2);
         tc_fence_after();
         for (int k = 0; k < ks; ++k)
           umma_i8(tmem, smem_desc(base + q_off + k * UK, 16, 1024, 2), smem_desc(base + k_off + k * UK, 16, 1024, 2),
@@ -172,7 +159,6 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
         ok = mbar_wait(bar_p, par, a.status);
         if (ok) { ok = mbar_wait(bar_v, par, a.status); v_flying = !ok; }
         if (!ok) break;
-        ATRACE(7);
         tc_fence_after();
         for (int k = 0; k < ks2; ++k) {
           const uint32_t pa = base + p_off + (k >> 2) * (128 * 128) + (k & 3) * UK;
@@ -187,9 +173,6 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
         item = next;
       }
       // end of work (or a wait that timed out): tell the other warps; nothing may be in flight at exit
-#ifdef IVIT_ATTN_TRACE
-      if (blockIdx.x < 64) g_attn_trace[blockIdx.x][10] = n;
-#endif
       publish(ok ? n : n + 1, -1);
       if (qk_flying) mbar_wait(bar_qk, qk_par, a.status);
       if (v_flying) mbar_wait(bar_v, v_par, a.status);
@@ -234,7 +217,6 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
       bool got_s = mbar_wait(bar_s, par, a.status);
       alive = alive && got_s;
       if (got_s) tc_fence_after();
-      if (st == 0) ATRACE(3);
       if (got_s && warp_ok) {
         // pass A: requantise the scores to int8 (Sec. 3.2), running maximum.  The two threads of a row take
         // alternate 16-column chunks (Npad / 16 is even: equal shares).  The chunk loops are rolled (the kernel's
@@ -280,7 +262,6 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
         part_max[half * 128 + trow] = mx;
       }
       asm volatile("bar.sync 1, 256;" ::: "memory");
-      if (st == 0) ATRACE(4);
       unsigned sum = 0;
       if (got_s && warp_ok) {
         mx = max(part_max[trow], part_max[128 + trow]);
@@ -312,7 +293,6 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
         part_sum[half * 128 + trow] = sum;
       }
       asm volatile("bar.sync 1, 256;" ::: "memory");
-      if (st == 0) ATRACE(5);
       if (got_s && warp_ok) {
         sum = part_sum[trow] + part_sum[128 + trow];
         // pass C: Eq. (IntDiv) with M = 45, k_out = 8: (floor(2^45 / sum) * e) >> 38 = umulhi(factor, e) >> 6
@@ -335,13 +315,11 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_p);
-      if (st == 0) ATRACE(6);
       // ---- output: O = sat8(rq(P V; pv_scale)), heads concatenated along the feature dimension ----
       const bool got_o = alive && mbar_wait(bar_o, par, a.status);
       alive = alive && got_o;
       if (got_o) {
         tc_fence_after();
-        if (st == 0) ATRACE(8);
         const long long pv_c = 1ll << (a.pv_s - 1);
         int8_t* orow = a.O + ((int64_t)b * a.T + r) * a.D + (int64_t)h * a.d;
         for (int c = half; c < a.d / 32; c += 2) {
@@ -370,7 +348,6 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0) {
-    ATRACE(9);
     // the last CTA to finish leaves the counters at zero for the next launch
     __threadfence();
     if (atomicAdd(a.sched + 1, 1u) == gridDim.x - 1) {

@@ -101,16 +101,6 @@ struct TcArgs {
   int* status;
 };
 
-#ifdef IVIT_TC_TRACE
-// debugging aid (compiled out by default): per-CTA, per-tile clock64() stamps of each role
-__device__ long long g_trace[148][40][8];
-#define IVIT_TRACE(tile_it, idx) do { if ((tile_it) < 40 && blockIdx.x < 148) g_trace[blockIdx.x][tile_it][idx] = clock64(); } while (0)
-__device__ long long g_trace2[148][4][16];
-#define IVIT_TRACE2(cond, ckk, idx) do { const int i_ = (idx); if ((cond) && i_ < 16) g_trace2[blockIdx.x][ckk][i_] = clock64(); } while (0)
-#else
-#define IVIT_TRACE2(cond, ckk, idx) do { } while (0)
-#define IVIT_TRACE(tile_it, idx) do { } while (0)
-#endif
 
 struct TileCoord {
   int64_t batch;
@@ -163,9 +153,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
                                                               const __grid_constant__ CUtensorMap tmO,
                                                               const __grid_constant__ CUtensorMap tmR, TcArgs a) {
   extern __shared__ __align__(1024) uint8_t smem_raw[];
-#ifdef IVIT_TC_TRACE
-  if (threadIdx.x == 0) { IVIT_TRACE(39, 0); long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); g_trace[blockIdx.x][39][4] = g; }
-#endif
   // carve: [stages x (P tile | Q tile)] [barriers] [tmem address, issued count]
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
@@ -215,36 +202,19 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       fence_async_smem();
     }
   }
-#ifdef IVIT_TC_TRACE
-  if (threadIdx.x == 64) IVIT_TRACE(38, 0);
-  if (threadIdx.x == 32) IVIT_TRACE(38, 1);
-#endif
   if (warp == 1) tmem_alloc(smem_u32(tmem_slot), (uint32_t)a.tmem_cols);
-#ifdef IVIT_TC_TRACE
-  if (threadIdx.x == 32) IVIT_TRACE(38, 2);
-#endif
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   // set-up done (barriers, tensor memory, descriptor prefetch): let the next kernel be scheduled, then wait
   // for the previous kernel's results before touching global memory
-#ifdef IVIT_TC_TRACE
-  if (threadIdx.x == 0) IVIT_TRACE(39, 1);
-#endif
   pdl_trigger();
   pdl_wait();
-#ifdef IVIT_TC_TRACE
-  if (threadIdx.x == 0) IVIT_TRACE(39, 2);
-#endif
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
-#ifdef IVIT_DBG_NOMMA
-    if (false) {
-#else
     if (lane == 0) {
-#endif
       int issued = 0;            // k-blocks issued so far, over all tiles of this CTA
       int s = 0, wrap = 0;       // ring slot of the next k-block and how often the ring has wrapped
       bool ok = true;
@@ -255,7 +225,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       const int pr = a.p_pos[0], pbi = a.p_pos[1], qr = a.q_pos[0], qbi = a.q_pos[1];
       for (int64_t t = t_begin; ok && t < t_end; ++t, ++pit, ti.next(a)) {
         const int p0 = ti.p0(), q0 = ti.q0(a);
-        IVIT_TRACE(pit, 0);
         const int pc1 = pr == 1 ? p0 : (pbi == 1 ? ti.bi : ti.bo), pc2 = pr == 2 ? p0 : (pbi == 2 ? ti.bi : ti.bo),
                   pc3 = pr == 3 ? p0 : (pbi == 3 ? ti.bi : ti.bo);
         bool bring_q = false;
@@ -309,11 +278,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       for (int64_t t = t_begin; ok && t < t_end; ++t, ++it) {
         const int buf = it & 1;
         bool last_of_q = false;
-#ifdef IVIT_DBG_NOMMA
-        if (false) {
-#else
         if (a.q_resident) {
-#endif
           // a new activation row block arrives k-block by k-block on the stage barriers of this tile
           cur_q = ti.q0(a);
           ti.next(a);
@@ -322,15 +287,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         // the epilogue must have drained this buffer (its use two tiles ago)
         if (it >= 2 && !mbar_wait(acce0 + 8 * buf, ((it >> 1) & 1) ^ 1, a.status)) { ok = false; break; }
         tc_fence_after();
-        IVIT_TRACE(it, 1);
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * a.BN);
         for (int kb = 0; kb < kblocks; ++kb) {
-#ifdef IVIT_DBG_NOMMA
-          continue;
-#endif
           if (!mbar_wait(full0 + 8 * s, wrap & 1, a.status)) { ok = false; break; }
           tc_fence_after();
-          if (kb == 0) IVIT_TRACE(it, 2);
           const uint32_t sp = base + s * stage_bytes, sq = a.q_resident ? qres + kb * a.q_stage_bytes : sp + BM * BK;
           uint32_t p_lo = desc_lo(sp, 16), q_lo = desc_lo(sq, 16);
           const int ksteps = kb == kblocks - 1 ? tail_steps : BK / UMMA_K;
@@ -345,7 +305,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         }
         if (ok) umma_commit(accf0 + 8 * buf);  // accumulator of this tile complete
         if (ok && last_of_q) umma_commit(qrese);   // the resident tile may be replaced once these MMAs are done
-        IVIT_TRACE(it, 3);
       }
       if (!ok) {
         // drain: copies that were issued but never consumed (only after a timeout)
@@ -444,7 +403,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     ti.init(a, t_begin);
     for (int64_t t = t_begin; t < t_end; ++t, ++it) {
       TileCoord tc;
-      if (et == 0) IVIT_TRACE(it, 6);
       tc.batch = ti.batch; tc.bo = ti.bo; tc.bi = ti.bi; tc.p0 = ti.p0(); tc.q0 = ti.q0(a);
       ti.next(a);   // ti now describes the next tile
       const int buf = it & 1;
@@ -458,10 +416,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       const int rnd_hi = cs >= 33 ? 1 << (cs - 33) : 0;
       if (dense && t + 1 < t_end) fetch_channel(ti.p0());
 
-      if (et == 0) IVIT_TRACE(it, 7);
       if (ok) ok = mbar_wait(accf0 + 8 * buf, (it >> 1) & 1, a.status);
       tc_fence_after();
-      if (et == 0) IVIT_TRACE(it, 4);
       const uint32_t t_row = tmem_base + ((uint32_t)(qd * 32) << 16) + (uint32_t)(buf * a.BN);
       const int64_t cols_left = a.Q - tc.q0;
       const int nck = (int)((cols_left < a.BN ? cols_left : a.BN) + 31) >> 5;   // chunks that hold output
@@ -643,12 +599,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
           }
         }
       }
-      if (et == 0) IVIT_TRACE(it, 0);
       // this warp has read everything it needs from the buffer: hand it back to the MMA warp
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(acce0 + 8 * buf);
-      if (et == 0) IVIT_TRACE(it, 5);
     }
     if (tma_out && lane == 0) tma_store_wait_all();
     // only after a timeout: residual bytes fetched for chunks that were never worked on may be in flight
@@ -662,9 +616,6 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     tc_fence_after();
     tmem_dealloc(tmem_base, (uint32_t)a.tmem_cols);
   }
-#ifdef IVIT_TC_TRACE
-  if (threadIdx.x == 0) { IVIT_TRACE(39, 3); long long g; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(g)); g_trace[blockIdx.x][39][5] = g; }
-#endif
 }
 
 // ---- host side ------------------------------------------------------------------------------
