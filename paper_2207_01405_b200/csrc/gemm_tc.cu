@@ -6,22 +6,26 @@
 //               mbarrier transaction counts);
 //   warp 1      owns tensor memory; one thread issues tcgen05.mma.kind::i8 (M = 128, N = BN,
 //               K = 32 per instruction) into one of two accumulator buffers;
-//   warps 2..17 epilogue: read the finished accumulator with tcgen05.ld (one TMEM lane per thread),
-//               requantise, add the residual, saturate and store - while the tensor core already
-//               works on the next tile in the other buffer.
+//   warps 2..17 epilogue (four per TMEM lane quarter): read the finished accumulator with tcgen05.ld (one
+//               TMEM lane per thread), requantise, add the residual, saturate and store - while the tensor
+//               core already works on the next tile in the other buffer.
 //
 // The 128 TMEM lanes of a tile hold the "P" operand's rows, the columns the "Q" operand's rows.
 //   * Dense layers (per-channel scale / bias):  P = weight rows (output channels), Q = activation
 //     rows.  A thread then owns ONE output channel: its multiplier, shift and bias stay in registers
-//     for the whole tile (no shared-memory traffic per value), and consecutive lanes touch
-//     consecutive channels of one output row, so residual loads and output stores coalesce.
+//     for the whole tile (no shared-memory traffic per value).  A warp turns its 32 channels x 32 rows
+//     into row-major bytes with 4x4 byte transposes (shuffles), stages them in a shared-memory slot
+//     of its own and stores the slot with a TMA store of its own; the residual bytes of the same
+//     32 x 32 piece arrive by TMA two chunks ahead.  No warp waits for another.
 //   * Batched MatMul (per-tensor scale): P = rows of A, Q = rows of B (K-major, Q K^T) or B is
 //     MN-major ([K, N] rows, P V; the V tile is consumed as stored, without a transpose).  A thread
 //     owns one output row and stores 32 consecutive int8 values per chunk.
 //
-// One CTA per SM walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...  Every device-side wait is
-// bounded: when one runs out the CTA records IVIT_ERR_DEVICE_TIMEOUT in the context's status
-// word, drains its outstanding copies, frees its tensor memory and returns.
+// One CTA per SM walks a contiguous range of tiles (channel blocks fastest, so that consecutive tiles
+// share their activation rows; for short K those rows stay resident in shared memory).  Every
+// device-side wait is bounded: when one runs out the thread records IVIT_ERR_DEVICE_TIMEOUT in the
+// context's status word, carries on without further waits, drains its outstanding copies, and the
+// CTA frees its tensor memory and returns.
 #include "tc_ptx.cuh"
 
 namespace ivit {
