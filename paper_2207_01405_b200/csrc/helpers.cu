@@ -30,6 +30,32 @@ __global__ void patchify_kernel(const int8_t* __restrict__ img, int64_t B, int C
   }
 }
 
+// P % 16 == 0, aligned image rows: one thread moves 16 bytes (px .. px+15 of one patch row) with 32-bit index
+// arithmetic; `segs` = P / 16 such pieces per patch row.
+__global__ void patchify_vec_kernel(const int8_t* __restrict__ img, int C, int Hi, int Wi, int P, int window,
+                                    int8_t* __restrict__ out, int64_t ldout, unsigned total_vecs) {
+  pdl_trigger();
+  pdl_wait();
+  const unsigned gh = Hi / P, gw = Wi / P, segs = P / 16;
+  const unsigned per_row = (unsigned)Wi / 16;          // 16-byte pieces per image row
+  for (unsigned t = blockIdx.x * blockDim.x + threadIdx.x; t < total_vecs; t += gridDim.x * blockDim.x) {
+    // t enumerates the image in memory order: consecutive threads read consecutive 16-byte pieces
+    const unsigned xv = t % per_row, line = t / per_row;          // line = (b * C + c) * Hi + y
+    const unsigned y = line % (unsigned)Hi, bc = line / (unsigned)Hi;
+    const unsigned c = bc % (unsigned)C, b = bc / (unsigned)C;
+    const unsigned gx = xv / segs, sx = xv % segs, gy = y / (unsigned)P, py = y % (unsigned)P;
+    const int4 v = __ldg(reinterpret_cast<const int4*>(img) + t);
+    unsigned row;
+    if (window > 0) {
+      const unsigned wy = gy / window, wx = gx / window, iy = gy % window, ix = gx % window;
+      row = (wy * (gw / window) + wx) * window * window + iy * window + ix;
+    } else {
+      row = gy * gw + gx;
+    }
+    *reinterpret_cast<int4*>(out + ((int64_t)b * gh * gw + row) * ldout + (c * P + py) * P + sx * 16) = v;
+  }
+}
+
 __global__ void gather_rows_kernel(const int8_t* __restrict__ src, int64_t ldsrc, const int32_t* __restrict__ index,
                                    int64_t n_rows, int vec_per_row, int8_t* __restrict__ dst, int64_t lddst) {
   pdl_trigger();
@@ -80,6 +106,12 @@ int launch_patchify(ivit_ctx* ctx, const int8_t* img, int64_t B, int64_t C, int6
   const int64_t total = B * C * Hi * Wi / 4;
   if (total == 0) return IVIT_OK;
   LaunchScope ls(ctx, KIND_MOVE, 2.0 * (double)total * 4);
+  if (P % 16 == 0 && Wi % 16 == 0 && ldout % 16 == 0 && total / 4 < 0x7fffffffLL && !(reinterpret_cast<uintptr_t>(img) & 15) &&
+      !(reinterpret_cast<uintptr_t>(out) & 15)) {
+    launch_k(patchify_vec_kernel, dim3(grid_for(ctx, total / 4, 256)), dim3(256), 0, ctx->stream, img, (int)C, (int)Hi, (int)Wi, (int)P,
+             (int)window, out, ldout, (unsigned)(total / 4));
+    return ls.done();
+  }
   launch_k(patchify_kernel, dim3(grid_for(ctx, total, 256)), dim3(256), 0, ctx->stream, img, B, (int)C, (int)Hi, (int)Wi, (int)P,
                                                                        (int)window, out, ldout, total);
   return ls.done();
