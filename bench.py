@@ -98,6 +98,38 @@ def measured_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "fallback"
 
 
+def gemm_probe(ctx, binding, peaks, dev):
+    """The Dense kernel alone on two tensor-bound shapes (ViT-B FC1 at batch 128, and 8192^3): back-to-back launches
+    between one pair of CUDA events, against the burst int8 peak (2 x the measured burst bf16 rate)."""
+    import numpy as np
+    import torch
+    from ivit_inputs import Scale
+    from ivit_inputs.gen import dyadic
+    out = []
+    rng = np.random.default_rng(0)
+    for M, N, K in ((25216, 3072, 768), (8192, 8192, 8192)):
+        A = torch.from_numpy(rng.integers(-127, 128, (M, K), dtype=np.int8)).to(dev)
+        W = torch.from_numpy(rng.integers(-127, 128, (N, K), dtype=np.int8)).to(dev)
+        sc = binding.DevScale(Scale(*dyadic(1.0 / (40.0 * 74.0 * np.sqrt(K)))), dev)
+        o = torch.empty((M, N), dtype=torch.int8, device=dev)
+        reps = 10
+        for _ in range(3):
+            ctx.linear(A, W, None, sc, out=o)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(reps):
+            ctx.linear(A, W, None, sc, out=o)
+        b.record()
+        torch.cuda.synchronize()
+        us = 1e3 * a.elapsed_time(b) / reps
+        tops = 2.0 * M * N * K / (us * 1e-6) / 1e12
+        out.append({"shape": f"{M}x{N}x{K}", "us": round(us, 2), "TOPS": round(tops, 1),
+                    "frac_of_burst_int8_peak": round(tops / (2.0 * peaks["bf16_tflops"]), 4)})
+        del A, W, o
+    return out
+
+
 def time_oracle(model, image, budget_s: float = 15.0):
     """Times the CPU oracle on a bounded sample of the workload's images; returns (images/s, n, seconds, threads)."""
     from oracle import api as O
@@ -290,6 +322,7 @@ def run_gpu(args):
         roofline = {"kernel": dom, "bound": "hbm", "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": round(achieved / peaks["hbm_gbs"], 4), "traffic": None, "peak_source": f"{peak_src} copy bandwidth"}
 
+    probe = gemm_probe(ctx, binding, peaks, dev)
     cpu_rate, cpu_n, cpu_s, cpu_threads = time_oracle(model, image)
     # the timed steps really computed the forward: spot-check one image against the oracle
     from oracle import api as O
@@ -311,6 +344,7 @@ def run_gpu(args):
         "roofline": roofline,
         "cpu_baseline": {"value": cpu_rate, "unit": "images/s", "cores": cpu_threads, "kind": "oracle",
                          "sample": f"{cpu_n} of {B} images ({cpu_s:.1f} s; images are independent)"},
+        "gemm_probe": probe,
         "int8_tops_whole_step": round(ops / (ms_total / args.steps * 1e-3) / 1e12, 2),
         "kernels": kernels,
         "parity_spot_check": ok,
