@@ -636,16 +636,25 @@ constexpr size_t kSmemFixed = 1024 + 8 * (2 * kMaxStages + 5 + 2 * kEpiWarps) + 
 bool g_attr_set = false;
 
 // Tile width along the TMEM columns: the candidate with the least (waves x tile cost).
-int pick_bn(int64_t extent, int64_t tiles_other, int sm_count) {
+// Tile width along the TMEM columns: the candidate with the least (rounds of tiles per CTA) x (time of a tile).
+// A tile's time is the larger of its operand traffic, (128 + bn) x K bytes at about 46 bytes per clock into an
+// SM's shared memory, and its epilogue, one 32-row chunk per epilogue part at a time (about 2000 clocks per round
+// of four chunks), plus a fixed cost per tile; the constants are measured on DeiT-S / ViT-B / ViT-L layer shapes.
+int pick_bn(int64_t extent, int64_t tiles_other, int64_t K, int sm_count) {
   if (extent <= 256) return (int)((extent + 31) / 32 * 32);
   int best = 0;
   double best_cost = 0;
   for (int bn : {256, 224, 192, 160, 128}) {
     const int64_t tiles = tiles_other * ((extent + bn - 1) / bn);
-    const double waves = (double)((tiles + sm_count - 1) / sm_count);
-    const double cost = waves * (bn + 24.0);
+    const double rounds = (double)((tiles + sm_count - 1) / sm_count);
+    const double feed = (double)K * (128.0 + bn) / 46.0;
+    const double epilogue = 2000.0 * ((bn + 127) / 128);
+    const double cost = rounds * ((feed > epilogue ? feed : epilogue) + 800.0);
     if (!best || cost < best_cost) { best = bn; best_cost = cost; }
   }
+#ifdef IVIT_TUNING
+  if (const char* f = getenv("IVIT_FORCE_BN")) return atoi(f);   // sweeps only
+#endif
   return best;
 }
 
@@ -671,7 +680,7 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
     a.lanes_are_channels = 1;
     a.P = g.N; a.Q = g.M;
     a.tiles_p = (int)((a.P + BM - 1) / BM);
-    a.BN = pick_bn(a.Q, a.tiles_p, ctx->sm_count);
+    a.BN = pick_bn(a.Q, a.tiles_p, g.K, ctx->sm_count);
     a.q_stage_bytes = a.BN * BK;
     if (!make_tensor_map(ctx, &tmP, g.B, g.K, g.N, 1, 1, g.ldb, 0, 0, BK, BM, CU_TENSOR_MAP_SWIZZLE_128B, a.p_pos) ||
         !make_tensor_map(ctx, &tmQ, g.A, g.K, g.M, 1, 1, g.lda, 0, 0, BK, a.BN, CU_TENSOR_MAP_SWIZZLE_128B, a.q_pos))
@@ -698,7 +707,7 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
                     swz, a.q_pos))
         return IVIT_ERR_UNSUPPORTED;
     } else {
-      a.BN = pick_bn(a.Q, (int64_t)a.tiles_p * batches, ctx->sm_count);
+      a.BN = pick_bn(a.Q, (int64_t)a.tiles_p * batches, g.K, ctx->sm_count);
       a.q_stage_bytes = a.BN * BK;
       if (!make_tensor_map(ctx, &tmQ, g.B, g.K, g.N, g.batches_inner, g.batches_outer, g.ldb, g.sBi, g.sBo, BK, a.BN,
                     CU_TENSOR_MAP_SWIZZLE_128B, a.q_pos))
