@@ -171,6 +171,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
   const uint32_t accf0 = empty0 + 8 * kMaxStages, acce0 = accf0 + 16, resf = acce0 + 16, qrese = resf + 16 * kEpiWarps;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + bars_off + 8 * (2 * kMaxStages + 5 + 2 * kEpiWarps));
   volatile int* issued_slot = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  // residual port: the requantised value of every int8 residual byte (256 entries, built below)
+  int8_t* res_tab = reinterpret_cast<int8_t*>(tmem_slot) + 32;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // this CTA's contiguous range of tiles
@@ -205,6 +207,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
       fence_async_smem();
     }
+    if (i >= 0 && i < 256 && a.epi.res) res_tab[i] = (int8_t)rq(i - 128, a.epi.res_scale.mult, clamp_shift(a.epi.res_scale.shift));
   }
   if (warp == 1) tmem_alloc(smem_u32(tmem_slot), (uint32_t)a.tmem_cols);
   tc_fence_before();
@@ -334,8 +337,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     const bool tma_res = MODE ? MODE == 2 : a.tma_res != 0;
     const bool ldg_res = MODE ? false : (e.res != nullptr && !a.tma_res);
     const bool out_i32 = MODE ? false : e.out_dtype == IVIT_I32;
-    const int rs_m = e.res_scale.mult, rs_s = clamp_shift(e.res_scale.shift);
-    const long long rs_c = 1ll << (rs_s - 1);
+    const int8_t* res_tab0 = res_tab + 128;   // entry of residual byte 0
     bool ok = true;
 
     // Dense orientation: constants of this thread's channel; fetched one tile ahead
@@ -460,19 +462,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
           if (tma_res) {
             // residual bytes of this chunk in shared memory: [row][32 channels]
             const uint8_t* rt = gen_base + (my_res - base) + (g & 1u) * 1024 + h * 512 + lane;
-            if (rs_s >= 32) {
 #pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                const int xr = (int)*reinterpret_cast<const int8_t*>(rt + j * 32);
-                v[j] += mad_wide_hi(xr, rs_m, rs_c) >> (rs_s - 32);
-              }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) {
-                const int xr = (int)*reinterpret_cast<const int8_t*>(rt + j * 32);
-                v[j] += (int)(mad_wide(xr, rs_m, rs_c) >> rs_s);
-              }
-            }
+            for (int j = 0; j < 16; ++j) v[j] += (int)res_tab0[(int)*reinterpret_cast<const int8_t*>(rt + j * 32)];
           } else if (ldg_res) {
             int64_t rr = (int64_t)((uint64_t)r0 % (uint64_t)e.res_rows);
 #pragma unroll
@@ -484,7 +475,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
                 if (++rr == e.res_rows) rr = 0;
               }
 #pragma unroll
-              for (int j = 0; j < 8; ++j) v[g + j] += (int)(mad_wide(xr[j], rs_m, rs_c) >> rs_s);
+              for (int j = 0; j < 8; ++j) v[g + j] += (int)res_tab0[xr[j]];
             }
           }
           if (out_i32) {
@@ -631,7 +622,7 @@ int pow2_at_least(int v) {
 }
 
 constexpr size_t kSmemBudget = 227 * 1024;
-constexpr size_t kSmemFixed = 1024 + 8 * (2 * kMaxStages + 5 + 2 * kEpiWarps) + 32;
+constexpr size_t kSmemFixed = 1024 + 8 * (2 * kMaxStages + 5 + 2 * kEpiWarps) + 32 + 256;
 
 bool g_attr_set = false;
 
