@@ -174,9 +174,55 @@ def merge_index(B: int, res: int, window: int) -> np.ndarray:
     return idx.reshape(-1)
 
 
+def _window_row(res: int, window: int, y: int, x: int) -> int:
+    """Row of token (y, x) of one image in window-major order."""
+    w = res // window
+    return ((y // window) * w + (x // window)) * window * window + (y % window) * window + (x % window)
+
+
+def shift_indices(B: int, res: int, window: int):
+    """Row permutations of a shifted-window block: the token grid is rolled by -(window // 2) in both directions
+    (the token at (y, x) of the rolled grid is the token at ((y + s) mod res, (x + s) mod res)), windows are then
+    taken on the rolled grid.  Returns (shift_index, unshift_index): X_rolled = X[shift_index],
+    X = X_rolled[unshift_index], both in window-major row order."""
+    s = window // 2
+    fwd = np.empty(res * res, dtype=np.int32)
+    for y in range(res):
+        for x in range(res):
+            fwd[_window_row(res, window, y, x)] = _window_row(res, window, (y + s) % res, (x + s) % res)
+    inv = np.empty_like(fwd)
+    inv[fwd] = np.arange(res * res, dtype=np.int32)
+    off = (np.arange(B, dtype=np.int32) * res * res)[:, None]
+    return (fwd[None, :] + off).reshape(-1), (inv[None, :] + off).reshape(-1)
+
+
+# added to the score accumulators of token pairs that the roll brought together from different sides of the
+# image: far below any score, so that the requantised score saturates at -128
+SHIFT_MASK = -(1 << 28)
+
+
+def shift_mask(res: int, window: int) -> np.ndarray:
+    """int32 [windows per image, T, T]: 0 where both tokens of a pair come from the same region of the rolled
+    grid, SHIFT_MASK elsewhere.  Regions: rows (and columns) [0, res-window), [res-window, res-s), [res-s, res)."""
+    s = window // 2
+    def band(v):
+        return 0 if v < res - window else (1 if v < res - s else 2)
+    w = res // window
+    T = window * window
+    m = np.zeros((w * w, T, T), dtype=np.int32)
+    for wy in range(w):
+        for wx in range(w):
+            reg = np.asarray([3 * band(wy * window + iy) + band(wx * window + ix)
+                              for iy in range(window) for ix in range(window)])
+            m[wy * w + wx] = np.where(reg[:, None] == reg[None, :], 0, SHIFT_MASK)
+    return m
+
+
 def make_swin(seed: int, B: int, img: int = 224, patch: int = 4, window: int = 7,
               dims=(96, 192, 384, 768), heads=(3, 6, 12, 24), depths=(2, 2, 6, 2),
-              classes: int = 1000) -> SwinParams:
+              classes: int = 1000, shifted: bool = False) -> SwinParams:
+    """shifted=True makes every second block of a stage a shifted-window block (cyclic roll by window // 2, mask
+    folded into the int32 score bias, one bias matrix per window position and head)."""
     ids = _Ids(seed)
     res = img // patch
     Wpe, bpe, pe_scale = _dense(ids, dims[0], 3 * patch * patch, 20.0, ACT_STD)
@@ -185,11 +231,21 @@ def make_swin(seed: int, B: int, img: int = 224, patch: int = 4, window: int = 7
     for s, (C, h, L) in enumerate(zip(dims, heads, depths)):
         r = res >> s
         nW = B * (r // window) ** 2
-        blocks = []
-        for _ in range(L):
-            blocks.append(make_block(ids, layer, nW, window * window, C, h, 4 * C, attn_bias_batches=h))
+        blocks, flags = [], []
+        for l in range(L):
+            blk = make_block(ids, layer, nW, window * window, C, h, 4 * C, attn_bias_batches=h)
+            sh = shifted and l % 2 == 1 and r > window
+            if sh:
+                # bias of window position w and head k: relative-position part of the head + mask of the position
+                m = shift_mask(r, window)
+                blk.attn_bias = (blk.attn_bias[None, :, :, :] + m[:, None, :, :]).reshape(-1, window * window, window * window)
+            blocks.append(blk)
+            flags.append(bool(sh))
             layer += 1
         st = SwinStage(C=C, heads=h, res=r, blocks=blocks)
+        if any(flags):
+            st.shifted = flags
+            st.shift_index, st.unshift_index = shift_indices(B, r, window)
         if s + 1 < len(dims):
             st.merge_index = merge_index(B, r, window)
             st.merge_ln_gamma, st.merge_ln_beta = _layernorm(ids, 4 * C, ACT_STD)
@@ -217,8 +273,9 @@ CONFIGS = {
 }
 
 
-def make_config(index: int, batch: int = None, depth: int = None):
-    """Parameters and input of workload `index`; `batch` / `depth` override the size (tests)."""
+def make_config(index: int, batch: int = None, depth: int = None, shifted: bool = False):
+    """Parameters and input of workload `index`; `batch` / `depth` override the size (tests); `shifted` builds the
+    Swin-shaped workload with shifted-window blocks."""
     c = dict(CONFIGS[index])
     B = batch if batch is not None else c["B"]
     if c["kind"] == "block":
@@ -229,4 +286,4 @@ def make_config(index: int, batch: int = None, depth: int = None):
         return make_vit(index, B, c["img"], c["D"], c["heads"], c["H"], L), make_image(index, B, c["img"])
     if depth is not None:
         raise ValueError("depth override is for ViT-family configs")
-    return make_swin(index, B, c["img"]), make_image(index, B, c["img"])
+    return make_swin(index, B, c["img"], shifted=shifted), make_image(index, B, c["img"])

@@ -105,6 +105,11 @@ class SwinStage:
     heads: int
     res: int                         # tokens per side of one image at this stage
     blocks: List[BlockParams]
+    # shifted-window blocks (every second block when the model is built with shifted=True): the rows are permuted
+    # into the cyclically shifted window order before such a block and back after it
+    shifted: Optional[List[bool]] = None       # per block
+    shift_index: Optional[np.ndarray] = None    # int32 [B*res*res]: source row of every row of the shifted order
+    unshift_index: Optional[np.ndarray] = None  # the inverse permutation
     # patch merging that follows the stage (None after the last stage)
     merge_index: Optional[np.ndarray] = None   # int32 [B*res*res]: source row of every C-wide slice
     merge_ln_gamma: Optional[Scale] = None

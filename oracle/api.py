@@ -334,14 +334,18 @@ def vit_forward(p, image, batch=None, return_tokens=False):
 
 
 def swin_forward(p, image):
-    """Swin-shaped forward (unshifted windows) composed from the oracle's operators; mirrors the model
+    """Swin-shaped forward (windows, optionally shifted in every second block) composed from the oracle's operators; mirrors the model
     description in ivit_inputs.params.SwinParams.  Returns int32 logits [B, classes]."""
     B = image.shape[0]
     X = linear(patchify(image, p.patch, window=p.window), p.Wpe, p.bpe, p.pe_scale)
     X = layernorm(X, p.pe_ln_gamma, p.pe_ln_beta, p.M_ln)
     for st in p.stages:
-        for blk in st.blocks:
-            X = block_forward(blk, X)
+        for i, blk in enumerate(st.blocks):
+            if st.shifted is not None and st.shifted[i]:
+                # shifted-window block: rows into the rolled window order, block, rows back
+                X = gather_rows(block_forward(blk, gather_rows(X, st.shift_index)), st.unshift_index)
+            else:
+                X = block_forward(blk, X)
         if st.merge_index is not None:
             G = gather_rows(X, st.merge_index, width=st.C).reshape(-1, 4 * st.C)
             G = layernorm(G, st.merge_ln_gamma, st.merge_ln_beta, p.M_ln)

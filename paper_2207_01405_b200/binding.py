@@ -446,7 +446,7 @@ class DeviceVit:
 
 
 class DeviceSwin:
-    """A Swin-shaped model (unshifted 7x7 windows) resident on the device."""
+    """A Swin-shaped model (7x7 windows, optionally shifted in every second block) resident on the device."""
 
     def __init__(self, p, device):
         self.p = p
@@ -457,7 +457,9 @@ class DeviceSwin:
         self.pe_ln_gamma, self.pe_ln_beta = DevScale(p.pe_ln_gamma, device), t(p.pe_ln_beta, np.int32)
         self.stages = []
         for st in p.stages:
-            d = {"blocks": [DeviceBlock(b, device) for b in st.blocks], "C": st.C}
+            d = {"blocks": [DeviceBlock(b, device) for b in st.blocks], "C": st.C, "shifted": st.shifted}
+            if st.shifted is not None:
+                d["shift_index"], d["unshift_index"] = t(st.shift_index, np.int32), t(st.unshift_index, np.int32)
             if st.merge_index is not None:
                 d["merge_index"] = t(st.merge_index, np.int32)
                 d["merge_ln_gamma"], d["merge_ln_beta"] = DevScale(st.merge_ln_gamma, device), t(st.merge_ln_beta, np.int32)
@@ -478,8 +480,13 @@ def swin_forward(ctx: Context, m: DeviceSwin, image: torch.Tensor) -> torch.Tens
     X = ctx.linear(ctx.patchify(image, p.patch, window=p.window), m.Wpe, m.bpe, m.pe_scale)
     X = ctx.layernorm(X, m.pe_ln_gamma, m.pe_ln_beta, p.M_ln)
     for st in m.stages:
-        for blk in st["blocks"]:
-            X = ctx.block_forward(blk, X, workspace=m.ws)
+        for i, blk in enumerate(st["blocks"]):
+            if st["shifted"] is not None and st["shifted"][i]:
+                # shifted-window block: rows into the rolled window order, block, rows back
+                X = ctx.block_forward(blk, ctx.gather_rows(X, st["shift_index"]), workspace=m.ws)
+                X = ctx.gather_rows(X, st["unshift_index"])
+            else:
+                X = ctx.block_forward(blk, X, workspace=m.ws)
         if "merge_index" in st:
             C_ = st["C"]
             G = ctx.gather_rows(X, st["merge_index"], width=C_).view(-1, 4 * C_)

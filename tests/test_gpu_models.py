@@ -39,6 +39,23 @@ def test_swin_tiny_shapes_bit_exact():
     assert c.poll_status() == 0
 
 
+def test_swin_shifted_windows_bit_exact():
+    """The Swin-shaped model with shifted-window blocks (cyclic roll as a row gather, mask folded into the int32
+    score bias, one bias matrix per window position and head), batch 2."""
+    g = _g()
+    c = g.ctx()
+    model, image = make_config(3, batch=2, shifted=True)
+    assert any(st.shifted and any(st.shifted) for st in model.stages)
+    dm = g.binding.DeviceSwin(model, "cuda")
+    logits = g.host(g.binding.swin_forward(c, dm, torch.from_numpy(image).cuda()))
+    want = O.swin_forward(model, image)
+    g.assert_equal(logits, want, "shifted swin logits")
+    # the shift changes the result
+    plain, _ = make_config(3, batch=2)
+    assert not np.array_equal(want, O.swin_forward(plain, image))
+    assert c.poll_status() == 0
+
+
 def test_vit_base_b128_full_size_sampled():
     """Config 2 at its full size (batch 128, 12 blocks); the oracle recomputes sampled images."""
     g = _g()
