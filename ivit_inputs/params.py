@@ -72,6 +72,7 @@ class BlockParams:
     b2: np.ndarray
     fc2_scale: Scale
     res2_scale: Scale
+    gelu_static_max: bool = False   # True: ShiftGELU variant with I_max fixed at I_p(127) (element-wise)
 
 
 @dataclass

@@ -39,6 +39,7 @@ class OBlock(C.Structure):
         ("W1", C.c_void_p), ("b1", C.c_void_p), ("fc1_scale", OScale),
         ("gelu", OExp), ("gelu_post", OScale),
         ("W2", C.c_void_p), ("b2", C.c_void_p), ("fc2_scale", OScale), ("res2_scale", OScale),
+        ("gelu_static_max", C.c_int32),
     ]
 
 
@@ -79,6 +80,7 @@ def lib():
                                  i64, i64, i64, i64, i64]
         L.orc_shiftmax.argtypes = [vp, i32, i64, vp, i64, i64, OScale, OExp, vp, i64, i64, i64]
         L.orc_shiftgelu.argtypes = [vp, i64, OExp, OScale, vp, i64, i64, i64]
+        L.orc_shiftgelu_static.argtypes = [vp, i64, OExp, OScale, vp, i64, i64, i64]
         L.orc_layernorm.argtypes = [vp, i32, i64, OScale, vp, i32, vp, i64, i64, i64]
         L.orc_block_forward.argtypes = [C.POINTER(OBlock), vp, vp]
         L.orc_attention.argtypes = [C.POINTER(OBlock), vp, vp]
@@ -225,13 +227,14 @@ def shiftmax(x, p, pre=None, bias32=None):
     return out
 
 
-def shiftgelu(x, p, post):
+def shiftgelu(x, p, post, static_max=False):
+    """Algorithm 2 per row; static_max=True: the variant with I_max fixed at I_p(127) (element-wise)."""
     k = _Keep()
     x = np.ascontiguousarray(x, dtype=np.int8)
     rows, cols = x.shape
     out = np.zeros((rows, cols), dtype=np.int8)
-    _chk(lib().orc_shiftgelu(x.ctypes.data, cols, _exp(p), k.scale(post), out.ctypes.data, cols, rows, cols),
-         "shiftgelu")
+    fn = lib().orc_shiftgelu_static if static_max else lib().orc_shiftgelu
+    _chk(fn(x.ctypes.data, cols, _exp(p), k.scale(post), out.ctypes.data, cols, rows, cols), "shiftgelu")
     return out
 
 
@@ -260,6 +263,7 @@ def _block_struct(p, k: _Keep) -> OBlock:
     b.W1, b.b1, b.fc1_scale = k.arr(p.W1, np.int8), k.arr(p.b1, np.int32), k.scale(p.fc1_scale)
     b.gelu, b.gelu_post = _exp(p.gelu), k.scale(p.gelu_post)
     b.W2, b.b2, b.fc2_scale, b.res2_scale = k.arr(p.W2, np.int8), k.arr(p.b2, np.int32), k.scale(p.fc2_scale), k.scale(p.res2_scale)
+    b.gelu_static_max = 1 if getattr(p, "gelu_static_max", False) else 0
     return b
 
 

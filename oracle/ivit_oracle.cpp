@@ -239,8 +239,21 @@ int orc_shiftmax(const void* in, int32_t in_dtype, int64_t ldin, const int32_t* 
   return 0;
 }
 
+static int shiftgelu_rows(const int8_t* in, int64_t ldin, orc_exp_params p, orc_scale post, int8_t* out,
+                          int64_t ldout, int64_t rows, int64_t cols, bool static_max);
+
 int orc_shiftgelu(const int8_t* in, int64_t ldin, orc_exp_params p, orc_scale post, int8_t* out,
                   int64_t ldout, int64_t rows, int64_t cols) {
+  return shiftgelu_rows(in, ldin, p, post, out, ldout, rows, cols, false);
+}
+
+int orc_shiftgelu_static(const int8_t* in, int64_t ldin, orc_exp_params p, orc_scale post, int8_t* out,
+                         int64_t ldout, int64_t rows, int64_t cols) {
+  return shiftgelu_rows(in, ldin, p, post, out, ldout, rows, cols, true);
+}
+
+static int shiftgelu_rows(const int8_t* in, int64_t ldin, orc_exp_params p, orc_scale post, int8_t* out,
+                          int64_t ldout, int64_t rows, int64_t cols, bool static_max) {
   if (!in || !out || cols < 1) return -1;
   if (!exp_params_ok(p, cols, true)) return -3;
   if (!scale_ok(post) || post.mult_c) return -2;
@@ -253,6 +266,7 @@ int orc_shiftgelu(const int8_t* in, int64_t ldin, orc_exp_params p, orc_scale po
       Ip[i] = x + asr(x, 1) + asr(x, 3) + asr(x, 4); /* 1.702 * I, (1.1011)b */
       if (Ip[i] > mx) mx = Ip[i];
     }
+    if (static_max) mx = 127 + asr(127, 1) + asr(127, 3) + asr(127, 4); /* I_p(127) = 212 */
     const int64_t e1 = shiftexp(-mx, p.I0, p.N);
     for (int64_t i = 0; i < cols; ++i) {
       const int64_t x = in[r * ldin + i];
@@ -333,7 +347,7 @@ int orc_block_forward(const orc_block_params* p, const int8_t* X, int8_t* Y) {
   if ((rc = orc_layernorm(Xh.data(), ORC_I8, D, p->ln2_gamma, p->ln2_beta, p->M_ln, A.data(), D, M, D))) return rc;
   if ((rc = orc_linear(A.data(), D, p->W1, D, p->b1, p->fc1_scale, nullptr, 0, 1, none, G.data(), H,
                        ORC_I8, 0, 0, M, H, D))) return rc;
-  if ((rc = orc_shiftgelu(G.data(), H, p->gelu, p->gelu_post, Hh.data(), H, M, H))) return rc;
+  if ((rc = shiftgelu_rows(G.data(), H, p->gelu, p->gelu_post, Hh.data(), H, M, H, p->gelu_static_max != 0))) return rc;
   if ((rc = orc_linear(Hh.data(), H, p->W2, H, p->b2, p->fc2_scale, Xh.data(), D, M, p->res2_scale, Y, D,
                        ORC_I8, 0, 0, M, D, H))) return rc;
   return 0;

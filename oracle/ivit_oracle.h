@@ -96,6 +96,11 @@ int orc_shiftmax(const void* in, int32_t in_dtype, int64_t ldin, const int32_t* 
 /* Algorithm 2 on each row (max over the row), then out = sat8(rq(I_in*I_div; post)). */
 int orc_shiftgelu(const int8_t* in, int64_t ldin, orc_exp_params p, orc_scale post, int8_t* out,
                   int64_t ldout, int64_t rows, int64_t cols);
+/* Variant of Algorithm 2 (not the paper's): I_max is the constant I_p(127) = 212, the largest value I_p can
+ * take for an int8 input, instead of the row maximum.  The sigmoid identity of Eq. (sigmoid) holds for any
+ * I_max >= max I_p; only the integer precision differs.  The function is then element-wise. */
+int orc_shiftgelu_static(const int8_t* in, int64_t ldin, orc_exp_params p, orc_scale post, int8_t* out,
+                         int64_t ldout, int64_t rows, int64_t cols);
 
 /* Sec. 3.5.  in_dtype ORC_I8 or ORC_I32 (|x| <= 2^20).
  *   mu = round-half-up(mean), y = x - mu, V = sum y^2, sd = isqrt(V),
@@ -118,6 +123,7 @@ typedef struct {
   const int8_t* W1; const int32_t* b1; orc_scale fc1_scale;
   orc_exp_params gelu; orc_scale gelu_post;
   const int8_t* W2; const int32_t* b2; orc_scale fc2_scale; orc_scale res2_scale;
+  int32_t gelu_static_max; /* 0: Algorithm 2 (row maximum); 1: the static-maximum variant above */
 } orc_block_params;
 
 /* X, Y: [B*T, D] int8, contiguous. */

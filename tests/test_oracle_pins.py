@@ -272,6 +272,36 @@ def test_shiftgelu_invariants():
     assert (o2 <= 0).all() and (o2 >= -8).all()
 
 
+@pytest.mark.parametrize("I0", [29, 32, 37])
+def test_shiftgelu_static_variant(I0):
+    """The static-maximum variant (not the paper's Algorithm 2): equal to Algorithm 2 on rows that contain 127
+    (there the row maximum is the constant), independent of the rest of the row everywhere, and within stated
+    distances of the float GELU and of Algorithm 2 (its coarser exponentials cost accuracy for small row maxima)."""
+    p = ExpParams(I0, 23)
+    post = Scale(2 ** 30, 37)
+    xs = np.arange(-128, 128)
+    full = xs.astype(np.int8)[None, :]
+    static_full = O.shiftgelu(full, p, post, static_max=True)
+    np.testing.assert_array_equal(static_full, O.shiftgelu(full, p, post))
+    # element-wise: any row gives the same value per input, also the closed form through the scalar helpers
+    rng = np.random.default_rng(I0)
+    rows = rng.integers(-128, 60, (5, 300)).astype(np.int8)
+    got = O.shiftgelu(rows, p, post, static_max=True)
+    np.testing.assert_array_equal(got, static_full[0][rows.astype(np.int64) + 128])
+    for x in (-128, -37, -1, 0, 1, 55, 127):
+        Ip = x + (x >> 1) + (x >> 3) + (x >> 4)
+        e, e1 = O.shiftexp(Ip - 212, I0, 23), O.shiftexp(-212, I0, 23)
+        div = O.intdiv(e, e + e1, 45, 8)
+        assert static_full[0][x + 128] == max(-128, min(127, exact_round_half_up(x * div, 2 ** 30, 37)))
+    xr = xs / I0
+    g_sig = xr / (1.0 + np.exp(-1.702 * xr))
+    assert np.abs(static_full[0] / I0 - g_sig).max() <= 0.035 + 0.5 / I0
+    # against Algorithm 2 on rows with a small maximum: a few output steps at most
+    low = np.clip(xs, -128, 20).astype(np.int8)[None, :]
+    d = np.abs(O.shiftgelu(low, p, post, static_max=True).astype(int) - O.shiftgelu(low, p, post).astype(int))
+    assert d.max() <= 2
+
+
 # ---------------------------------------------------------------- integer square root (Sec. 3.5)
 
 def test_isqrt_equals_floor_sqrt_below_2_24():
