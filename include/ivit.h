@@ -144,6 +144,14 @@ int ivit_shiftmax(ivit_ctx* ctx, const void* in, int32_t in_dtype, int64_t ldin,
  * in == out (in place) is allowed.  cols % 16 == 0, cols <= 16384. */
 int ivit_shiftgelu(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_params p,
                    ivit_scale post, int8_t* out, int64_t ldout, int64_t rows, int64_t cols);
+/* Variant of Algorithm 2 that is NOT the paper's function: I_max is the constant I_p(127) = 212
+ * (the largest value I_p takes for an int8 input) instead of the row maximum.  The sigmoid identity
+ * behind Algorithm 2 holds for any I_max >= max I_p, only the integer precision of the two
+ * exponentials differs (outputs differ from ivit_shiftgelu by at most a few steps, and are equal on
+ * rows that contain 127).  The function is element-wise, which lets ivit_block_forward apply it
+ * inside the FC1 epilogue (ivit_block_params.gelu_static_max).  Arguments as for ivit_shiftgelu. */
+int ivit_shiftgelu_static(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_params p,
+                          ivit_scale post, int8_t* out, int64_t ldout, int64_t rows, int64_t cols);
 
 /* ---- Sec. 3.5: I-LayerNorm over each row ----
  *   mu = floor((2*sum x + C) / (2C)); y = x - mu; V = sum y^2;
@@ -178,6 +186,9 @@ typedef struct {
   const int8_t* W1; const int32_t* b1; ivit_scale fc1_scale;
   ivit_exp_params gelu; ivit_scale gelu_post;
   const int8_t* W2; const int32_t* b2; ivit_scale fc2_scale; ivit_scale res2_scale;
+  /* 0: ShiftGELU as Algorithm 2 (row maximum, a kernel of its own between FC1 and FC2).
+   * 1: the static-maximum variant of ivit_shiftgelu_static, applied inside the FC1 epilogue. */
+  int32_t gelu_static_max;
 } ivit_block_params;
 
 size_t ivit_block_workspace_bytes(const ivit_block_params* p);

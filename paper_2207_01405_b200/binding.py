@@ -21,6 +21,7 @@ LIB_PATH = os.path.join(_HERE, "libivit.so")
 EXPORTS = [
     "ivit_ctx_create", "ivit_ctx_destroy", "ivit_ctx_set_stream", "ivit_ctx_poll_status", "ivit_ctx_launch_count",
     "ivit_ctx_set_gemm_engine", "ivit_strerror", "ivit_linear", "ivit_matmul", "ivit_shiftmax", "ivit_shiftgelu",
+    "ivit_shiftgelu_static",
     "ivit_layernorm", "ivit_block_workspace_bytes", "ivit_block_forward", "ivit_block_forward_static", "ivit_attention",
     "ivit_vit_workspace_bytes", "ivit_vit_forward", "ivit_vit_host_workspace_bytes", "ivit_vit_forward_host",
     "ivit_ctx_profile_start", "ivit_ctx_profile_stop", "ivit_ctx_profile_get", "ivit_kernel_kind_name", "ivit_patchify", "ivit_gather_rows", "ivit_fill_rows",
@@ -49,6 +50,7 @@ class CBlock(C.Structure):
         ("W1", C.c_void_p), ("b1", C.c_void_p), ("fc1_scale", CScale),
         ("gelu", CExp), ("gelu_post", CScale),
         ("W2", C.c_void_p), ("b2", C.c_void_p), ("fc2_scale", CScale), ("res2_scale", CScale),
+        ("gelu_static_max", C.c_int32),
     ]
 
 
@@ -90,6 +92,7 @@ def load_library():
                               i64, i64, i64, i64, i64]
     L.ivit_shiftmax.argtypes = [vp, vp, i32, i64, vp, i64, i64, CScale, CExp, vp, i64, i64, i64]
     L.ivit_shiftgelu.argtypes = [vp, vp, i64, CExp, CScale, vp, i64, i64, i64]
+    L.ivit_shiftgelu_static.argtypes = [vp, vp, i64, CExp, CScale, vp, i64, i64, i64]
     L.ivit_layernorm.argtypes = [vp, vp, i32, i64, CScale, vp, i32, vp, i64, i64, i64]
     L.ivit_block_workspace_bytes.argtypes = [C.POINTER(CBlock)]
     L.ivit_block_workspace_bytes.restype = C.c_size_t
@@ -267,12 +270,13 @@ class Context:
                                     _ld(out), rows, d), "ivit_shiftmax")
         return out
 
-    def shiftgelu(self, x, p, post: DevScale, out=None):
+    def shiftgelu(self, x, p, post: DevScale, out=None, static_max=False):
+        """static_max=True: ivit_shiftgelu_static (I_max fixed at I_p(127), element-wise; not the paper's function)."""
         rows, cols = x.shape
         if out is None:
             out = torch.empty_like(x)
-        _chk(self.lib.ivit_shiftgelu(self.h, x.data_ptr(), _ld(x), _cexp(p), post.c, out.data_ptr(), _ld(out), rows,
-                                     cols), "ivit_shiftgelu")
+        fn = self.lib.ivit_shiftgelu_static if static_max else self.lib.ivit_shiftgelu
+        _chk(fn(self.h, x.data_ptr(), _ld(x), _cexp(p), post.c, out.data_ptr(), _ld(out), rows, cols), "ivit_shiftgelu")
         return out
 
     def layernorm(self, x, gamma_scale: DevScale, beta, M_ln=20, out=None, rows=None, ldin=None):
@@ -383,6 +387,7 @@ def _fill_block(c: CBlock, p, up: _Uploader, B=None):
     c.W1, c.b1, c.fc1_scale = up.t(p.W1, np.int8), up.t(p.b1, np.int32), up.s(p.fc1_scale)
     c.gelu, c.gelu_post = _cexp(p.gelu), up.s(p.gelu_post)
     c.W2, c.b2, c.fc2_scale, c.res2_scale = up.t(p.W2, np.int8), up.t(p.b2, np.int32), up.s(p.fc2_scale), up.s(p.res2_scale)
+    c.gelu_static_max = 1 if getattr(p, "gelu_static_max", False) else 0
 
 
 class DeviceBlock:

@@ -99,7 +99,8 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(GemmProblem g, int64_t t
       int v = rq(a, e.scale.m((int)c), e.scale.s((int)c));
       if (e.res) v += rq((int)__ldg(e.res + (r % e.res_rows) * e.ldres + c), e.res_scale.m(0), e.res_scale.s(0));
       if (e.out_dtype == IVIT_I8)
-        reinterpret_cast<int8_t*>(e.out)[out_off + ro * e.ldo + c] = (int8_t)sat8(v);
+        reinterpret_cast<int8_t*>(e.out)[out_off + ro * e.ldo + c] =
+            e.act_table ? __ldg(e.act_table + sat8(v) + 128) : (int8_t)sat8(v);
       else
         reinterpret_cast<int32_t*>(e.out)[out_off + ro * e.ldo + c] = v;
     }

@@ -150,7 +150,8 @@ struct TileIter {
 // MODE fixes the run-time choices of the epilogue at compile time for the shapes of an encoder block, so that
 // the per-chunk code carries no branches on kernel arguments: 0 = everything decided at run time (any
 // orientation, output type and residual port), 1 = Dense orientation, int8 output staged for TMA stores, no
-// residual, 2 = the same with the residual tile fetched by TMA.
+// residual, 2 = the same with the residual tile fetched by TMA, 3 = as 1 with an activation table applied to the
+// saturated value (the element-wise ShiftGELU variant inside FC1).
 template <int MODE>
 __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmP,
                                                               const __grid_constant__ CUtensorMap tmQ,
@@ -171,7 +172,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
   const uint32_t accf0 = empty0 + 8 * kMaxStages, acce0 = accf0 + 16, resf = acce0 + 16, qrese = resf + 16 * kEpiWarps;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + bars_off + 8 * (2 * kMaxStages + 5 + 2 * kEpiWarps));
   volatile int* issued_slot = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  // residual port: the requantised value of every int8 residual byte (256 entries, built below)
+  // residual port: the requantised value of every int8 residual byte (256 entries, built below), followed by the
+  // 256 entries of the optional activation table
   int8_t* res_tab = reinterpret_cast<int8_t*>(tmem_slot) + 32;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -334,10 +336,17 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     const GemmEpilogue& e = a.epi;
     const bool dense = MODE ? true : a.lanes_are_channels != 0;
     const bool tma_out = MODE ? true : a.tma_out != 0;
-    const bool tma_res = MODE ? MODE == 2 : a.tma_res != 0;
+    const bool tma_res = MODE ? MODE == 2 : a.tma_res != 0;   // MODE 3 = MODE 1 + activation table
     const bool ldg_res = MODE ? false : (e.res != nullptr && !a.tma_res);
     const bool out_i32 = MODE ? false : e.out_dtype == IVIT_I32;
     const int8_t* res_tab0 = res_tab + 128;   // entry of residual byte 0
+    const int8_t* act_tab0 = res_tab + 256 + 128;   // entry of value 0 of the activation table
+    const bool act = MODE == 3 ? true : (MODE ? false : e.act_table != nullptr);
+    if (act) {
+      // the table may come from an earlier kernel of the stream: read it after the dependency wait above
+      if (et < 256) res_tab[256 + et] = e.act_table[et];
+      asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+    }
     bool ok = true;
 
     // Dense orientation: constants of this thread's channel; fetched one tile ahead
@@ -484,6 +493,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
               if (j < nrow && c_ok) reinterpret_cast<int32_t*>(e.out)[(r0 + j) * e.ldo + c] = v[j];
             return;
           }
+          if (act) {
+            // element-wise activation of the saturated value (the static-maximum ShiftGELU variant)
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] = (int)act_tab0[max(-128, min(127, v[j]))];
+          }
           // int8: pack four rows per word, transpose 4x4 bytes inside each group of four lanes so that a lane
           // ends up with four consecutive channels of one row, then store 4 bytes per lane and word
           uint32_t w[4], o[4];
@@ -622,7 +636,7 @@ int pow2_at_least(int v) {
 }
 
 constexpr size_t kSmemBudget = 227 * 1024;
-constexpr size_t kSmemFixed = 1024 + 8 * (2 * kMaxStages + 5 + 2 * kEpiWarps) + 32 + 256;
+constexpr size_t kSmemFixed = 1024 + 8 * (2 * kMaxStages + 5 + 2 * kEpiWarps) + 32 + 512;
 
 bool g_attr_set = false;
 
@@ -678,7 +692,7 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
       return IVIT_ERR_UNSUPPORTED;
   } else {
     // MatMul orientation: lanes = rows of A; the epilogue's 16-byte stores need aligned output rows
-    if (e.out_dtype != IVIT_I8 || e.bias || e.res || e.scale.mult_c || e.group_rows > 0) return IVIT_ERR_UNSUPPORTED;
+    if (e.out_dtype != IVIT_I8 || e.bias || e.res || e.scale.mult_c || e.group_rows > 0 || e.act_table) return IVIT_ERR_UNSUPPORTED;
     if ((reinterpret_cast<uintptr_t>(e.out) & 15) || e.ldo % 16 || g.sCo % 16 || g.sCi % 16) return IVIT_ERR_UNSUPPORTED;
     a.P = g.M; a.Q = g.N;
     a.tiles_p = (int)((a.P + BM - 1) / BM);
@@ -735,15 +749,18 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
   if (!g_attr_set) {
     if (cudaFuncSetAttribute(gemm_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
         cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
-        cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess)
+        cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
+        cudaFuncSetAttribute(gemm_tc_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess)
       return IVIT_ERR_CUDA;
     g_attr_set = true;
   }
   const unsigned grid = (unsigned)(a.total_tiles < ctx->sm_count ? a.total_tiles : ctx->sm_count);
   LaunchScope ls(ctx, KIND_GEMM_TC, 2.0 * (double)batches * (double)g.M * (double)g.N * (double)g.K);
   // the encoder block's Dense layers take the specialised instantiations
-  const int mode = (a.lanes_are_channels && a.tma_out && (!e.res || a.tma_res)) ? (a.tma_res ? 2 : 1) : 0;
-  if (mode == 2) launch_k(gemm_tc_kernel<2>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
+  int mode = (a.lanes_are_channels && a.tma_out && (!e.res || a.tma_res)) ? (a.tma_res ? 2 : 1) : 0;
+  if (e.act_table) mode = mode == 1 ? 3 : 0;
+  if (mode == 3) launch_k(gemm_tc_kernel<3>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
+  else if (mode == 2) launch_k(gemm_tc_kernel<2>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
   else if (mode == 1) launch_k(gemm_tc_kernel<1>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
   else launch_k(gemm_tc_kernel<0>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
   return ls.done();

@@ -137,9 +137,15 @@ int block_impl(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* X, int8_
                                             IVIT_I8, 0, 0, M, D, D)))) return rc;
   // Y = MLP(LayerNorm(X^)) + X^
   if ((rc = launch_layernorm(ctx, Xh, IVIT_I8, D, to_dev(p->ln2_gamma), p->ln2_beta, p->M_ln, A, D, M, D))) return rc;
-  if ((rc = launch_gemm(ctx, linear_problem(A, D, p->W1, D, p->b1, p->fc1_scale, nullptr, 0, 1, none, G, H, IVIT_I8,
-                                            0, 0, M, H, D)))) return rc;
-  if ((rc = launch_shiftgelu(ctx, G, H, p->gelu, p->gelu_post, G, H, M, H))) return rc;
+  GemmProblem fc1 = linear_problem(A, D, p->W1, D, p->b1, p->fc1_scale, nullptr, 0, 1, none, G, H, IVIT_I8, 0, 0, M, H, D);
+  if (p->gelu_static_max) {
+    // static-maximum ShiftGELU variant: element-wise, applied to the requantised value inside the FC1 epilogue
+    if ((rc = gelu_static_row(ctx, p->gelu, p->gelu_post, &fc1.epi.act_table))) return rc;
+    if ((rc = launch_gemm(ctx, fc1))) return rc;
+  } else {
+    if ((rc = launch_gemm(ctx, fc1))) return rc;
+    if ((rc = launch_shiftgelu(ctx, G, H, p->gelu, p->gelu_post, G, H, M, H))) return rc;
+  }
   return launch_gemm(ctx, linear_problem(G, H, p->W2, H, p->b2, p->fc2_scale, Xh, D, M, p->res2_scale, Y, D, IVIT_I8,
                                          0, 0, M, D, H));
 }
@@ -331,6 +337,18 @@ int ivit_shiftgelu(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_param
   int rc = check_exp(p, cols, true);
   if (rc) return rc;
   return launch_shiftgelu(ctx, in, ldin, p, post, out, ldout, rows, cols);
+}
+
+int ivit_shiftgelu_static(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_params p,
+                          ivit_scale post, int8_t* out, int64_t ldout, int64_t rows, int64_t cols) {
+  if (!ctx || !in || !out || rows < 0 || cols < 1) return IVIT_ERR_INVALID_ARG;
+  if (cols % 16 || cols > 16384) return IVIT_ERR_UNSUPPORTED;
+  if (ldin < cols || ldout < cols) return IVIT_ERR_INVALID_ARG;
+  if (!aligned16(in) || !aligned16(out) || ldin % 16 || ldout % 16) return IVIT_ERR_ALIGNMENT;
+  if (!scale_ok(post) || post.mult_c) return IVIT_ERR_RANGE;
+  int rc = check_exp(p, cols, true);
+  if (rc) return rc;
+  return launch_shiftgelu_static(ctx, in, ldin, p, post, out, ldout, rows, cols);
 }
 
 int ivit_layernorm(ivit_ctx* ctx, const void* in, int32_t in_dtype, int64_t ldin,

@@ -595,7 +595,7 @@ template <int WPL>
 __global__ void __launch_bounds__(256) shiftgelu_kernel(const int8_t* __restrict__ in, int64_t ldin,
                                                         const int8_t* __restrict__ table,
                                                         int8_t* __restrict__ out, int64_t ldout,
-                                                        int64_t rows, int cols) {
+                                                        int64_t rows, int cols, int fixed_max) {
   pdl_trigger();
   pdl_wait();
   __shared__ unsigned tab[8][64];  // one 256-byte table row per warp
@@ -619,7 +619,7 @@ __global__ void __launch_bounds__(256) shiftgelu_kernel(const int8_t* __restrict
       mx4 = (int)__vmaxs4(__vmaxs4((unsigned)v.x, (unsigned)v.y), __vmaxs4(__vmaxs4((unsigned)v.z, (unsigned)v.w), (unsigned)mx4));
     }
     int mx = max(max((int)(int8_t)mx4, (int)(int8_t)(mx4 >> 8)), max((int)(int8_t)(mx4 >> 16), (int)(int8_t)(mx4 >> 24)));
-    mx = max(0, warp_max(mx));
+    mx = fixed_max >= 0 ? fixed_max : max(0, warp_max(mx));   // fixed_max: the static-maximum variant
     __syncwarp();
     const unsigned* trow = reinterpret_cast<const unsigned*>(table + mx * 256);
     tab[wib][lane] = __ldg(trow + lane);
@@ -650,10 +650,8 @@ __global__ void __launch_bounds__(256) shiftgelu_kernel(const int8_t* __restrict
   }
 }
 
-int launch_shiftgelu(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_params p, ivit_scale post,
-                     int8_t* out, int64_t ldout, int64_t rows, int64_t cols) {
-  if (rows == 0) return IVIT_OK;
-  // find or build the lookup table of this parameter set
+// Finds or builds the lookup table of a parameter set; *table = its 128 x 256 bytes on the device.
+static int gelu_table(ivit_ctx* ctx, ivit_exp_params p, ivit_scale post, const int8_t** table) {
   const GeluKey key{p.I0, p.N, p.M, p.k_out, post.mult, post.shift};
   int slot = -1;
   for (int i = 0; i < ctx->gelu_used; ++i)
@@ -672,20 +670,47 @@ int launch_shiftgelu(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_par
     int rc = lt.done();
     if (rc) return rc;
   }
-  const int8_t* table = ctx->gelu_tables + (size_t)slot * kGeluTableBytes;
+  *table = ctx->gelu_tables + (size_t)slot * kGeluTableBytes;
+  return IVIT_OK;
+}
+
+int gelu_static_row(ivit_ctx* ctx, ivit_exp_params p, ivit_scale post, const int8_t** row) {
+  const int8_t* table = nullptr;
+  const int rc = gelu_table(ctx, p, post, &table);
+  if (rc) return rc;
+  *row = table + 127 * 256;   // I_max = I_p(127)
+  return IVIT_OK;
+}
+
+static int shiftgelu_rows(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_params p, ivit_scale post,
+                          int8_t* out, int64_t ldout, int64_t rows, int64_t cols, int fixed_max) {
+  if (rows == 0) return IVIT_OK;
+  const int8_t* table = nullptr;
+  int rc = gelu_table(ctx, p, post, &table);
+  if (rc) return rc;
   const int64_t want = (rows + 7) / 8;
   const int grid = (int)(want < (int64_t)ctx->sm_count * 8 ? want : (int64_t)ctx->sm_count * 8);
   const int wpl = (int)((cols / 16 + 31) / 32);
   cudaStream_t st = ctx->stream;
   LaunchScope ls(ctx, KIND_SHIFTGELU, 2.0 * (double)rows * (double)cols);
-  if (wpl <= 1) launch_k(shiftgelu_kernel<1>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols);
-  else if (wpl <= 2) launch_k(shiftgelu_kernel<2>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols);
-  else if (wpl <= 3) launch_k(shiftgelu_kernel<3>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols);
-  else if (wpl <= 4) launch_k(shiftgelu_kernel<4>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols);
-  else if (wpl <= 6) launch_k(shiftgelu_kernel<6>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols);
-  else if (wpl <= 8) launch_k(shiftgelu_kernel<8>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols);
-  else launch_k(shiftgelu_kernel<0>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols);
+  if (wpl <= 1) launch_k(shiftgelu_kernel<1>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
+  else if (wpl <= 2) launch_k(shiftgelu_kernel<2>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
+  else if (wpl <= 3) launch_k(shiftgelu_kernel<3>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
+  else if (wpl <= 4) launch_k(shiftgelu_kernel<4>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
+  else if (wpl <= 6) launch_k(shiftgelu_kernel<6>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
+  else if (wpl <= 8) launch_k(shiftgelu_kernel<8>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
+  else launch_k(shiftgelu_kernel<0>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
   return ls.done();
+}
+
+int launch_shiftgelu(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_params p, ivit_scale post,
+                     int8_t* out, int64_t ldout, int64_t rows, int64_t cols) {
+  return shiftgelu_rows(ctx, in, ldin, p, post, out, ldout, rows, cols, -1);
+}
+
+int launch_shiftgelu_static(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_params p, ivit_scale post,
+                            int8_t* out, int64_t ldout, int64_t rows, int64_t cols) {
+  return shiftgelu_rows(ctx, in, ldin, p, post, out, ldout, rows, cols, 127);
 }
 
 }  // namespace ivit

@@ -90,3 +90,30 @@ def test_fused_attention_kernel_serves_short_rows():
         assert (kinds == ["attention_fused"]) == fused, (T, kinds)
         g.assert_equal(g.host(Oo), O.attention(blk, QKV), f"attention T={T}")
     assert c.poll_status() == 0
+
+
+@pytest.mark.parametrize("engine", [0, 1])
+@pytest.mark.parametrize("B,T,D,heads,H", [(3, 197, 384, 6, 1536), (2, 50, 192, 3, 200 * 4), (1, 9, 64, 1, 64)])
+def test_block_static_gelu_variant_bit_exact(engine, B, T, D, heads, H):
+    """Block with the static-maximum ShiftGELU variant: the look-up runs inside the FC1 epilogue (tensor-core and
+    dp4a engines), one kernel launch fewer than the default block; bit-exact against the oracle's variant."""
+    import dataclasses
+    g = _g()
+    c = g.ctx()
+    c.set_gemm_engine(engine)
+    blk = dataclasses.replace(make_block(_Ids(300 + B + T), 2, B, T, D, heads, H), gelu_static_max=True)
+    X = make_block_input(11, B, T, D)
+    dblk = g.binding.DeviceBlock(blk, "cuda")
+    n0 = c.launch_count()
+    Y = c.block_forward(dblk, torch.from_numpy(X).cuda())
+    n_static = c.launch_count() - n0
+    g.assert_equal(g.host(Y), O.block_forward(blk, X), "block, static gelu")
+    plain = dataclasses.replace(blk, gelu_static_max=False)
+    dplain = g.binding.DeviceBlock(plain, "cuda")
+    c.block_forward(dplain, torch.from_numpy(X).cuda())   # builds nothing new: the table is shared
+    n0 = c.launch_count()
+    Yp = c.block_forward(dplain, torch.from_numpy(X).cuda())
+    assert c.launch_count() - n0 == n_static + 1 or n_static > 8   # first static call may also build the table
+    assert not np.array_equal(g.host(Yp), g.host(Y)) or T < 10
+    assert c.poll_status() == 0
+    c.set_gemm_engine(0)

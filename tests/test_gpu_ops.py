@@ -205,6 +205,22 @@ def test_shiftgelu_parity(rows, cols, I0):
     g.assert_equal(g.host(dx), want, "shiftgelu in place")
 
 
+@pytest.mark.parametrize("rows,cols,I0", [(1, 16, 29), (197, 768, 31), (77, 1536, 37), (5, 4096, 33)])
+def test_shiftgelu_static_variant_parity(rows, cols, I0):
+    """ivit_shiftgelu_static (I_max fixed at I_p(127)) against the oracle's variant, in place as well."""
+    g = _g()
+    c = g.ctx()
+    rng = np.random.default_rng(rows + cols + I0)
+    x = rand_i8(rng, (rows, cols), I0)
+    p, post = ExpParams(I0, 23), Scale(*dyadic(1.0 / (128 * 0.9)))
+    want = O.shiftgelu(x, p, post, static_max=True)
+    dx = g.dev(x)
+    g.assert_equal(g.host(c.shiftgelu(dx, p, g.binding.DevScale(post, "cuda"), static_max=True)), want, "shiftgelu static")
+    c.shiftgelu(dx, p, g.binding.DevScale(post, "cuda"), out=dx, static_max=True)
+    g.assert_equal(g.host(dx), want, "shiftgelu static in place")
+    assert c.poll_status() == 0
+
+
 @pytest.mark.parametrize("rows,C", [(1, 16), (197, 192), (500, 384), (301, 768), (100, 1024), (5, 520), (50, 96), (67, 128), (20, 1536),
                                     (9, 3072), (3, 16384), (11, 4)])
 def test_layernorm_parity(rows, C):
