@@ -104,16 +104,17 @@ def test_block_static_gelu_variant_bit_exact(engine, B, T, D, heads, H):
     blk = dataclasses.replace(make_block(_Ids(300 + B + T), 2, B, T, D, heads, H), gelu_static_max=True)
     X = make_block_input(11, B, T, D)
     dblk = g.binding.DeviceBlock(blk, "cuda")
+    Y = c.block_forward(dblk, torch.from_numpy(X).cuda())     # the first call may also build the look-up table
+    g.assert_equal(g.host(Y), O.block_forward(blk, X), "block, static gelu")
     n0 = c.launch_count()
     Y = c.block_forward(dblk, torch.from_numpy(X).cuda())
     n_static = c.launch_count() - n0
-    g.assert_equal(g.host(Y), O.block_forward(blk, X), "block, static gelu")
+    g.assert_equal(g.host(Y), O.block_forward(blk, X), "block, static gelu, second call")
     plain = dataclasses.replace(blk, gelu_static_max=False)
     dplain = g.binding.DeviceBlock(plain, "cuda")
-    c.block_forward(dplain, torch.from_numpy(X).cuda())   # builds nothing new: the table is shared
     n0 = c.launch_count()
-    Yp = c.block_forward(dplain, torch.from_numpy(X).cuda())
-    assert c.launch_count() - n0 == n_static + 1 or n_static > 8   # first static call may also build the table
-    assert not np.array_equal(g.host(Yp), g.host(Y)) or T < 10
+    Yp = c.block_forward(dplain, torch.from_numpy(X).cuda())   # the table of these parameters exists already
+    assert c.launch_count() - n0 == n_static + 1
+    g.assert_equal(g.host(Yp), O.block_forward(plain, X), "block, Algorithm 2")
     assert c.poll_status() == 0
     c.set_gemm_engine(0)
