@@ -261,7 +261,8 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
         mx = max(-128, min(127, mx));
         part_max[half * 128 + trow] = mx;
       }
-      asm volatile("bar.sync 1, 256;" ::: "memory");
+      // only the two warps that share these 32 rows exchange partial results: a barrier of their own
+      asm volatile("bar.sync %0, 64;" ::"r"(2 + qd) : "memory");
       unsigned sum = 0;
       if (got_s && warp_ok) {
         mx = max(part_max[trow], part_max[128 + trow]);
@@ -292,7 +293,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
         tmem_st_wait();
         part_sum[half * 128 + trow] = sum;
       }
-      asm volatile("bar.sync 1, 256;" ::: "memory");
+      asm volatile("bar.sync %0, 64;" ::"r"(2 + qd) : "memory");
       if (got_s && warp_ok) {
         sum = part_sum[trow] + part_sum[128 + trow];
         // pass C: Eq. (IntDiv) with M = 45, k_out = 8: (floor(2^45 / sum) * e) >> 38 = umulhi(factor, e) >> 6
