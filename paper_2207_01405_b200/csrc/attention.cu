@@ -328,8 +328,14 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
           int v[32];
           tmem_ld32(t_row + c * 32, v);
           if (row_ok) {
+            if (a.pv_s >= 33) {   // high product word plus 2^(s-33), shifted by s - 32
+              const int pv_rnd = 1 << (a.pv_s - 33), pv_sh = a.pv_s - 32;
 #pragma unroll
-            for (int j = 0; j < 32; ++j) v[j] = (int)(((long long)v[j] * a.pv_m + pv_c) >> a.pv_s);
+              for (int j = 0; j < 32; ++j) v[j] = mad_hi(v[j], a.pv_m, pv_rnd) >> pv_sh;
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) v[j] = (int)(((long long)v[j] * a.pv_m + pv_c) >> a.pv_s);
+            }
             int4 w0, w1;
             w0.x = (int)pack_sat8(v[0], v[1], v[2], v[3]);     w0.y = (int)pack_sat8(v[4], v[5], v[6], v[7]);
             w0.z = (int)pack_sat8(v[8], v[9], v[10], v[11]);   w0.w = (int)pack_sat8(v[12], v[13], v[14], v[15]);
