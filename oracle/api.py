@@ -79,6 +79,7 @@ def lib():
         L.orc_matmul.argtypes = [vp, i64, i64, i64, vp, i64, i64, i64, i32, vp, i64, i64, OScale, vp, i64, i64, i64,
                                  i64, i64, i64, i64, i64]
         L.orc_shiftmax.argtypes = [vp, i32, i64, vp, i64, i64, OScale, OExp, vp, i64, i64, i64]
+        L.orc_shiftmax_direct.argtypes = [vp, i64, OExp, vp, i64, i64, i64]
         L.orc_shiftgelu.argtypes = [vp, i64, OExp, OScale, vp, i64, i64, i64]
         L.orc_shiftgelu_static.argtypes = [vp, i64, OExp, OScale, vp, i64, i64, i64]
         L.orc_layernorm.argtypes = [vp, i32, i64, OScale, vp, i32, vp, i64, i64, i64]
@@ -224,6 +225,15 @@ def shiftmax(x, p, pre=None, bias32=None):
     br = 1 if bias32 is None else bias32.shape[0]
     _chk(lib().orc_shiftmax(x.ctypes.data, in_dtype, d, k.arr(bias32, np.int32), d, br, k.scale(pre), _exp(p),
                             out.ctypes.data, d, rows, d), "shiftmax")
+    return out
+
+
+def shiftmax_direct(x, p):
+    """Algorithm 1 on rows of int32 scores, no requantisation in front (x [rows, d] int32)."""
+    x = np.ascontiguousarray(x, dtype=np.int32)
+    rows, d = x.shape
+    out = np.zeros((rows, d), dtype=np.int8)
+    _chk(lib().orc_shiftmax_direct(x.ctypes.data, d, _exp(p), out.ctypes.data, d, rows, d), "shiftmax_direct")
     return out
 
 

@@ -51,6 +51,7 @@ inline int64_t shiftexp(int64_t I, int64_t I0, int N) {
   int64_t r = -(Ip + q * I0);             /* decimal part, 0 <= r < I0 */
   int64_t Ib = asr(-r, 1) + I0;           /* Eq. (linear): 2^x ~ 1 + x/2 */
   if (q <= N) return Ib * ((int64_t)1 << (N - q)); /* Ib << (N - q) */
+  if (q - N >= 63) return 0;                         /* every bit of Ib (< 2^63) is shifted out */
   return asr(Ib, (int)(q - N));
 }
 
@@ -97,7 +98,7 @@ inline int64_t isqrt_printed(int64_t n) {
 bool exp_params_ok(const orc_exp_params& p, int64_t row_len, bool gelu) {
   if (p.I0 < 1 || p.I0 > (1 << 15)) return false;
   if (p.N < 0 || p.N > 24) return false;
-  if (p.k_out != 8) return false;
+  if (p.k_out < 2 || p.k_out > 8) return false; /* the output is stored as int8 */
   if (p.M < 32 || p.M > 60) return false;
   const int64_t top = (int64_t)p.I0 << p.N;
   if (gelu) {
@@ -229,6 +230,34 @@ int orc_shiftmax(const void* in, int32_t in_dtype, int64_t ldin, const int32_t* 
     int64_t sum = 0;
     for (int64_t i = 0; i < d; ++i) {
       e[i] = shiftexp(x[i] - mx, p.I0, p.N); /* I_delta = I_in - max(I_in) */
+      sum += e[i];
+    }
+    for (int64_t i = 0; i < d; ++i) {
+      int64_t o = intdiv(e[i], sum, p.M, p.k_out);
+      out[r * ldout + i] = (int8_t)(o > omax ? omax : o);
+    }
+  }
+  return 0;
+}
+
+/* Algorithm 1 taken literally on wide inputs: no requantisation in front, I0 = round(1 / S_in) as large as
+ * the score scale makes it, 64-bit exponentials and sums, M chosen by the caller. */
+int orc_shiftmax_direct(const int32_t* in, int64_t ldin, orc_exp_params p, int8_t* out, int64_t ldout,
+                        int64_t rows, int64_t d) {
+  if (!in || !out || d < 1) return -1;
+  if (p.I0 < 1 || p.I0 > (1 << 28) || p.N < 0 || p.N > 24) return -3;
+  if (p.k_out < 2 || p.k_out > 8 || p.M < 32 || p.M > 62) return -3;
+  /* largest possible sum d * I0 * 2^N must leave the reciprocal floor(2^M / sum) at least 13 bits */
+  if ((__int128)d * p.I0 * ((__int128)1 << p.N) > ((__int128)1 << (p.M - 13))) return -3;
+  const int64_t omax = ((int64_t)1 << (p.k_out - 1)) - 1;
+#pragma omp parallel for schedule(static)
+  for (int64_t r = 0; r < rows; ++r) {
+    std::vector<int64_t> e(d);
+    int64_t mx = in[r * ldin];
+    for (int64_t i = 1; i < d; ++i) mx = in[r * ldin + i] > mx ? in[r * ldin + i] : mx;
+    int64_t sum = 0;
+    for (int64_t i = 0; i < d; ++i) {
+      e[i] = shiftexp((int64_t)in[r * ldin + i] - mx, p.I0, p.N); /* I_delta = I_in - max(I_in) */
       sum += e[i];
     }
     for (int64_t i = 0; i < d; ++i) {

@@ -93,6 +93,12 @@ int orc_shiftmax(const void* in, int32_t in_dtype, int64_t ldin, const int32_t* 
                  int64_t ldbias, int64_t bias_rows, orc_scale pre, orc_exp_params p, int8_t* out,
                  int64_t ldout, int64_t rows, int64_t d);
 
+/* Algorithm 1 on each row of int32 scores with nothing in front: I_delta = in - max(in) (up to 33 bits),
+ * ShiftExp with I0 = round(1 / S_in) <= 2^28, 64-bit sum, IntDiv with the caller's M (32..62) and k_out (2..8);
+ * out int8 in [0, 2^(k_out-1) - 1].  Requires d * I0 * 2^N <= 2^(M-13). */
+int orc_shiftmax_direct(const int32_t* in, int64_t ldin, orc_exp_params p, int8_t* out, int64_t ldout,
+                        int64_t rows, int64_t d);
+
 /* Algorithm 2 on each row (max over the row), then out = sat8(rq(I_in*I_div; post)). */
 int orc_shiftgelu(const int8_t* in, int64_t ldin, orc_exp_params p, orc_scale post, int8_t* out,
                   int64_t ldout, int64_t rows, int64_t cols);

@@ -215,6 +215,117 @@ def test_shiftmax_int32_input_equals_requant_then_int8():
     assert np.array_equal(O.shiftmax(acc, p, pre=pre, bias32=bias), O.shiftmax(x8, p))
 
 
+# ---------------------------------------------------------------- Algorithm 1 with k_out < 8 and on wide inputs
+
+@pytest.mark.parametrize("k_out", [2, 4, 6, 7])
+def test_shiftmax_k_out_is_a_truncation_of_the_8_bit_result(k_out):
+    """Eq. (IntDiv) shifts by M - (k_out - 1): lowering k_out by one drops one more low bit of the same product, so
+    out_k = out_8 >> (8 - k_out), the clamp to 2^(k_out-1) - 1 included (127 >> j is the smaller format's maximum)."""
+    rng = np.random.default_rng(40 + k_out)
+    rows = np.clip(np.rint(rng.standard_normal((50, 97)) * 30), -128, 127).astype(np.int8)
+    rows[0, :] = -5
+    rows[1, 1:] = -128
+    rows[1, 0] = 127
+    o8 = O.shiftmax(rows, ExpParams(13, 15)).astype(np.int64)
+    ok = O.shiftmax(rows, ExpParams(13, 15, 45, k_out)).astype(np.int64)
+    assert np.array_equal(ok, o8 >> (8 - k_out))
+    assert ok.max() <= 2 ** (k_out - 1) - 1 and ok[1, 0] == 2 ** (k_out - 1) - 1
+    assert O.shiftmax(np.array([[3]], dtype=np.int8), ExpParams(13, 15, 45, k_out))[0, 0] == 2 ** (k_out - 1) - 1
+
+
+def test_shiftgelu_k_out_against_float_gelu():
+    """Algorithm 2 with a 6-bit sigmoid: S_out of the sigmoid is 1/32, folded into the output ratio."""
+    I0 = 32
+    xs = np.arange(-128, 128)
+    row = xs.astype(np.int8)[None, :]
+    out = O.shiftgelu(row, ExpParams(I0, 23, 45, 6), Scale(2 ** 30, 35))[0].astype(np.float64)   # ratio 1/32
+    xr = xs / I0
+    g_sig = xr / (1.0 + np.exp(-1.702 * xr))
+    # the sigmoid is truncated to a multiple of 1/32: up to |x| / 32 further below the 8-bit result
+    assert (np.abs(out / I0 - g_sig) <= 0.035 + 0.5 / I0 + np.abs(xr) / 32).all()
+    o8 = O.shiftgelu(row, ExpParams(I0, 23), Scale(2 ** 30, 37))[0].astype(np.int64)
+    assert (np.abs(out.astype(np.int64)) <= np.abs(o8) + 1).all()
+
+
+def test_shiftexp_wide_exact_powers_of_two():
+    """I = -16 m gives I_p = -16m - 8m + m = -23 m exactly, so with I0 = 23 t and I = -16 t q the exponent is the
+    integer -q and ShiftExp must return (I0 << N) >> q with no fractional part, for any magnitude of t."""
+    for t in (1, 7, 1000, 10 ** 6, (1 << 28) // 23):
+        I0 = 23 * t
+        for N in (0, 5, 24):
+            for q in (0, 1, 2, 9, 24, 40, 52, 53, 70, 200):
+                if 16 * t * q < 2 ** 33:
+                    assert O.shiftexp(-16 * t * q, I0, N) == ((I0 << N) >> q), (t, N, q)
+    # half-way in the exponent: I_p = -(q I0 + r) with r = I0 / 2 -> I_b = I0 - ceil(r / 2)
+    assert O.shiftexp(-8 * 1000, 23 * 1000, 4) == (23000 - 5750) << 4
+    # far below the range: every bit shifted out, also when the shift count passes 63
+    assert O.shiftexp(-(2 ** 33 - 2), 1, 0) == 0
+
+
+@pytest.mark.parametrize("I0,N,M", [(1000, 15, 50), (65536, 10, 50), (1 << 24, 4, 56), (1 << 28, 0, 62)])
+def test_shiftmax_direct_vs_float_softmax(I0, N, M):
+    rng = np.random.default_rng(I0 % 1000 + N)
+    p = ExpParams(I0, N, M, 8)
+    for d in (2, 3, 49, 197, 577):
+        # real-valued scores of a few units, at scale 1 / I0 (clipped to int32)
+        x = np.clip(np.rint(rng.standard_normal((40, d)) * 2.5 * I0), -2 ** 31, 2 ** 31 - 1).astype(np.int32)
+        out = O.shiftmax_direct(x, p).astype(np.int64)
+        assert out.min() >= 0 and out.max() <= 127
+        sm = float_softmax(x.astype(np.float64) / I0)
+        assert np.abs(out / 128.0 - sm).max() <= 0.026, (d, np.abs(out / 128.0 - sm).max())
+        s = out.sum(axis=1)
+        assert (s <= 128).all() and (s >= 128 - d).all()
+        assert (out[np.arange(40), x.argmax(axis=1)] == out.max(axis=1)).all()
+        # shift invariance (the same offset on a row) and permutation equivariance
+        off = rng.integers(-1000, 1000, (40, 1))
+        narrow = np.clip(x.astype(np.int64), -2 ** 31 + 1000, 2 ** 31 - 1001)
+        assert np.array_equal(O.shiftmax_direct((narrow + off).astype(np.int32), p),
+                              O.shiftmax_direct(narrow.astype(np.int32), p))
+        perm = rng.permutation(d)
+        assert np.array_equal(O.shiftmax_direct(x[:, perm], p), out[:, perm])
+
+
+def test_shiftmax_direct_special_rows_and_extremes():
+    lo, hi = -2 ** 31, 2 ** 31 - 1
+    for I0, N, M, k in [(1, 20, 45, 8), (23, 15, 45, 8), (40000, 8, 48, 8), (1 << 28, 0, 62, 8), (5000, 12, 45, 5)]:
+        p = ExpParams(I0, N, M, k)
+        omax = 2 ** (k - 1) - 1
+        assert O.shiftmax_direct(np.array([[hi]], dtype=np.int32), p)[0, 0] == omax
+        assert O.shiftmax_direct(np.array([[lo]], dtype=np.int32), p)[0, 0] == omax
+        for d in (2, 3, 4, 7, 49):
+            for v in (lo, -12345, hi):
+                o = O.shiftmax_direct(np.full((1, d), v, dtype=np.int32), p)[0]
+                assert (o == o[0]).all() and o[0] in ((omax + 1) // d, (omax + 1) // d - 1)
+        # the whole int32 range inside one row: I_delta needs 33 bits; the maximum takes everything
+        row = np.full((1, 50), lo, dtype=np.int32)
+        row[0, 17] = hi
+        row[0, 3] = 0
+        o = O.shiftmax_direct(row, p)[0]
+        assert o[17] == omax and o.sum() == omax
+    # two entries one exact octave apart (see test_shiftexp_wide_exact_powers_of_two): 2/3 and 1/3 of 128
+    o = O.shiftmax_direct(np.array([[0, -16 * 1000]], dtype=np.int32), ExpParams(23 * 1000, 10, 45, 8))[0]
+    assert list(o) == [85, 42]
+    o = O.shiftmax_direct(np.array([[-16 * 3 * 500, 7, 7 - 16 * 500]], dtype=np.int32), ExpParams(23 * 500, 10, 45, 8))[0]
+    assert list(o) == [9, 78, 39]   # floor(128 * {1, 8, 4} / 13)
+
+
+def test_shiftmax_direct_on_int8_values_equals_the_int8_form():
+    rng = np.random.default_rng(77)
+    for d, I0, k in [(197, 11, 8), (64, 30, 8), (50, 13, 6)]:
+        rows = np.clip(np.rint(rng.standard_normal((33, d)) * 40), -128, 127).astype(np.int8)
+        p = ExpParams(I0, 15, 45, k)
+        assert np.array_equal(O.shiftmax_direct(rows.astype(np.int32), p), O.shiftmax(rows, p))
+
+
+def test_shiftmax_direct_rejects_out_of_range_parameters():
+    x = np.zeros((1, 8), dtype=np.int32)
+    for bad in [ExpParams(0, 10, 45, 8), ExpParams((1 << 28) + 1, 0, 62, 8), ExpParams(100, 25, 62, 8),
+                ExpParams(100, 10, 63, 8), ExpParams(100, 10, 31, 8), ExpParams(100, 10, 45, 9),
+                ExpParams(100, 10, 45, 1), ExpParams(1 << 20, 10, 45, 8)]:
+        with pytest.raises(Exception):
+            O.shiftmax_direct(x, bad)
+
+
 # ---------------------------------------------------------------- ShiftGELU (Algorithm 2)
 
 def test_gelu_shift_constant():
