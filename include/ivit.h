@@ -69,10 +69,13 @@ typedef struct {
 
 /* Constants of Algorithm 1 / Algorithm 2: I0 = round(1 / S_in); N = the
  * left pre-shift of ShiftExp (footnote of Algorithm 1); M = width of the
- * reciprocal in Eq. (IntDiv); k_out = output bit width (only 8 is built).
+ * reciprocal in Eq. (IntDiv); k_out = output bit width (results are stored
+ * as int8 in [0, 2^(k_out-1) - 1], scale 1 / 2^(k_out-1)).
  * Bounds (IVIT_ERR_RANGE otherwise): 1 <= I0 <= 2^15, 0 <= N <= 24, M == 45,
- * k_out == 8; Shiftmax: row_len * I0 * 2^N < 2^32 and I0 * 2^N >= 2^14;
- * ShiftGELU: 2 * I0 * 2^N < 2^32. */
+ * 2 <= k_out <= 8; Shiftmax: row_len * I0 * 2^N < 2^32 and I0 * 2^N >= 2^14;
+ * ShiftGELU: 2 * I0 * 2^N < 2^32.  ivit_shiftmax_direct has wider bounds of
+ * its own.  The fused attention kernel is built for k_out == 8; with another
+ * k_out, ivit_attention and the block run the unfused sequence of kernels. */
 typedef struct {
   int32_t I0, N, M, k_out;
 } ivit_exp_params;
@@ -130,12 +133,25 @@ int ivit_matmul(ivit_ctx* ctx, const int8_t* A, int64_t lda, int64_t sAo, int64_
  * in_dtype IVIT_I8: rows of int8 scores.  IVIT_I32: rows of int32
  * accumulators, x8 = sat8(rq(in32 + bias32[row % bias_rows, :]; pre)) first
  * (bias32 may be NULL), which is bit-identical to requantising to int8 and
- * then calling the int8 form.  out int8 in [0, 127], scale 1/128
- * (Eq. (IntDiv), S_out = 1/2^(k_out-1)).  Columns d .. roundup(d,16)-1 of out
+ * then calling the int8 form.  out int8 in [0, 2^(k_out-1) - 1]
+ * (Eq. (IntDiv), S_out = 1/2^(k_out-1); [0, 127] at k_out = 8).  Columns d .. roundup(d,16)-1 of out
  * are written as 0.  1 <= d <= 8192. */
 int ivit_shiftmax(ivit_ctx* ctx, const void* in, int32_t in_dtype, int64_t ldin,
                   const int32_t* bias32, int64_t ldbias, int64_t bias_rows, ivit_scale pre,
                   ivit_exp_params p, int8_t* out, int64_t ldout, int64_t rows, int64_t d);
+
+/* ---- Sec. 3.3, Algorithm 1 on int32 scores with no requantisation in front ----
+ * The general form of the algorithm: in is int32 [rows, ldin] (for instance
+ * the accumulators of Q K^T at scale S_in), I_delta = in - max(in) takes up to
+ * 33 bits, I0 = round(1 / S_in) may be as large as 2^28, exponentials and
+ * their sum are 64-bit, and the caller chooses M.  out int8 [rows, ldout] in
+ * [0, 2^(k_out-1) - 1]; columns d .. roundup(d,16)-1 are written as 0.
+ * Bounds (IVIT_ERR_RANGE otherwise): 1 <= I0 <= 2^28, 0 <= N <= 24,
+ * 32 <= M <= 62, 2 <= k_out <= 8, d * I0 * 2^N <= 2^(M-13) (so that the
+ * reciprocal floor(2^M / sum) keeps at least 13 bits).  1 <= d <= 8192,
+ * ldin % 4 == 0, ldout % 16 == 0, both pointers 16-byte aligned (device). */
+int ivit_shiftmax_direct(ivit_ctx* ctx, const int32_t* in, int64_t ldin, ivit_exp_params p,
+                         int8_t* out, int64_t ldout, int64_t rows, int64_t d);
 
 /* ---- Sec. 3.4, Algorithm 2: ShiftGELU over each row, then requantisation ----
  *   I_p = x + (x>>1) + (x>>3) + (x>>4); I_max = max(0, max_row I_p);

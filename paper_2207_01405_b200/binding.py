@@ -22,6 +22,7 @@ EXPORTS = [
     "ivit_ctx_create", "ivit_ctx_destroy", "ivit_ctx_set_stream", "ivit_ctx_poll_status", "ivit_ctx_launch_count",
     "ivit_ctx_set_gemm_engine", "ivit_strerror", "ivit_linear", "ivit_matmul", "ivit_shiftmax", "ivit_shiftgelu",
     "ivit_shiftgelu_static",
+    "ivit_shiftmax_direct",
     "ivit_layernorm", "ivit_block_workspace_bytes", "ivit_block_forward", "ivit_block_forward_static", "ivit_attention",
     "ivit_vit_workspace_bytes", "ivit_vit_forward", "ivit_vit_host_workspace_bytes", "ivit_vit_forward_host",
     "ivit_ctx_profile_start", "ivit_ctx_profile_stop", "ivit_ctx_profile_get", "ivit_kernel_kind_name", "ivit_patchify", "ivit_gather_rows", "ivit_fill_rows",
@@ -93,6 +94,7 @@ def load_library():
     L.ivit_shiftmax.argtypes = [vp, vp, i32, i64, vp, i64, i64, CScale, CExp, vp, i64, i64, i64]
     L.ivit_shiftgelu.argtypes = [vp, vp, i64, CExp, CScale, vp, i64, i64, i64]
     L.ivit_shiftgelu_static.argtypes = [vp, vp, i64, CExp, CScale, vp, i64, i64, i64]
+    L.ivit_shiftmax_direct.argtypes = [vp, vp, i64, CExp, vp, i64, i64, i64]
     L.ivit_layernorm.argtypes = [vp, vp, i32, i64, CScale, vp, i32, vp, i64, i64, i64]
     L.ivit_block_workspace_bytes.argtypes = [C.POINTER(CBlock)]
     L.ivit_block_workspace_bytes.restype = C.c_size_t
@@ -268,6 +270,16 @@ class Context:
                                     _ld(bias32) if bias32 is not None else 0,
                                     bias32.shape[0] if bias32 is not None else 1, pre_c, _cexp(p), out.data_ptr(),
                                     _ld(out), rows, d), "ivit_shiftmax")
+        return out
+
+    def shiftmax_direct(self, x, p, out=None):
+        """ivit_shiftmax_direct: Algorithm 1 on int32 scores [rows, d] with no requantisation in front."""
+        rows, d = x.shape
+        if out is None:
+            ldo = (d + 15) // 16 * 16
+            out = torch.empty((rows, ldo), dtype=torch.int8, device=x.device)[:, :d]
+        _chk(self.lib.ivit_shiftmax_direct(self.h, x.data_ptr(), _ld(x), _cexp(p), out.data_ptr(), _ld(out), rows, d),
+             "ivit_shiftmax_direct")
         return out
 
     def shiftgelu(self, x, p, post: DevScale, out=None, static_max=False):

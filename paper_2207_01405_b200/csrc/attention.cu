@@ -379,6 +379,7 @@ int launch_attention_fused(ivit_ctx* ctx, const ivit_block_params* p, const int8
   if (!ctx->tmap_encode) return IVIT_ERR_UNSUPPORTED;
   const int64_t B = p->B, T = p->T, D = p->D, h = p->heads, d = D / h;
   if (T > 256 || (d != 32 && d != 64 && d != 128) || B * h > 2147483647LL / 4) return IVIT_ERR_UNSUPPORTED;
+  if (p->smax.k_out != 8) return IVIT_ERR_UNSUPPORTED;   // the fused kernel has the 8-bit IntDiv shift built in
   if ((reinterpret_cast<uintptr_t>(QKV) & 15) || (reinterpret_cast<uintptr_t>(O) & 15)) return IVIT_ERR_UNSUPPORTED;
   if (B == 0) return IVIT_OK;
   AttnArgs a{};

@@ -182,6 +182,8 @@ int launch_layernorm(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, 
 int launch_shiftmax(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, const int32_t* bias32,
                     int64_t ldbias, int64_t bias_rows, ScaleDev pre, ivit_exp_params p, int8_t* out,
                     int64_t ldout, int64_t rows, int64_t d);
+int launch_shiftmax_direct(ivit_ctx* ctx, const int32_t* in, int64_t ldin, ivit_exp_params p, int8_t* out,
+                           int64_t ldout, int64_t rows, int64_t d);
 // Row `127` of the ShiftGELU table of (p, post) on the device (built on first use): the static-maximum variant.
 int gelu_static_row(ivit_ctx* ctx, ivit_exp_params p, ivit_scale post, const int8_t** row);
 int launch_shiftgelu_static(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_params p, ivit_scale post,

@@ -15,7 +15,7 @@ inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 inline int64_t round16(int64_t v) { return (v + 15) / 16 * 16; }
 
 int check_exp(ivit_exp_params p, int64_t row_len, bool gelu) {
-  if (p.I0 < 1 || p.I0 > (1 << 15) || p.N < 0 || p.N > 24 || p.M != 45 || p.k_out != 8) return IVIT_ERR_RANGE;
+  if (p.I0 < 1 || p.I0 > (1 << 15) || p.N < 0 || p.N > 24 || p.M != 45 || p.k_out < 2 || p.k_out > 8) return IVIT_ERR_RANGE;
   const int64_t top = (int64_t)p.I0 << p.N;
   if (gelu) {
     if (2 * top > 4294967295LL) return IVIT_ERR_RANGE;
@@ -325,6 +325,19 @@ int ivit_shiftmax(ivit_ctx* ctx, const void* in, int32_t in_dtype, int64_t ldin,
     if (bias32 && (!aligned16(bias32) || ldbias % 4)) return IVIT_ERR_ALIGNMENT;
   }
   return launch_shiftmax(ctx, in, in_dtype, ldin, bias32, ldbias, bias_rows, to_dev(pre), p, out, ldout, rows, d);
+}
+
+int ivit_shiftmax_direct(ivit_ctx* ctx, const int32_t* in, int64_t ldin, ivit_exp_params p, int8_t* out,
+                         int64_t ldout, int64_t rows, int64_t d) {
+  if (!ctx || !in || !out || rows < 0 || d < 1) return IVIT_ERR_INVALID_ARG;
+  if (d > 8192) return IVIT_ERR_UNSUPPORTED;
+  if (ldin < d || ldout < round16(d)) return IVIT_ERR_INVALID_ARG;
+  if (!aligned16(in) || !aligned16(out) || ldout % 16 || ldin % 4) return IVIT_ERR_ALIGNMENT;
+  if (p.I0 < 1 || p.I0 > (1 << 28) || p.N < 0 || p.N > 24 || p.k_out < 2 || p.k_out > 8 || p.M < 32 || p.M > 62)
+    return IVIT_ERR_RANGE;
+  // the largest possible sum d * I0 * 2^N leaves the reciprocal floor(2^M / sum) at least 13 bits
+  if (((int64_t)p.I0 << p.N) > (((int64_t)1 << (p.M - 13)) / d)) return IVIT_ERR_RANGE;
+  return launch_shiftmax_direct(ctx, in, ldin, p, out, ldout, rows, d);
 }
 
 int ivit_shiftgelu(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_params p,

@@ -498,9 +498,11 @@ __global__ void __launch_bounds__(256) shiftmax_kernel(RowLoader<FROM_I32> ld, i
       sum -= (unsigned)(32 * iters * 4 - d) * exp_tab[mxu];
       if (lane == q) { my_sum = sum; my_mxu = mxu; }
     }
-    // Eq. (IntDiv): one reciprocal per row (lane q for row q), M = 45, k_out = 8:
-    // (floor(2^45 / sum) * e) >> 38 == umulhi(factor, e) >> 6 since factor <= 2^31.
+    // Eq. (IntDiv): one reciprocal per row (lane q for row q), M = 45:
+    // (floor(2^45 / sum) * e) >> (45 - (k_out - 1)) == umulhi(factor, e) >> (14 - k_out) since factor <= 2^31.
     const unsigned my_factor = (unsigned)((1ull << 45) / (unsigned long long)my_sum);
+    const int osh = 14 - p.k_out;
+    const int omax = (1 << (p.k_out - 1)) - 1;   // the one possible 2^(k_out-1) is clamped
 #pragma unroll
     for (int q = 0; q < R; ++q) {
       const unsigned factor = __shfl_sync(0xffffffffu, my_factor, q);
@@ -523,9 +525,8 @@ __global__ void __launch_bounds__(256) shiftmax_kernel(RowLoader<FROM_I32> ld, i
             e2 = *reinterpret_cast<const unsigned*>(tmx - 4 * (int)__byte_perm(v, 0, 0x4442));
             e3 = *reinterpret_cast<const unsigned*>(tmx - 4 * (int)(v >> 24));
           }
-          // values are <= 128: the saturating pack clamps the one possible 128 to 127
-          unsigned packed = pack_sat8_u((int)(__umulhi(factor, e0) >> 6), (int)(__umulhi(factor, e1) >> 6),
-                                        (int)(__umulhi(factor, e2) >> 6), (int)(__umulhi(factor, e3) >> 6));
+          unsigned packed = pack_sat8_u(min((int)(__umulhi(factor, e0) >> osh), omax), min((int)(__umulhi(factor, e1) >> osh), omax),
+                                        min((int)(__umulhi(factor, e2) >> osh), omax), min((int)(__umulhi(factor, e3) >> osh), omax));
           // positions past d are written as zero
           if (idx >= nwords) packed = 0;
           else if (idx == nwords - 1 && npad) packed &= 0xffffffffu >> (8 * npad);
@@ -564,6 +565,129 @@ int launch_shiftmax(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, c
   return ls.done();
 }
 
+// ------------------------------------------------------------------ Shiftmax on int32 scores (Algorithm 1, wide form)
+
+struct DirectConsts {
+  unsigned I0;
+  int N;
+  int osh;                       // M - (k_out - 1)
+  int omax;                      // 2^(k_out-1) - 1
+  int M;
+  unsigned long long magic;      // reciprocal of I0 scaled by 2^64, rounded up (unused when I0 == 1)
+  unsigned long long zero_from;  // I0 * (N + 29): from here on every bit of I_b < 2^29 is shifted out
+};
+
+// ShiftExp(I - I_max) for nd = I_max - I (0 .. 2^32 - 1).  The arithmetic shifts of the negative I_delta round
+// towards -inf, so -I_p = nd + ceil(nd / 2) - ceil(nd / 16).  Below zero_from the quotient by I0 is < 53 and
+// (-I_p) * I0 < 2^64, which makes the multiply-high by floor(2^64 / I0) + 1 the exact floor quotient.
+__device__ __forceinline__ unsigned long long shiftexp_wide(unsigned nd, const DirectConsts& c) {
+  const unsigned up2 = (nd >> 1) + (nd & 1u);
+  const unsigned up16 = (nd >> 4) + ((nd & 15u) != 0u);
+  const unsigned long long n = (unsigned long long)nd + up2 - up16;
+  if (n >= c.zero_from) return 0ull;
+  const unsigned q = c.I0 == 1u ? (unsigned)n : (unsigned)__umul64hi(n, c.magic);
+  const unsigned r = (unsigned)(n - (unsigned long long)q * c.I0);   // 0 <= r < I0
+  const unsigned Ib = c.I0 - ((r + 1) >> 1);                         // ((-r) >> 1) + I0
+  return q <= (unsigned)c.N ? (unsigned long long)Ib << (c.N - q) : (unsigned long long)(Ib >> (q - c.N));
+}
+
+__device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// One warp per row.  WPL groups of four scores per lane stay in registers as their exponentials
+// (d <= 128 * WPL); WPL == 0 reads the row three times instead.
+template <int WPL>
+__global__ void __launch_bounds__(256) shiftmax_direct_kernel(const int32_t* __restrict__ in, int64_t ldin,
+                                                              DirectConsts c, int8_t* __restrict__ out,
+                                                              int64_t ldout, int64_t rows, int d) {
+  pdl_trigger();
+  pdl_wait();
+  const int lane = threadIdx.x & 31;
+  const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  const int ngroups = (d + 3) >> 2;                // int4 groups that hold scores
+  const int nwords_out = ((d + 15) >> 4) << 2;     // output words, zero-filled up to the next multiple of 16 columns
+  constexpr int W = WPL > 0 ? WPL : 1;
+  const int iters = WPL > 0 ? WPL : (nwords_out + 31) / 32;
+  for (int64_t r = warp; r < rows; r += nwarps) {
+    const int4* src = reinterpret_cast<const int4*>(in + r * ldin);
+    // pass 1: row maximum (positions past d never count)
+    int mx = INT_MIN;
+    int4 x[W];
+#pragma unroll
+    for (int i = 0; i < iters; ++i) {
+      const int g = lane + 32 * i;
+      int4 v = make_int4(INT_MIN, INT_MIN, INT_MIN, INT_MIN);
+      if (g < ngroups) {
+        v = __ldg(src + g);
+        if (4 * g + 1 >= d) v.y = INT_MIN;
+        if (4 * g + 2 >= d) v.z = INT_MIN;
+        if (4 * g + 3 >= d) v.w = INT_MIN;
+      }
+      if (WPL > 0) x[i] = v;
+      mx = max(max(mx, max(v.x, v.y)), max(v.z, v.w));
+    }
+    mx = __reduce_max_sync(0xffffffffu, mx);
+    // exponentials of group g (0 for positions past d)
+    auto exps = [&](int g, const int4& v, unsigned long long* e) {
+      e[0] = 4 * g + 0 < d ? shiftexp_wide((unsigned)mx - (unsigned)v.x, c) : 0ull;
+      e[1] = 4 * g + 1 < d ? shiftexp_wide((unsigned)mx - (unsigned)v.y, c) : 0ull;
+      e[2] = 4 * g + 2 < d ? shiftexp_wide((unsigned)mx - (unsigned)v.z, c) : 0ull;
+      e[3] = 4 * g + 3 < d ? shiftexp_wide((unsigned)mx - (unsigned)v.w, c) : 0ull;
+    };
+    // pass 2: sum
+    unsigned long long e[W][4];
+    unsigned long long sum = 0;
+#pragma unroll
+    for (int i = 0; i < iters; ++i) {
+      const int g = lane + 32 * i;
+      unsigned long long t[4] = {0ull, 0ull, 0ull, 0ull};
+      if (g < ngroups) exps(g, WPL > 0 ? x[i] : __ldg(src + g), t);
+      if (WPL > 0) { e[i][0] = t[0]; e[i][1] = t[1]; e[i][2] = t[2]; e[i][3] = t[3]; }
+      sum += (t[0] + t[1]) + (t[2] + t[3]);
+    }
+    sum = warp_sum_u64(sum);                                   // >= I0 * 2^N: the maximum contributes exactly that
+    const unsigned long long factor = (1ull << c.M) / sum;     // Eq. (IntDiv); factor * e <= 2^M < 2^63
+    // pass 3: outputs
+    int* dst = reinterpret_cast<int*>(out + r * ldout);
+#pragma unroll
+    for (int i = 0; i < iters; ++i) {
+      const int g = lane + 32 * i;
+      if (g < nwords_out) {
+        unsigned long long t[4] = {0ull, 0ull, 0ull, 0ull};
+        if (WPL > 0) { t[0] = e[i][0]; t[1] = e[i][1]; t[2] = e[i][2]; t[3] = e[i][3]; }
+        else if (g < ngroups) exps(g, __ldg(src + g), t);
+        const int o0 = min((int)((factor * t[0]) >> c.osh), c.omax), o1 = min((int)((factor * t[1]) >> c.osh), c.omax);
+        const int o2 = min((int)((factor * t[2]) >> c.osh), c.omax), o3 = min((int)((factor * t[3]) >> c.osh), c.omax);
+        dst[g] = (int)pack_sat8_u(o0, o1, o2, o3);
+      }
+    }
+  }
+}
+
+int launch_shiftmax_direct(ivit_ctx* ctx, const int32_t* in, int64_t ldin, ivit_exp_params p, int8_t* out,
+                           int64_t ldout, int64_t rows, int64_t d) {
+  if (rows == 0) return IVIT_OK;
+  DirectConsts c;
+  c.I0 = (unsigned)p.I0; c.N = p.N; c.M = p.M;
+  c.osh = p.M - (p.k_out - 1);
+  c.omax = (1 << (p.k_out - 1)) - 1;
+  // floor((2^64 - 1) / I0) + 1: floor(2^64 / I0) + 1, or exactly 2^64 / I0 when I0 is a power of two (both give the floor quotient)
+  c.magic = p.I0 > 1 ? ~0ull / (unsigned long long)p.I0 + 1ull : 0ull;
+  c.zero_from = (unsigned long long)p.I0 * (unsigned long long)(p.N + 29);
+  const int64_t want = (rows + 7) / 8;
+  const int grid = (int)(want < (int64_t)ctx->sm_count * 8 ? want : (int64_t)ctx->sm_count * 8);
+  LaunchScope ls(ctx, KIND_SHIFTMAX, (double)rows * (double)d * 5.0);
+  const int wpl = (int)(((d + 15) / 16 * 4 + 31) / 32);
+  if (wpl <= 2) launch_k(shiftmax_direct_kernel<2>, dim3(grid), dim3(256), 0, ctx->stream, in, ldin, c, out, ldout, rows, (int)d);
+  else if (wpl <= 5) launch_k(shiftmax_direct_kernel<5>, dim3(grid), dim3(256), 0, ctx->stream, in, ldin, c, out, ldout, rows, (int)d);
+  else launch_k(shiftmax_direct_kernel<0>, dim3(grid), dim3(256), 0, ctx->stream, in, ldin, c, out, ldout, rows, (int)d);
+  return ls.done();
+}
+
 // ------------------------------------------------------------------ ShiftGELU
 
 // Because the input is int8 and the row statistic is I_max = max(0, I_p(max_row x)), the output
@@ -584,7 +708,7 @@ __global__ void shiftgelu_table_kernel(ivit_exp_params p, int post_m, int post_s
     int div = 0;
     if (den != 0) {
       const unsigned long long f = (1ull << 45) / den;  // Eq. (IntDiv), M = 45
-      div = (int)((f * e) >> 38);                         // k_out = 8; f*e <= 2^45
+      div = (int)((f * e) >> (46 - p.k_out));             // f*e <= 2^45
     }
     out = sat8(rq(x * div, post_m, post_s));
   }

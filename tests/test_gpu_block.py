@@ -118,3 +118,28 @@ def test_block_static_gelu_variant_bit_exact(engine, B, T, D, heads, H):
     g.assert_equal(g.host(Yp), O.block_forward(plain, X), "block, Algorithm 2")
     assert c.poll_status() == 0
     c.set_gemm_engine(0)
+
+
+@pytest.mark.parametrize("k_out", [6, 4])
+def test_block_other_output_width_bit_exact(k_out):
+    """A block whose Shiftmax and ShiftGELU use k_out < 8: the attention core runs as separate kernels (the fused one
+    is built for 8 bits); P*V and the GELU output ratios absorb the coarser scale 1 / 2^(k_out-1)."""
+    import dataclasses
+    from ivit_inputs import ExpParams, Scale
+    g = _g()
+    c = g.ctx()
+    blk = make_block(_Ids(500 + k_out), 1, 2, 197, 192, 3, 768)
+    up = 8 - k_out
+    blk = dataclasses.replace(
+        blk,
+        smax=ExpParams(blk.smax.I0, blk.smax.N, 45, k_out), gelu=ExpParams(blk.gelu.I0, blk.gelu.N, 45, k_out),
+        pv_scale=Scale(blk.pv_scale.mult, max(31, blk.pv_scale.shift - up)),
+        gelu_post=Scale(blk.gelu_post.mult, max(31, blk.gelu_post.shift - up)))
+    X = make_block_input(13, 2, 197, 192)
+    dblk = g.binding.DeviceBlock(blk, "cuda")
+    Y = c.block_forward(dblk, torch.from_numpy(X).cuda())
+    want = O.block_forward(blk, X)
+    g.assert_equal(g.host(Y), want, f"block k_out={k_out}")
+    assert len(np.unique(want)) > 50
+    assert c.poll_status() == 0
+

@@ -159,6 +159,87 @@ def test_shiftmax_parity(rows, d, I0):
     g.assert_equal(g.host(out), O.shiftmax(acc, p, pre=pre, bias32=bias), "shiftmax i32")
 
 
+@pytest.mark.parametrize("k_out", [2, 5, 7])
+def test_shiftmax_and_gelu_other_output_widths(k_out):
+    """Algorithm 1 / 2 with k_out < 8 (Eq. (IntDiv) shifts by M - (k_out - 1)), both Shiftmax entry forms and ShiftGELU."""
+    g = _g()
+    c = g.ctx()
+    rng = np.random.default_rng(900 + k_out)
+    for rows, d, I0 in [(60, 197, 11), (7, 49, 20), (3, 1, 16), (5, 3000, 4)]:
+        x = rand_i8(rng, (rows, d), 32)
+        x[1 % rows, :] = 5
+        p = ExpParams(I0, 15, 45, k_out)
+        got = g.host(c.shiftmax(g.dev(x), p))
+        g.assert_equal(got, O.shiftmax(x, p), f"shiftmax i8 k_out={k_out}")
+        assert got.max() <= 2 ** (k_out - 1) - 1
+        acc = (rng.standard_normal((rows, d)) * 9000).astype(np.int32)
+        pre = Scale(*dyadic(30.0 / 8192))
+        out = c.shiftmax(g.dev(acc, 4), p, pre=g.binding.DevScale(pre, "cuda"))
+        g.assert_equal(g.host(out), O.shiftmax(acc, p, pre=pre), f"shiftmax i32 k_out={k_out}")
+    xg = rand_i8(rng, (37, 304), 45)
+    xg[0, :256] = np.arange(-128, 128).astype(np.int8)
+    pg = ExpParams(32, 23, 45, k_out)
+    post = Scale(*dyadic(1.0 / (2 ** (k_out - 1) * 0.8)))
+    g.assert_equal(g.host(c.shiftgelu(g.dev(xg), pg, g.binding.DevScale(post, "cuda"))), O.shiftgelu(xg, pg, post),
+                   f"shiftgelu k_out={k_out}")
+    g.assert_equal(g.host(c.shiftgelu(g.dev(xg), pg, g.binding.DevScale(post, "cuda"), static_max=True)),
+                   O.shiftgelu(xg, pg, post, static_max=True), f"shiftgelu static k_out={k_out}")
+    assert c.poll_status() == 0
+
+
+@pytest.mark.parametrize("rows,d", [(1, 1), (3, 2), (50, 49), (400, 197), (130, 577), (33, 64), (9, 1024), (5, 3000),
+                                    (6, 8192), (40, 255), (40, 257), (12, 640), (12, 641)])
+@pytest.mark.parametrize("I0,N,M,k_out", [(1, 20, 52, 8), (23000, 10, 52, 8), (65536, 8, 52, 8), (1 << 24, 4, 62, 8),
+                                           (1 << 28, 0, 62, 8), (1000, 15, 55, 5), (11, 15, 45, 8)])
+def test_shiftmax_direct_parity(rows, d, I0, N, M, k_out):
+    """ivit_shiftmax_direct (Algorithm 1 on int32 scores, nothing in front) against the oracle: every register
+    variant of the kernel, ragged rows, scores of a few units at scale 1 / I0, the full int32 range in one row,
+    exact octaves, constant rows, and poisoned padding between d and the row stride."""
+    g = _g()
+    c = g.ctx()
+    if d * I0 * 2 ** N > 2 ** (M - 13):
+        with pytest.raises(Exception):
+            c.shiftmax_direct(torch.zeros((rows, (d + 3) // 4 * 4), dtype=torch.int32, device="cuda")[:, :d],
+                              ExpParams(I0, N, M, k_out))
+        return
+    rng = np.random.default_rng(rows * 31 + d + N)
+    p = ExpParams(I0, N, M, k_out)
+    x = np.clip(np.rint(rng.standard_normal((rows, d)) * 2.5 * I0), -2 ** 31, 2 ** 31 - 1).astype(np.int32)
+    x[0, :] = np.clip(-16 * max(1, I0 // 23) * rng.integers(0, 60, d), -2 ** 31, 0)   # whole octaves when 23 divides I0
+    if rows > 1:
+        x[1, :] = 123456                                                   # constant row
+    if rows > 2:
+        x[2, :] = rng.choice(np.array([-2 ** 31, 2 ** 31 - 1, 0, -1, 2 ** 31 - 2], dtype=np.int64), d).astype(np.int32)
+    if rows > 3:
+        x[3, :] = -2 ** 31                                                 # the most negative value everywhere
+    if rows > 4:
+        x[4, :] = np.clip(2 ** 31 - 1 - rng.integers(0, 40 * I0 + 2, d), -2 ** 31, 2 ** 31 - 1)   # steps below the int32 maximum
+    ld = (d + 3) // 4 * 4 + 8
+    buf = torch.full((rows, ld), 2 ** 31 - 1, dtype=torch.int32, device="cuda")   # padding larger than any score
+    buf[:, :d] = torch.from_numpy(x).cuda()
+    out = c.shiftmax_direct(buf[:, :d], p)
+    g.assert_equal(g.host(out), O.shiftmax_direct(x, p), "shiftmax direct")
+    base = out._base if out._base is not None else out
+    assert (g.host(base)[:, d:((d + 15) // 16) * 16] == 0).all()
+    assert c.poll_status() == 0
+
+
+def test_shiftmax_direct_argument_checks():
+    g = _g()
+    c = g.ctx()
+    x = torch.zeros((4, 64), dtype=torch.int32, device="cuda")
+    ok = ExpParams(1000, 10, 50, 8)
+    c.shiftmax_direct(x, ok)
+    for bad in [ExpParams(0, 10, 50, 8), ExpParams((1 << 28) + 1, 0, 62, 8), ExpParams(1000, 25, 62, 8),
+                ExpParams(1000, 10, 63, 8), ExpParams(1000, 10, 31, 8), ExpParams(1000, 10, 50, 9),
+                ExpParams(1000, 10, 50, 1), ExpParams(1 << 20, 10, 45, 8)]:
+        with pytest.raises(Exception):
+            c.shiftmax_direct(x, bad)
+    with pytest.raises(Exception):
+        c.shiftmax_direct(torch.zeros((4, 66), dtype=torch.int32, device="cuda")[:, 1:65], ok)   # misaligned rows
+    assert c.poll_status() == 0
+
+
 def test_shiftexp_and_gelu_exhaustive_domain():
     """All 256 int8 inputs against every possible row maximum, several I0: the whole ShiftGELU domain."""
     g = _g()
