@@ -68,6 +68,69 @@ def test_vit_base_b128_full_size_sampled():
     assert c.poll_status() == 0
 
 
+def test_deit_small_b64_full_size_graph_replay_sampled():
+    """Config 1 at its full size in the launch configuration the benchmark times: the whole forward captured into
+    one CUDA graph on a side stream and replayed (twice, the second time on a changed input buffer); sampled images
+    are recomputed by the oracle."""
+    g = _g()
+    dev = torch.device("cuda", 0)
+    c = g.binding.Context(0)
+    side = torch.cuda.Stream(device=dev)
+    model, image = make_config(1)
+    dm = g.binding.DeviceVit(model, dev)
+    ws = dm.host_workspace()
+    with torch.cuda.stream(side):
+        c.set_stream(side)
+        d_image = torch.from_numpy(image).to(dev)
+        d_logits = torch.zeros((model.B, model.classes), dtype=torch.int32, device=dev)
+        for _ in range(2):                     # tables, attributes and tensor maps exist before the capture
+            c.vit_forward(dm, d_image, logits=d_logits, workspace=ws)
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            c.vit_forward(dm, d_image, logits=d_logits, workspace=ws)
+        d_logits.zero_()
+        graph.replay()
+        side.synchronize()
+        logits = g.host(d_logits)
+        for i in (0, 37, 63):
+            g.assert_equal(logits[i:i + 1], O.vit_forward(model, image[i:i + 1]), f"replay 1, image {i}")
+        # same graph, new pixels in the same buffer
+        image2 = np.ascontiguousarray(image[::-1])
+        d_image.copy_(torch.from_numpy(image2).to(dev))
+        graph.replay()
+        side.synchronize()
+        logits2 = g.host(d_logits)
+        g.assert_equal(logits2, logits[::-1], "replay 2 (batch reversed)")
+    assert c.poll_status() == 0
+
+
+def test_vit_large_384_b32_full_size_sampled():
+    """Config 4 at its full size (batch 32, 24 blocks, 577 tokens: attention composed from MatMul and Shiftmax
+    kernels); the oracle recomputes one sampled image."""
+    g = _g()
+    c = g.ctx()
+    model, image = make_config(4)
+    dm = g.binding.DeviceVit(model, "cuda")
+    logits = g.host(c.vit_forward(dm, torch.from_numpy(image).cuda()))
+    g.assert_equal(logits[31:32], O.vit_forward(model, image[31:32]), "image 31")
+    assert c.poll_status() == 0
+
+
+def test_swin_tiny_b64_full_size_sampled():
+    """Config 3 at its full size (batch 64); the oracle recomputes sampled images."""
+    g = _g()
+    c = g.ctx()
+    model, image = make_config(3)
+    dm = g.binding.DeviceSwin(model, "cuda")
+    logits = g.host(g.binding.swin_forward(c, dm, torch.from_numpy(image).cuda()))
+    one, _ = make_config(3, batch=1)      # the same weights with the window counts of a single image
+    assert np.array_equal(one.Wpe, model.Wpe)
+    for i in (0, 63):
+        g.assert_equal(logits[i:i + 1], O.swin_forward(one, image[i:i + 1]), f"image {i}")
+    assert c.poll_status() == 0
+
+
 def test_host_forward_back_to_back_calls():
     """ivit_vit_forward_host enqueued four times without a synchronisation in between: the input copy of a call
     overlaps the compute of the call before it (two staging buffers), and every call must still see its own image."""
