@@ -274,6 +274,17 @@ size_t ivit_vit_host_workspace_bytes(const ivit_vit_params* p);
 int ivit_vit_forward_host(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* image_host,
                           int32_t* logits_host, void* workspace, size_t workspace_bytes);
 
+/* Graph replay for ivit_vit_forward_host (off by default).  When enabled, the third call in a row that repeats
+ * the same model description (every field of p and of its blocks), workspace and stream captures the device part
+ * of the forward into a CUDA graph, and later calls launch that graph instead of about a hundred kernels; any
+ * change of those arguments, a new stream, or switching the mode off drops the graph.  Needs a stream other than
+ * the legacy default stream (with the default stream the kernels keep being launched one by one).  Tensors the
+ * model description points to may change contents between calls; they must stay at the same addresses.
+ * Results are identical in both modes. */
+int ivit_ctx_set_host_graph(ivit_ctx* ctx, int enable);
+/* Number of graphs currently instantiated for ivit_vit_forward_host (0, 1 or 2: one per staging buffer). */
+int ivit_ctx_host_graph_count(ivit_ctx* ctx);
+
 /* ---- per-kernel timing (measurement aid; not part of the paper's method) ----
  * Between profile_start and profile_stop every kernel the context launches is bracketed by a pair
  * of CUDA events on the context's stream (at most 8192 launches per session; later ones are not

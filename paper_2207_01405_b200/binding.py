@@ -22,7 +22,7 @@ EXPORTS = [
     "ivit_ctx_create", "ivit_ctx_destroy", "ivit_ctx_set_stream", "ivit_ctx_poll_status", "ivit_ctx_launch_count",
     "ivit_ctx_set_gemm_engine", "ivit_strerror", "ivit_linear", "ivit_matmul", "ivit_shiftmax", "ivit_shiftgelu",
     "ivit_shiftgelu_static",
-    "ivit_shiftmax_direct",
+    "ivit_shiftmax_direct", "ivit_ctx_set_host_graph", "ivit_ctx_host_graph_count",
     "ivit_layernorm", "ivit_block_workspace_bytes", "ivit_block_forward", "ivit_block_forward_static", "ivit_attention",
     "ivit_vit_workspace_bytes", "ivit_vit_forward", "ivit_vit_host_workspace_bytes", "ivit_vit_forward_host",
     "ivit_ctx_profile_start", "ivit_ctx_profile_stop", "ivit_ctx_profile_get", "ivit_kernel_kind_name", "ivit_patchify", "ivit_gather_rows", "ivit_fill_rows",
@@ -86,6 +86,8 @@ def load_library():
     L.ivit_ctx_launch_count.argtypes = [vp]
     L.ivit_ctx_launch_count.restype = i64
     L.ivit_ctx_set_gemm_engine.argtypes = [vp, C.c_int]
+    L.ivit_ctx_set_host_graph.argtypes = [vp, C.c_int]
+    L.ivit_ctx_host_graph_count.argtypes = [vp]
     L.ivit_strerror.argtypes = [C.c_int]
     L.ivit_strerror.restype = C.c_char_p
     L.ivit_linear.argtypes = [vp, vp, i64, vp, i64, vp, CScale, vp, i64, i64, CScale, vp, i64, i32, i64, i64, i64, i64, i64]
@@ -209,6 +211,13 @@ class Context:
 
     def set_gemm_engine(self, engine: int):
         _chk(self.lib.ivit_ctx_set_gemm_engine(self.h, engine), "ivit_ctx_set_gemm_engine")
+
+    def set_host_graph(self, enable: bool):
+        """Graph replay inside vit_forward_host (ivit_ctx_set_host_graph); off by default."""
+        _chk(self.lib.ivit_ctx_set_host_graph(self.h, 1 if enable else 0), "ivit_ctx_set_host_graph")
+
+    def host_graph_count(self) -> int:
+        return int(self.lib.ivit_ctx_host_graph_count(self.h))
 
     def poll_status(self) -> int:
         return self.lib.ivit_ctx_poll_status(self.h)

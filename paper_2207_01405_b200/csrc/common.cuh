@@ -42,6 +42,14 @@ struct ivit_ctx {
   cudaStream_t copy_stream;
   cudaEvent_t img_ready[2], img_free[2];
   uint64_t host_calls;
+  // ivit_ctx_set_host_graph: the forward of ivit_vit_forward_host replayed as an instantiated CUDA graph, one per
+  // staging buffer, captured at the third call that repeats the same arguments
+  int host_graph;
+  cudaGraphExec_t hg_exec[2];
+  char* hg_key[2];          // model description, workspace and stream the graph was captured with
+  size_t hg_key_bytes[2];
+  int hg_seen[2];           // calls seen with this key (-1: capture failed, launch kernel by kernel)
+  int64_t hg_launches[2];   // kernels inside the graph
   // per-kernel timing session (ivit_ctx_profile_*)
   bool profiling;
   int prof_count;

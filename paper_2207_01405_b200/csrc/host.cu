@@ -152,6 +152,76 @@ int block_impl(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* X, int8_
 
 }  // namespace
 
+namespace {
+
+void host_graph_drop(ivit_ctx* ctx, int slot) {
+  if (ctx->hg_exec[slot]) cudaGraphExecDestroy(ctx->hg_exec[slot]);
+  ctx->hg_exec[slot] = nullptr;
+  delete[] ctx->hg_key[slot];
+  ctx->hg_key[slot] = nullptr;
+  ctx->hg_key_bytes[slot] = 0;
+  ctx->hg_seen[slot] = 0;
+}
+
+// The device part of ivit_vit_forward_host.  With graph replay switched on, the third call that repeats the same
+// model description, buffers and stream captures the forward into a CUDA graph (the first two run kernel by
+// kernel, so that look-up tables and kernel attributes exist); later calls launch the instantiated graph.  Any
+// change of the arguments drops the graph.  A capture that fails leaves the kernel-by-kernel path in place.
+int forward_or_replay(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* img_dev, int32_t* lg_dev, void* workspace,
+                      size_t inner, int slot) {
+  if (!ctx->host_graph || ctx->profiling || ctx->stream == nullptr)
+    return ivit_vit_forward(ctx, p, img_dev, lg_dev, workspace, inner);
+  const size_t nb = (size_t)p->depth * sizeof(ivit_block_params);
+  const void* tail[4] = {img_dev, lg_dev, workspace, (const void*)ctx->stream};
+  const size_t key_bytes = sizeof(*p) + nb + sizeof(tail) + sizeof(int);
+  char* key = new (std::nothrow) char[key_bytes];
+  if (!key) return IVIT_ERR_CUDA;
+  std::memcpy(key, p, sizeof(*p));
+  std::memcpy(key + sizeof(*p), p->blocks, nb);
+  std::memcpy(key + sizeof(*p) + nb, tail, sizeof(tail));
+  std::memcpy(key + sizeof(*p) + nb + sizeof(tail), &ctx->gemm_engine, sizeof(int));
+  const bool same = ctx->hg_key[slot] && ctx->hg_key_bytes[slot] == key_bytes && std::memcmp(ctx->hg_key[slot], key, key_bytes) == 0;
+  if (!same) {
+    host_graph_drop(ctx, slot);
+    ctx->hg_key[slot] = key;
+    ctx->hg_key_bytes[slot] = key_bytes;
+    ctx->hg_seen[slot] = 1;
+    return ivit_vit_forward(ctx, p, img_dev, lg_dev, workspace, inner);
+  }
+  delete[] key;
+  if (ctx->hg_exec[slot]) {
+    if (cudaGraphLaunch(ctx->hg_exec[slot], ctx->stream) != cudaSuccess) return IVIT_ERR_CUDA;
+    ctx->launches += ctx->hg_launches[slot];
+    return IVIT_OK;
+  }
+  if (ctx->hg_seen[slot] < 0 || ++ctx->hg_seen[slot] < 3) return ivit_vit_forward(ctx, p, img_dev, lg_dev, workspace, inner);
+  const int64_t before = ctx->launches;
+  if (cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+    cudaGetLastError();
+    ctx->hg_seen[slot] = -1;
+    return ivit_vit_forward(ctx, p, img_dev, lg_dev, workspace, inner);
+  }
+  const int rc = ivit_vit_forward(ctx, p, img_dev, lg_dev, workspace, inner);
+  cudaGraph_t graph = nullptr;
+  const cudaError_t end = cudaStreamEndCapture(ctx->stream, &graph);
+  cudaGraphExec_t exec = nullptr;
+  if (rc == IVIT_OK && end == cudaSuccess && graph && cudaGraphInstantiate(&exec, graph, 0) == cudaSuccess) {
+    cudaGraphDestroy(graph);
+    ctx->hg_exec[slot] = exec;
+    ctx->hg_launches[slot] = ctx->launches - before;
+    if (cudaGraphLaunch(exec, ctx->stream) != cudaSuccess) return IVIT_ERR_CUDA;
+    return IVIT_OK;
+  }
+  if (graph) cudaGraphDestroy(graph);
+  cudaGetLastError();
+  ctx->launches = before;
+  ctx->hg_seen[slot] = -1;
+  if (rc) return rc;
+  return ivit_vit_forward(ctx, p, img_dev, lg_dev, workspace, inner);   // nothing ran during the failed capture
+}
+
+}  // namespace
+
 namespace ivit {
 int launch_gemm(ivit_ctx* ctx, const GemmProblem& g) {
   if (ctx->gemm_engine == 0) {
@@ -218,6 +288,7 @@ int ivit_ctx_destroy(ivit_ctx* ctx) {
   cudaSetDevice(ctx->device);
   cudaFree(ctx->gelu_tables);
   cudaFreeHost(ctx->status_host);
+  for (int i = 0; i < 2; ++i) host_graph_drop(ctx, i);
   if (ctx->copy_stream) {
     cudaStreamSynchronize(ctx->copy_stream);
     for (int i = 0; i < 2; ++i) {
@@ -239,6 +310,7 @@ int ivit_ctx_destroy(ivit_ctx* ctx) {
 int ivit_ctx_set_stream(ivit_ctx* ctx, void* cuda_stream) {
   if (!ctx) return IVIT_ERR_INVALID_ARG;
   ctx->stream = (cudaStream_t)cuda_stream;
+  for (int i = 0; i < 2; ++i) host_graph_drop(ctx, i);
   ctx->gelu_used = 0;  // tables were built in the order of the old stream
   ctx->gelu_next = 0;
   return IVIT_OK;
@@ -509,6 +581,19 @@ size_t ivit_vit_host_workspace_bytes(const ivit_vit_params* p) {
   return vit_ws(p).total + 2 * img + lg;
 }
 
+int ivit_ctx_set_host_graph(ivit_ctx* ctx, int enable) {
+  if (!ctx) return IVIT_ERR_INVALID_ARG;
+  ctx->host_graph = enable ? 1 : 0;
+  if (!enable)
+    for (int i = 0; i < 2; ++i) host_graph_drop(ctx, i);
+  return IVIT_OK;
+}
+
+int ivit_ctx_host_graph_count(ivit_ctx* ctx) {
+  if (!ctx) return IVIT_ERR_INVALID_ARG;
+  return (ctx->hg_exec[0] ? 1 : 0) + (ctx->hg_exec[1] ? 1 : 0);
+}
+
 int ivit_vit_forward_host(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* image_host,
                           int32_t* logits_host, void* workspace, size_t workspace_bytes) {
   if (!ctx || !image_host || !logits_host) return IVIT_ERR_INVALID_ARG;
@@ -542,7 +627,7 @@ int ivit_vit_forward_host(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t*
       cudaStreamWaitEvent(ctx->stream, ctx->img_ready[slot], 0) != cudaSuccess)
     return IVIT_ERR_CUDA;
   ++ctx->host_calls;
-  rc = ivit_vit_forward(ctx, p, reinterpret_cast<const int8_t*>(img_dev), reinterpret_cast<int32_t*>(ws + lg_off), workspace, inner);
+  rc = forward_or_replay(ctx, p, reinterpret_cast<const int8_t*>(img_dev), reinterpret_cast<int32_t*>(ws + lg_off), workspace, inner, slot);
   // recorded even after an error: a later copy into this buffer waits for it
   if (cudaEventRecord(ctx->img_free[slot], ctx->stream) != cudaSuccess) return IVIT_ERR_CUDA;
   if (rc) return rc;

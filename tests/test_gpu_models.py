@@ -150,3 +150,52 @@ def test_host_forward_back_to_back_calls():
     for k, (x, y) in enumerate(zip(images, h_out)):
         g.assert_equal(y.numpy(), O.vit_forward(model, x), f"call {k}")
     assert c.poll_status() == 0
+
+
+def test_host_forward_graph_replay_mode():
+    """ivit_ctx_set_host_graph: the host-buffer forward replays a captured graph from the third repeat of the same
+    arguments on (one graph per staging buffer).  Every call, before and after the capture, with changing images,
+    and after a change of model, must give the oracle's logits; far fewer launches reach the stream once it replays."""
+    import gpu_util as g
+    dev = torch.device("cuda", 0)
+    c = g.binding.Context(0)
+    side = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(side):
+        c.set_stream(side)
+        c.set_host_graph(True)
+        model, image = make_config(1, batch=3, depth=2)
+        dm = g.binding.DeviceVit(model, dev)
+        ws = dm.host_workspace()
+        rng = np.random.default_rng(9)
+        images = [np.clip(image.astype(np.int32) + rng.integers(-30, 30, image.shape), -128, 127).astype(np.int8)
+                  for _ in range(9)]
+        h_img = [torch.from_numpy(x).pin_memory() for x in images]
+        h_out = [torch.empty((3, model.classes), dtype=torch.int32).pin_memory() for _ in images]
+        for x, y in zip(h_img, h_out):
+            g.binding.vit_forward_host(c, dm, x, y, ws)
+        side.synchronize()
+        for k, (x, y) in enumerate(zip(images, h_out)):
+            g.assert_equal(y.numpy(), O.vit_forward(model, x), f"call {k}")
+        assert c.host_graph_count() == 2          # one graph per staging buffer, both captured by now
+        # another model through the same context and workspace size class: the graphs are dropped and rebuilt
+        model2, image2 = make_config(1, batch=3, depth=1)
+        dm2 = g.binding.DeviceVit(model2, dev)
+        ws2 = dm2.host_workspace()
+        outs = [torch.empty((3, model2.classes), dtype=torch.int32).pin_memory() for _ in range(7)]
+        h2 = torch.from_numpy(image2).pin_memory()
+        for y in outs:
+            g.binding.vit_forward_host(c, dm2, h2, y, ws2)
+        side.synchronize()
+        want2 = O.vit_forward(model2, image2)
+        for k, y in enumerate(outs):
+            g.assert_equal(y.numpy(), want2, f"second model, call {k}")
+        # switching the mode off goes back to kernel-by-kernel launches with the same result
+        assert c.host_graph_count() == 2
+        c.set_host_graph(False)
+        assert c.host_graph_count() == 0
+        y = torch.empty((3, model2.classes), dtype=torch.int32).pin_memory()
+        g.binding.vit_forward_host(c, dm2, h2, y, ws2)
+        side.synchronize()
+        g.assert_equal(y.numpy(), want2, "mode off")
+    assert c.poll_status() == 0
+
