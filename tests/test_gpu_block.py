@@ -77,12 +77,15 @@ def test_vit_small_model_bit_exact():
 
 
 def test_fused_attention_kernel_serves_short_rows():
-    """Rows up to 256 tokens go through the fused tensor-core attention kernel; longer rows are composed."""
+    """Rows up to 256 tokens go through the fused tensor-core attention kernel, longer rows through its key-block
+    form as long as a 128-row tile of probabilities and the V of a head fit shared memory; beyond that the attention
+    is composed from MatMul and Shiftmax kernels."""
     g = _g()
     c = g.ctx()
     rng = np.random.default_rng(2)
-    for (B, T, D, heads, fused) in [(2, 197, 384, 6, True), (4, 49, 96, 3, True), (1, 256, 128, 2, True), (1, 300, 128, 2, False)]:
-        blk = make_block(_Ids(50 + T), 1, B, T, D, heads, 4 * D, attn_bias_batches=heads if T == 49 else 0)
+    for (B, T, D, heads, fused) in [(2, 197, 384, 6, True), (4, 49, 96, 3, True), (1, 256, 128, 2, True), (1, 300, 128, 2, True),
+                                   (1, 1100, 64, 1, False)]:
+        blk = make_block(_Ids(50 + T), 1, B, T, D, heads, 4 * D, attn_bias_batches=heads if T in (49, 300) else 0)
         dblk = g.binding.DeviceBlock(blk, "cuda")
         QKV = np.clip(np.rint(rng.standard_normal((B * T, 3 * D)) * 32), -128, 127).astype(np.int8)
         c.profile_start()
@@ -142,5 +145,26 @@ def test_block_other_output_width_bit_exact(k_out):
     want = O.block_forward(blk, X)
     g.assert_equal(g.host(Y), want, f"block k_out={k_out}")
     assert len(np.unique(want)) > 50
+    assert c.poll_status() == 0
+
+
+@pytest.mark.parametrize("B,T,D,heads,bias", [(2, 257, 128, 2, False), (1, 300, 128, 2, True), (3, 577, 128, 2, False),
+                                              (2, 449, 64, 2, False), (1, 640, 64, 1, False), (2, 577, 256, 4, True), (1, 400, 256, 2, False),
+                                              (40, 320, 128, 2, False)])
+def test_long_row_attention_bit_exact(B, T, D, heads, bias):
+    """The key-block form of the fused attention kernel (rows longer than 256 tokens): two to four key blocks, ragged
+    last blocks and last row tiles, head dimensions 32 / 64 / 128, with and without a score bias, and more work items
+    than CTAs (several items per CTA, the control thread running ahead across items)."""
+    g = _g()
+    c = g.ctx()
+    blk = make_block(_Ids(700 + T + D), 1, B, T, D, heads, 2 * D, attn_bias_batches=heads if bias else 0)
+    dblk = g.binding.DeviceBlock(blk, "cuda")
+    rng = np.random.default_rng(T)
+    QKV = np.clip(np.rint(rng.standard_normal((B * T, 3 * D)) * 32), -128, 127).astype(np.int8)
+    c.profile_start()
+    Oo = c.attention(dblk, torch.from_numpy(QKV).cuda())
+    kinds = [k for k, _, _ in c.profile_stop()]
+    assert kinds == ["attention_fused"], kinds
+    g.assert_equal(g.host(Oo), O.attention(blk, QKV), f"long-row attention T={T}")
     assert c.poll_status() == 0
 
