@@ -13,6 +13,7 @@
 //           that the second MMA consumes as its A operand.
 // V is consumed as stored ([token, d] rows, MN-major B operand).  Every wait is bounded.
 #include "tc_ptx.cuh"
+#include <cstdlib>
 
 namespace ivit {
 
@@ -549,9 +550,9 @@ __global__ void __launch_bounds__(kLongThreads, 1) attention_long_kernel(const _
         if (next >= 0) {
           load_q(next); q_fly = true; q_par = (n + 1) & 1u;
           // The item barrier may run one phase ahead of its readers at most: every Shiftmax warp has taken item n
-          // once it has handed back the score buffer of that item's first key block.
-          const uint32_t g0 = g - (uint32_t)nblk;
-          ok = mbar_wait(bar_f + 8 * (g0 & 1u), (g0 >> 1) & 1u, a.status);
+          // once it has handed back the score buffer of that item's last key block (the latest phase of that
+          // barrier: the block that completes it next has not been issued yet).
+          ok = mbar_wait(bar_f + 8 * ((g - 1) & 1u), ((g - 1) >> 1) & 1u, a.status);
           if (!ok) break;
           publish(n + 1, next);
           issue_block(next, 0, n + 1, -1);   // nblk >= 2: the block after it belongs to the same item
@@ -811,7 +812,10 @@ static int launch_attention_long(ivit_ctx* ctx, const ivit_block_params* p, cons
   a.Npad = (int)((T + 31) / 32 * 32);
   a.tiles_m = (int)((T + 127) / 128);
   a.tmem_cols = 512;
-  const int nb_max = ((512 - (int)d) / 2) / 32 * 32 > 224 ? 224 : ((512 - (int)d) / 2) / 32 * 32;   // two score buffers + d output columns
+  int nb_max = ((512 - (int)d) / 2) / 32 * 32 > 224 ? 224 : ((512 - (int)d) / 2) / 32 * 32;   // two score buffers + d output columns
+#ifdef IVIT_TUNING
+  if (const char* e = getenv("IVIT_ATTN_LONG")) { const int f = atoi(e); if (f >= 32 && f < nb_max) nb_max = f; }   // stress runs only
+#endif
   la.nblk = (a.Npad + nb_max - 1) / nb_max;
   la.NB = ((a.Npad + la.nblk - 1) / la.nblk + 31) / 32 * 32;
   la.nv = (a.Npad + 255) / 256;
@@ -858,6 +862,9 @@ int launch_attention_fused(ivit_ctx* ctx, const ivit_block_params* p, const int8
   if (p->smax.k_out != 8) return IVIT_ERR_UNSUPPORTED;   // the fused kernels have the 8-bit IntDiv shift built in
   if ((reinterpret_cast<uintptr_t>(QKV) & 15) || (reinterpret_cast<uintptr_t>(O) & 15)) return IVIT_ERR_UNSUPPORTED;
   if (B == 0) return IVIT_OK;
+#ifdef IVIT_TUNING
+  if (getenv("IVIT_ATTN_LONG") && T > 64) return launch_attention_long(ctx, p, QKV, O);   // stress runs only
+#endif
   if (T > 256) return launch_attention_long(ctx, p, QKV, O);
   AttnArgs a{};
   a.T = (int)T; a.d = (int)d; a.heads = (int)h; a.D = D;
