@@ -29,6 +29,8 @@ struct AttnArgs {
   int tiles_m;                      // ceil(T / 128)
   int bh;                           // images (or windows) x heads
   int items;                        // bh * tiles_m
+  int G, R;                         // G windows of at most R = 128 / G tokens share one tile (G = 1: one image or window per tile)
+  int Btot;                         // images or windows in the tensor
   int tmem_cols;
   int qk_m, qk_s, pv_m, pv_s;
   ivit_exp_params smax;
@@ -106,9 +108,9 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
         const int h = bhid % a.heads, b = bhid / a.heads;
         mbar_expect_tx(bar_qk, 128 * 128 + a.Npad * 128);
         int c[4];
-        c[0] = 0; c[a.q_pos[0]] = tile * 128; c[a.q_pos[1]] = h; c[a.q_pos[2]] = b;
+        c[0] = 0; c[a.q_pos[0]] = tile * 128; c[a.q_pos[1]] = h; c[a.q_pos[2]] = b * a.G;
         tma_load_4d(base + q_off, &tmQ, bar_qk, c[0], c[1], c[2], c[3]);
-        c[0] = 0; c[a.k_pos[0]] = 0; c[a.k_pos[1]] = h; c[a.k_pos[2]] = b;
+        c[0] = 0; c[a.k_pos[0]] = 0; c[a.k_pos[1]] = h; c[a.k_pos[2]] = b * a.G;
         tma_load_4d(base + k_off, &tmK, bar_qk, c[0], c[1], c[2], c[3]);
       };
       auto load_v = [&](int item) {
@@ -116,7 +118,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
         const int h = bhid % a.heads, b = bhid / a.heads;
         mbar_expect_tx(bar_v, a.Npad * a.d);
         int c[4];
-        c[0] = 0; c[a.v_pos[0]] = 0; c[a.v_pos[1]] = h; c[a.v_pos[2]] = b;
+        c[0] = 0; c[a.v_pos[0]] = 0; c[a.v_pos[1]] = h; c[a.v_pos[2]] = b * a.G;
         tma_load_4d(base + v_off, &tmV, bar_v, c[0], c[1], c[2], c[3]);
       };
       auto draw = [&]() {
@@ -207,12 +209,18 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
       const int item = got_item ? item_ring[par] : -1;
       if (item < 0) break;
       const int tile = item / a.bh, bhid = item - tile * a.bh;
-      const int h = bhid % a.heads, b = bhid / a.heads;
+      const int h = bhid % a.heads;
+      // G > 1: the tile holds G windows of R rows each (window `slot` in rows and columns slot R .. slot R + R - 1 of
+      // the block-diagonal score tile); a warp's 32 rows lie inside one window
+      const int slot = a.G > 1 ? trow / a.R : 0;
+      const int b = (bhid / a.heads) * a.G + slot;  // image / window of this row
       const int m0 = tile * 128;
-      const int r = m0 + trow;                      // token (row) inside this image / window
-      const bool row_ok = r < a.T;
-      const bool warp_ok = m0 + qd * 32 < a.T;      // warps whose 32 rows all lie past T only keep the barriers
-      const int32_t* brow = a.bias ? a.bias + (((int64_t)bhid % a.bias_batches) * a.T + (row_ok ? r : 0)) * (int64_t)a.T : nullptr;
+      const int r = m0 + trow - slot * a.R;         // token (row) inside this image / window
+      const bool row_ok = r < a.T && b < a.Btot;
+      const bool warp_ok = m0 + qd * 32 - slot * a.R < a.T && b < a.Btot;   // warps whose 32 rows all lie past T only keep the barriers
+      const int col0 = slot * a.R;                  // first score column of this row's window
+      const int c_lo = col0 >> 4, c_hi = a.G > 1 ? c_lo + (a.R >> 4) : nch;   // this row's 16-column chunks
+      const int32_t* brow = a.bias ? a.bias + ((((int64_t)b * a.heads + h) % a.bias_batches) * a.T + (row_ok ? r : 0)) * (int64_t)a.T - col0 : nullptr;
 
       int mx = -128;
       bool got_s = mbar_wait(bar_s, par, a.status);
@@ -224,13 +232,13 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
         // code stays within the instruction cache); what a later pass needs of a chunk waits in the chunk's own
         // tensor-memory columns.
 #pragma unroll 1
-        for (int c = half; c < nch; c += 2) {
+        for (int c = c_lo + half; c < c_hi; c += 2) {
           int v[16];
           tmem_ld16(t_row + c * 16, v);
           if (brow) {
 #pragma unroll
             for (int j = 0; j < 16; ++j)
-              if (c * 16 + j < a.T) v[j] += __ldg(brow + c * 16 + j);
+              if (c * 16 + j - col0 < a.T) v[j] += __ldg(brow + c * 16 + j);
           }
           if (qk_hi) {          // the usual case: high product word plus 2^(s-33), shifted by s - 32
 #pragma unroll
@@ -240,10 +248,10 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
             for (int j = 0; j < 16; ++j) v[j] = (int)(((long long)v[j] * a.qk_m + qk_c) >> a.qk_s);
           }
           // columns past T (only in the last two chunks) never win the maximum and look up a valid table entry
-          if (c >= nch - 2) {
+          if (c >= c_hi - 2) {
 #pragma unroll
             for (int j = 0; j < 16; ++j)
-              if (c * 16 + j >= a.T) v[j] = -128;
+              if (c * 16 + j - col0 >= a.T) v[j] = -128;
           }
           // running maximum on the unsaturated values (saturation is monotone: it is applied to the result)
           int m = v[0];
@@ -271,7 +279,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
         // entry (I_max - I) of the table = word at tab + 4*(I_max + 128) - 4*(I + 128)
         const uint8_t* tmx = reinterpret_cast<const uint8_t*>(tab) + 4 * (mx + 128);
 #pragma unroll 1
-        for (int c = half; c < nch; c += 2) {
+        for (int c = c_lo + half; c < c_hi; c += 2) {
           int ev[16];
           uint32_t xs[4];
           tmem_ld4(t_row + c * 16, xs);
@@ -282,10 +290,10 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
             for (int bb = 0; bb < 4; ++bb)
               ev[4 * k + bb] = (int)*reinterpret_cast<const unsigned*>(tmx - 4 * (int)__byte_perm(w, 0, 0x4440 + bb));
           }
-          if (c >= nch - 2) {   // columns past T contribute nothing
+          if (c >= c_hi - 2) {   // columns past T contribute nothing
 #pragma unroll
             for (int j = 0; j < 16; ++j)
-              if (c * 16 + j >= a.T) ev[j] = 0;
+              if (c * 16 + j - col0 >= a.T) ev[j] = 0;
           }
 #pragma unroll
           for (int j = 0; j < 16; ++j) sum += (unsigned)ev[j];
@@ -300,7 +308,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
         // pass C: Eq. (IntDiv) with M = 45, k_out = 8: (floor(2^45 / sum) * e) >> 38 = umulhi(factor, e) >> 6
         const unsigned factor = (unsigned)((1ull << 45) / (unsigned long long)(sum ? sum : 1u));
 #pragma unroll 1
-        for (int c = half; c < nch; c += 2) {
+        for (int c = c_lo + half; c < c_hi; c += 2) {
           int ev[16];
           tmem_ld16(t_row + c * 16, ev);
           uint32_t w[4];
@@ -311,6 +319,11 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
           // A operand of P V: row = tile row, k-block = 128 columns, 16-byte pieces XOR (row & 7)
           uint8_t* prow = gen + p_off + (c >> 3) * (128 * 128) + trow * 128;
           *reinterpret_cast<uint4*>(prow + ((((c & 7)) ^ (trow & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+        if (a.G > 1) {   // the other windows' columns of this row: probability 0, so that P V stays inside the window
+          for (int c = half; c < nch; c += 2)
+            if (c < c_lo || c >= c_hi)
+              *reinterpret_cast<uint4*>(gen + p_off + trow * 128 + ((((c & 7)) ^ (trow & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
         }
         fence_async_smem();
       }
@@ -812,6 +825,7 @@ static int launch_attention_long(ivit_ctx* ctx, const ivit_block_params* p, cons
   a.Npad = (int)((T + 31) / 32 * 32);
   a.tiles_m = (int)((T + 127) / 128);
   a.tmem_cols = 512;
+  a.G = 1; a.R = 128; a.Btot = (int)B;
   int nb_max = ((512 - (int)d) / 2) / 32 * 32 > 224 ? 224 : ((512 - (int)d) / 2) / 32 * 32;   // two score buffers + d output columns
 #ifdef IVIT_TUNING
   if (const char* e = getenv("IVIT_ATTN_LONG")) { const int f = atoi(e); if (f >= 32 && f < nb_max) nb_max = f; }   // stress runs only
@@ -870,6 +884,14 @@ int launch_attention_fused(ivit_ctx* ctx, const ivit_block_params* p, const int8
   a.T = (int)T; a.d = (int)d; a.heads = (int)h; a.D = D;
   a.Npad = (int)((T + 31) / 32 * 32);
   a.tiles_m = (int)((T + 127) / 128);
+  // Short rows (window attention): 2 windows of up to 64 tokens, or 4 of up to 32, share one 128-row tile.  The
+  // score tile is then block-diagonal; the probabilities outside a row's own window are written as 0.
+  a.G = 1; a.R = 128; a.Btot = (int)B;
+  if (T <= 64 && B >= 2) {
+    a.G = T <= 32 ? 4 : 2;
+    a.R = 128 / a.G;
+    a.Npad = 128;
+  }
   a.tmem_cols = 32;
   while (a.tmem_cols < a.Npad) a.tmem_cols <<= 1;
   a.qk_m = p->qk_scale.mult; a.qk_s = clamp_shift(p->qk_scale.shift);
@@ -881,9 +903,10 @@ int launch_attention_fused(ivit_ctx* ctx, const ivit_block_params* p, const int8
   const int64_t ldq = 3 * D;
   CUtensorMap tmQ, tmK, tmV;
   const CUtensorMapSwizzle vsw = d == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : (d == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
-  if (!make_tensor_map(ctx, &tmQ, QKV, d, T, h, B, ldq, d, T * ldq, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B, a.q_pos) ||
-      !make_tensor_map(ctx, &tmK, QKV + D, d, T, h, B, ldq, d, T * ldq, 128, a.Npad, CU_TENSOR_MAP_SWIZZLE_128B, a.k_pos) ||
-      !make_tensor_map(ctx, &tmV, QKV + 2 * D, d, T, h, B, ldq, d, T * ldq, (int)d, a.Npad, vsw, a.v_pos))
+  // boxes: a.R rows of a.G consecutive images / windows (G = 1: 128 query rows, Npad key / value rows of one image)
+  if (!make_tensor_map(ctx, &tmQ, QKV, d, T, h, B, ldq, d, T * ldq, 128, a.G > 1 ? a.R : 128, CU_TENSOR_MAP_SWIZZLE_128B, a.q_pos, a.G) ||
+      !make_tensor_map(ctx, &tmK, QKV + D, d, T, h, B, ldq, d, T * ldq, 128, a.G > 1 ? a.R : a.Npad, CU_TENSOR_MAP_SWIZZLE_128B, a.k_pos, a.G) ||
+      !make_tensor_map(ctx, &tmV, QKV + 2 * D, d, T, h, B, ldq, d, T * ldq, (int)d, a.G > 1 ? a.R : a.Npad, vsw, a.v_pos, a.G))
     return IVIT_ERR_UNSUPPORTED;
   const uint32_t v_off = 128 * 128 + a.Npad * 128;
   const uint32_t p_off = (v_off + a.Npad * a.d + 1023u) & ~1023u;
@@ -893,8 +916,8 @@ int launch_attention_fused(ivit_ctx* ctx, const ivit_block_params* p, const int8
       return IVIT_ERR_CUDA;
     g_attn_attr = true;
   }
-  a.bh = (int)(B * h);
-  a.items = (int)(B * h * a.tiles_m);
+  a.bh = (int)((B + a.G - 1) / a.G * h);
+  a.items = a.bh * a.tiles_m;
   a.sched = ctx->sched_dev + 2 * ctx->attn_gen;
   a.sched_other = ctx->sched_dev + 2 * (ctx->attn_gen ^ 1);
   ctx->attn_gen ^= 1;

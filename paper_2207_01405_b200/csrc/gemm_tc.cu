@@ -40,10 +40,10 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 // coordinate.  Byte strides must be multiples of 16.
 bool make_tensor_map(ivit_ctx* ctx, CUtensorMap* map, const int8_t* ptr, int64_t inner, int64_t rows, int64_t bi, int64_t bo,
               int64_t row_stride, int64_t si, int64_t so, int box_inner, int box_rows, CUtensorMapSwizzle swz,
-              int pos[3]) {
+              int pos[3], int box_bo) {
   if ((reinterpret_cast<uintptr_t>(ptr) & 15) || row_stride % 16) return false;
   struct Dim { int64_t size, stride; int box, which; };
-  Dim d[3] = {{rows, row_stride, box_rows, 0}, {bi, si, 1, 1}, {bo, so, 1, 2}};
+  Dim d[3] = {{rows, row_stride, box_rows, 0}, {bi, si, 1, 1}, {bo, so, box_bo, 2}};
   // size-1 dimensions never contribute to an address: give them the largest stride so they sort last
   int64_t big = row_stride;
   for (int i = 1; i < 3; ++i)

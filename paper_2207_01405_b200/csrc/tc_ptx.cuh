@@ -16,7 +16,7 @@ constexpr uint32_t kSuspendHintNs = 2000;      // suspend-time hint of one poll
 // receive the tensor-map dimension (1..3) holding the row, inner-batch and outer-batch coordinate.
 bool make_tensor_map(ivit_ctx* ctx, CUtensorMap* map, const int8_t* ptr, int64_t inner, int64_t rows, int64_t bi,
                      int64_t bo, int64_t row_stride, int64_t si, int64_t so, int box_inner, int box_rows,
-                     CUtensorMapSwizzle swz, int pos[3]);
+                     CUtensorMapSwizzle swz, int pos[3], int box_bo = 1);
 
 // ---- PTX wrappers -------------------------------------------------------------------------
 

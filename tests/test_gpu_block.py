@@ -31,7 +31,9 @@ def test_config0_block_bit_exact(engine):
 @pytest.mark.parametrize("B,T,D,heads,H,bias", [(3, 197, 384, 6, 1536, False), (2, 577, 256, 4, 512, False),
                                                 (16, 49, 96, 3, 384, True), (2, 49, 768, 24, 3072, True),
                                                 (1, 1, 64, 1, 64, False), (2, 130, 256, 2, 512, False),
-                                                (3, 256, 128, 4, 256, True), (2, 31, 64, 2, 128, False)])
+                                                (3, 256, 128, 4, 256, True), (2, 31, 64, 2, 128, False),
+                                                (5, 49, 96, 3, 96, True), (7, 20, 64, 2, 64, True), (3, 64, 64, 1, 64, False),
+                                                (9, 33, 128, 4, 128, False), (600, 49, 96, 3, 96, True), (13, 32, 64, 2, 64, False)])
 def test_block_shapes_bit_exact(B, T, D, heads, H, bias):
     g = _g()
     c = g.ctx()
