@@ -152,7 +152,8 @@ def test_block_other_output_width_bit_exact(k_out):
 
 @pytest.mark.parametrize("B,T,D,heads,bias", [(2, 257, 128, 2, False), (1, 300, 128, 2, True), (3, 577, 128, 2, False),
                                               (2, 449, 64, 2, False), (1, 640, 64, 1, False), (2, 577, 256, 4, True), (1, 400, 256, 2, False),
-                                              (40, 320, 128, 2, False)])
+                                              (40, 320, 128, 2, False), (1, 768, 64, 1, False), (1, 512, 128, 1, True),
+                                              (2, 896, 32, 1, False)])
 def test_long_row_attention_bit_exact(B, T, D, heads, bias):
     """The key-block form of the fused attention kernel (rows longer than 256 tokens): two to four key blocks, ragged
     last blocks and last row tiles, head dimensions 32 / 64 / 128, with and without a score bias, and more work items
