@@ -92,13 +92,12 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
   tc_fence_after();
   const uint32_t tmem = *tmem_slot;
   pdl_trigger();
-  pdl_wait();   // the QKV tensor comes from the previous kernel
+  // The ShiftExp table depends on parameters only: the Shiftmax threads build it before they wait for the previous
+  // kernel (whose QKV tensor the control thread loads and whose successors' buffers the output overwrites).
+  if (warp == 0) pdl_wait();
   // Launches alternate between two pairs of counters.  A launch leaves its own pair at zero when its last CTA
-  // finishes, and also zeroes the other pair here, so that a launch that was cut short cannot poison the next.
-  if (blockIdx.x == 0 && threadIdx.x == 32) {
-    a.sched_other[0] = 0;
-    a.sched_other[1] = 0;
-  }
+  // finishes, and also zeroes the other pair (below, after the wait), so that a launch that was cut short cannot
+  // poison the next.
 
   // item -> (tile, image/window * heads + head): all first tiles before all second tiles
   if (warp == 0) {
@@ -185,6 +184,11 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
     //      take the even / odd 32-column chunks of the same 32 rows ----
     const int st = threadIdx.x - 32;   // 0..255
     tab[st] = shiftexp(-st, a.smax.I0, a.smax.N);
+    pdl_wait();
+    if (blockIdx.x == 0 && threadIdx.x == 32) {
+      a.sched_other[0] = 0;
+      a.sched_other[1] = 0;
+    }
     const int qd = warp & 3;
     const int half = (warp - 1) >> 2;
     const int trow = qd * 32 + lane;              // row inside the tile
@@ -455,11 +459,7 @@ __global__ void __launch_bounds__(kLongThreads, 1) attention_long_kernel(const _
   const uint32_t tmem = *tmem_slot;
   const uint32_t o_col = 2u * (uint32_t)NB;   // output accumulator behind the two score buffers
   pdl_trigger();
-  pdl_wait();   // the QKV tensor comes from the previous kernel
-  if (blockIdx.x == 0 && threadIdx.x == 32) {
-    a.sched_other[0] = 0;
-    a.sched_other[1] = 0;
-  }
+  if (warp == 0) pdl_wait();   // the QKV tensor comes from the previous kernel; the other warps build their table first
 
   if (warp == 0) {
     if (lane == 0) {
@@ -603,6 +603,11 @@ __global__ void __launch_bounds__(kLongThreads, 1) attention_long_kernel(const _
     //      quarters of every key block of the same 32 rows ----
     const int st = threadIdx.x - 32;   // 0..511
     if (st < 256) tab[st] = shiftexp(-st, a.smax.I0, a.smax.N);
+    pdl_wait();
+    if (blockIdx.x == 0 && threadIdx.x == 32) {
+      a.sched_other[0] = 0;
+      a.sched_other[1] = 0;
+    }
     const int qd = warp & 3;
     const int part = (warp - 1) >> 2;             // 0..3
     const int trow = qd * 32 + lane;              // row inside the tile

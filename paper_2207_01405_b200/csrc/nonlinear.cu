@@ -135,7 +135,8 @@ __global__ void __launch_bounds__(128, SMEMC ? 4 : 6) layernorm_i8_batched_kerne
                                                                       int64_t rows, int C, unsigned mean_magic, int vec) {
   extern __shared__ int4 ln_consts[];   // SMEMC: [3][C / 4] multipliers, shifts, addends (or betas)
   pdl_trigger();
-  pdl_wait();
+  // the per-channel constants are parameters, not results of the previous kernel: they are fetched before the
+  // wait for that kernel (below, in front of the first row load)
   const int lane = threadIdx.x & 31;
   const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
@@ -213,6 +214,7 @@ __global__ void __launch_bounds__(128, SMEMC ? 4 : 6) layernorm_i8_batched_kerne
       for (int i = 0; i < WR; ++i) to_fast(ps[i], pb[i]);
     }
   }
+  pdl_wait();
   for (int64_t r0 = warp * ROWS; r0 < rows; r0 += nwarps * ROWS) {
     int w[ROWS][WPL];
     int my_s1 = 0, my_s2 = 0;
