@@ -49,6 +49,8 @@ constexpr uint32_t kItemWaitRounds = 16;   // the item barrier outlasts every bo
 // full 128-row tiles first.  One control thread issues the TMA loads and the MMAs; the loads of the next item
 // are issued as soon as the MMAs that read the shared-memory operands of the current one have completed, so
 // they overlap the Shiftmax passes.  Barriers are used once per item: the parity of a wait is the item count.
+// kPack: several windows share the tile (AttnArgs::G > 1); the plain form carries none of that index arithmetic.
+template <bool kPack>
 __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid_constant__ CUtensorMap tmQ,
                                                                  const __grid_constant__ CUtensorMap tmK,
                                                                  const __grid_constant__ CUtensorMap tmV, AttnArgs a) {
@@ -107,9 +109,9 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
         const int h = bhid % a.heads, b = bhid / a.heads;
         mbar_expect_tx(bar_qk, 128 * 128 + a.Npad * 128);
         int c[4];
-        c[0] = 0; c[a.q_pos[0]] = tile * 128; c[a.q_pos[1]] = h; c[a.q_pos[2]] = b * a.G;
+        c[0] = 0; c[a.q_pos[0]] = tile * 128; c[a.q_pos[1]] = h; c[a.q_pos[2]] = kPack ? b * a.G : b;
         tma_load_4d(base + q_off, &tmQ, bar_qk, c[0], c[1], c[2], c[3]);
-        c[0] = 0; c[a.k_pos[0]] = 0; c[a.k_pos[1]] = h; c[a.k_pos[2]] = b * a.G;
+        c[0] = 0; c[a.k_pos[0]] = 0; c[a.k_pos[1]] = h; c[a.k_pos[2]] = kPack ? b * a.G : b;
         tma_load_4d(base + k_off, &tmK, bar_qk, c[0], c[1], c[2], c[3]);
       };
       auto load_v = [&](int item) {
@@ -117,7 +119,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
         const int h = bhid % a.heads, b = bhid / a.heads;
         mbar_expect_tx(bar_v, a.Npad * a.d);
         int c[4];
-        c[0] = 0; c[a.v_pos[0]] = 0; c[a.v_pos[1]] = h; c[a.v_pos[2]] = b * a.G;
+        c[0] = 0; c[a.v_pos[0]] = 0; c[a.v_pos[1]] = h; c[a.v_pos[2]] = kPack ? b * a.G : b;
         tma_load_4d(base + v_off, &tmV, bar_v, c[0], c[1], c[2], c[3]);
       };
       auto draw = [&]() {
@@ -216,14 +218,14 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
       const int h = bhid % a.heads;
       // G > 1: the tile holds G windows of R rows each (window `slot` in rows and columns slot R .. slot R + R - 1 of
       // the block-diagonal score tile); a warp's 32 rows lie inside one window
-      const int slot = a.G > 1 ? trow / a.R : 0;
-      const int b = (bhid / a.heads) * a.G + slot;  // image / window of this row
+      const int slot = kPack ? trow / a.R : 0;
+      const int b = kPack ? (bhid / a.heads) * a.G + slot : bhid / a.heads;   // image / window of this row
       const int m0 = tile * 128;
-      const int r = m0 + trow - slot * a.R;         // token (row) inside this image / window
-      const bool row_ok = r < a.T && b < a.Btot;
-      const bool warp_ok = m0 + qd * 32 - slot * a.R < a.T && b < a.Btot;   // warps whose 32 rows all lie past T only keep the barriers
-      const int col0 = slot * a.R;                  // first score column of this row's window
-      const int c_lo = col0 >> 4, c_hi = a.G > 1 ? c_lo + (a.R >> 4) : nch;   // this row's 16-column chunks
+      const int col0 = kPack ? slot * a.R : 0;      // first row and first score column of this row's window in the tile
+      const int r = m0 + trow - col0;               // token (row) inside this image / window
+      const bool row_ok = r < a.T && (!kPack || b < a.Btot);
+      const bool warp_ok = m0 + qd * 32 - col0 < a.T && (!kPack || b < a.Btot);   // warps whose 32 rows all lie past T only keep the barriers
+      const int c_lo = col0 >> 4, c_hi = kPack ? c_lo + (a.R >> 4) : nch;   // this row's 16-column chunks
       const int32_t* brow = a.bias ? a.bias + ((((int64_t)b * a.heads + h) % a.bias_batches) * a.T + (row_ok ? r : 0)) * (int64_t)a.T - col0 : nullptr;
 
       int mx = -128;
@@ -324,7 +326,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
           uint8_t* prow = gen + p_off + (c >> 3) * (128 * 128) + trow * 128;
           *reinterpret_cast<uint4*>(prow + ((((c & 7)) ^ (trow & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
         }
-        if (a.G > 1) {   // the other windows' columns of this row: probability 0, so that P V stays inside the window
+        if (kPack) {   // the other windows' columns of this row: probability 0, so that P V stays inside the window
           for (int c = half; c < nch; c += 2)
             if (c < c_lo || c >= c_hi)
               *reinterpret_cast<uint4*>(gen + p_off + trow * 128 + ((((c & 7)) ^ (trow & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
@@ -917,7 +919,8 @@ int launch_attention_fused(ivit_ctx* ctx, const ivit_block_params* p, const int8
   const uint32_t p_off = (v_off + a.Npad * a.d + 1023u) & ~1023u;
   const size_t smem = 1024 + p_off + (size_t)((a.Npad + 127) / 128) * 128 * 128 + 1024 + 2048 + 16 + 64 + 16;
   if (!g_attn_attr) {
-    if (cudaFuncSetAttribute(attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+    if (cudaFuncSetAttribute(attention_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(attention_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
       return IVIT_ERR_CUDA;
     g_attn_attr = true;
   }
@@ -929,7 +932,8 @@ int launch_attention_fused(ivit_ctx* ctx, const ivit_block_params* p, const int8
   const int64_t slots = 2 * (int64_t)ctx->sm_count;
   const int64_t grid = a.items < slots ? a.items : slots;
   LaunchScope ls(ctx, KIND_ATTENTION, 4.0 * (double)(B * h) * (double)T * (double)T * (double)d);
-  launch_k(attention_kernel, dim3((unsigned)grid), dim3(kAttnThreads), smem, ctx->stream, tmQ, tmK, tmV, a);
+  if (a.G > 1) launch_k(attention_kernel<true>, dim3((unsigned)grid), dim3(kAttnThreads), smem, ctx->stream, tmQ, tmK, tmV, a);
+  else launch_k(attention_kernel<false>, dim3((unsigned)grid), dim3(kAttnThreads), smem, ctx->stream, tmQ, tmK, tmV, a);
   return ls.done();
 }
 
