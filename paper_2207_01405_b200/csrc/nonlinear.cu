@@ -2,6 +2,7 @@
 // One warp owns one row; rows are read once from HBM as coalesced 32-bit words and
 // kept in registers between the reduction and the output pass.
 #include "common.cuh"
+#include <type_traits>
 
 namespace ivit {
 
@@ -577,6 +578,9 @@ struct DirectConsts {
   int M;
   unsigned long long magic;      // reciprocal of I0 scaled by 2^64, rounded up (unused when I0 == 1)
   unsigned long long zero_from;  // I0 * (N + 29): from here on every bit of I_b < 2^29 is shifted out
+  // 32-bit form (taken when exponentials, their sum and the reciprocal all fit 32 bits and zero_from <= 2^31)
+  unsigned nd_cut;               // I_max - I >= nd_cut implies -I_p >= zero_from; below it -I_p fits 32 bits
+  unsigned m_hi, m_lo;           // the two words of magic
 };
 
 // ShiftExp(I - I_max) for nd = I_max - I (0 .. 2^32 - 1).  The arithmetic shifts of the negative I_delta round
@@ -593,6 +597,17 @@ __device__ __forceinline__ unsigned long long shiftexp_wide(unsigned nd, const D
   return q <= (unsigned)c.N ? (unsigned long long)Ib << (c.N - q) : (unsigned long long)(Ib >> (q - c.N));
 }
 
+// The same in 32-bit arithmetic: the quotient is the high word of n * magic, taken from two 32-bit products.
+__device__ __forceinline__ unsigned shiftexp_narrow(unsigned nd, const DirectConsts& c) {
+  if (nd >= c.nd_cut) return 0u;
+  const unsigned n = nd + ((nd >> 1) + (nd & 1u)) - ((nd >> 4) + ((nd & 15u) != 0u));
+  if (n >= (unsigned)c.zero_from) return 0u;
+  const unsigned q = c.I0 == 1u ? n : (unsigned)(((unsigned long long)n * c.m_hi + __umulhi(n, c.m_lo)) >> 32);
+  const unsigned r = n - q * c.I0;
+  const unsigned Ib = c.I0 - ((r + 1) >> 1);
+  return q <= (unsigned)c.N ? Ib << (c.N - q) : Ib >> (q - c.N);
+}
+
 __device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -601,7 +616,8 @@ __device__ __forceinline__ unsigned long long warp_sum_u64(unsigned long long v)
 
 // One warp per row.  WPL groups of four scores per lane stay in registers as their exponentials
 // (d <= 128 * WPL); WPL == 0 reads the row three times instead.
-template <int WPL>
+// NARROW: every exponential, the row sum and the reciprocal fit 32 bits (checked by the launcher).
+template <int WPL, bool NARROW>
 __global__ void __launch_bounds__(256) shiftmax_direct_kernel(const int32_t* __restrict__ in, int64_t ldin,
                                                               DirectConsts c, int8_t* __restrict__ out,
                                                               int64_t ldout, int64_t rows, int d) {
@@ -634,37 +650,48 @@ __global__ void __launch_bounds__(256) shiftmax_direct_kernel(const int32_t* __r
     }
     mx = __reduce_max_sync(0xffffffffu, mx);
     // exponentials of group g (0 for positions past d)
-    auto exps = [&](int g, const int4& v, unsigned long long* e) {
-      e[0] = 4 * g + 0 < d ? shiftexp_wide((unsigned)mx - (unsigned)v.x, c) : 0ull;
-      e[1] = 4 * g + 1 < d ? shiftexp_wide((unsigned)mx - (unsigned)v.y, c) : 0ull;
-      e[2] = 4 * g + 2 < d ? shiftexp_wide((unsigned)mx - (unsigned)v.z, c) : 0ull;
-      e[3] = 4 * g + 3 < d ? shiftexp_wide((unsigned)mx - (unsigned)v.w, c) : 0ull;
+    using E = typename std::conditional<NARROW, unsigned, unsigned long long>::type;
+    auto one = [&](int v) -> E {
+      if constexpr (NARROW) return shiftexp_narrow((unsigned)mx - (unsigned)v, c);
+      else return shiftexp_wide((unsigned)mx - (unsigned)v, c);
+    };
+    auto exps = [&](int g, const int4& v, E* e) {
+      e[0] = 4 * g + 0 < d ? one(v.x) : (E)0;
+      e[1] = 4 * g + 1 < d ? one(v.y) : (E)0;
+      e[2] = 4 * g + 2 < d ? one(v.z) : (E)0;
+      e[3] = 4 * g + 3 < d ? one(v.w) : (E)0;
     };
     // pass 2: sum
-    unsigned long long e[W][4];
-    unsigned long long sum = 0;
+    E e[W][4];
+    E sum = 0;
 #pragma unroll
     for (int i = 0; i < iters; ++i) {
       const int g = lane + 32 * i;
-      unsigned long long t[4] = {0ull, 0ull, 0ull, 0ull};
+      E t[4] = {0, 0, 0, 0};
       if (g < ngroups) exps(g, WPL > 0 ? x[i] : __ldg(src + g), t);
       if (WPL > 0) { e[i][0] = t[0]; e[i][1] = t[1]; e[i][2] = t[2]; e[i][3] = t[3]; }
       sum += (t[0] + t[1]) + (t[2] + t[3]);
     }
-    sum = warp_sum_u64(sum);                                   // >= I0 * 2^N: the maximum contributes exactly that
-    const unsigned long long factor = (1ull << c.M) / sum;     // Eq. (IntDiv); factor * e <= 2^M < 2^63
+    // the row sum is >= I0 * 2^N: the maximum contributes exactly that
+    if constexpr (NARROW) sum = __reduce_add_sync(0xffffffffu, sum);
+    else sum = warp_sum_u64(sum);
+    // Eq. (IntDiv); factor * e <= 2^M < 2^63.  NARROW: factor < 2^32 and M - (k_out - 1) >= 32, so the product's
+    // high word shifted by the rest is the same value.
+    const E factor = (E)((1ull << c.M) / (unsigned long long)sum);
+    auto prob = [&](E t) -> int {
+      if constexpr (NARROW) return min((int)(__umulhi(factor, t) >> (c.osh - 32)), c.omax);
+      else return min((int)((factor * t) >> c.osh), c.omax);
+    };
     // pass 3: outputs
     int* dst = reinterpret_cast<int*>(out + r * ldout);
 #pragma unroll
     for (int i = 0; i < iters; ++i) {
       const int g = lane + 32 * i;
       if (g < nwords_out) {
-        unsigned long long t[4] = {0ull, 0ull, 0ull, 0ull};
+        E t[4] = {0, 0, 0, 0};
         if (WPL > 0) { t[0] = e[i][0]; t[1] = e[i][1]; t[2] = e[i][2]; t[3] = e[i][3]; }
         else if (g < ngroups) exps(g, __ldg(src + g), t);
-        const int o0 = min((int)((factor * t[0]) >> c.osh), c.omax), o1 = min((int)((factor * t[1]) >> c.osh), c.omax);
-        const int o2 = min((int)((factor * t[2]) >> c.osh), c.omax), o3 = min((int)((factor * t[3]) >> c.osh), c.omax);
-        dst[g] = (int)pack_sat8_u(o0, o1, o2, o3);
+        dst[g] = (int)pack_sat8_u(prob(t[0]), prob(t[1]), prob(t[2]), prob(t[3]));
       }
     }
   }
@@ -680,13 +707,25 @@ int launch_shiftmax_direct(ivit_ctx* ctx, const int32_t* in, int64_t ldin, ivit_
   // floor((2^64 - 1) / I0) + 1: floor(2^64 / I0) + 1, or exactly 2^64 / I0 when I0 is a power of two (both give the floor quotient)
   c.magic = p.I0 > 1 ? ~0ull / (unsigned long long)p.I0 + 1ull : 0ull;
   c.zero_from = (unsigned long long)p.I0 * (unsigned long long)(p.N + 29);
+  c.m_hi = (unsigned)(c.magic >> 32); c.m_lo = (unsigned)c.magic;
+  // -I_p >= (23 / 16) nd - 1: from nd_cut on it is at least zero_from; below it -I_p <= 1.5 nd_cut + 1 < 2^32
+  c.nd_cut = (unsigned)(((c.zero_from + 1) * 16 + 22) / 23);
+  const unsigned long long top = (unsigned long long)p.I0 << p.N;   // the largest exponential
+  const bool narrow = c.zero_from <= (1ull << 31) && top * (unsigned long long)d < (1ull << 32) && c.osh >= 32 &&
+                      (p.M <= 32 || top > (1ull << (p.M - 32)));
   const int64_t want = (rows + 7) / 8;
   const int grid = (int)(want < (int64_t)ctx->sm_count * 8 ? want : (int64_t)ctx->sm_count * 8);
   LaunchScope ls(ctx, KIND_SHIFTMAX, (double)rows * (double)d * 5.0);
   const int wpl = (int)(((d + 15) / 16 * 4 + 31) / 32);
-  if (wpl <= 2) launch_k(shiftmax_direct_kernel<2>, dim3(grid), dim3(256), 0, ctx->stream, in, ldin, c, out, ldout, rows, (int)d);
-  else if (wpl <= 5) launch_k(shiftmax_direct_kernel<5>, dim3(grid), dim3(256), 0, ctx->stream, in, ldin, c, out, ldout, rows, (int)d);
-  else launch_k(shiftmax_direct_kernel<0>, dim3(grid), dim3(256), 0, ctx->stream, in, ldin, c, out, ldout, rows, (int)d);
+  if (narrow) {
+    if (wpl <= 2) launch_k(shiftmax_direct_kernel<2, true>, dim3(grid), dim3(256), 0, ctx->stream, in, ldin, c, out, ldout, rows, (int)d);
+    else if (wpl <= 5) launch_k(shiftmax_direct_kernel<5, true>, dim3(grid), dim3(256), 0, ctx->stream, in, ldin, c, out, ldout, rows, (int)d);
+    else launch_k(shiftmax_direct_kernel<0, true>, dim3(grid), dim3(256), 0, ctx->stream, in, ldin, c, out, ldout, rows, (int)d);
+  } else {
+    if (wpl <= 2) launch_k(shiftmax_direct_kernel<2, false>, dim3(grid), dim3(256), 0, ctx->stream, in, ldin, c, out, ldout, rows, (int)d);
+    else if (wpl <= 5) launch_k(shiftmax_direct_kernel<5, false>, dim3(grid), dim3(256), 0, ctx->stream, in, ldin, c, out, ldout, rows, (int)d);
+    else launch_k(shiftmax_direct_kernel<0, false>, dim3(grid), dim3(256), 0, ctx->stream, in, ldin, c, out, ldout, rows, (int)d);
+  }
   return ls.done();
 }
 
