@@ -1,6 +1,5 @@
 """Parity at the benchmark's full size: DeiT-S, batch 64, 12 blocks, in the launch configuration
 bench.py times.  Images are independent, so the oracle recomputes a sample of them one by one."""
-import numpy as np
 import pytest
 import torch
 

@@ -6,7 +6,6 @@ a fixed device array inside the library instead of a caller-provided workspace. 
 same bytes as ivit_block_forward, call after call, because the shared array keeps the previous
 call's contents.  This file sorts last so that a run stopping at the first failure has already run
 every other test; it passes alone in a fresh process as well."""
-import numpy as np
 import pytest
 import torch
 
