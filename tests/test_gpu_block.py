@@ -171,3 +171,25 @@ def test_long_row_attention_bit_exact(B, T, D, heads, bias):
     g.assert_equal(g.host(Oo), O.attention(blk, QKV), f"long-row attention T={T}")
     assert c.poll_status() == 0
 
+
+def test_attention_random_shapes():
+    """Thirty seeded random attention problems (fused short-row, window-packed and key-block kernels, and the composed
+    path for head dimensions the fused kernels do not take): random batch, row length, heads and head dimension, with
+    and without a score bias; every output element against the oracle."""
+    g = _g()
+    c = g.ctx()
+    rng = np.random.default_rng(77)
+    for case in range(30):
+        d = int(rng.choice([16, 32, 48, 64, 128]))
+        heads = int(rng.integers(1, 4))
+        T = int(rng.choice([int(rng.integers(1, 70)), int(rng.integers(70, 257)), int(rng.integers(257, 520))]))
+        B = int(rng.integers(1, 6)) if T > 64 else int(rng.integers(1, 40))
+        bias = bool(rng.random() < 0.4)
+        D = heads * d
+        blk = make_block(_Ids(2000 + case), 1, B, T, D, heads, 2 * D, attn_bias_batches=heads if bias else 0)
+        dblk = g.binding.DeviceBlock(blk, "cuda")
+        QKV = np.clip(np.rint(rng.standard_normal((B * T, 3 * D)) * 32), -128, 127).astype(np.int8)
+        got = g.host(c.attention(dblk, torch.from_numpy(QKV).cuda()))
+        g.assert_equal(got, O.attention(blk, QKV), f"case {case}: B={B} T={T} heads={heads} d={d} bias={bias}")
+    assert c.poll_status() == 0
+

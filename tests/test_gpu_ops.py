@@ -52,6 +52,34 @@ def test_linear_parity(engine, M, N, K):
     assert c.poll_status() == 0
 
 
+def test_linear_random_shapes():
+    """Forty seeded random Dense problems on the tensor-core engine: ragged M, N and K (N a multiple of 4, K of 16),
+    with and without bias, with the residual port in its three forms (none, full rows, wrapped rows), saturating
+    scales included; every output element against the oracle."""
+    g = _g()
+    c = g.ctx()
+    c.set_gemm_engine(0)
+    rng = np.random.default_rng(2024)
+    for case in range(40):
+        M = int(rng.integers(1, 900))
+        N = 4 * int(rng.integers(1, 160))
+        K = 16 * int(rng.integers(1, 50))
+        A, W = rand_i8(rng, (M, K)), rand_i8(rng, (N, K))
+        bias = rng.integers(-30000, 30000, N).astype(np.int32) if rng.random() < 0.7 else None
+        acc_std = np.sqrt(K) * 40 * 40
+        scale = scale_channels(rng.uniform(10, 120, N) / acc_std)     # the upper end saturates a good share of outputs
+        mode = int(rng.integers(0, 3))
+        res = None if mode == 0 else rand_i8(rng, (M if mode == 1 else int(rng.integers(1, M + 1)), N))
+        rs = Scale(*dyadic(float(rng.uniform(0.2, 0.99))))
+        got = c.linear(g.dev(A), g.dev(W), None if bias is None else torch.from_numpy(bias).cuda(),
+                       g.binding.DevScale(scale, "cuda"), res=None if res is None else g.dev(res),
+                       res_scale=None if res is None else g.binding.DevScale(rs, "cuda"),
+                       out=g.dev(np.zeros((M, N), np.int8)))
+        want = O.linear(A, W, bias, scale, res=res, res_scale=None if res is None else rs)
+        g.assert_equal(g.host(got), want, f"case {case}: M={M} N={N} K={K} bias={bias is not None} res mode {mode}")
+    assert c.poll_status() == 0
+
+
 @pytest.mark.parametrize("M,N,K", [(130, 200, 48), (197, 384, 1536), (393, 1000, 384), (33, 36, 96), (700, 384, 384)])
 def test_linear_residual_full_rows(M, N, K):
     """Residual with one row per output row (the encoder block's form): the residual tile is staged by TMA."""
