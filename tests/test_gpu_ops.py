@@ -354,6 +354,47 @@ def test_layernorm_parity(rows, C):
     g.assert_equal(g.host(got), O.layernorm(x32, scale, beta), "layernorm i32")
 
 
+def test_row_kernels_random_shapes():
+    """Seeded random shapes for the row kernels: I-LayerNorm (int8 and int32 input, per-channel and per-tensor scale),
+    Shiftmax (int8 input), ShiftGELU and its static variant; every output element against the oracle."""
+    g = _g()
+    c = g.ctx()
+    rng = np.random.default_rng(4242)
+    for case in range(25):
+        rows = int(rng.integers(1, 700))
+        C = 4 * int(rng.integers(1, 520))
+        x = rand_i8(rng, (rows, C), float(rng.uniform(3, 50))) + rng.integers(-40, 40, (rows, 1)).astype(np.int8)
+        per_channel = rng.random() < 0.7
+        ratio = 32 * np.sqrt(C) / 2.0 ** 20
+        scale = scale_channels((1 + 0.2 * rng.standard_normal(C)).clip(0.2) * ratio) if per_channel else Scale(*dyadic(ratio))
+        beta = rng.integers(-30, 30, C).astype(np.int32) if rng.random() < 0.7 else None
+        dbeta = None if beta is None else torch.from_numpy(beta).cuda()
+        got = c.layernorm(g.dev(x), g.binding.DevScale(scale, "cuda"), dbeta)
+        g.assert_equal(g.host(got), O.layernorm(x, scale, beta), f"layernorm case {case}: rows={rows} C={C}")
+        x32 = (rng.standard_normal((rows, C)) * float(rng.uniform(100, 100000))).astype(np.int32)
+        got = c.layernorm(g.dev(x32, 4), g.binding.DevScale(scale, "cuda"), dbeta)
+        g.assert_equal(g.host(got), O.layernorm(x32, scale, beta), f"layernorm i32 case {case}: rows={rows} C={C}")
+    for case in range(25):
+        rows = int(rng.integers(1, 500))
+        d = int(rng.integers(1, 1500))
+        I0 = int(rng.integers(4, 40))
+        x = rand_i8(rng, (rows, d), float(rng.uniform(5, 60)))
+        p = ExpParams(I0, 15)
+        g.assert_equal(g.host(c.shiftmax(g.dev(x), p)), O.shiftmax(x, p), f"shiftmax case {case}: rows={rows} d={d} I0={I0}")
+    for case in range(15):
+        rows = int(rng.integers(1, 400))
+        cols = 16 * int(rng.integers(1, 260))
+        I0 = int(rng.integers(20, 45))
+        x = rand_i8(rng, (rows, cols), float(rng.uniform(10, 60)))
+        p = ExpParams(I0, 23)
+        post = Scale(*dyadic(1.0 / (128 * float(rng.uniform(0.6, 1.2)))))
+        dpost = g.binding.DevScale(post, "cuda")
+        g.assert_equal(g.host(c.shiftgelu(g.dev(x), p, dpost)), O.shiftgelu(x, p, post), f"shiftgelu case {case}")
+        g.assert_equal(g.host(c.shiftgelu(g.dev(x), p, dpost, static_max=True)), O.shiftgelu(x, p, post, static_max=True),
+                       f"shiftgelu static case {case}")
+    assert c.poll_status() == 0
+
+
 def test_helpers_parity():
     g = _g()
     c = g.ctx()
