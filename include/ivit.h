@@ -74,8 +74,7 @@ typedef struct {
  * Bounds (IVIT_ERR_RANGE otherwise): 1 <= I0 <= 2^15, 0 <= N <= 24, M == 45,
  * 2 <= k_out <= 8; Shiftmax: row_len * I0 * 2^N < 2^32 and I0 * 2^N >= 2^14;
  * ShiftGELU: 2 * I0 * 2^N < 2^32.  ivit_shiftmax_direct has wider bounds of
- * its own.  The fused attention kernel is built for k_out == 8; with another
- * k_out, ivit_attention and the block run the unfused sequence of kernels. */
+ * its own. */
 typedef struct {
   int32_t I0, N, M, k_out;
 } ivit_exp_params;

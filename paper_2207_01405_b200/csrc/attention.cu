@@ -23,6 +23,17 @@ constexpr int kAttnThreads = 288;   // warp 0: TMA + MMA issue + TMEM owner; war
 constexpr int UK = 32;              // K of one tcgen05.mma.kind::i8
 
 
+// Eq. (IntDiv) with M = 45 for four exponentials: (floor(2^45 / sum) * e) >> (45 - (k_out - 1)) = umulhi(factor, e) >> (14 - k_out),
+// clamped to 2^(k_out-1) - 1 and packed.  K8: k_out = 8, where the saturating pack does the clamp (values are <= 128).
+template <bool K8>
+__device__ __forceinline__ uint32_t prob_word(unsigned factor, int e0, int e1, int e2, int e3, int osh, int omax) {
+  if (K8)
+    return pack_sat8((int)(__umulhi(factor, (unsigned)e0) >> 6), (int)(__umulhi(factor, (unsigned)e1) >> 6),
+                     (int)(__umulhi(factor, (unsigned)e2) >> 6), (int)(__umulhi(factor, (unsigned)e3) >> 6));
+  return pack_sat8(min((int)(__umulhi(factor, (unsigned)e0) >> osh), omax), min((int)(__umulhi(factor, (unsigned)e1) >> osh), omax),
+                   min((int)(__umulhi(factor, (unsigned)e2) >> osh), omax), min((int)(__umulhi(factor, (unsigned)e3) >> osh), omax));
+}
+
 struct AttnArgs {
   int T, d, heads, Npad;            // Npad = T rounded up to 32 (score columns and P.V contraction length)
   int64_t D;                        // heads * d
@@ -50,7 +61,7 @@ constexpr uint32_t kItemWaitRounds = 16;   // the item barrier outlasts every bo
 // are issued as soon as the MMAs that read the shared-memory operands of the current one have completed, so
 // they overlap the Shiftmax passes.  Barriers are used once per item: the parity of a wait is the item count.
 // kPack: several windows share the tile (AttnArgs::G > 1); the plain form carries none of that index arithmetic.
-template <bool kPack>
+template <bool kPack, bool K8>
 __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid_constant__ CUtensorMap tmQ,
                                                                  const __grid_constant__ CUtensorMap tmK,
                                                                  const __grid_constant__ CUtensorMap tmV, AttnArgs a) {
@@ -311,7 +322,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
       asm volatile("bar.sync %0, 64;" ::"r"(2 + qd) : "memory");
       if (got_s && warp_ok) {
         sum = part_sum[trow] + part_sum[128 + trow];
-        // pass C: Eq. (IntDiv) with M = 45, k_out = 8: (floor(2^45 / sum) * e) >> 38 = umulhi(factor, e) >> 6
+        // pass C: Eq. (IntDiv) with M = 45 (prob_word)
         const unsigned factor = (unsigned)((1ull << 45) / (unsigned long long)(sum ? sum : 1u));
 #pragma unroll 1
         for (int c = c_lo + half; c < c_hi; c += 2) {
@@ -319,9 +330,8 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
           tmem_ld16(t_row + c * 16, ev);
           uint32_t w[4];
 #pragma unroll
-          for (int k = 0; k < 4; ++k)   // values are <= 128: the saturating pack clamps the one possible 128 to 127
-            w[k] = pack_sat8((int)(__umulhi(factor, (unsigned)ev[4 * k]) >> 6), (int)(__umulhi(factor, (unsigned)ev[4 * k + 1]) >> 6),
-                             (int)(__umulhi(factor, (unsigned)ev[4 * k + 2]) >> 6), (int)(__umulhi(factor, (unsigned)ev[4 * k + 3]) >> 6));
+          for (int k = 0; k < 4; ++k)
+            w[k] = prob_word<K8>(factor, ev[4 * k], ev[4 * k + 1], ev[4 * k + 2], ev[4 * k + 3], 14 - a.smax.k_out, (1 << (a.smax.k_out - 1)) - 1);
           // A operand of P V: row = tile row, k-block = 128 columns, 16-byte pieces XOR (row & 7)
           uint8_t* prow = gen + p_off + (c >> 3) * (128 * 128) + trow * 128;
           *reinterpret_cast<uint4*>(prow + ((((c & 7)) ^ (trow & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
@@ -411,6 +421,7 @@ struct LongArgs {
 __device__ __forceinline__ void tmem_ld_cols(uint32_t addr, int (&v)[16]) { tmem_ld16(addr, v); }
 __device__ __forceinline__ void tmem_ld_cols(uint32_t addr, int (&v)[8]) { tmem_ld8_issue(addr, v); tmem_ld_wait8(v); }
 
+template <bool K8>
 __global__ void __launch_bounds__(kLongThreads, 1) attention_long_kernel(const __grid_constant__ CUtensorMap tmQ,
                                                                         const __grid_constant__ CUtensorMap tmK,
                                                                         const __grid_constant__ CUtensorMap tmV, LongArgs la) {
@@ -735,7 +746,7 @@ __global__ void __launch_bounds__(kLongThreads, 1) attention_long_kernel(const _
       asm volatile("bar.sync %0, 128;" ::"r"(2 + qd) : "memory");
       if (alive && warp_ok) {
         sum = (part_sum[trow] + part_sum[128 + trow]) + (part_sum[256 + trow] + part_sum[384 + trow]);
-        // pass C: Eq. (IntDiv) with M = 45, k_out = 8: (floor(2^45 / sum) * e) >> 38 = umulhi(factor, e) >> 6,
+        // pass C: Eq. (IntDiv) with M = 45 (prob_word),
         // the parked score bytes turned into probabilities in place
         const unsigned factor = (unsigned)((1ull << 45) / (unsigned long long)(sum ? sum : 1u));
         for (int j = 0; j < nblk; ++j) {
@@ -755,9 +766,8 @@ __global__ void __launch_bounds__(kLongThreads, 1) attention_long_kernel(const _
                 if (col + i >= a.T) ev[i] = 0;
             }
 #pragma unroll
-            for (int k = 0; k < W / 4; ++k)   // values are <= 128: the saturating pack clamps the one possible 128 to 127
-              xs[k] = pack_sat8((int)(__umulhi(factor, (unsigned)ev[4 * k]) >> 6), (int)(__umulhi(factor, (unsigned)ev[4 * k + 1]) >> 6),
-                                (int)(__umulhi(factor, (unsigned)ev[4 * k + 2]) >> 6), (int)(__umulhi(factor, (unsigned)ev[4 * k + 3]) >> 6));
+            for (int k = 0; k < W / 4; ++k)
+              xs[k] = prob_word<K8>(factor, ev[4 * k], ev[4 * k + 1], ev[4 * k + 2], ev[4 * k + 3], 14 - a.smax.k_out, (1 << (a.smax.k_out - 1)) - 1);
             if constexpr (W == 16) *reinterpret_cast<uint4*>(p_addr(col)) = make_uint4(xs[0], xs[1], xs[2], xs[3]);
             else *reinterpret_cast<uint2*>(p_addr(col)) = make_uint2(xs[0], xs[1]);
           });
@@ -859,7 +869,8 @@ static int launch_attention_long(ivit_ctx* ctx, const ivit_block_params* p, cons
       !make_tensor_map(ctx, &tmV, QKV + 2 * D, d, T, h, B, ldq, d, T * ldq, (int)d, 256, vsw, a.v_pos))
     return IVIT_ERR_UNSUPPORTED;
   if (!g_attn_long_attr) {
-    if (cudaFuncSetAttribute(attention_long_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+    if (cudaFuncSetAttribute(attention_long_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(attention_long_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
       return IVIT_ERR_CUDA;
     g_attn_long_attr = true;
   }
@@ -870,7 +881,8 @@ static int launch_attention_long(ivit_ctx* ctx, const ivit_block_params* p, cons
   ctx->attn_gen ^= 1;
   const int64_t grid = a.items < ctx->sm_count ? a.items : ctx->sm_count;
   LaunchScope ls(ctx, KIND_ATTENTION, 4.0 * (double)(B * h) * (double)T * (double)T * (double)d);
-  launch_k(attention_long_kernel, dim3((unsigned)grid), dim3(kLongThreads), smem, ctx->stream, tmQ, tmK, tmV, la);
+  if (p->smax.k_out == 8) launch_k(attention_long_kernel<true>, dim3((unsigned)grid), dim3(kLongThreads), smem, ctx->stream, tmQ, tmK, tmV, la);
+  else launch_k(attention_long_kernel<false>, dim3((unsigned)grid), dim3(kLongThreads), smem, ctx->stream, tmQ, tmK, tmV, la);
   return ls.done();
 }
 
@@ -880,7 +892,6 @@ int launch_attention_fused(ivit_ctx* ctx, const ivit_block_params* p, const int8
   if (!ctx->tmap_encode) return IVIT_ERR_UNSUPPORTED;
   const int64_t B = p->B, T = p->T, D = p->D, h = p->heads, d = D / h;
   if ((d != 32 && d != 64 && d != 128) || B * h > 2147483647LL / 8) return IVIT_ERR_UNSUPPORTED;
-  if (p->smax.k_out != 8) return IVIT_ERR_UNSUPPORTED;   // the fused kernels have the 8-bit IntDiv shift built in
   if ((reinterpret_cast<uintptr_t>(QKV) & 15) || (reinterpret_cast<uintptr_t>(O) & 15)) return IVIT_ERR_UNSUPPORTED;
   if (B == 0) return IVIT_OK;
 #ifdef IVIT_TUNING
@@ -919,8 +930,10 @@ int launch_attention_fused(ivit_ctx* ctx, const ivit_block_params* p, const int8
   const uint32_t p_off = (v_off + a.Npad * a.d + 1023u) & ~1023u;
   const size_t smem = 1024 + p_off + (size_t)((a.Npad + 127) / 128) * 128 * 128 + 1024 + 2048 + 16 + 64 + 16;
   if (!g_attn_attr) {
-    if (cudaFuncSetAttribute(attention_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-        cudaFuncSetAttribute(attention_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+    if (cudaFuncSetAttribute(attention_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(attention_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(attention_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+        cudaFuncSetAttribute(attention_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
       return IVIT_ERR_CUDA;
     g_attn_attr = true;
   }
@@ -932,8 +945,14 @@ int launch_attention_fused(ivit_ctx* ctx, const ivit_block_params* p, const int8
   const int64_t slots = 2 * (int64_t)ctx->sm_count;
   const int64_t grid = a.items < slots ? a.items : slots;
   LaunchScope ls(ctx, KIND_ATTENTION, 4.0 * (double)(B * h) * (double)T * (double)T * (double)d);
-  if (a.G > 1) launch_k(attention_kernel<true>, dim3((unsigned)grid), dim3(kAttnThreads), smem, ctx->stream, tmQ, tmK, tmV, a);
-  else launch_k(attention_kernel<false>, dim3((unsigned)grid), dim3(kAttnThreads), smem, ctx->stream, tmQ, tmK, tmV, a);
+  const bool k8 = p->smax.k_out == 8;
+  if (a.G > 1) {
+    if (k8) launch_k(attention_kernel<true, true>, dim3((unsigned)grid), dim3(kAttnThreads), smem, ctx->stream, tmQ, tmK, tmV, a);
+    else launch_k(attention_kernel<true, false>, dim3((unsigned)grid), dim3(kAttnThreads), smem, ctx->stream, tmQ, tmK, tmV, a);
+  } else {
+    if (k8) launch_k(attention_kernel<false, true>, dim3((unsigned)grid), dim3(kAttnThreads), smem, ctx->stream, tmQ, tmK, tmV, a);
+    else launch_k(attention_kernel<false, false>, dim3((unsigned)grid), dim3(kAttnThreads), smem, ctx->stream, tmQ, tmK, tmV, a);
+  }
   return ls.done();
 }
 

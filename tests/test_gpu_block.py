@@ -128,8 +128,8 @@ def test_block_static_gelu_variant_bit_exact(engine, B, T, D, heads, H):
 
 @pytest.mark.parametrize("k_out", [6, 4])
 def test_block_other_output_width_bit_exact(k_out):
-    """A block whose Shiftmax and ShiftGELU use k_out < 8: the attention core runs as separate kernels (the fused one
-    is built for 8 bits); P*V and the GELU output ratios absorb the coarser scale 1 / 2^(k_out-1)."""
+    """A block whose Shiftmax and ShiftGELU use k_out < 8 (the fused attention kernel has a variant for it); P*V and
+    the GELU output ratios absorb the coarser scale 1 / 2^(k_out-1)."""
     import dataclasses
     from ivit_inputs import ExpParams, Scale
     g = _g()
@@ -176,6 +176,8 @@ def test_attention_random_shapes():
     """Thirty seeded random attention problems (fused short-row, window-packed and key-block kernels, and the composed
     path for head dimensions the fused kernels do not take): random batch, row length, heads and head dimension, with
     and without a score bias; every output element against the oracle."""
+    import dataclasses
+    from ivit_inputs import ExpParams, Scale
     g = _g()
     c = g.ctx()
     rng = np.random.default_rng(77)
@@ -187,9 +189,13 @@ def test_attention_random_shapes():
         bias = bool(rng.random() < 0.4)
         D = heads * d
         blk = make_block(_Ids(2000 + case), 1, B, T, D, heads, 2 * D, attn_bias_batches=heads if bias else 0)
+        k_out = int(rng.choice([8, 8, 7, 5, 3]))          # Eq. (IntDiv) output width of the Shiftmax inside
+        if k_out != 8:
+            blk = dataclasses.replace(blk, smax=ExpParams(blk.smax.I0, blk.smax.N, 45, k_out),
+                                      pv_scale=Scale(blk.pv_scale.mult, max(31, blk.pv_scale.shift - (8 - k_out))))
         dblk = g.binding.DeviceBlock(blk, "cuda")
         QKV = np.clip(np.rint(rng.standard_normal((B * T, 3 * D)) * 32), -128, 127).astype(np.int8)
         got = g.host(c.attention(dblk, torch.from_numpy(QKV).cuda()))
-        g.assert_equal(got, O.attention(blk, QKV), f"case {case}: B={B} T={T} heads={heads} d={d} bias={bias}")
+        g.assert_equal(got, O.attention(blk, QKV), f"case {case}: B={B} T={T} heads={heads} d={d} bias={bias} k_out={k_out}")
     assert c.poll_status() == 0
 
