@@ -654,7 +654,7 @@ int pick_bn(int64_t extent, int64_t tiles_other, int64_t K, int sm_count) {
     const double rounds = (double)((tiles + sm_count - 1) / sm_count);
     const double feed = (double)K * (128.0 + bn) / 46.0;
     const double epilogue = 2000.0 * ((bn + 127) / 128);
-    const double cost = rounds * ((feed > epilogue ? feed : epilogue) + 800.0);
+    const double cost = rounds * ((feed > epilogue ? feed : epilogue) + 1200.0);
     if (!best || cost < best_cost) { best = bn; best_cost = cost; }
   }
 #ifdef IVIT_TUNING
