@@ -14,10 +14,14 @@
  *
  * Parity status: every primitive below is pinned by CPU tests against closed
  * forms, exact rational arithmetic, brute force or a float reference with a
- * committed numeric bound.  orc_block_forward and orc_vit_forward are a
- * composition of pinned primitives; beyond a float shadow-model agreement
- * check their composition has no published activation dump to compare with:
- * "parity unpinned" for the block/model composition order itself.
+ * committed numeric bound.  orc_block_forward, orc_vit_forward and the Python
+ * composition oracle.api.swin_forward are pinned as compositions: each equals
+ * the same model written out in the test from the pinned primitives with
+ * plain numpy indexing (raster-order tokens, windows cut by slicing, np.roll
+ * for the shifted windows, a strided slice for patch merging), mutations of
+ * the outer layers are shown to break that equality, and a float64 shadow of
+ * the block and of the whole ViT agrees within stated bounds.  There is no
+ * published activation dump to compare with.
  */
 #ifndef IVIT_ORACLE_H
 #define IVIT_ORACLE_H

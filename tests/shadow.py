@@ -49,3 +49,25 @@ def block_forward_float(p, X):
     gelu = xr * 0.5 * (1.0 + _erf(xr / math.sqrt(2.0)))
     Hh = gelu * p.gelu.I0 * 128.0 * p.gelu_post.ratio()
     return dense(Hh, p.W2, p.b2, p.fc2_scale) + Xh * p.res2_scale.ratio()
+
+
+def vit_forward_float(model, image):
+    """Float64 shadow of the whole ViT-family model: patch embedding (+ position embedding), class row, blocks,
+    final LayerNorm of the class rows, classifier.  Returns logits in the units of the int32 logits."""
+    import copy
+    B, T, D, P = image.shape[0], model.T, model.D, model.patch
+    g = model.img // P
+    x = image.astype(np.float64).reshape(B, 3, g, P, g, P).transpose(0, 2, 4, 1, 3, 5).reshape(B, g * g, 3 * P * P)
+    E = (x @ model.Wpe.astype(np.float64).T + model.bpe[None, None, :]) * model.pe_scale.ratio()[None, None, :]
+    E = E + model.pos.astype(np.float64)[None] * model.pos_scale.ratio()
+    X = np.concatenate([np.broadcast_to(model.cls.astype(np.float64), (B, 1, D)), E], axis=1).reshape(B * T, D)
+    for blk in model.blocks:
+        bb = copy.copy(blk)
+        bb.B = B
+        X = block_forward_float(bb, X)
+    Z = X.reshape(B, T, D)[:, 0]
+    mu = Z.mean(axis=1, keepdims=True)
+    sd = np.sqrt(((Z - mu) ** 2).mean(axis=1, keepdims=True))
+    gsc = model.lnf_gamma.ratio() * 2.0 ** model.blocks[0].M_ln / math.sqrt(D)
+    Z = (Z - mu) / sd * gsc[None, :] + model.lnf_beta[None, :]
+    return (Z @ model.Whead.astype(np.float64).T + model.bhead[None, :]) * model.head_scale.ratio()[None, :]
