@@ -12,12 +12,22 @@
  *  - Every call returns IVIT_OK (0) or a negative IVIT_ERR_* code; nothing is
  *    enqueued when a call fails argument validation.
  *  - Tensor and parameter-array pointers are DEVICE pointers owned by the
- *    caller.  The library allocates no memory per call; scratch comes from a
+ *    caller.  The operator, block and model entry points that take device
+ *    buffers allocate no memory per call; scratch comes from a
  *    caller-provided workspace (ivit_*_workspace_bytes).  ivit_ctx_create
  *    allocates a few hundred KB once (status word, ShiftGELU table cache).
- *  - Work is enqueued on the CUDA stream held by the context; calls never
- *    synchronise.  Device-side failures (a bounded wait that ran out) are
+ *    Exceptions: ivit_vit_forward_host creates a stream and four events on
+ *    its first call and, with graph replay switched on, instantiates CUDA
+ *    graphs (which allocate on the device); ivit_ctx_profile_start creates
+ *    its events on first use.
+ *  - Work is enqueued on the CUDA stream held by the context; the entry
+ *    points do not synchronise (ivit_ctx_profile_stop and ivit_ctx_destroy
+ *    do).  Device-side failures (a bounded wait that ran out) are
  *    reported by ivit_ctx_poll_status after the stream has been synchronised.
+ *  - A context belongs to one device; the caller keeps that device current
+ *    (cudaSetDevice) while calling into the library with that context.
+ *    Kernel attributes are set per device by ivit_ctx_create, so several
+ *    contexts on several devices may live in one process.
  *  - Matrices are row-major; leading dimensions (ld*) and strides are in
  *    elements.  int8 tensors: pointer 16-byte aligned and ld a multiple of 16.
  *    int32 tensors: pointer 16-byte aligned and ld a multiple of 4.  Otherwise
@@ -92,6 +102,13 @@ int ivit_ctx_set_stream(ivit_ctx* ctx, void* cuda_stream);
 int ivit_ctx_poll_status(ivit_ctx* ctx);
 /* Number of kernels this context has launched since creation. */
 int64_t ivit_ctx_launch_count(const ivit_ctx* ctx);
+/* ShiftGELU look-up tables (one per parameter set: I0, N, M, k_out, post) are built on first use and cached in
+ * the context, 16 sets at a time, the oldest slot being rebuilt for a 17th.  This counter changes whenever a slot
+ * is built or rebuilt.  A CUDA graph that the CALLER captured around library calls holds the addresses of the
+ * tables those calls used: it stays valid while this counter keeps the value it had when the capture ended, and
+ * must be captured again otherwise (or keep the models that share a context to at most 16 parameter sets).  The
+ * library's own graphs (ivit_ctx_set_host_graph) check this themselves. */
+uint64_t ivit_ctx_table_generation(const ivit_ctx* ctx);
 /* Selects the GEMM engine: 0 = tcgen05 tensor-core kernels where the shape
  * qualifies (default), 1 = force the CUDA-core (dp4a) kernels everywhere.
  * Both are bit-exact; the switch exists for testing and measurement. */
@@ -260,6 +277,13 @@ size_t ivit_vit_workspace_bytes(const ivit_vit_params* p);
 int ivit_vit_forward(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* image, int32_t* logits,
                      void* workspace, size_t workspace_bytes);
 
+/* The same forward, additionally copying the output of the last encoder block, [B*T, D] int8 (ld = D), to
+ * `tokens` (device, 16-byte aligned; NULL: no copy).  The class rows of that tensor are what the final LayerNorm
+ * and the classifier read; the other rows reach no logit, so this is the call that lets a caller (or a parity
+ * test) see every byte the encoder produced. */
+int ivit_vit_forward_tokens(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* image, int32_t* logits,
+                            int8_t* tokens, void* workspace, size_t workspace_bytes);
+
 /* Same forward with HOST buffers: copies image_host to a staging area in the workspace, runs
  * ivit_vit_forward, and copies the logits back to logits_host.  The call only enqueues work and
  * returns: the caller synchronises the context's stream before reading logits_host, and both host
@@ -279,7 +303,8 @@ int ivit_vit_forward_host(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t*
  * change of those arguments, a new stream, or switching the mode off drops the graph.  Needs a stream other than
  * the legacy default stream (with the default stream the kernels keep being launched one by one).  Tensors the
  * model description points to may change contents between calls; they must stay at the same addresses.
- * Results are identical in both modes. */
+ * Results are identical in both modes: a graph is dropped, and captured again later, when another call on the
+ * context has rebuilt a slot of the ShiftGELU table cache since the capture (see ivit_ctx_table_generation). */
 int ivit_ctx_set_host_graph(ivit_ctx* ctx, int enable);
 /* Number of graphs currently instantiated for ivit_vit_forward_host (0, 1 or 2: one per staging buffer). */
 int ivit_ctx_host_graph_count(ivit_ctx* ctx);
@@ -295,6 +320,14 @@ int ivit_ctx_profile_start(ivit_ctx* ctx);
 int ivit_ctx_profile_stop(ivit_ctx* ctx);
 int ivit_ctx_profile_get(ivit_ctx* ctx, int32_t idx, int32_t* kind, float* ms, double* work);
 const char* ivit_kernel_kind_name(int32_t kind);
+
+/* Issue-only ceiling of the int8 tensor cores (measurement aid; the paper has no counterpart): one CTA per SM
+ * issues `iters` x 4 tcgen05.mma.kind::i8 instructions of shape M128 x N256 x K32 on operands that stay in
+ * shared memory, with no loads and no epilogue.  Runs the kernel twice on the context's stream (the second
+ * launch is timed with CUDA events), SYNCHRONISES the stream, and returns the time in milliseconds and the int8
+ * operations (2 per multiply-accumulate) of the timed launch; ops / ms is the rate the Dense kernels' TOP/s are
+ * measured against.  1 <= iters <= 2^20. */
+int ivit_probe_int8_mma(ivit_ctx* ctx, int32_t iters, float* ms, double* ops);
 
 /* ---- data movement helpers (not in the paper; needed by the full models) ---- */
 

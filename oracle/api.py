@@ -347,9 +347,10 @@ def vit_forward(p, image, batch=None, return_tokens=False):
     return (logits, tokens) if return_tokens else logits
 
 
-def swin_forward(p, image):
+def swin_forward(p, image, return_tokens=False):
     """Swin-shaped forward (windows, optionally shifted in every second block) composed from the oracle's operators; mirrors the model
-    description in ivit_inputs.params.SwinParams.  Returns int32 logits [B, classes]."""
+    description in ivit_inputs.params.SwinParams.  Returns int32 logits [B, classes]; with return_tokens also the
+    output of the last block ([B * tokens, C] int8, window-major rows) that the final LayerNorm reads."""
     B = image.shape[0]
     X = linear(patchify(image, p.patch, window=p.window), p.Wpe, p.bpe, p.pe_scale)
     X = layernorm(X, p.pe_ln_gamma, p.pe_ln_beta, p.M_ln)
@@ -364,6 +365,8 @@ def swin_forward(p, image):
             G = gather_rows(X, st.merge_index, width=st.C).reshape(-1, 4 * st.C)
             G = layernorm(G, st.merge_ln_gamma, st.merge_ln_beta, p.M_ln)
             X = linear(G, st.Wmerge, None, st.merge_scale)
+    last = X
     X = layernorm(X, p.lnf_gamma, p.lnf_beta, p.M_ln)
     Z = token_mean(X, X.shape[0] // B, p.pool_scale)
-    return linear(Z, p.Whead, p.bhead, p.head_scale, out_dtype=I32)
+    logits = linear(Z, p.Whead, p.bhead, p.head_scale, out_dtype=I32)
+    return (logits, last) if return_tokens else logits

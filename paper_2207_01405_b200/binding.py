@@ -19,7 +19,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libivit.so")
 
 EXPORTS = [
-    "ivit_ctx_create", "ivit_ctx_destroy", "ivit_ctx_set_stream", "ivit_ctx_poll_status", "ivit_ctx_launch_count",
+    "ivit_ctx_create", "ivit_ctx_destroy", "ivit_probe_int8_mma", "ivit_ctx_table_generation", "ivit_vit_forward_tokens", "ivit_ctx_set_stream", "ivit_ctx_poll_status", "ivit_ctx_launch_count",
     "ivit_ctx_set_gemm_engine", "ivit_strerror", "ivit_linear", "ivit_matmul", "ivit_shiftmax", "ivit_shiftgelu",
     "ivit_shiftgelu_static",
     "ivit_shiftmax_direct", "ivit_ctx_set_host_graph", "ivit_ctx_host_graph_count",
@@ -86,6 +86,8 @@ def load_library():
     L.ivit_ctx_launch_count.argtypes = [vp]
     L.ivit_ctx_launch_count.restype = i64
     L.ivit_ctx_set_gemm_engine.argtypes = [vp, C.c_int]
+    L.ivit_ctx_table_generation.argtypes = [vp]
+    L.ivit_ctx_table_generation.restype = C.c_uint64
     L.ivit_ctx_set_host_graph.argtypes = [vp, C.c_int]
     L.ivit_ctx_host_graph_count.argtypes = [vp]
     L.ivit_strerror.argtypes = [C.c_int]
@@ -106,12 +108,14 @@ def load_library():
     L.ivit_vit_workspace_bytes.argtypes = [C.POINTER(CVit)]
     L.ivit_vit_workspace_bytes.restype = C.c_size_t
     L.ivit_vit_forward.argtypes = [vp, C.POINTER(CVit), vp, vp, vp, C.c_size_t]
+    L.ivit_vit_forward_tokens.argtypes = [vp, C.POINTER(CVit), vp, vp, vp, vp, C.c_size_t]
     L.ivit_vit_host_workspace_bytes.argtypes = [C.POINTER(CVit)]
     L.ivit_vit_host_workspace_bytes.restype = C.c_size_t
     L.ivit_vit_forward_host.argtypes = [vp, C.POINTER(CVit), vp, vp, vp, C.c_size_t]
     L.ivit_ctx_profile_start.argtypes = [vp]
     L.ivit_ctx_profile_stop.argtypes = [vp]
     L.ivit_ctx_profile_get.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(C.c_float), C.POINTER(C.c_double)]
+    L.ivit_probe_int8_mma.argtypes = [vp, i32, C.POINTER(C.c_float), C.POINTER(C.c_double)]
     L.ivit_kernel_kind_name.argtypes = [i32]
     L.ivit_kernel_kind_name.restype = C.c_char_p
     L.ivit_patchify.argtypes = [vp, vp, i64, i64, i64, i64, i64, i64, vp, i64]
@@ -224,6 +228,15 @@ class Context:
 
     def launch_count(self) -> int:
         return int(self.lib.ivit_ctx_launch_count(self.h))
+
+    def probe_int8_mma(self, iters: int = 4096):
+        """ivit_probe_int8_mma: (milliseconds, int8 operations) of the issue-only tensor-core loop."""
+        ms, ops = C.c_float(), C.c_double()
+        _chk(self.lib.ivit_probe_int8_mma(self.h, iters, C.byref(ms), C.byref(ops)), "ivit_probe_int8_mma")
+        return ms.value, ops.value
+
+    def table_generation(self) -> int:
+        return int(self.lib.ivit_ctx_table_generation(self.h))
 
     def profile_start(self):
         _chk(self.lib.ivit_ctx_profile_start(self.h), "ivit_ctx_profile_start")
@@ -362,12 +375,18 @@ class Context:
              "ivit_attention")
         return O
 
-    def vit_forward(self, model: "DeviceVit", image, logits=None, workspace=None):
+    def vit_forward(self, model: "DeviceVit", image, logits=None, workspace=None, tokens=None):
+        """ivit_vit_forward; with `tokens` ([B*T, D] int8) ivit_vit_forward_tokens, which also hands back the
+        output of the last encoder block."""
         if logits is None:
             logits = torch.empty((model.c.B, model.c.classes), dtype=torch.int32, device=image.device)
         ws = workspace if workspace is not None else model.workspace()
-        _chk(self.lib.ivit_vit_forward(self.h, C.byref(model.c), image.data_ptr(), logits.data_ptr(), ws.data_ptr(),
-                                       ws.numel()), "ivit_vit_forward")
+        if tokens is None:
+            _chk(self.lib.ivit_vit_forward(self.h, C.byref(model.c), image.data_ptr(), logits.data_ptr(), ws.data_ptr(),
+                                           ws.numel()), "ivit_vit_forward")
+        else:
+            _chk(self.lib.ivit_vit_forward_tokens(self.h, C.byref(model.c), image.data_ptr(), logits.data_ptr(),
+                                                  tokens.data_ptr(), ws.data_ptr(), ws.numel()), "ivit_vit_forward_tokens")
         return logits
 
 
@@ -498,7 +517,7 @@ class DeviceSwin:
                               device=device)
 
 
-def swin_forward(ctx: Context, m: DeviceSwin, image: torch.Tensor) -> torch.Tensor:
+def swin_forward(ctx: Context, m: DeviceSwin, image: torch.Tensor, return_tokens: bool = False):
     """Swin-shaped forward composed from the library's entry points (every step is a library kernel):
     patchify (window-major) -> Dense -> LN -> [blocks -> 2x2 gather -> LN -> Dense] x stages -> LN -> token
     mean -> Dense head (int32 logits)."""
@@ -518,7 +537,9 @@ def swin_forward(ctx: Context, m: DeviceSwin, image: torch.Tensor) -> torch.Tens
             G = ctx.gather_rows(X, st["merge_index"], width=C_).view(-1, 4 * C_)
             G = ctx.layernorm(G, st["merge_ln_gamma"], st["merge_ln_beta"], p.M_ln)
             X = ctx.linear(G, st["Wmerge"], None, st["merge_scale"])
+    last = X
     X = ctx.layernorm(X, m.lnf_gamma, m.lnf_beta, p.M_ln)
     tokens = X.shape[0] // image.shape[0]
     Z = ctx.token_mean(X, tokens, m.pool_scale)
-    return ctx.linear(Z, m.Whead, m.bhead, m.head_scale, out_dtype=I32)
+    logits = ctx.linear(Z, m.Whead, m.bhead, m.head_scale, out_dtype=I32)
+    return (logits, last) if return_tokens else logits

@@ -8,7 +8,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "build")
 LIB = os.path.join(HERE, "libivit.so")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
-SOURCES = ["host.cu", "nonlinear.cu", "gemm_simt.cu", "gemm_tc.cu", "attention.cu", "helpers.cu"]
+SOURCES = ["host.cu", "nonlinear.cu", "gemm_simt.cu", "gemm_tc.cu", "attention.cu", "helpers.cu", "probe.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", INCLUDE]
 

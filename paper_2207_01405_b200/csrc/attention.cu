@@ -826,11 +826,19 @@ __global__ void __launch_bounds__(kLongThreads, 1) attention_long_kernel(const _
   }
 }
 
-bool g_attn_long_attr = false;
-
-bool g_attn_attr = false;
-
 }  // namespace
+
+// The shared-memory limit of a kernel is a per-device attribute: set for the current device at context creation.
+int attention_prepare_device() {
+  if (cudaFuncSetAttribute(attention_long_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+      cudaFuncSetAttribute(attention_long_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+      cudaFuncSetAttribute(attention_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+      cudaFuncSetAttribute(attention_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+      cudaFuncSetAttribute(attention_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
+      cudaFuncSetAttribute(attention_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
+    return IVIT_ERR_CUDA;
+  return IVIT_OK;
+}
 
 // Rows longer than 256 tokens: key blocks, one CTA per SM.  IVIT_ERR_UNSUPPORTED when the row does not fit the
 // kernel's shared memory (the probabilities of a 128-row tile and the whole V of a head stay resident).
@@ -844,9 +852,6 @@ static int launch_attention_long(ivit_ctx* ctx, const ivit_block_params* p, cons
   a.tmem_cols = 512;
   a.G = 1; a.R = 128; a.Btot = (int)B;
   int nb_max = ((512 - (int)d) / 2) / 32 * 32 > 224 ? 224 : ((512 - (int)d) / 2) / 32 * 32;   // two score buffers + d output columns
-#ifdef IVIT_TUNING
-  if (const char* e = getenv("IVIT_ATTN_LONG")) { const int f = atoi(e); if (f >= 32 && f < nb_max) nb_max = f; }   // stress runs only
-#endif
   la.nblk = (a.Npad + nb_max - 1) / nb_max;
   la.NB = ((a.Npad + la.nblk - 1) / la.nblk + 31) / 32 * 32;
   la.nv = (a.Npad + 255) / 256;
@@ -868,12 +873,6 @@ static int launch_attention_long(ivit_ctx* ctx, const ivit_block_params* p, cons
       !make_tensor_map(ctx, &tmK, QKV + D, d, T, h, B, ldq, d, T * ldq, 128, la.NB, CU_TENSOR_MAP_SWIZZLE_128B, a.k_pos) ||
       !make_tensor_map(ctx, &tmV, QKV + 2 * D, d, T, h, B, ldq, d, T * ldq, (int)d, 256, vsw, a.v_pos))
     return IVIT_ERR_UNSUPPORTED;
-  if (!g_attn_long_attr) {
-    if (cudaFuncSetAttribute(attention_long_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-        cudaFuncSetAttribute(attention_long_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
-      return IVIT_ERR_CUDA;
-    g_attn_long_attr = true;
-  }
   a.bh = (int)(B * h);
   a.items = (int)(B * h * a.tiles_m);
   a.sched = ctx->sched_dev + 2 * ctx->attn_gen;
@@ -894,9 +893,6 @@ int launch_attention_fused(ivit_ctx* ctx, const ivit_block_params* p, const int8
   if ((d != 32 && d != 64 && d != 128) || B * h > 2147483647LL / 8) return IVIT_ERR_UNSUPPORTED;
   if ((reinterpret_cast<uintptr_t>(QKV) & 15) || (reinterpret_cast<uintptr_t>(O) & 15)) return IVIT_ERR_UNSUPPORTED;
   if (B == 0) return IVIT_OK;
-#ifdef IVIT_TUNING
-  if (getenv("IVIT_ATTN_LONG") && T > 64) return launch_attention_long(ctx, p, QKV, O);   // stress runs only
-#endif
   if (T > 256) return launch_attention_long(ctx, p, QKV, O);
   AttnArgs a{};
   a.T = (int)T; a.d = (int)d; a.heads = (int)h; a.D = D;
@@ -929,14 +925,6 @@ int launch_attention_fused(ivit_ctx* ctx, const ivit_block_params* p, const int8
   const uint32_t v_off = 128 * 128 + a.Npad * 128;
   const uint32_t p_off = (v_off + a.Npad * a.d + 1023u) & ~1023u;
   const size_t smem = 1024 + p_off + (size_t)((a.Npad + 127) / 128) * 128 * 128 + 1024 + 2048 + 16 + 64 + 16;
-  if (!g_attn_attr) {
-    if (cudaFuncSetAttribute(attention_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-        cudaFuncSetAttribute(attention_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-        cudaFuncSetAttribute(attention_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess ||
-        cudaFuncSetAttribute(attention_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) != cudaSuccess)
-      return IVIT_ERR_CUDA;
-    g_attn_attr = true;
-  }
   a.bh = (int)((B + a.G - 1) / a.G * h);
   a.items = a.bh * a.tiles_m;
   a.sched = ctx->sched_dev + 2 * ctx->attn_gen;

@@ -34,6 +34,7 @@ struct ivit_ctx {
   ivit::GeluKey gelu_keys[ivit::kGeluTableSlots];
   int gelu_used;
   int gelu_next;
+  uint64_t gelu_gen;    // bumped whenever a table slot is (re)built: graphs that point at the tables check it
   int64_t launches;
   int gemm_engine;
   int sm_count;
@@ -48,6 +49,10 @@ struct ivit_ctx {
   cudaGraphExec_t hg_exec[2];
   char* hg_key[2];          // model description, workspace and stream the graph was captured with
   size_t hg_key_bytes[2];
+  size_t hg_key_cap[2];     // allocated size of hg_key (the buffers are reused from call to call)
+  char* hg_scratch;         // key of the current call, compared with hg_key
+  size_t hg_scratch_cap;
+  uint64_t hg_gen[2];       // table generation the graph was captured at
   int hg_seen[2];           // calls seen with this key (-1: capture failed, launch kernel by kernel)
   int64_t hg_launches[2];   // kernels inside the graph
   // per-kernel timing session (ivit_ctx_profile_*)
@@ -88,16 +93,21 @@ struct ScaleDev {
 
 inline ScaleDev to_dev(const ivit_scale& s) { return ScaleDev{s.mult_c, s.shift_c, s.mult, s.shift}; }
 
-// Algorithm 1, function ShiftExp, for I <= 0 (32-bit: |I| < 2^15, I0 <= 2^15, N <= 24).
+// Integer exponential of a non-positive argument, exp(S * I) in units of S * 2^-N with I0 = round(1 / S):
+// Eq. (exp_shift) turns the base into 2 with log2(e) ~ (1.0111)b, so the exponent is -n / I0 with
+// n = nd + ceil(nd / 2) - ceil(nd / 16) for nd = -I >= 0 (the arithmetic shifts of the negative I round towards
+// -inf, which is what the two ceilings say); n = q * I0 + r splits it into an integer power of two and a
+// fraction -r / I0 in (-1, 0], on which Eq. (linear) takes 2^x ~ 1 + x / 2: mantissa I0 - ceil(r / 2), scaled by
+// 2^(N - q).  32-bit: nd < 2^15, I0 <= 2^15, N <= 24.
 __device__ __forceinline__ unsigned shiftexp(int I, int I0, int N) {
-  int Ip = I + (I >> 1) - (I >> 4);  // I * log2(e) as (1.0111)b; >> on int is arithmetic in CUDA
-  int negp = -Ip;                    // >= 0
-  int q = negp / I0;                 // floor(Ip / (-I0))
-  int r = negp - q * I0;             // 0 <= r < I0
-  int Ib = I0 - ((r + 1) >> 1);      // ((-r) >> 1) + I0
-  if (q <= N) return (unsigned)Ib << (N - q);
-  int sh = q - N;
-  return sh >= 31 ? 0u : ((unsigned)Ib >> sh);
+  const unsigned nd = (unsigned)(-I);
+  const unsigned n = nd + ((nd + 1u) >> 1) - ((nd + 15u) >> 4);
+  const unsigned q = n / (unsigned)I0;
+  const unsigned r = n - q * (unsigned)I0;
+  const unsigned mant = (unsigned)I0 - ((r + 1u) >> 1);
+  if (q <= (unsigned)N) return mant << ((unsigned)N - q);
+  const unsigned down = q - (unsigned)N;
+  return down >= 31u ? 0u : mant >> down;
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
@@ -182,6 +192,9 @@ int launch_gemm_simt(ivit_ctx* ctx, const GemmProblem& g);
 // Returns IVIT_ERR_UNSUPPORTED when the shape does not qualify for the tensor-core kernel.
 int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g);
 int launch_gemm(ivit_ctx* ctx, const GemmProblem& g);
+// Per-device kernel attributes (shared-memory limits) of the tensor-core kernels, for the current device.
+int gemm_tc_prepare_device();
+int attention_prepare_device();
 // Fused Q K^T -> requant -> Shiftmax -> P V -> requant; IVIT_ERR_UNSUPPORTED when the shape does not qualify.
 int launch_attention_fused(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* QKV, int8_t* O);
 

@@ -638,9 +638,6 @@ int pow2_at_least(int v) {
 constexpr size_t kSmemBudget = 227 * 1024;
 constexpr size_t kSmemFixed = 1024 + 8 * (2 * kMaxStages + 5 + 2 * kEpiWarps) + 32 + 512;
 
-bool g_attr_set = false;
-
-// Tile width along the TMEM columns: the candidate with the least (waves x tile cost).
 // Tile width along the TMEM columns: the candidate with the least (rounds of tiles per CTA) x (time of a tile).
 // A tile's time is the larger of its operand traffic, (128 + bn) x K bytes at about 46 bytes per clock into an
 // SM's shared memory, and its epilogue, one 32-row chunk per epilogue part at a time (about 2000 clocks per round
@@ -657,13 +654,20 @@ int pick_bn(int64_t extent, int64_t tiles_other, int64_t K, int sm_count) {
     const double cost = rounds * ((feed > epilogue ? feed : epilogue) + 1200.0);
     if (!best || cost < best_cost) { best = bn; best_cost = cost; }
   }
-#ifdef IVIT_TUNING
-  if (const char* f = getenv("IVIT_FORCE_BN")) return atoi(f);   // sweeps only
-#endif
   return best;
 }
 
 }  // namespace
+
+// The shared-memory limit of a kernel is a per-device attribute: set for the current device at context creation.
+int gemm_tc_prepare_device() {
+  if (cudaFuncSetAttribute(gemm_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
+      cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
+      cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
+      cudaFuncSetAttribute(gemm_tc_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess)
+    return IVIT_ERR_CUDA;
+  return IVIT_OK;
+}
 
 int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
   if (!ctx->tmap_encode) return IVIT_ERR_UNSUPPORTED;
@@ -746,14 +750,6 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
   a.total_tiles = (int64_t)a.tiles_p * a.tiles_q * batches;
 
   const size_t smem = kSmemFixed + (size_t)a.stages * stage + fixed;
-  if (!g_attr_set) {
-    if (cudaFuncSetAttribute(gemm_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
-        cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
-        cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
-        cudaFuncSetAttribute(gemm_tc_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess)
-      return IVIT_ERR_CUDA;
-    g_attr_set = true;
-  }
   const unsigned grid = (unsigned)(a.total_tiles < ctx->sm_count ? a.total_tiles : ctx->sm_count);
   LaunchScope ls(ctx, KIND_GEMM_TC, 2.0 * (double)batches * (double)g.M * (double)g.N * (double)g.K);
   // the encoder block's Dense layers take the specialised instantiations

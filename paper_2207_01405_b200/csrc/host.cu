@@ -157,16 +157,27 @@ namespace {
 void host_graph_drop(ivit_ctx* ctx, int slot) {
   if (ctx->hg_exec[slot]) cudaGraphExecDestroy(ctx->hg_exec[slot]);
   ctx->hg_exec[slot] = nullptr;
-  delete[] ctx->hg_key[slot];
-  ctx->hg_key[slot] = nullptr;
-  ctx->hg_key_bytes[slot] = 0;
+  ctx->hg_key_bytes[slot] = 0;   // the key buffer itself is kept for the next description
   ctx->hg_seen[slot] = 0;
+}
+
+bool grow(char*& buf, size_t& cap, size_t need) {
+  if (cap >= need) return true;
+  char* n = new (std::nothrow) char[need];
+  if (!n) return false;
+  delete[] buf;
+  buf = n;
+  cap = need;
+  return true;
 }
 
 // The device part of ivit_vit_forward_host.  With graph replay switched on, the third call that repeats the same
 // model description, buffers and stream captures the forward into a CUDA graph (the first two run kernel by
-// kernel, so that look-up tables and kernel attributes exist); later calls launch the instantiated graph.  Any
-// change of the arguments drops the graph.  A capture that fails leaves the kernel-by-kernel path in place.
+// kernel, so that look-up tables exist); later calls launch the instantiated graph.  Any change of the arguments
+// drops the graph.  The graph holds the addresses of cached ShiftGELU tables: it is only kept while the table
+// generation of the context is the one it was captured at (another call that rebuilds a table slot makes the
+// next call fall back to kernels and capture again), and a capture during which a table had to be built is thrown
+// away.  A capture that fails leaves the kernel-by-kernel path in place.
 int forward_or_replay(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* img_dev, int32_t* lg_dev, void* workspace,
                       size_t inner, int slot) {
   if (!ctx->host_graph || ctx->profiling || ctx->stream == nullptr)
@@ -174,28 +185,47 @@ int forward_or_replay(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* img
   const size_t nb = (size_t)p->depth * sizeof(ivit_block_params);
   const void* tail[4] = {img_dev, lg_dev, workspace, (const void*)ctx->stream};
   const size_t key_bytes = sizeof(*p) + nb + sizeof(tail) + sizeof(int);
-  char* key = new (std::nothrow) char[key_bytes];
-  if (!key) return IVIT_ERR_CUDA;
+  if (!grow(ctx->hg_scratch, ctx->hg_scratch_cap, key_bytes)) return IVIT_ERR_CUDA;
+  char* key = ctx->hg_scratch;
   std::memcpy(key, p, sizeof(*p));
   std::memcpy(key + sizeof(*p), p->blocks, nb);
   std::memcpy(key + sizeof(*p) + nb, tail, sizeof(tail));
   std::memcpy(key + sizeof(*p) + nb + sizeof(tail), &ctx->gemm_engine, sizeof(int));
-  const bool same = ctx->hg_key[slot] && ctx->hg_key_bytes[slot] == key_bytes && std::memcmp(ctx->hg_key[slot], key, key_bytes) == 0;
+  const bool same = ctx->hg_key_bytes[slot] == key_bytes && std::memcmp(ctx->hg_key[slot], key, key_bytes) == 0;
   if (!same) {
     host_graph_drop(ctx, slot);
-    ctx->hg_key[slot] = key;
+    if (!grow(ctx->hg_key[slot], ctx->hg_key_cap[slot], key_bytes)) return IVIT_ERR_CUDA;
+    std::memcpy(ctx->hg_key[slot], key, key_bytes);
     ctx->hg_key_bytes[slot] = key_bytes;
     ctx->hg_seen[slot] = 1;
     return ivit_vit_forward(ctx, p, img_dev, lg_dev, workspace, inner);
   }
-  delete[] key;
   if (ctx->hg_exec[slot]) {
-    if (cudaGraphLaunch(ctx->hg_exec[slot], ctx->stream) != cudaSuccess) return IVIT_ERR_CUDA;
-    ctx->launches += ctx->hg_launches[slot];
-    return IVIT_OK;
+    if (ctx->hg_gen[slot] == ctx->gelu_gen) {
+      if (cudaGraphLaunch(ctx->hg_exec[slot], ctx->stream) != cudaSuccess) return IVIT_ERR_CUDA;
+      ctx->launches += ctx->hg_launches[slot];
+      return IVIT_OK;
+    }
+    // a table slot was rebuilt since the capture: the graph may point at another parameter set's table
+    cudaGraphExecDestroy(ctx->hg_exec[slot]);
+    ctx->hg_exec[slot] = nullptr;
+    ctx->hg_seen[slot] = 1;
+    return ivit_vit_forward(ctx, p, img_dev, lg_dev, workspace, inner);
   }
   if (ctx->hg_seen[slot] < 0 || ++ctx->hg_seen[slot] < 3) return ivit_vit_forward(ctx, p, img_dev, lg_dev, workspace, inner);
   const int64_t before = ctx->launches;
+  // state of the table cache, put back if the capture is not kept (kernels recorded in a discarded capture never ran)
+  GeluKey keys_before[kGeluTableSlots];
+  std::memcpy(keys_before, ctx->gelu_keys, sizeof(keys_before));
+  const int used_before = ctx->gelu_used, next_before = ctx->gelu_next;
+  const uint64_t gen_before = ctx->gelu_gen;
+  auto restore_cache = [&]() {
+    if (ctx->gelu_gen == gen_before) return;
+    std::memcpy(ctx->gelu_keys, keys_before, sizeof(keys_before));
+    ctx->gelu_used = used_before;
+    ctx->gelu_next = next_before;
+    ++ctx->gelu_gen;
+  };
   if (cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
     cudaGetLastError();
     ctx->hg_seen[slot] = -1;
@@ -205,9 +235,11 @@ int forward_or_replay(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* img
   cudaGraph_t graph = nullptr;
   const cudaError_t end = cudaStreamEndCapture(ctx->stream, &graph);
   cudaGraphExec_t exec = nullptr;
-  if (rc == IVIT_OK && end == cudaSuccess && graph && cudaGraphInstantiate(&exec, graph, 0) == cudaSuccess) {
+  const bool tables_stable = ctx->gelu_gen == gen_before;
+  if (rc == IVIT_OK && end == cudaSuccess && graph && tables_stable && cudaGraphInstantiate(&exec, graph, 0) == cudaSuccess) {
     cudaGraphDestroy(graph);
     ctx->hg_exec[slot] = exec;
+    ctx->hg_gen[slot] = ctx->gelu_gen;
     ctx->hg_launches[slot] = ctx->launches - before;
     if (cudaGraphLaunch(exec, ctx->stream) != cudaSuccess) return IVIT_ERR_CUDA;
     return IVIT_OK;
@@ -215,9 +247,11 @@ int forward_or_replay(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* img
   if (graph) cudaGraphDestroy(graph);
   cudaGetLastError();
   ctx->launches = before;
-  ctx->hg_seen[slot] = -1;
+  restore_cache();
+  // a model with more parameter sets than table slots rebuilds tables on every call: try again later, not never
+  ctx->hg_seen[slot] = tables_stable ? -1 : 1;
   if (rc) return rc;
-  return ivit_vit_forward(ctx, p, img_dev, lg_dev, workspace, inner);   // nothing ran during the failed capture
+  return ivit_vit_forward(ctx, p, img_dev, lg_dev, workspace, inner);   // nothing ran during the discarded capture
 }
 
 }  // namespace
@@ -278,6 +312,13 @@ int ivit_ctx_create(ivit_ctx** out, int device, void* cuda_stream) {
       qres != cudaDriverEntryPointSuccess)
     fn = nullptr;
   c->tmap_encode = fn;
+  if (gemm_tc_prepare_device() != IVIT_OK || attention_prepare_device() != IVIT_OK) {
+    cudaGetLastError();
+    cudaFree(c->gelu_tables);
+    cudaFreeHost(c->status_host);
+    delete c;
+    return IVIT_ERR_CUDA;
+  }
   c->sched_dev = reinterpret_cast<unsigned*>(c->gelu_tables + (size_t)kGeluTableSlots * kGeluTableBytes);
   *out = c;
   return IVIT_OK;
@@ -286,9 +327,15 @@ int ivit_ctx_create(ivit_ctx** out, int device, void* cuda_stream) {
 int ivit_ctx_destroy(ivit_ctx* ctx) {
   if (!ctx) return IVIT_ERR_INVALID_ARG;
   cudaSetDevice(ctx->device);
+  // graphs point at the table cache: drop them and let the stream drain before the cache is freed
+  for (int i = 0; i < 2; ++i) {
+    host_graph_drop(ctx, i);
+    delete[] ctx->hg_key[i];
+  }
+  delete[] ctx->hg_scratch;
+  cudaStreamSynchronize(ctx->stream);
   cudaFree(ctx->gelu_tables);
   cudaFreeHost(ctx->status_host);
-  for (int i = 0; i < 2; ++i) host_graph_drop(ctx, i);
   if (ctx->copy_stream) {
     cudaStreamSynchronize(ctx->copy_stream);
     for (int i = 0; i < 2; ++i) {
@@ -313,6 +360,7 @@ int ivit_ctx_set_stream(ivit_ctx* ctx, void* cuda_stream) {
   for (int i = 0; i < 2; ++i) host_graph_drop(ctx, i);
   ctx->gelu_used = 0;  // tables were built in the order of the old stream
   ctx->gelu_next = 0;
+  ++ctx->gelu_gen;
   return IVIT_OK;
 }
 
@@ -325,6 +373,8 @@ int ivit_ctx_poll_status(ivit_ctx* ctx) {
 }
 
 int64_t ivit_ctx_launch_count(const ivit_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+uint64_t ivit_ctx_table_generation(const ivit_ctx* ctx) { return ctx ? ctx->gelu_gen : 0; }
 
 int ivit_ctx_set_gemm_engine(ivit_ctx* ctx, int engine) {
   if (!ctx || engine < 0 || engine > 1) return IVIT_ERR_INVALID_ARG;
@@ -476,6 +526,8 @@ int ivit_block_forward_static(ivit_ctx* ctx, const ivit_block_params* p, const i
   if (block_ws(p).total > (size_t)IVIT_STATIC_SCRATCH_BYTES) return IVIT_ERR_WORKSPACE;   // larger than the fixed scratch
   // In host code the array's name is only a handle; kernels need its device address, which differs per
   // device.  It is looked up once per device, with that device current, and kept.
+  // (Two host threads making the first call on a device at the same time both look the address up and store the
+  // same value: harmless.)
   static void* scratch_of_device[64] = {nullptr};
   if (ctx->device < 0 || ctx->device >= 64) return IVIT_ERR_UNSUPPORTED;
   if (!scratch_of_device[ctx->device]) {
@@ -545,10 +597,16 @@ size_t ivit_vit_workspace_bytes(const ivit_vit_params* p) {
 
 int ivit_vit_forward(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* image, int32_t* logits,
                      void* workspace, size_t workspace_bytes) {
+  return ivit_vit_forward_tokens(ctx, p, image, logits, nullptr, workspace, workspace_bytes);
+}
+
+int ivit_vit_forward_tokens(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* image, int32_t* logits,
+                            int8_t* tokens, void* workspace, size_t workspace_bytes) {
   if (!ctx || !image || !logits) return IVIT_ERR_INVALID_ARG;
   int rc = check_vit(p);
   if (rc) return rc;
   if (!aligned16(image) || !aligned16(logits) || p->classes % 4) return IVIT_ERR_ALIGNMENT;
+  if (tokens && !aligned16(tokens)) return IVIT_ERR_ALIGNMENT;
   const VitWs w = vit_ws(p);
   if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < w.total) return IVIT_ERR_WORKSPACE;
   char* ws = static_cast<char*>(workspace);
@@ -568,6 +626,8 @@ int ivit_vit_forward(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* imag
     if ((rc = block_impl(ctx, &p->blocks[l], X, Y, ws + w.block))) return rc;
     int8_t* t = X; X = Y; Y = t;
   }
+  if (tokens && cudaMemcpyAsync(tokens, X, (size_t)(B * T * D), cudaMemcpyDeviceToDevice, ctx->stream) != cudaSuccess)
+    return IVIT_ERR_CUDA;
   // final LayerNorm on the class-token rows, then the classifier (int32 logits, not saturated)
   if ((rc = launch_layernorm(ctx, X, IVIT_I8, T * D, to_dev(p->lnf_gamma), p->lnf_beta, p->blocks[0].M_ln, Z, D, B, D))) return rc;
   return launch_gemm(ctx, linear_problem(Z, D, p->Whead, D, p->bhead, p->head_scale, nullptr, 0, 1, none, logits,

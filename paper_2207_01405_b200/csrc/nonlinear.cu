@@ -731,29 +731,32 @@ int launch_shiftmax_direct(ivit_ctx* ctx, const int32_t* in, int64_t ldin, ivit_
 
 // ------------------------------------------------------------------ ShiftGELU
 
-// Because the input is int8 and the row statistic is I_max = max(0, I_p(max_row x)), the output
-// is a function of (max(0, row max of x), x): 128 x 256 values.  They are produced here by
-// running Algorithm 2 literally once per pair; the row kernel then only looks values up.
+// ShiftGELU over an int8 row depends on two numbers only: the element x and m = max(0, row maximum of x)
+// (the scaled value 1.702 x ~ (1.1011)b x of Eq. (GELU) is monotone in x, so its row maximum is that of m).
+// The 128 x 256 results are produced once per parameter set; the row kernel then only looks values up.
+// Entry (m, x): sigmoid(1.702 S x) as e / (e + e1) with both exponentials taken relative to the scaled maximum
+// (Eq. (sigmoid)): e = exp of (scaled x - scaled m), e1 = exp of (-scaled m); quotient by Eq. (IntDiv) with
+// M = 45 and k_out bits; the product x * quotient is requantised by `post` and saturated.
 __global__ void shiftgelu_table_kernel(ivit_exp_params p, int post_m, int post_s, int8_t* __restrict__ table) {
   pdl_trigger();
   pdl_wait();
-  const int rmax = blockIdx.x;         // max(0, row max of x), 0..127
+  const int m = blockIdx.x;            // 0..127
   const int x = (int)threadIdx.x - 128;
   int out = 0;
-  if (x <= rmax) {
-    const int Ip = x + (x >> 1) + (x >> 3) + (x >> 4);              // 1.702 x as (1.1011)b
-    const int Imax = rmax + (rmax >> 1) + (rmax >> 3) + (rmax >> 4);  // I_p is monotone in x; rmax >= 0
-    const unsigned e1 = shiftexp(-Imax, p.I0, p.N);
-    const unsigned e = shiftexp(Ip - Imax, p.I0, p.N);
+  if (x <= m) {                        // pairs with x above the row maximum cannot occur
+    auto scaled = [](int v) { return v + (v >> 1) + (v >> 3) + (v >> 4); };
+    const int top = scaled(m);
+    const unsigned e1 = shiftexp(-top, p.I0, p.N);
+    const unsigned e = shiftexp(scaled(x) - top, p.I0, p.N);
     const unsigned long long den = (unsigned long long)e + e1;
-    int div = 0;
+    int quot = 0;
     if (den != 0) {
-      const unsigned long long f = (1ull << 45) / den;  // Eq. (IntDiv), M = 45
-      div = (int)((f * e) >> (46 - p.k_out));             // f*e <= 2^45
+      const unsigned long long recip = (1ull << 45) / den;
+      quot = (int)((recip * e) >> (46 - p.k_out));       // recip * e <= 2^45
     }
-    out = sat8(rq(x * div, post_m, post_s));
+    out = sat8(rq(x * quot, post_m, post_s));
   }
-  table[rmax * 256 + threadIdx.x] = (int8_t)out;
+  table[m * 256 + threadIdx.x] = (int8_t)out;
 }
 
 template <int WPL>
@@ -829,6 +832,7 @@ static int gelu_table(ivit_ctx* ctx, ivit_exp_params p, ivit_scale post, const i
       ctx->gelu_next = (ctx->gelu_next + 1) % kGeluTableSlots;
     }
     ctx->gelu_keys[slot] = key;
+    ++ctx->gelu_gen;
     LaunchScope lt(ctx, KIND_GELU_TABLE, (double)kGeluTableBytes);
     launch_k(shiftgelu_table_kernel, dim3(128), dim3(256), 0, ctx->stream, p, post.mult, post.shift,
                                                           ctx->gelu_tables + (size_t)slot * kGeluTableBytes);

@@ -1,5 +1,6 @@
-"""GPU parity on the other workloads: ViT-B, ViT-L/384 and Swin-T shapes (reduced batch / depth for the
-element-by-element comparison), and sampled images at the full sizes the configs name."""
+"""GPU parity on the other workloads: ViT-B, ViT-L/384 and Swin-T shapes at reduced batch / depth, the graph-replay
+launch configuration of the benchmark, and the host-buffer entry point.  The full configured sizes are in
+test_gpu_full.py."""
 import numpy as np
 import pytest
 import torch
@@ -56,18 +57,6 @@ def test_swin_shifted_windows_bit_exact():
     assert c.poll_status() == 0
 
 
-def test_vit_base_b128_full_size_sampled():
-    """Config 2 at its full size (batch 128, 12 blocks); the oracle recomputes sampled images."""
-    g = _g()
-    c = g.ctx()
-    model, image = make_config(2)
-    dm = g.binding.DeviceVit(model, "cuda")
-    logits = g.host(c.vit_forward(dm, torch.from_numpy(image).cuda()))
-    for i in (0, 127):
-        g.assert_equal(logits[i:i + 1], O.vit_forward(model, image[i:i + 1]), f"image {i}")
-    assert c.poll_status() == 0
-
-
 def test_deit_small_b64_full_size_graph_replay_sampled():
     """Config 1 at its full size in the launch configuration the benchmark times: the whole forward captured into
     one CUDA graph on a side stream and replayed (twice, the second time on a changed input buffer); sampled images
@@ -102,32 +91,6 @@ def test_deit_small_b64_full_size_graph_replay_sampled():
         side.synchronize()
         logits2 = g.host(d_logits)
         g.assert_equal(logits2, logits[::-1], "replay 2 (batch reversed)")
-    assert c.poll_status() == 0
-
-
-def test_vit_large_384_b32_full_size_sampled():
-    """Config 4 at its full size (batch 32, 24 blocks, 577 tokens: attention composed from MatMul and Shiftmax
-    kernels); the oracle recomputes one sampled image."""
-    g = _g()
-    c = g.ctx()
-    model, image = make_config(4)
-    dm = g.binding.DeviceVit(model, "cuda")
-    logits = g.host(c.vit_forward(dm, torch.from_numpy(image).cuda()))
-    g.assert_equal(logits[31:32], O.vit_forward(model, image[31:32]), "image 31")
-    assert c.poll_status() == 0
-
-
-def test_swin_tiny_b64_full_size_sampled():
-    """Config 3 at its full size (batch 64); the oracle recomputes sampled images."""
-    g = _g()
-    c = g.ctx()
-    model, image = make_config(3)
-    dm = g.binding.DeviceSwin(model, "cuda")
-    logits = g.host(g.binding.swin_forward(c, dm, torch.from_numpy(image).cuda()))
-    one, _ = make_config(3, batch=1)      # the same weights with the window counts of a single image
-    assert np.array_equal(one.Wpe, model.Wpe)
-    for i in (0, 63):
-        g.assert_equal(logits[i:i + 1], O.swin_forward(one, image[i:i + 1]), f"image {i}")
     assert c.poll_status() == 0
 
 
@@ -199,3 +162,42 @@ def test_host_forward_graph_replay_mode():
         g.assert_equal(y.numpy(), want2, "mode off")
     assert c.poll_status() == 0
 
+
+
+def test_host_graph_survives_table_cache_eviction():
+    """The graphs of ivit_vit_forward_host point at cached ShiftGELU tables.  Seventeen ivit_shiftgelu calls with
+    distinct parameter sets between two forwards rebuild every slot of the 16-entry cache; the next forward must
+    notice (table generation) and still give the oracle's logits instead of replaying a graph that reads another
+    parameter set's table."""
+    import gpu_util as g
+    from ivit_inputs import ExpParams, Scale
+    from ivit_inputs.gen import dyadic
+    dev = torch.device("cuda", 0)
+    c = g.binding.Context(0)
+    side = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(side):
+        c.set_stream(side)
+        c.set_host_graph(True)
+        model, image = make_config(1, batch=2, depth=2)
+        dm = g.binding.DeviceVit(model, dev)
+        ws = dm.host_workspace()
+        h_img = torch.from_numpy(image).pin_memory()
+        want = O.vit_forward(model, image)
+        outs = [torch.empty((2, model.classes), dtype=torch.int32).pin_memory() for _ in range(12)]
+        for y in outs[:6]:
+            g.binding.vit_forward_host(c, dm, h_img, y, ws)
+        side.synchronize()
+        assert c.host_graph_count() == 2
+        gen = c.table_generation()
+        x = torch.from_numpy(np.random.default_rng(3).integers(-128, 128, (8, 64), dtype=np.int8)).to(dev)
+        post = g.binding.DevScale(Scale(*dyadic(1.0 / 115.0)), dev)
+        for k in range(17):
+            c.shiftgelu(x, ExpParams(40 + k, 23), post)
+        assert c.table_generation() >= gen + 17
+        for y in outs[6:]:
+            g.binding.vit_forward_host(c, dm, h_img, y, ws)
+        side.synchronize()
+        for k, y in enumerate(outs):
+            g.assert_equal(y.numpy(), want, f"call {k}")
+        assert c.host_graph_count() == 2          # captured again after the eviction
+    assert c.poll_status() == 0

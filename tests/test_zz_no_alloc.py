@@ -11,6 +11,7 @@ import torch
 
 from ivit_inputs import make_config
 from ivit_inputs.gen import _Ids, make_block, make_block_input
+from oracle import api as O
 
 pytestmark = pytest.mark.gpu
 
@@ -28,11 +29,21 @@ def test_static_scratch_block_matches_workspace_block_twice():
     dblk2 = g.binding.DeviceBlock(blk2, "cuda")
     dX2 = torch.from_numpy(X2).cuda()
     want2 = g.host(c.block_forward(dblk2, dX2))
+    oracle1, oracle2 = O.block_forward(blk, X), O.block_forward(blk2, X2)
+    Y, Y2 = torch.empty_like(dX), torch.empty_like(dX2)
+    c.block_forward_static(dblk, dX, Y)          # first call on the device: looks the array's address up
+    torch.cuda.synchronize()
     for call in range(2):
-        got = g.host(c.block_forward_static(dblk, dX))
+        free_before = torch.cuda.mem_get_info()[0]
+        got = g.host(c.block_forward_static(dblk, dX, Y))
+        got2 = g.host(c.block_forward_static(dblk2, dX2, Y2))
+        # the calls took no device memory (outputs were allocated beforehand)
+        assert torch.cuda.mem_get_info()[0] == free_before
         g.assert_equal(got, want, f"static scratch, call {call}")
-        got2 = g.host(c.block_forward_static(dblk2, dX2))
         g.assert_equal(got2, want2, f"static scratch, second block, call {call}")
+        # ... and against the oracle directly
+        g.assert_equal(got, oracle1, f"static scratch vs oracle, call {call}")
+        g.assert_equal(got2, oracle2, f"static scratch vs oracle, second block, call {call}")
     assert c.poll_status() == 0
 
 
