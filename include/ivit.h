@@ -113,6 +113,14 @@ uint64_t ivit_ctx_table_generation(const ivit_ctx* ctx);
  * qualifies (default), 1 = force the CUDA-core (dp4a) kernels everywhere.
  * Both are bit-exact; the switch exists for testing and measurement. */
 int ivit_ctx_set_gemm_engine(ivit_ctx* ctx, int engine);
+/* Row-operator fusion (off by default).  1: inside ivit_block_forward and the model forwards, LayerNorm 2, ShiftGELU
+ * (Algorithm 2 with its row maximum) and the LayerNorm 1 of the following block run inside the Dense kernel that
+ * produces their input rows, where the shapes allow it: the kernel's warps count the finished channel tiles of every
+ * block of rows and, after their last tile, run the operator on slices of the completed rows.  0: every operator
+ * is a kernel of its own.  Both give the same bytes.  On the measured workloads the separate kernels, whose launch
+ * overlaps the previous kernel's tail, are as fast or faster, which is why they are the default.  (2 / 4 switch on
+ * the LayerNorm / ShiftGELU part alone, for measurements.) */
+int ivit_ctx_set_row_fusion(ivit_ctx* ctx, int enable);
 const char* ivit_strerror(int code);
 
 /* ---- Sec. 3.2: Dense layer with dyadic requantisation ----
@@ -187,7 +195,8 @@ int ivit_shiftgelu_static(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_ex
 
 /* ---- Sec. 3.5: I-LayerNorm over each row ----
  *   mu = floor((2*sum x + C) / (2C)); y = x - mu; V = sum y^2;
- *   sd = integer sqrt of V by Eq. (iterative) (10 guarded iterations);
+ *   sd = integer sqrt of V: the value of Eq. (iterative) with 10 guarded iterations, floor(sqrt(V)) (int8 rows
+ *        of up to 1024 channels take it bit by bit without divisions, see ivit_isqrt_range);
  *   F = sd ? floor(2^M_ln / sd) : 0;
  *   out[c] = sat8( rq(y[c] * F; gamma_scale[c]) + beta[c] )
  * gamma_scale per-channel or per-tensor; beta int32 [C] or NULL.
@@ -297,6 +306,54 @@ size_t ivit_vit_host_workspace_bytes(const ivit_vit_params* p);
 int ivit_vit_forward_host(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* image_host,
                           int32_t* logits_host, void* workspace, size_t workspace_bytes);
 
+/* ---- Swin-shaped forward (window attention, patch merging, token pooling) ----
+ * The paper names Swin as a benchmark model without describing its outer layers; they are instances of the
+ * operators above.  Token rows are WINDOW-MAJOR everywhere (windows of one image in raster order, raster order
+ * inside a window), so that every window is a contiguous run of window^2 rows:
+ *   patches (window-major) -> Dense(Wpe) -> LayerNorm -> for every stage [ blocks -> (not after the last stage)
+ *   2x2 merge: gather_rows(merge_index) viewed as [rows / 4, 4C] -> LayerNorm -> Dense(Wmerge) ] ->
+ *   LayerNorm -> token mean (rq with pool_scale, sat8) -> Dense(Whead) -> int32 logits (not saturated).
+ * A block with shifted[i] != 0 is a shifted-window block: its input rows are permuted by shift_index before
+ * the block and its output rows by unshift_index after it (the cyclic roll as a row gather; the attention mask
+ * is part of the block's attn_bias).  Every block of stage s has B * (res / window)^2 windows of window^2
+ * tokens, D = C, and the heads / MLP width the caller chose. */
+typedef struct {
+  int64_t C, res, depth;                      /* channels, tokens per image side, blocks */
+  const ivit_block_params* blocks;            /* HOST array of depth entries */
+  const uint8_t* shifted;                     /* HOST array of depth flags, or NULL (no shifted block) */
+  const int32_t* shift_index;                 /* device int32 [B*res*res] or NULL */
+  const int32_t* unshift_index;               /* device int32 [B*res*res] or NULL */
+  const int32_t* merge_index;                 /* device int32 [B*res*res]; NULL after the last stage */
+  ivit_scale merge_ln_gamma; const int32_t* merge_ln_beta;   /* 4C channels */
+  const int8_t* Wmerge; ivit_scale merge_scale;              /* [2C, 4C], no bias */
+} ivit_swin_stage;
+
+typedef struct {
+  int64_t B, img, patch, window, classes, n_stages;
+  int32_t M_ln;
+  const int8_t* Wpe; const int32_t* bpe; ivit_scale pe_scale;   /* [C0, 3*patch*patch] */
+  ivit_scale pe_ln_gamma; const int32_t* pe_ln_beta;
+  const ivit_swin_stage* stages;                                /* HOST array of n_stages entries */
+  ivit_scale lnf_gamma; const int32_t* lnf_beta;
+  ivit_scale pool_scale;                                        /* per-tensor, 1 / tokens folded in */
+  const int8_t* Whead; const int32_t* bhead; ivit_scale head_scale;   /* [classes, C_last] */
+} ivit_swin_params;
+
+size_t ivit_swin_workspace_bytes(const ivit_swin_params* p);
+/* image [B,3,img,img] int8 (device) -> logits [B, classes] int32 (device, ld = classes).  tokens: NULL, or a
+ * device buffer [B * res_last^2, C_last] int8 that receives the output of the last block (what the final
+ * LayerNorm reads).  Nothing is allocated: every intermediate lives in the workspace (device, 256-byte aligned,
+ * at least ivit_swin_workspace_bytes(p)). */
+int ivit_swin_forward(ivit_ctx* ctx, const ivit_swin_params* p, const int8_t* image, int32_t* logits,
+                      int8_t* tokens, void* workspace, size_t workspace_bytes);
+/* The same with HOST buffers: image_host is copied to a staging area of the workspace on the context's stream,
+ * the forward runs, the logits are copied back to logits_host; the call only enqueues (synchronise the stream
+ * before reading logits_host; keep both host buffers valid until then; pinned memory makes the copies
+ * asynchronous).  workspace must hold ivit_swin_host_workspace_bytes(p). */
+size_t ivit_swin_host_workspace_bytes(const ivit_swin_params* p);
+int ivit_swin_forward_host(ivit_ctx* ctx, const ivit_swin_params* p, const int8_t* image_host,
+                           int32_t* logits_host, void* workspace, size_t workspace_bytes);
+
 /* Graph replay for ivit_vit_forward_host (off by default).  When enabled, the third call in a row that repeats
  * the same model description (every field of p and of its blocks), workspace and stream captures the device part
  * of the forward into a CUDA graph, and later calls launch that graph instead of about a hundred kernels; any
@@ -328,6 +385,12 @@ const char* ivit_kernel_kind_name(int32_t kind);
  * operations (2 per multiply-accumulate) of the timed launch; ops / ms is the rate the Dense kernels' TOP/s are
  * measured against.  1 <= iters <= 2^20. */
 int ivit_probe_int8_mma(ivit_ctx* ctx, int32_t iters, float* ms, double* ops);
+
+/* Verification aid for Sec. 3.5: out[i] = the integer square root that the I-LayerNorm kernels compute for the
+ * radicand n0 + i, i < count (device uint16 array; n0 + count <= 2^26, the largest sum of squared deviations of
+ * an int8 row of 1024 channels).  The kernels take the root bit by bit instead of running Eq. (iterative); a test
+ * compares this routine with the iteration over the whole range. */
+int ivit_isqrt_range(ivit_ctx* ctx, uint32_t n0, uint32_t count, uint16_t* out);
 
 /* ---- data movement helpers (not in the paper; needed by the full models) ---- */
 

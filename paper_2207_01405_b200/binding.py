@@ -19,7 +19,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libivit.so")
 
 EXPORTS = [
-    "ivit_ctx_create", "ivit_ctx_destroy", "ivit_probe_int8_mma", "ivit_ctx_table_generation", "ivit_vit_forward_tokens", "ivit_ctx_set_stream", "ivit_ctx_poll_status", "ivit_ctx_launch_count",
+    "ivit_ctx_create", "ivit_ctx_destroy", "ivit_swin_workspace_bytes", "ivit_swin_forward", "ivit_swin_host_workspace_bytes", "ivit_swin_forward_host", "ivit_isqrt_range", "ivit_ctx_set_row_fusion", "ivit_probe_int8_mma", "ivit_ctx_table_generation", "ivit_vit_forward_tokens", "ivit_ctx_set_stream", "ivit_ctx_poll_status", "ivit_ctx_launch_count",
     "ivit_ctx_set_gemm_engine", "ivit_strerror", "ivit_linear", "ivit_matmul", "ivit_shiftmax", "ivit_shiftgelu",
     "ivit_shiftgelu_static",
     "ivit_shiftmax_direct", "ivit_ctx_set_host_graph", "ivit_ctx_host_graph_count",
@@ -67,6 +67,28 @@ class CVit(C.Structure):
     ]
 
 
+class CSwinStage(C.Structure):
+    _fields_ = [
+        ("C", C.c_int64), ("res", C.c_int64), ("depth", C.c_int64),
+        ("blocks", C.POINTER(CBlock)), ("shifted", C.c_void_p),
+        ("shift_index", C.c_void_p), ("unshift_index", C.c_void_p), ("merge_index", C.c_void_p),
+        ("merge_ln_gamma", CScale), ("merge_ln_beta", C.c_void_p),
+        ("Wmerge", C.c_void_p), ("merge_scale", CScale),
+    ]
+
+
+class CSwin(C.Structure):
+    _fields_ = [
+        ("B", C.c_int64), ("img", C.c_int64), ("patch", C.c_int64), ("window", C.c_int64), ("classes", C.c_int64),
+        ("n_stages", C.c_int64), ("M_ln", C.c_int32),
+        ("Wpe", C.c_void_p), ("bpe", C.c_void_p), ("pe_scale", CScale),
+        ("pe_ln_gamma", CScale), ("pe_ln_beta", C.c_void_p),
+        ("stages", C.POINTER(CSwinStage)),
+        ("lnf_gamma", CScale), ("lnf_beta", C.c_void_p), ("pool_scale", CScale),
+        ("Whead", C.c_void_p), ("bhead", C.c_void_p), ("head_scale", CScale),
+    ]
+
+
 _lib = None
 
 
@@ -86,6 +108,7 @@ def load_library():
     L.ivit_ctx_launch_count.argtypes = [vp]
     L.ivit_ctx_launch_count.restype = i64
     L.ivit_ctx_set_gemm_engine.argtypes = [vp, C.c_int]
+    L.ivit_ctx_set_row_fusion.argtypes = [vp, C.c_int]
     L.ivit_ctx_table_generation.argtypes = [vp]
     L.ivit_ctx_table_generation.restype = C.c_uint64
     L.ivit_ctx_set_host_graph.argtypes = [vp, C.c_int]
@@ -109,6 +132,12 @@ def load_library():
     L.ivit_vit_workspace_bytes.restype = C.c_size_t
     L.ivit_vit_forward.argtypes = [vp, C.POINTER(CVit), vp, vp, vp, C.c_size_t]
     L.ivit_vit_forward_tokens.argtypes = [vp, C.POINTER(CVit), vp, vp, vp, vp, C.c_size_t]
+    L.ivit_swin_workspace_bytes.argtypes = [C.POINTER(CSwin)]
+    L.ivit_swin_workspace_bytes.restype = C.c_size_t
+    L.ivit_swin_host_workspace_bytes.argtypes = [C.POINTER(CSwin)]
+    L.ivit_swin_host_workspace_bytes.restype = C.c_size_t
+    L.ivit_swin_forward.argtypes = [vp, C.POINTER(CSwin), vp, vp, vp, vp, C.c_size_t]
+    L.ivit_swin_forward_host.argtypes = [vp, C.POINTER(CSwin), vp, vp, vp, C.c_size_t]
     L.ivit_vit_host_workspace_bytes.argtypes = [C.POINTER(CVit)]
     L.ivit_vit_host_workspace_bytes.restype = C.c_size_t
     L.ivit_vit_forward_host.argtypes = [vp, C.POINTER(CVit), vp, vp, vp, C.c_size_t]
@@ -116,6 +145,7 @@ def load_library():
     L.ivit_ctx_profile_stop.argtypes = [vp]
     L.ivit_ctx_profile_get.argtypes = [vp, i32, C.POINTER(i32), C.POINTER(C.c_float), C.POINTER(C.c_double)]
     L.ivit_probe_int8_mma.argtypes = [vp, i32, C.POINTER(C.c_float), C.POINTER(C.c_double)]
+    L.ivit_isqrt_range.argtypes = [vp, C.c_uint32, C.c_uint32, vp]
     L.ivit_kernel_kind_name.argtypes = [i32]
     L.ivit_kernel_kind_name.restype = C.c_char_p
     L.ivit_patchify.argtypes = [vp, vp, i64, i64, i64, i64, i64, i64, vp, i64]
@@ -216,6 +246,10 @@ class Context:
     def set_gemm_engine(self, engine: int):
         _chk(self.lib.ivit_ctx_set_gemm_engine(self.h, engine), "ivit_ctx_set_gemm_engine")
 
+    def set_row_fusion(self, enable: bool):
+        """ivit_ctx_set_row_fusion: LayerNorm / ShiftGELU in the tail of the producing Dense kernel (default) or alone."""
+        _chk(self.lib.ivit_ctx_set_row_fusion(self.h, 1 if enable else 0), "ivit_ctx_set_row_fusion")
+
     def set_host_graph(self, enable: bool):
         """Graph replay inside vit_forward_host (ivit_ctx_set_host_graph); off by default."""
         _chk(self.lib.ivit_ctx_set_host_graph(self.h, 1 if enable else 0), "ivit_ctx_set_host_graph")
@@ -234,6 +268,12 @@ class Context:
         ms, ops = C.c_float(), C.c_double()
         _chk(self.lib.ivit_probe_int8_mma(self.h, iters, C.byref(ms), C.byref(ops)), "ivit_probe_int8_mma")
         return ms.value, ops.value
+
+    def isqrt_range(self, n0: int, count: int) -> torch.Tensor:
+        """ivit_isqrt_range: the I-LayerNorm kernels' integer square root of n0 .. n0 + count - 1 (uint16 on device)."""
+        out = torch.empty(count, dtype=torch.uint16, device=self.device)
+        _chk(self.lib.ivit_isqrt_range(self.h, n0, count, out.data_ptr()), "ivit_isqrt_range")
+        return out
 
     def table_generation(self) -> int:
         return int(self.lib.ivit_ctx_table_generation(self.h))
@@ -491,55 +531,76 @@ class DeviceVit:
 
 
 class DeviceSwin:
-    """A Swin-shaped model (7x7 windows, optionally shifted in every second block) resident on the device."""
+    """A Swin-shaped model (7x7 windows, optionally shifted in every second block) resident on the device: the
+    ivit_swin_params description and everything it points at."""
 
     def __init__(self, p, device):
         self.p = p
         self.device = device
         self.up = _Uploader(device)
-        t = lambda a, dt: None if a is None else torch.from_numpy(np.ascontiguousarray(a, dtype=dt)).to(device)
-        self.Wpe, self.bpe, self.pe_scale = t(p.Wpe, np.int8), t(p.bpe, np.int32), DevScale(p.pe_scale, device)
-        self.pe_ln_gamma, self.pe_ln_beta = DevScale(p.pe_ln_gamma, device), t(p.pe_ln_beta, np.int32)
-        self.stages = []
-        for st in p.stages:
-            d = {"blocks": [DeviceBlock(b, device) for b in st.blocks], "C": st.C, "shifted": st.shifted}
+        up = self.up
+        self.block_arrays, self.flag_arrays = [], []
+        self.stages = (CSwinStage * len(p.stages))()
+        for i, st in enumerate(p.stages):
+            blocks = (CBlock * len(st.blocks))()
+            for j, b in enumerate(st.blocks):
+                _fill_block(blocks[j], b, up)
+            self.block_arrays.append(blocks)
+            cs = self.stages[i]
+            cs.C, cs.res, cs.depth = st.C, st.res, len(st.blocks)
+            cs.blocks = C.cast(blocks, C.POINTER(CBlock))
+            cs.shifted = None
             if st.shifted is not None:
-                d["shift_index"], d["unshift_index"] = t(st.shift_index, np.int32), t(st.unshift_index, np.int32)
+                flags = (C.c_uint8 * len(st.blocks))(*[1 if f else 0 for f in st.shifted])
+                self.flag_arrays.append(flags)
+                cs.shifted = C.cast(flags, C.c_void_p)
+                cs.shift_index, cs.unshift_index = up.t(st.shift_index, np.int32), up.t(st.unshift_index, np.int32)
             if st.merge_index is not None:
-                d["merge_index"] = t(st.merge_index, np.int32)
-                d["merge_ln_gamma"], d["merge_ln_beta"] = DevScale(st.merge_ln_gamma, device), t(st.merge_ln_beta, np.int32)
-                d["Wmerge"], d["merge_scale"] = t(st.Wmerge, np.int8), DevScale(st.merge_scale, device)
-            self.stages.append(d)
-        self.lnf_gamma, self.lnf_beta = DevScale(p.lnf_gamma, device), t(p.lnf_beta, np.int32)
-        self.pool_scale = DevScale(p.pool_scale, device)
-        self.Whead, self.bhead, self.head_scale = t(p.Whead, np.int8), t(p.bhead, np.int32), DevScale(p.head_scale, device)
-        self.ws = torch.empty(max(b.workspace_bytes() for s in self.stages for b in s["blocks"]), dtype=torch.uint8,
-                              device=device)
+                cs.merge_index = up.t(st.merge_index, np.int32)
+                cs.merge_ln_gamma, cs.merge_ln_beta = up.s(st.merge_ln_gamma), up.t(st.merge_ln_beta, np.int32)
+                cs.Wmerge, cs.merge_scale = up.t(st.Wmerge, np.int8), up.s(st.merge_scale)
+        c = CSwin()
+        c.B, c.img, c.patch, c.window, c.classes, c.n_stages, c.M_ln = p.B, p.img, p.patch, p.window, p.classes, len(p.stages), p.M_ln
+        c.Wpe, c.bpe, c.pe_scale = up.t(p.Wpe, np.int8), up.t(p.bpe, np.int32), up.s(p.pe_scale)
+        c.pe_ln_gamma, c.pe_ln_beta = up.s(p.pe_ln_gamma), up.t(p.pe_ln_beta, np.int32)
+        c.stages = C.cast(self.stages, C.POINTER(CSwinStage))
+        c.lnf_gamma, c.lnf_beta, c.pool_scale = up.s(p.lnf_gamma), up.t(p.lnf_beta, np.int32), up.s(p.pool_scale)
+        c.Whead, c.bhead, c.head_scale = up.t(p.Whead, np.int8), up.t(p.bhead, np.int32), up.s(p.head_scale)
+        self.c = c
+        self.tokens_shape = (p.B * p.stages[-1].res ** 2, p.stages[-1].C)
+        self._ws = None
+
+    def workspace_bytes(self) -> int:
+        n = load_library().ivit_swin_workspace_bytes(C.byref(self.c))
+        if n == 0:
+            raise ValueError("ivit_swin_workspace_bytes rejected the model parameters")
+        return int(n)
+
+    def workspace(self) -> torch.Tensor:
+        if self._ws is None:
+            self._ws = torch.empty(self.workspace_bytes(), dtype=torch.uint8, device=self.device)
+        return self._ws
+
+    def host_workspace(self) -> torch.Tensor:
+        n = load_library().ivit_swin_host_workspace_bytes(C.byref(self.c))
+        if n == 0:
+            raise ValueError("ivit_swin_host_workspace_bytes rejected the model parameters")
+        return torch.empty(int(n), dtype=torch.uint8, device=self.device)
 
 
-def swin_forward(ctx: Context, m: DeviceSwin, image: torch.Tensor, return_tokens: bool = False):
-    """Swin-shaped forward composed from the library's entry points (every step is a library kernel):
-    patchify (window-major) -> Dense -> LN -> [blocks -> 2x2 gather -> LN -> Dense] x stages -> LN -> token
-    mean -> Dense head (int32 logits)."""
-    p = m.p
-    X = ctx.linear(ctx.patchify(image, p.patch, window=p.window), m.Wpe, m.bpe, m.pe_scale)
-    X = ctx.layernorm(X, m.pe_ln_gamma, m.pe_ln_beta, p.M_ln)
-    for st in m.stages:
-        for i, blk in enumerate(st["blocks"]):
-            if st["shifted"] is not None and st["shifted"][i]:
-                # shifted-window block: rows into the rolled window order, block, rows back
-                X = ctx.block_forward(blk, ctx.gather_rows(X, st["shift_index"]), workspace=m.ws)
-                X = ctx.gather_rows(X, st["unshift_index"])
-            else:
-                X = ctx.block_forward(blk, X, workspace=m.ws)
-        if "merge_index" in st:
-            C_ = st["C"]
-            G = ctx.gather_rows(X, st["merge_index"], width=C_).view(-1, 4 * C_)
-            G = ctx.layernorm(G, st["merge_ln_gamma"], st["merge_ln_beta"], p.M_ln)
-            X = ctx.linear(G, st["Wmerge"], None, st["merge_scale"])
-    last = X
-    X = ctx.layernorm(X, m.lnf_gamma, m.lnf_beta, p.M_ln)
-    tokens = X.shape[0] // image.shape[0]
-    Z = ctx.token_mean(X, tokens, m.pool_scale)
-    logits = ctx.linear(Z, m.Whead, m.bhead, m.head_scale, out_dtype=I32)
-    return (logits, last) if return_tokens else logits
+def swin_forward(ctx: Context, m: DeviceSwin, image: torch.Tensor, return_tokens: bool = False, logits=None, workspace=None):
+    """ivit_swin_forward: image [B,3,img,img] int8 on the device -> int32 logits [B, classes]; with return_tokens
+    also the output of the last block ([B * tokens, C] int8, window-major rows)."""
+    if logits is None:
+        logits = torch.empty((m.c.B, m.c.classes), dtype=torch.int32, device=image.device)
+    tokens = torch.empty(m.tokens_shape, dtype=torch.int8, device=image.device) if return_tokens else None
+    ws = workspace if workspace is not None else m.workspace()
+    _chk(ctx.lib.ivit_swin_forward(ctx.h, C.byref(m.c), image.data_ptr(), logits.data_ptr(), _ptr(tokens), ws.data_ptr(),
+                                   ws.numel()), "ivit_swin_forward")
+    return (logits, tokens) if return_tokens else logits
+
+
+def swin_forward_host(ctx: Context, m: DeviceSwin, image_host: torch.Tensor, logits_host: torch.Tensor, workspace):
+    """ivit_swin_forward_host: host image -> host logits, copies enqueued on the context's stream."""
+    _chk(ctx.lib.ivit_swin_forward_host(ctx.h, C.byref(m.c), image_host.data_ptr(), logits_host.data_ptr(),
+                                        workspace.data_ptr(), workspace.numel()), "ivit_swin_forward_host")

@@ -12,6 +12,11 @@ constexpr int kProfMax = 8192;
 enum KernelKind { KIND_GEMM_TC = 0, KIND_GEMM_SIMT, KIND_LAYERNORM, KIND_SHIFTMAX, KIND_SHIFTGELU, KIND_GELU_TABLE,
                   KIND_ATTENTION, KIND_MOVE, KIND_COUNT };
 constexpr int kGeluTableSlots = 16;
+constexpr int kRowCounters = 4096;     // row blocks a Dense launch with a row operator may have
+constexpr int kRowStateStride = 32;    // words between the counters (and between the flags) of neighbouring row blocks: one 128-byte line each
+constexpr size_t kRowStateBytes = 4 * (32 + 2 * (size_t)kRowCounters * kRowStateStride);
+constexpr int kGeluTailRows = 2;      // rows a warp of the Dense kernel works on together in the ShiftGELU tail
+constexpr int kGeluTailSmem = 16 * kGeluTailRows * 256;
 constexpr int kGeluTableBytes = 128 * 256;  // [max(0,row max of x)] [x + 128] -> int8 output
 
 struct GeluKey {
@@ -30,6 +35,9 @@ struct ivit_ctx {
   int* status_dev;   // device view of the same word
   int8_t* gelu_tables;  // kGeluTableSlots tables on the device
   unsigned* sched_dev;  // two pairs of work counters of the attention kernel (behind the tables), used alternately
+  unsigned* rowblk_dev; // row-operator state of the Dense kernels: kRowStateBytes (zero between launches)
+  int row_fusion;       // non-zero (bit 0 LayerNorm, bit 1 ShiftGELU; default 0): LayerNorm / ShiftGELU run in the tail of the Dense kernel that produces their rows
+  int rowop_fused;      // set by the Dense launcher when the kernel it launched runs the requested row operator
   int attn_gen;         // pair of the next launch
   ivit::GeluKey gelu_keys[ivit::kGeluTableSlots];
   int gelu_used;
@@ -163,6 +171,23 @@ inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
 
 // launchers implemented in the kernel files ---------------------------------------------
 
+// What a Dense launch does with a block of output rows once all its channel tiles are stored (see rowops.cuh).
+struct RowOpArgs {
+  int kind;              // 0: nothing; 1: I-LayerNorm of the rows into ln_out; 2: ShiftGELU of the rows, in place
+  unsigned* counters;    // [2] CTAs finished; from word 32 on one arrival counter per row block, then one ready flag per
+                         // row block, each on a 128-byte line of its own; all zero between launches
+  // kind 1
+  ScaleDev gs;           // per-channel (or per-tensor) multiplier and shift of the affine requantisation
+  const int32_t* beta;
+  int M_ln;
+  int8_t* ln_out;
+  int64_t ld_ln;
+  unsigned mean_magic;   // floor(2^32 / 2C) + 1
+  int vec;               // per-channel arrays aligned for 16-byte loads
+  // kind 2
+  const int8_t* table;   // 128 x 256 bytes: [max(0, row maximum)][x + 128]
+};
+
 struct GemmEpilogue {
   const int32_t* bias;       // [N] (linear) or nullptr
   const int32_t* bias32;     // [bias_batches, Ma, ldbias] (matmul) or nullptr
@@ -176,6 +201,8 @@ struct GemmEpilogue {
   int out_dtype;
   int64_t group_rows, group_stride;
   const int8_t* act_table;   // int8 outputs only: out = act_table[sat8(value) + 128] (256 entries on the device) or nullptr
+  RowOpArgs rop;             // row operator wanted on the finished output rows (kind 0: none); the launcher sets
+                             // ctx->rowop_fused when the kernel it launched runs it, else the caller launches it
 };
 
 struct GemmProblem {
@@ -205,6 +232,8 @@ int launch_shiftmax(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, c
                     int64_t ldout, int64_t rows, int64_t d);
 int launch_shiftmax_direct(ivit_ctx* ctx, const int32_t* in, int64_t ldin, ivit_exp_params p, int8_t* out,
                            int64_t ldout, int64_t rows, int64_t d);
+// The 128 x 256 ShiftGELU table of (p, post) on the device (built on first use, cached in the context).
+int gelu_table_for(ivit_ctx* ctx, ivit_exp_params p, ivit_scale post, const int8_t** table);
 // Row `127` of the ShiftGELU table of (p, post) on the device (built on first use): the static-maximum variant.
 int gelu_static_row(ivit_ctx* ctx, ivit_exp_params p, ivit_scale post, const int8_t** row);
 int launch_shiftgelu_static(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_exp_params p, ivit_scale post,

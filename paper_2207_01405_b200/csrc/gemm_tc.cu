@@ -27,6 +27,7 @@
 // context's status word, carries on without further waits, drains its outstanding copies, and the
 // CTA frees its tensor memory and returns.
 #include "tc_ptx.cuh"
+#include "rowops.cuh"
 
 namespace ivit {
 
@@ -75,10 +76,7 @@ constexpr int BM = 128;          // TMEM lanes of a tile (UMMA M, cta_group::1)
 constexpr int BK = 128;          // bytes (= int8 elements) of K per pipeline stage
 constexpr int UMMA_K = 32;       // K of one tcgen05.mma.kind::i8
 constexpr int kMaxStages = 8;
-#ifndef IVIT_EPI_WARPS
-#define IVIT_EPI_WARPS 16
-#endif
-constexpr int kEpiWarps = IVIT_EPI_WARPS;
+constexpr int kEpiWarps = 16;
 constexpr int kEpiThreads = 32 * kEpiWarps;
 constexpr int kFirstEpiWarp = 2;   // warp 0: TMA loads, warp 1: MMA
 constexpr int kThreads = 32 * kFirstEpiWarp + kEpiThreads;
@@ -102,6 +100,7 @@ struct TcArgs {
   int tma_res;       // ... and the residual tile of the same shape is fetched by TMA into shared memory
   int q_resident;    // Dense orientation, short K: all k-blocks of the Q (activation row) tile stay in shared
                      // memory while the CTA walks the channel blocks; only weight tiles stream through the ring
+  RowOpArgs rop;     // row operator on finished blocks of output rows (Dense orientation, staged int8 output)
   int* status;
 };
 
@@ -152,7 +151,15 @@ struct TileIter {
 // orientation, output type and residual port), 1 = Dense orientation, int8 output staged for TMA stores, no
 // residual, 2 = the same with the residual tile fetched by TMA, 3 = as 1 with an activation table applied to the
 // saturated value (the element-wise ShiftGELU variant inside FC1).
-template <int MODE>
+// ROP != 0 (MODE 1 or 2 only): a row operator on the output, run by this same kernel: 1 = I-LayerNorm into a second
+// tensor (the input of the next Dense layer), 2 = ShiftGELU in place (Algorithm 2 with its row maximum).  Both need
+// whole output rows, i.e. every channel tile of a block of rows, and those tiles may belong to several CTAs.  So
+// every epilogue warp, once its stores of a row block are complete, adds its tiles to the block's arrival counter;
+// the warp that completes the count raises the block's ready flag.  The rows are cut into slices (one batch of the
+// row routine each) that are dealt to all epilogue warps of the grid in a fixed order; a warp works on its slices
+// after its CTA's last tile, straight out of L2, waiting (bounded) only for the ready flag of the slice's block.
+// The last CTA to finish leaves counters and flags at zero for the next launch.
+template <int MODE, int ROP>
 __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmP,
                                                               const __grid_constant__ CUtensorMap tmQ,
                                                               const __grid_constant__ CUtensorMap tmO,
@@ -175,6 +182,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
   // residual port: the requantised value of every int8 residual byte (256 entries, built below), followed by the
   // 256 entries of the optional activation table
   int8_t* res_tab = reinterpret_cast<int8_t*>(tmem_slot) + 32;
+  volatile uint32_t* rop_flag = tmem_slot + 2;                                // row operator: a flag the CTA agrees on
+  uint8_t* rop_smem = gen_base + bars_off + 1024;   // ROP == 1: LayerNorm constants; ROP == 2: table rows, per warp
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // this CTA's contiguous range of tiles
@@ -196,6 +205,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     } else if (i == 2 * kMaxStages + 4 + 2 * kEpiWarps) {
       mbar_init(qrese, 1);
       *issued_slot = 0;
+      *rop_flag = 1u;
     } else if (i == 2 * kMaxStages + 5 + 2 * kEpiWarps) {
       prefetch_tmap(&tmP);
     } else if (i == 2 * kMaxStages + 6 + 2 * kEpiWarps) {
@@ -219,7 +229,18 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
   // set-up done (barriers, tensor memory, descriptor prefetch): let the next kernel be scheduled, then wait
   // for the previous kernel's results before touching global memory
   pdl_trigger();
-  pdl_wait();
+  if (ROP == 1 && warp >= kFirstEpiWarp) {
+    // I-LayerNorm constants of all channels into shared memory: parameters, read before the wait for the previous
+    // kernel.  The form (fast / general, see LnConsts) is agreed on by all epilogue threads.
+    const int et0 = (int)threadIdx.x - 32 * kFirstEpiWarp, nwords = (int)(a.P >> 2);
+    int4* sm_m = reinterpret_cast<int4*>(rop_smem);
+    if (!ln_stage_consts(a.rop.gs, a.rop.beta, nwords, a.rop.vec, sm_m, sm_m + nwords, sm_m + 2 * nwords, et0, kEpiThreads))
+      atomicAnd(const_cast<uint32_t*>(rop_flag), 0u);
+    asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
+    if (*rop_flag) ln_fold_consts(nwords, sm_m + nwords, sm_m + 2 * nwords, et0, kEpiThreads);
+    asm volatile("bar.sync 2, %0;" ::"n"(kEpiThreads) : "memory");
+  }
+  if (warp != 0) pdl_wait();
 
   if (warp == 0) {
     // ---------------- TMA producer ----------------
@@ -232,6 +253,19 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       ti.init(a, t_begin);
       // which tensor-map coordinate (1..3) carries the row / inner batch / outer batch index
       const int pr = a.p_pos[0], pbi = a.p_pos[1], qr = a.q_pos[0], qbi = a.q_pos[1];
+      // Dense orientation: the P operand is the weight matrix, which no kernel writes.  The weight k-blocks of the
+      // first tile are requested before the wait for the previous kernel (whose last CTAs may still be running
+      // elsewhere); the activation k-blocks that complete the same stage barriers follow after the wait.
+      int pre = 0;
+      if (a.lanes_are_channels && t_begin < t_end) {
+        pre = kblocks < a.stages ? kblocks : a.stages;
+        for (int kb = 0; kb < pre; ++kb) {
+          mbar_expect_tx(full0 + 8 * kb, BM * BK + a.q_stage_bytes);
+          tma_load_4d(base + kb * stage_bytes, &tmP, full0 + 8 * kb, kb * BK, pr == 1 ? ti.p0() : 0, pr == 2 ? ti.p0() : 0,
+                      pr == 3 ? ti.p0() : 0);
+        }
+      }
+      pdl_wait();
       for (int64_t t = t_begin; ok && t < t_end; ++t, ++pit, ti.next(a)) {
         const int p0 = ti.p0(), q0 = ti.q0(a);
         const int pc1 = pr == 1 ? p0 : (pbi == 1 ? ti.bi : ti.bo), pc2 = pr == 2 ? p0 : (pbi == 2 ? ti.bi : ti.bo),
@@ -248,11 +282,12 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         for (int kb = 0; kb < kblocks; ++kb) {
           if (wrap > 0 && !mbar_wait(empty0 + 8 * s, (wrap & 1) ^ 1, a.status)) { ok = false; break; }
           const uint32_t sp = base + s * stage_bytes, sq = sp + BM * BK;
-          mbar_expect_tx(full0 + 8 * s, stage_bytes + (bring_q ? a.q_stage_bytes : 0));
+          const bool early = t == t_begin && kb < pre;   // barrier armed and weights requested before the wait
+          if (!early) mbar_expect_tx(full0 + 8 * s, stage_bytes + (bring_q ? a.q_stage_bytes : 0));
           if (bring_q)
             tma_load_4d(qres + kb * a.q_stage_bytes, &tmQ, full0 + 8 * s, kb * BK, qr == 1 ? q0 : 0, qr == 2 ? q0 : 0,
                         qr == 3 ? q0 : 0);
-          tma_load_4d(sp, &tmP, full0 + 8 * s, kb * BK, pc1, pc2, pc3);
+          if (!early) tma_load_4d(sp, &tmP, full0 + 8 * s, kb * BK, pc1, pc2, pc3);
           if (!a.q_resident) {
             const int qrow = a.q_mn ? kb * BK : q0;     // MN-major: rows of the map are k, the inner index is n
             const int qc0 = a.q_mn ? q0 : kb * BK;
@@ -414,6 +449,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     }
 
     int it = 0;
+    int tiles_in_q = 0;   // ROP: tiles of the current block of output rows that this CTA has finished
     TileIter ti;
     ti.init(a, t_begin);
     for (int64_t t = t_begin; t < t_end; ++t, ++it) {
@@ -612,6 +648,91 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(acce0 + 8 * buf);
+      if (ROP) {
+        ++tiles_in_q;
+        if (t + 1 >= t_end || ti.q0(a) != tc.q0) {
+          // this warp's last tile of the row block: see the stores complete, release them, count the tiles
+          if (lane == 0) {
+            unsigned* q_state = a.rop.counters;
+            const unsigned qblk = (unsigned)tc.q0 / (unsigned)a.BN;
+            tma_store_wait_all();
+            asm volatile("fence.proxy.async;" ::: "memory");
+            __threadfence();
+            unsigned* cnt = q_state + 32 + qblk * kRowStateStride;
+            const unsigned old = atomicAdd(cnt, (unsigned)tiles_in_q);
+            if (old + (unsigned)tiles_in_q == (unsigned)(a.tiles_p * kEpiWarps)) {
+              *cnt = 0u;
+              __threadfence();
+              asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(cnt + kRowCounters * kRowStateStride), "r"(1u) : "memory");
+            }
+          }
+          tiles_in_q = 0;
+        }
+      }
+    }
+    if (ROP && ok) {
+      // ---- row operator on this warp's slices ----
+      unsigned* q_state = a.rop.counters;
+      constexpr int kSlice = ROP == 1 ? 8 : 2;                       // rows of a slice: one batch of the row routine
+      const unsigned spb = (unsigned)(a.BN + kSlice - 1) / kSlice;   // slices per row block
+      const unsigned total = (unsigned)a.tiles_q * spb;
+      const unsigned nwarps = gridDim.x * kEpiWarps;
+      const int C = (int)a.P;
+      const int nwords = C >> 2;
+      const int4* sm_m = reinterpret_cast<const int4*>(rop_smem);
+      const LnConsts lk{sm_m, sm_m + nwords, sm_m + 2 * nwords, *rop_flag != 0u};
+      unsigned* tab = reinterpret_cast<unsigned*>(rop_smem) + ew * (kGeluTailRows * 64);
+      for (unsigned sl = (unsigned)ew * gridDim.x + blockIdx.x; sl < total; sl += nwarps) {
+        const unsigned blk = sl / spb, j = sl - blk * spb;
+        const int64_t q0 = (int64_t)blk * a.BN;
+        const int64_t left = a.Q - q0;
+        const int in_blk = (int)(left < a.BN ? left : a.BN);
+        const int r0 = (int)j * kSlice;
+        if (r0 >= in_blk) continue;
+        unsigned rdy = 0;
+        if (lane == 0) {
+          // polls back off: thousands of warps may wait for a handful of flags
+          const unsigned* flag = q_state + 32 + (kRowCounters + blk) * kRowStateStride;
+          unsigned pause = 64;
+          for (uint32_t spin = 0; spin < kSpinLimit; ++spin) {
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(rdy) : "l"(flag) : "memory");
+            if (rdy) break;
+            __nanosleep(pause);
+            if (pause < 2048) pause <<= 1;
+          }
+          if (!rdy) {
+            *reinterpret_cast<volatile int*>(a.status) = IVIT_ERR_DEVICE_TIMEOUT;
+            __threadfence_system();
+          }
+        }
+        rdy = __shfl_sync(0xffffffffu, rdy, 0);
+        if (!rdy) break;
+        const int nrows = in_blk - r0 < kSlice ? in_blk - r0 : kSlice;
+        int8_t* rows0 = reinterpret_cast<int8_t*>(e.out) + (q0 + r0) * e.ldo;
+        if (ROP == 1) {
+          int8_t* dst = a.rop.ln_out + (q0 + r0) * a.rop.ld_ln;
+          if (C <= 384) {
+            layernorm_rows<3, 8, true>(rows0, e.ldo, nrows, C, a.rop.M_ln, a.rop.mean_magic, lk, dst, a.rop.ld_ln, lane);
+          } else if (C <= 512) {
+            layernorm_rows<4, 8, true>(rows0, e.ldo, nrows, C, a.rop.M_ln, a.rop.mean_magic, lk, dst, a.rop.ld_ln, lane);
+          } else {
+            for (int h = 0; h < nrows; h += 4)
+              layernorm_rows<8, 4, true>(rows0 + (int64_t)h * e.ldo, e.ldo, nrows - h < 4 ? nrows - h : 4, C, a.rop.M_ln,
+                                         a.rop.mean_magic, lk, dst + (int64_t)h * a.rop.ld_ln, a.rop.ld_ln, lane);
+          }
+        } else {
+          if (C <= 1536) {
+            shiftgelu_rows<3, 2, true>(rows0, e.ldo, nrows, C, a.rop.table, tab, rows0, e.ldo, lane);
+          } else {
+            for (int h = 0; h < nrows; ++h) {
+              shiftgelu_rows<8, 1, true>(rows0 + (int64_t)h * e.ldo, e.ldo, 1, C, a.rop.table, tab, rows0 + (int64_t)h * e.ldo,
+                                         e.ldo, lane);
+              __syncwarp();
+            }
+          }
+          __syncwarp();
+        }
+      }
     }
     if (tma_out && lane == 0) tma_store_wait_all();
     // only after a timeout: residual bytes fetched for chunks that were never worked on may be in flight
@@ -625,6 +746,20 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     tc_fence_after();
     tmem_dealloc(tmem_base, (uint32_t)a.tmem_cols);
   }
+  if (ROP) {
+    // the last CTA to get here finds every other CTA out of the queue: it leaves the queue state at zero
+    unsigned* q_state = a.rop.counters;
+    if (threadIdx.x == 0) {
+      __threadfence();
+      *rop_flag = atomicAdd(q_state + 2, 1u) == gridDim.x - 1 ? 1u : 0u;
+    }
+    __syncthreads();
+    if (*rop_flag) {
+      for (int i = threadIdx.x; i < a.tiles_q; i += kThreads) q_state[32 + (kRowCounters + i) * kRowStateStride] = 0u;
+      if (threadIdx.x == 0) q_state[2] = 0u;
+      __threadfence();
+    }
+  }
 }
 
 // ---- host side ------------------------------------------------------------------------------
@@ -636,7 +771,11 @@ int pow2_at_least(int v) {
 }
 
 constexpr size_t kSmemBudget = 227 * 1024;
-constexpr size_t kSmemFixed = 1024 + 8 * (2 * kMaxStages + 5 + 2 * kEpiWarps) + 32 + 512;
+// alignment slack + one KB of barriers, tensor-memory slot, flags and the two 256-entry tables of the residual /
+// activation port; a row operator's shared memory follows it
+constexpr size_t kSmemFixed = 1024 + 1024;
+static_assert(8 * (2 * kMaxStages + 5 + 2 * kEpiWarps) + 32 + 512 <= 1024, "barrier block");
+
 
 // Tile width along the TMEM columns: the candidate with the least (rounds of tiles per CTA) x (time of a tile).
 // A tile's time is the larger of its operand traffic, (128 + bn) x K bytes at about 46 bytes per clock into an
@@ -661,10 +800,13 @@ int pick_bn(int64_t extent, int64_t tiles_other, int64_t K, int sm_count) {
 
 // The shared-memory limit of a kernel is a per-device attribute: set for the current device at context creation.
 int gemm_tc_prepare_device() {
-  if (cudaFuncSetAttribute(gemm_tc_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
-      cudaFuncSetAttribute(gemm_tc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
-      cudaFuncSetAttribute(gemm_tc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
-      cudaFuncSetAttribute(gemm_tc_kernel<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess)
+  if (cudaFuncSetAttribute(gemm_tc_kernel<0, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
+      cudaFuncSetAttribute(gemm_tc_kernel<1, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
+      cudaFuncSetAttribute(gemm_tc_kernel<2, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
+      cudaFuncSetAttribute(gemm_tc_kernel<3, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
+      cudaFuncSetAttribute(gemm_tc_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
+      cudaFuncSetAttribute(gemm_tc_kernel<2, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
+      cudaFuncSetAttribute(gemm_tc_kernel<1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess)
     return IVIT_ERR_CUDA;
   return IVIT_OK;
 }
@@ -735,30 +877,49 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
     a.tma_res = make_tensor_map(ctx, &tmR, e.res, g.N, g.M, 1, 1, e.ldres, 0, 0, 32, 32, CU_TENSOR_MAP_SWIZZLE_NONE,
                                 rpos) ? 1 : 0;
   }
+  // The row operator runs in this kernel when the epilogue is one of the specialised forms (staged int8 output,
+  // residual absent or fetched by TMA), the rows fit the tail routines and there is a counter per row block.
+  int rop = 0;
+  if (e.rop.kind && a.lanes_are_channels && a.tma_out && (!e.res || a.tma_res) && !e.act_table && ctx->row_fusion) {
+    const int64_t blocks_q = (a.Q + a.BN - 1) / a.BN;
+    if (blocks_q <= kRowCounters && e.rop.kind == 1 && g.N <= 1024 && (ctx->row_fusion & 1)) rop = 1;
+    if (blocks_q <= kRowCounters && e.rop.kind == 2 && g.N % 16 == 0 && g.N <= 4096 && !e.res && (ctx->row_fusion & 2)) rop = 2;
+  }
+  a.rop = e.rop;
+  a.rop.kind = rop;
+  a.rop.counters = ctx->rowblk_dev;
+  a.rop.mean_magic = (unsigned)(0x100000000ull / (unsigned long long)(2 * g.N)) + 1u;
+  a.rop.vec = e.rop.gs.mult_c && e.rop.gs.shift_c && !(reinterpret_cast<uintptr_t>(e.rop.gs.mult_c) & 15) &&
+              !(reinterpret_cast<uintptr_t>(e.rop.gs.shift_c) & 3) && !(reinterpret_cast<uintptr_t>(e.rop.beta) & 15);
+  const size_t rop_bytes = rop == 1 ? ((size_t)g.N * 12 + 1023) / 1024 * 1024 : (rop == 2 ? (size_t)kGeluTailSmem : 0);
   const size_t out_stage = (a.tma_out ? (size_t)kEpiWarps * 2048 : 0) + (a.tma_res ? (size_t)kEpiWarps * 2048 : 0);
   // short K: keep the activation tile resident if that still leaves four weight stages
   const size_t kblocks = (size_t)((g.K + BK - 1) / BK);
   const size_t qres_bytes = kblocks * a.q_stage_bytes;
-  a.q_resident = (dense && kSmemFixed + out_stage + qres_bytes + 4 * (size_t)BM * BK <= kSmemBudget) ? 1 : 0;
+  a.q_resident = (dense && kSmemFixed + rop_bytes + out_stage + qres_bytes + 4 * (size_t)BM * BK <= kSmemBudget) ? 1 : 0;
   const size_t stage = (size_t)BM * BK + (a.q_resident ? 0 : a.q_stage_bytes);
   const size_t fixed = out_stage + (a.q_resident ? qres_bytes : 0);
-  int stages = (int)((kSmemBudget - kSmemFixed - fixed) / stage);
+  int stages = (int)((kSmemBudget - kSmemFixed - rop_bytes - fixed) / stage);
   a.stages = stages > kMaxStages ? kMaxStages : stages;
   if (a.stages < 2) return IVIT_ERR_UNSUPPORTED;
   a.tmem_cols = pow2_at_least(2 * a.BN);
   a.tiles_q = (int)((a.Q + a.BN - 1) / a.BN);
   a.total_tiles = (int64_t)a.tiles_p * a.tiles_q * batches;
 
-  const size_t smem = kSmemFixed + (size_t)a.stages * stage + fixed;
+  const size_t smem = kSmemFixed + rop_bytes + (size_t)a.stages * stage + fixed;
   const unsigned grid = (unsigned)(a.total_tiles < ctx->sm_count ? a.total_tiles : ctx->sm_count);
   LaunchScope ls(ctx, KIND_GEMM_TC, 2.0 * (double)batches * (double)g.M * (double)g.N * (double)g.K);
   // the encoder block's Dense layers take the specialised instantiations
   int mode = (a.lanes_are_channels && a.tma_out && (!e.res || a.tma_res)) ? (a.tma_res ? 2 : 1) : 0;
   if (e.act_table) mode = mode == 1 ? 3 : 0;
-  if (mode == 3) launch_k(gemm_tc_kernel<3>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
-  else if (mode == 2) launch_k(gemm_tc_kernel<2>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
-  else if (mode == 1) launch_k(gemm_tc_kernel<1>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
-  else launch_k(gemm_tc_kernel<0>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
+  if (rop == 1 && mode == 2) launch_k(gemm_tc_kernel<2, 1>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
+  else if (rop == 1 && mode == 1) launch_k(gemm_tc_kernel<1, 1>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
+  else if (rop == 2 && mode == 1) launch_k(gemm_tc_kernel<1, 2>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
+  else if (mode == 3) launch_k(gemm_tc_kernel<3, 0>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
+  else if (mode == 2) launch_k(gemm_tc_kernel<2, 0>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
+  else if (mode == 1) launch_k(gemm_tc_kernel<1, 0>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
+  else launch_k(gemm_tc_kernel<0, 0>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
+  ctx->rowop_fused = (rop != 0 && (mode == 1 || mode == 2)) ? 1 : 0;
   return ls.done();
 }
 

@@ -118,7 +118,22 @@ int attention_impl(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* QKV,
   return launch_gemm(ctx, pv);
 }
 
-int block_impl(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* X, int8_t* Y, char* ws) {
+// Asks the Dense launch `g` to run I-LayerNorm (gamma, beta) on its finished output rows, writing `out` (ld = C).
+void want_layernorm(GemmProblem& g, const ivit_scale& gamma, const int32_t* beta, int M_ln, int8_t* out, int64_t ld) {
+  g.epi.rop.kind = 1;
+  g.epi.rop.gs = to_dev(gamma);
+  g.epi.rop.beta = beta;
+  g.epi.rop.M_ln = M_ln;
+  g.epi.rop.ln_out = out;
+  g.epi.rop.ld_ln = ld;
+}
+
+// One encoder block.  a_ready: LayerNorm 1 of X already sits in the workspace (the previous block's last Dense
+// layer produced it); next: the block that follows on Y with the same shape, or nullptr - its LayerNorm 1 is then
+// run in the tail of this block's last Dense layer, where that is possible.  *a_next_ready tells the caller whether
+// it was.  Row operators that a Dense kernel cannot take on run as kernels of their own, with the same result.
+int block_impl(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* X, int8_t* Y, char* ws, bool a_ready = false,
+               const ivit_block_params* next = nullptr, bool* a_next_ready = nullptr) {
   const BlockWs w = block_ws(p);
   const int64_t M = p->B * p->T, D = p->D, H = p->H;
   int8_t* A = reinterpret_cast<int8_t*>(ws + w.A);
@@ -128,26 +143,42 @@ int block_impl(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* X, int8_
   int8_t* G = reinterpret_cast<int8_t*>(ws + w.G);
   const ivit_scale none{nullptr, nullptr, 1, 1};
   int rc;
+  if (a_next_ready) *a_next_ready = false;
   // X^ = MSA(LayerNorm(X)) + X
-  if ((rc = launch_layernorm(ctx, X, IVIT_I8, D, to_dev(p->ln1_gamma), p->ln1_beta, p->M_ln, A, D, M, D))) return rc;
+  if (!a_ready && (rc = launch_layernorm(ctx, X, IVIT_I8, D, to_dev(p->ln1_gamma), p->ln1_beta, p->M_ln, A, D, M, D))) return rc;
   if ((rc = launch_gemm(ctx, linear_problem(A, D, p->Wqkv, D, p->bqkv, p->qkv_scale, nullptr, 0, 1, none, QKV, 3 * D,
                                             IVIT_I8, 0, 0, M, 3 * D, D)))) return rc;
   if ((rc = attention_impl(ctx, p, QKV, O, ws, w))) return rc;
-  if ((rc = launch_gemm(ctx, linear_problem(O, D, p->Wo, D, p->bo, p->o_scale, X, D, M, p->res1_scale, Xh, D,
-                                            IVIT_I8, 0, 0, M, D, D)))) return rc;
+  // output projection + residual; LayerNorm 2 of its rows in the kernel's tail
+  GemmProblem proj = linear_problem(O, D, p->Wo, D, p->bo, p->o_scale, X, D, M, p->res1_scale, Xh, D, IVIT_I8, 0, 0, M, D, D);
+  want_layernorm(proj, p->ln2_gamma, p->ln2_beta, p->M_ln, A, D);
+  ctx->rowop_fused = 0;
+  if ((rc = launch_gemm(ctx, proj))) return rc;
   // Y = MLP(LayerNorm(X^)) + X^
-  if ((rc = launch_layernorm(ctx, Xh, IVIT_I8, D, to_dev(p->ln2_gamma), p->ln2_beta, p->M_ln, A, D, M, D))) return rc;
+  if (!ctx->rowop_fused &&
+      (rc = launch_layernorm(ctx, Xh, IVIT_I8, D, to_dev(p->ln2_gamma), p->ln2_beta, p->M_ln, A, D, M, D))) return rc;
   GemmProblem fc1 = linear_problem(A, D, p->W1, D, p->b1, p->fc1_scale, nullptr, 0, 1, none, G, H, IVIT_I8, 0, 0, M, H, D);
   if (p->gelu_static_max) {
     // static-maximum ShiftGELU variant: element-wise, applied to the requantised value inside the FC1 epilogue
     if ((rc = gelu_static_row(ctx, p->gelu, p->gelu_post, &fc1.epi.act_table))) return rc;
     if ((rc = launch_gemm(ctx, fc1))) return rc;
   } else {
+    // Algorithm 2 needs the maximum of a token's whole MLP row: ShiftGELU of a block of rows runs once all the
+    // channel tiles of those rows are stored, in the FC1 kernel's tail
+    if (ctx->row_fusion & 2) {
+      if ((rc = gelu_table_for(ctx, p->gelu, p->gelu_post, &fc1.epi.rop.table))) return rc;
+      fc1.epi.rop.kind = 2;
+    }
+    ctx->rowop_fused = 0;
     if ((rc = launch_gemm(ctx, fc1))) return rc;
-    if ((rc = launch_shiftgelu(ctx, G, H, p->gelu, p->gelu_post, G, H, M, H))) return rc;
+    if (!ctx->rowop_fused && (rc = launch_shiftgelu(ctx, G, H, p->gelu, p->gelu_post, G, H, M, H))) return rc;
   }
-  return launch_gemm(ctx, linear_problem(G, H, p->W2, H, p->b2, p->fc2_scale, Xh, D, M, p->res2_scale, Y, D, IVIT_I8,
-                                         0, 0, M, D, H));
+  GemmProblem fc2 = linear_problem(G, H, p->W2, H, p->b2, p->fc2_scale, Xh, D, M, p->res2_scale, Y, D, IVIT_I8, 0, 0, M, D, H);
+  if (next) want_layernorm(fc2, next->ln1_gamma, next->ln1_beta, next->M_ln, A, D);
+  ctx->rowop_fused = 0;
+  if ((rc = launch_gemm(ctx, fc2))) return rc;
+  if (a_next_ready) *a_next_ready = next && ctx->rowop_fused;
+  return IVIT_OK;
 }
 
 }  // namespace
@@ -300,8 +331,8 @@ int ivit_ctx_create(ivit_ctx** out, int device, void* cuda_stream) {
   if (cudaHostAlloc((void**)&c->status_host, sizeof(int), cudaHostAllocMapped) != cudaSuccess) { delete c; return IVIT_ERR_CUDA; }
   *c->status_host = 0;
   if (cudaHostGetDevicePointer((void**)&c->status_dev, c->status_host, 0) != cudaSuccess ||
-      cudaMalloc((void**)&c->gelu_tables, (size_t)kGeluTableSlots * kGeluTableBytes + 64) != cudaSuccess ||
-      cudaMemset(c->gelu_tables + (size_t)kGeluTableSlots * kGeluTableBytes, 0, 64) != cudaSuccess) {
+      cudaMalloc((void**)&c->gelu_tables, (size_t)kGeluTableSlots * kGeluTableBytes + 128 + kRowStateBytes) != cudaSuccess ||
+      cudaMemset(c->gelu_tables + (size_t)kGeluTableSlots * kGeluTableBytes, 0, 128 + kRowStateBytes) != cudaSuccess) {
     cudaFreeHost(c->status_host);
     delete c;
     return IVIT_ERR_CUDA;
@@ -320,6 +351,8 @@ int ivit_ctx_create(ivit_ctx** out, int device, void* cuda_stream) {
     return IVIT_ERR_CUDA;
   }
   c->sched_dev = reinterpret_cast<unsigned*>(c->gelu_tables + (size_t)kGeluTableSlots * kGeluTableBytes);
+  c->rowblk_dev = c->sched_dev + 32;
+  c->row_fusion = 0;
   *out = c;
   return IVIT_OK;
 }
@@ -368,13 +401,26 @@ int ivit_ctx_poll_status(ivit_ctx* ctx) {
   if (!ctx) return IVIT_ERR_INVALID_ARG;
   volatile int* s = ctx->status_host;
   const int v = *s;
-  if (v != 0) { *s = 0; return v; }
+  if (v != 0) {
+    *s = 0;
+    // a kernel that gave up may have left work counters behind: zero them for the launches that follow
+    cudaMemsetAsync(ctx->sched_dev, 0, 128 + kRowStateBytes, ctx->stream);
+    return v;
+  }
   return IVIT_OK;
 }
 
 int64_t ivit_ctx_launch_count(const ivit_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
 uint64_t ivit_ctx_table_generation(const ivit_ctx* ctx) { return ctx ? ctx->gelu_gen : 0; }
+
+int ivit_ctx_set_row_fusion(ivit_ctx* ctx, int enable) {
+  if (!ctx) return IVIT_ERR_INVALID_ARG;
+  // 1: every row operator; 2: I-LayerNorm only, 4: ShiftGELU only (for measurements)
+  ctx->row_fusion = enable == 1 ? 3 : (enable == 2 ? 1 : (enable == 4 ? 2 : 0));
+  for (int i = 0; i < 2; ++i) host_graph_drop(ctx, i);
+  return IVIT_OK;
+}
 
 int ivit_ctx_set_gemm_engine(ivit_ctx* ctx, int engine) {
   if (!ctx || engine < 0 || engine > 1) return IVIT_ERR_INVALID_ARG;
@@ -622,8 +668,10 @@ int ivit_vit_forward_tokens(ivit_ctx* ctx, const ivit_vit_params* p, const int8_
   if ((rc = launch_gemm(ctx, linear_problem(patches, Kpe, p->Wpe, Kpe, p->bpe, p->pe_scale, p->pos, D, np,
                                             p->pos_scale, X + D, D, IVIT_I8, np, T, B * np, D, Kpe)))) return rc;
   if ((rc = launch_fill_rows(ctx, p->cls, D, X, T * D, B))) return rc;
+  bool a_ready = false;   // LayerNorm 1 of the next block already produced by the previous block's last Dense layer
   for (int64_t l = 0; l < p->depth; ++l) {
-    if ((rc = block_impl(ctx, &p->blocks[l], X, Y, ws + w.block))) return rc;
+    const ivit_block_params* next = l + 1 < p->depth ? &p->blocks[l + 1] : nullptr;
+    if ((rc = block_impl(ctx, &p->blocks[l], X, Y, ws + w.block, a_ready, next, &a_ready))) return rc;
     int8_t* t = X; X = Y; Y = t;
   }
   if (tokens && cudaMemcpyAsync(tokens, X, (size_t)(B * T * D), cudaMemcpyDeviceToDevice, ctx->stream) != cudaSuccess)
@@ -639,6 +687,177 @@ size_t ivit_vit_host_workspace_bytes(const ivit_vit_params* p) {
   const size_t img = align_up((size_t)(p->B * 3 * p->img * p->img), 256);
   const size_t lg = align_up((size_t)(p->B * p->classes) * 4, 256);
   return vit_ws(p).total + 2 * img + lg;
+}
+
+// ---- Swin-shaped forward -------------------------------------------------------------------------------
+
+static int check_swin(const ivit_swin_params* p) {
+  if (!p || p->B < 0 || p->n_stages < 1 || !p->stages || p->patch < 4 || p->patch % 4 || p->window < 1 || p->classes < 1)
+    return IVIT_ERR_INVALID_ARG;
+  if (p->img % p->patch || !p->Wpe || !p->Whead) return IVIT_ERR_INVALID_ARG;
+  if (p->M_ln < 8 || p->M_ln > 29) return IVIT_ERR_RANGE;
+  if (!scale_ok(p->pe_scale) || !scale_ok(p->pe_ln_gamma) || !scale_ok(p->lnf_gamma) || !scale_ok(p->pool_scale) ||
+      p->pool_scale.mult_c || !scale_ok(p->head_scale))
+    return IVIT_ERR_RANGE;
+  int64_t res = p->img / p->patch;
+  for (int64_t s = 0; s < p->n_stages; ++s) {
+    const ivit_swin_stage* st = &p->stages[s];
+    if (st->res != res || st->C < 16 || st->C % 16 || st->depth < 1 || !st->blocks || res % p->window) return IVIT_ERR_INVALID_ARG;
+    const int64_t windows = p->B * (res / p->window) * (res / p->window);
+    for (int64_t l = 0; l < st->depth; ++l) {
+      const ivit_block_params* b = &st->blocks[l];
+      int rc = check_block(b);
+      if (rc) return rc;
+      if (b->B != windows || b->T != p->window * p->window || b->D != st->C) return IVIT_ERR_INVALID_ARG;
+      if (st->shifted && st->shifted[l] && (!st->shift_index || !st->unshift_index)) return IVIT_ERR_INVALID_ARG;
+    }
+    const bool last = s + 1 == p->n_stages;
+    if (last != (st->merge_index == nullptr)) return IVIT_ERR_INVALID_ARG;
+    if (!last) {
+      if (!st->Wmerge || res % 2) return IVIT_ERR_INVALID_ARG;
+      if (!scale_ok(st->merge_ln_gamma) || !scale_ok(st->merge_scale)) return IVIT_ERR_RANGE;
+      if (p->stages[s + 1].C != 2 * st->C) return IVIT_ERR_INVALID_ARG;
+      res /= 2;
+    }
+  }
+  return IVIT_OK;
+}
+
+struct SwinWs { size_t patches, P[3], Z, block, total; };
+static SwinWs swin_ws(const ivit_swin_params* p) {
+  SwinWs w;
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+  const int64_t res0 = p->img / p->patch;
+  const size_t Kpe = (size_t)(3 * p->patch * p->patch);
+  w.patches = take((size_t)(p->B * res0 * res0) * Kpe);
+  // the token tensor is largest in stage 0 (every merge halves its bytes); three buffers of that size
+  const size_t tok = (size_t)(p->B * res0 * res0 * p->stages[0].C);
+  for (int i = 0; i < 3; ++i) w.P[i] = take(tok);
+  w.Z = take((size_t)(p->B * p->stages[p->n_stages - 1].C));
+  size_t blk = 0;
+  for (int64_t s = 0; s < p->n_stages; ++s)
+    for (int64_t l = 0; l < p->stages[s].depth; ++l) {
+      const size_t b = block_ws(&p->stages[s].blocks[l]).total;
+      blk = b > blk ? b : blk;
+    }
+  w.block = take(blk);
+  w.total = off;
+  return w;
+}
+
+size_t ivit_swin_workspace_bytes(const ivit_swin_params* p) {
+  if (check_swin(p) != IVIT_OK) return 0;
+  return swin_ws(p).total;
+}
+
+// Dense layer followed by I-LayerNorm of its output rows (in the Dense kernel's tail where that is possible).
+static int dense_then_layernorm(ivit_ctx* ctx, GemmProblem g, const ivit_scale& gamma, const int32_t* beta, int M_ln,
+                                int8_t* ln_out) {
+  const int64_t M = g.M, N = g.N;
+  want_layernorm(g, gamma, beta, M_ln, ln_out, N);
+  ctx->rowop_fused = 0;
+  int rc = launch_gemm(ctx, g);
+  if (rc) return rc;
+  if (ctx->rowop_fused) return IVIT_OK;
+  return launch_layernorm(ctx, g.epi.out, IVIT_I8, g.epi.ldo, to_dev(gamma), beta, M_ln, ln_out, N, M, N);
+}
+
+int ivit_swin_forward(ivit_ctx* ctx, const ivit_swin_params* p, const int8_t* image, int32_t* logits,
+                      int8_t* tokens, void* workspace, size_t workspace_bytes) {
+  if (!ctx || !image || !logits) return IVIT_ERR_INVALID_ARG;
+  int rc = check_swin(p);
+  if (rc) return rc;
+  if (!aligned16(image) || !aligned16(logits) || p->classes % 4 || (tokens && !aligned16(tokens))) return IVIT_ERR_ALIGNMENT;
+  const SwinWs w = swin_ws(p);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < w.total) return IVIT_ERR_WORKSPACE;
+  char* ws = static_cast<char*>(workspace);
+  const ivit_scale none{nullptr, nullptr, 1, 1};
+  const int64_t B = p->B, Kpe = 3 * p->patch * p->patch;
+  int64_t res = p->img / p->patch, rows = B * res * res;
+  int8_t* patches = reinterpret_cast<int8_t*>(ws + w.patches);
+  int8_t* cur = reinterpret_cast<int8_t*>(ws + w.P[0]);
+  int8_t* other = reinterpret_cast<int8_t*>(ws + w.P[1]);
+  int8_t* third = reinterpret_cast<int8_t*>(ws + w.P[2]);
+  int8_t* Z = reinterpret_cast<int8_t*>(ws + w.Z);
+  char* wsb = ws + w.block;
+  if ((rc = launch_patchify(ctx, image, B, 3, p->img, p->img, p->patch, p->window, patches, Kpe))) return rc;
+  const int64_t C0 = p->stages[0].C;
+  if ((rc = dense_then_layernorm(ctx, linear_problem(patches, Kpe, p->Wpe, Kpe, p->bpe, p->pe_scale, nullptr, 0, 1, none, other,
+                                                      C0, IVIT_I8, 0, 0, rows, C0, Kpe),
+                                 p->pe_ln_gamma, p->pe_ln_beta, p->M_ln, cur))) return rc;
+  // the final LayerNorm, dressed as the LayerNorm 1 of a block that follows the last one
+  ivit_block_params fin{};
+  fin.ln1_gamma = p->lnf_gamma; fin.ln1_beta = p->lnf_beta; fin.M_ln = p->M_ln;
+  bool a_ready = false;   // the LayerNorm output that the next block (or the pooling) reads sits in the block workspace
+  for (int64_t s = 0; s < p->n_stages; ++s) {
+    const ivit_swin_stage* st = &p->stages[s];
+    const int64_t C = st->C;
+    for (int64_t l = 0; l < st->depth; ++l) {
+      const bool sh = st->shifted && st->shifted[l];
+      const bool sh_next = l + 1 < st->depth && st->shifted && st->shifted[l + 1];
+      // LayerNorm 1 of the next block comes out of this block's last Dense layer when the next block reads this
+      // block's output rows as they are (no row permutation in between)
+      const ivit_block_params* next = (l + 1 < st->depth && !sh && !sh_next) ? &st->blocks[l + 1] : nullptr;
+      if (l + 1 == st->depth && s + 1 == p->n_stages && !sh) next = &fin;
+      if (sh) {
+        if ((rc = launch_gather_rows(ctx, cur, C, st->shift_index, rows, C, third, C))) return rc;
+        if ((rc = block_impl(ctx, &st->blocks[l], third, other, wsb, false, nullptr, nullptr))) return rc;
+        if ((rc = launch_gather_rows(ctx, other, C, st->unshift_index, rows, C, cur, C))) return rc;
+        a_ready = false;
+      } else {
+        if ((rc = block_impl(ctx, &st->blocks[l], cur, other, wsb, a_ready, next, &a_ready))) return rc;
+        int8_t* t = cur; cur = other; other = t;
+      }
+    }
+    if (st->merge_index) {
+      // 2x2 patch merging: four C-wide slices per output row, LayerNorm over 4C, Dense to 2C
+      if ((rc = launch_gather_rows(ctx, cur, C, st->merge_index, rows, C, other, C))) return rc;
+      rows /= 4;
+      res /= 2;
+      if ((rc = launch_layernorm(ctx, other, IVIT_I8, 4 * C, to_dev(st->merge_ln_gamma), st->merge_ln_beta, p->M_ln, third,
+                                 4 * C, rows, 4 * C))) return rc;
+      // ... followed by LayerNorm 1 of the next stage's first block (into the block workspace, where it expects it)
+      const ivit_block_params* nb = &p->stages[s + 1].blocks[0];
+      if ((rc = dense_then_layernorm(ctx, linear_problem(third, 4 * C, st->Wmerge, 4 * C, nullptr, st->merge_scale, nullptr, 0, 1,
+                                                          none, cur, 2 * C, IVIT_I8, 0, 0, rows, 2 * C, 4 * C),
+                                     nb->ln1_gamma, nb->ln1_beta, nb->M_ln, reinterpret_cast<int8_t*>(wsb)))) return rc;
+      a_ready = !(p->stages[s + 1].shifted && p->stages[s + 1].shifted[0]);
+    }
+  }
+  const int64_t Cl = p->stages[p->n_stages - 1].C;
+  if (tokens && cudaMemcpyAsync(tokens, cur, (size_t)(rows * Cl), cudaMemcpyDeviceToDevice, ctx->stream) != cudaSuccess)
+    return IVIT_ERR_CUDA;
+  const int8_t* normed = reinterpret_cast<const int8_t*>(wsb);
+  if (!a_ready) {
+    if ((rc = launch_layernorm(ctx, cur, IVIT_I8, Cl, to_dev(p->lnf_gamma), p->lnf_beta, p->M_ln, other, Cl, rows, Cl))) return rc;
+    normed = other;
+  }
+  if ((rc = launch_token_mean(ctx, normed, Cl, B, rows / (B > 0 ? B : 1), Cl, to_dev(p->pool_scale), Z, Cl))) return rc;
+  return launch_gemm(ctx, linear_problem(Z, Cl, p->Whead, Cl, p->bhead, p->head_scale, nullptr, 0, 1, none, logits, p->classes,
+                                         IVIT_I32, 0, 0, B, p->classes, Cl));
+}
+
+size_t ivit_swin_host_workspace_bytes(const ivit_swin_params* p) {
+  if (check_swin(p) != IVIT_OK) return 0;
+  return swin_ws(p).total + align_up((size_t)(p->B * 3 * p->img * p->img), 256) + align_up((size_t)(p->B * p->classes) * 4, 256);
+}
+
+int ivit_swin_forward_host(ivit_ctx* ctx, const ivit_swin_params* p, const int8_t* image_host, int32_t* logits_host,
+                           void* workspace, size_t workspace_bytes) {
+  if (!ctx || !image_host || !logits_host) return IVIT_ERR_INVALID_ARG;
+  int rc = check_swin(p);
+  if (rc) return rc;
+  const size_t img_bytes = (size_t)(p->B * 3 * p->img * p->img), lg_bytes = (size_t)(p->B * p->classes) * 4;
+  const size_t inner = swin_ws(p).total, lg_off = inner + align_up(img_bytes, 256);
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < lg_off + align_up(lg_bytes, 256))
+    return IVIT_ERR_WORKSPACE;
+  char* ws = static_cast<char*>(workspace);
+  if (cudaMemcpyAsync(ws + inner, image_host, img_bytes, cudaMemcpyHostToDevice, ctx->stream) != cudaSuccess) return IVIT_ERR_CUDA;
+  if ((rc = ivit_swin_forward(ctx, p, reinterpret_cast<const int8_t*>(ws + inner), reinterpret_cast<int32_t*>(ws + lg_off), nullptr,
+                              workspace, inner))) return rc;
+  if (cudaMemcpyAsync(logits_host, ws + lg_off, lg_bytes, cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess) return IVIT_ERR_CUDA;
+  return IVIT_OK;
 }
 
 int ivit_ctx_set_host_graph(ivit_ctx* ctx, int enable) {

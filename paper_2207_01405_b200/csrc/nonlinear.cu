@@ -1,7 +1,7 @@
 // I-LayerNorm (Sec. 3.5), Shiftmax (Algorithm 1) and ShiftGELU (Algorithm 2) kernels, sm_100a.
 // One warp owns one row; rows are read once from HBM as coalesced 32-bit words and
 // kept in registers between the reduction and the output pass.
-#include "common.cuh"
+#include "rowops.cuh"
 #include <type_traits>
 
 namespace ivit {
@@ -122,175 +122,32 @@ __global__ void __launch_bounds__(256) layernorm_i8_kernel(const int8_t* __restr
   }
 }
 
-// Batched form: a warp owns ROWS consecutive rows.  The rows' sums are reduced together, the
-// per-row scalars (mean, integer square root, reciprocal) are then computed by ROWS different lanes
-// at once instead of redundantly by all 32, and the per-channel constants of the lane's channels
-// are loaded once for all ROWS rows: v = ((x*F - mu*F) * m + 2^(s-1)) >> s + beta.
-// mean_magic = floor(2^32 / (2C)) + 1 turns the mean's division into a multiplication (exact for the
-// numerators of int8 rows of up to 1024 channels, which stay below 2^19).
-// SMEMC: the per-channel constants live in shared memory (rows too wide for registers), set up once per block.
-template <int WPL, int ROWS, bool SMEMC>
-__global__ void __launch_bounds__(128, SMEMC ? 4 : 6) layernorm_i8_batched_kernel(const int8_t* __restrict__ in, int64_t ldin,
-                                                                      ScaleDev gs, const int32_t* __restrict__ beta,
-                                                                      int M_ln, int8_t* __restrict__ out, int64_t ldout,
-                                                                      int64_t rows, int C, unsigned mean_magic, int vec) {
-  extern __shared__ int4 ln_consts[];   // SMEMC: [3][C / 4] multipliers, shifts, addends (or betas)
+// Rows of up to 1024 channels: a warp takes R rows at a time (layernorm_rows); the per-channel constants are
+// prepared once per block in shared memory, before the wait for the previous kernel (they are parameters, not
+// results).
+template <int WPL, int R>
+__global__ void __launch_bounds__(128) layernorm_rows_kernel(const int8_t* __restrict__ in, int64_t ldin, ScaleDev gs,
+                                                             const int32_t* __restrict__ beta, int M_ln,
+                                                             int8_t* __restrict__ out, int64_t ldout, int64_t rows, int C,
+                                                             unsigned mean_magic, int vec) {
+  extern __shared__ int4 ln_consts[];   // [3][C / 4]: multipliers, shifts, addends (or betas)
   pdl_trigger();
-  // the per-channel constants are parameters, not results of the previous kernel: they are fetched before the
-  // wait for that kernel (below, in front of the first row load)
+  const int nwords = C >> 2;
+  int4* sm_m = ln_consts;
+  int4* sm_s = ln_consts + nwords;
+  int4* sm_b = ln_consts + 2 * nwords;
+  bool fast = ln_stage_consts(gs, beta, nwords, vec, sm_m, sm_s, sm_b, threadIdx.x, blockDim.x);
+  fast = __syncthreads_and(fast) != 0;
+  if (fast) ln_fold_consts(nwords, sm_s, sm_b, threadIdx.x, blockDim.x);
+  __syncthreads();
+  const LnConsts k{sm_m, sm_s, sm_b, fast};
+  pdl_wait();
   const int lane = threadIdx.x & 31;
   const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
-  const int nwords = C >> 2;
-  // constants of four channels (one word of the row)
-  auto load_consts = [&](int idx, int (&m)[4], int (&sft)[4], int (&b)[4]) {
-    if (vec) {
-      // per-channel arrays aligned for one 16-byte (4-byte for the shifts) load per word of four channels
-      int4 m4 = make_int4(1, 1, 1, 1), b4 = make_int4(0, 0, 0, 0);
-      uchar4 s4 = make_uchar4(40, 40, 40, 40);
-      if (idx < nwords) {
-        m4 = __ldg(reinterpret_cast<const int4*>(gs.mult_c) + idx);
-        s4 = __ldg(reinterpret_cast<const uchar4*>(gs.shift_c) + idx);
-        if (beta) b4 = __ldg(reinterpret_cast<const int4*>(beta) + idx);
-      }
-      m[0] = m4.x; m[1] = m4.y; m[2] = m4.z; m[3] = m4.w;
-      sft[0] = clamp_shift(s4.x); sft[1] = clamp_shift(s4.y); sft[2] = clamp_shift(s4.z); sft[3] = clamp_shift(s4.w);
-      b[0] = b4.x; b[1] = b4.y; b[2] = b4.z; b[3] = b4.w;
-    } else {
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const int c = idx * 4 + k;
-        m[k] = idx < nwords ? gs.m(c) : 1;
-        sft[k] = idx < nwords ? gs.s(c) : 40;
-        b[k] = (idx < nwords && beta) ? __ldg(beta + c) : 0;
-      }
-    }
-  };
-  // Fast form, taken when it is exact for every channel: with s >= 33 the rounding constant 2^(s-1) is a
-  // multiple of 2^32, so (yF m + 2^(s-1)) >> s = (hi32(yF m) + 2^(s-33)) >> (s - 32), and beta joins the
-  // constant as beta 2^(s-32) when that stays far from 32 bits (|hi32| < 2^21 here).
-  auto fast_ok = [](const int (&sft)[4], const int (&b)[4]) {
-    bool f = true;
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      const int sh = sft[k] - 32;
-      f = f && sh >= 1 && b[k] > -(1 << (29 - sh)) && b[k] < (1 << (29 - sh));
-    }
-    return f;
-  };
-  // the fast form keeps s - 32 and the combined constant instead of s and beta
-  auto to_fast = [](int (&sft)[4], int (&b)[4]) {
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-      sft[k] -= 32;
-      b[k] = (1 << (sft[k] - 1)) + b[k] * (1 << sft[k]);
-    }
-  };
-  constexpr int WR = SMEMC ? 1 : WPL;
-  int pm[WR][4], ps[WR][4], pb[WR][4];   // registers: the constants of this lane's channels
-  bool fast = true;
-  if (SMEMC) {
-    for (int idx = threadIdx.x; idx < nwords; idx += blockDim.x) {
-      load_consts(idx, pm[0], ps[0], pb[0]);
-      fast = fast && fast_ok(ps[0], pb[0]);
-    }
-    fast = __syncthreads_and(fast) != 0;
-    for (int idx = threadIdx.x; idx < nwords; idx += blockDim.x) {
-      load_consts(idx, pm[0], ps[0], pb[0]);
-      if (fast) to_fast(ps[0], pb[0]);
-      ln_consts[idx] = make_int4(pm[0][0], pm[0][1], pm[0][2], pm[0][3]);
-      ln_consts[nwords + idx] = make_int4(ps[0][0], ps[0][1], ps[0][2], ps[0][3]);
-      ln_consts[2 * nwords + idx] = make_int4(pb[0][0], pb[0][1], pb[0][2], pb[0][3]);
-    }
-    __syncthreads();
-  } else {
-#pragma unroll
-    for (int i = 0; i < WR; ++i) {
-      load_consts(lane + 32 * i, pm[i], ps[i], pb[i]);
-      fast = fast && fast_ok(ps[i], pb[i]);
-    }
-    fast = __all_sync(0xffffffffu, fast);
-    if (fast) {
-#pragma unroll
-      for (int i = 0; i < WR; ++i) to_fast(ps[i], pb[i]);
-    }
-  }
-  pdl_wait();
-  for (int64_t r0 = warp * ROWS; r0 < rows; r0 += nwarps * ROWS) {
-    int w[ROWS][WPL];
-    int my_s1 = 0, my_s2 = 0;
-#pragma unroll
-    for (int r = 0; r < ROWS; ++r) {
-      const bool ok = r0 + r < rows;
-      const int* src = reinterpret_cast<const int*>(in + (r0 + r) * ldin);
-#pragma unroll
-      for (int i = 0; i < WPL; ++i) {
-        const int idx = lane + 32 * i;
-        w[r][i] = (ok && idx < nwords) ? __ldg(src + idx) : 0;
-      }
-    }
-#pragma unroll
-    for (int r = 0; r < ROWS; ++r) {
-      int s1 = 0, s2 = 0;
-#pragma unroll
-      for (int i = 0; i < WPL; ++i) {
-        s1 = __dp4a(w[r][i], 0x01010101, s1);
-        s2 = __dp4a(w[r][i], w[r][i], s2);
-      }
-      s1 = __reduce_add_sync(0xffffffffu, s1);
-      s2 = __reduce_add_sync(0xffffffffu, s2);
-      if (lane == r) { my_s1 = s1; my_s2 = s2; }
-    }
-    // lane r (< ROWS) holds the sums of row r0 + r: mean (round half up) = floor((2 S1 + C) / 2C), taken on the
-    // numerator shifted by 256 C to make it positive; sum of squared deviations = sum x^2 - 2 mu sum x + C mu^2
-    // (every term below 2^26 for int8 rows of up to 1024 channels); integer square root; reciprocal
-    const int mu = (int)__umulhi((unsigned)(2 * my_s1 + 257 * C), mean_magic) - 128;
-    const int V = my_s2 - 2 * mu * my_s1 + C * mu * mu;
-    const unsigned sd = isqrt_u32((unsigned)V);
-    const int F = sd == 0 ? 0 : (int)((1u << M_ln) / sd);
-    const int muF = (int)((unsigned)mu * (unsigned)F);
-#pragma unroll
-    for (int r = 0; r < ROWS; ++r) {
-      const int Fr = __shfl_sync(0xffffffffu, F, r);
-      const int muFr = __shfl_sync(0xffffffffu, muF, r);
-      if (r0 + r < rows) {
-        int* dst = reinterpret_cast<int*>(out + (r0 + r) * ldout);
-#pragma unroll
-        for (int i = 0; i < WPL; ++i) {
-          const int idx = lane + 32 * i;
-          if (idx < nwords) {
-            int cm[4], cs[4], cb[4];
-            if (SMEMC) {
-              const int4 m4 = ln_consts[idx], s4 = ln_consts[nwords + idx], b4 = ln_consts[2 * nwords + idx];
-              cm[0] = m4.x; cm[1] = m4.y; cm[2] = m4.z; cm[3] = m4.w;
-              cs[0] = s4.x; cs[1] = s4.y; cs[2] = s4.z; cs[3] = s4.w;
-              cb[0] = b4.x; cb[1] = b4.y; cb[2] = b4.z; cb[3] = b4.w;
-            } else {
-#pragma unroll
-              for (int b = 0; b < 4; ++b) { cm[b] = pm[SMEMC ? 0 : i][b]; cs[b] = ps[SMEMC ? 0 : i][b]; cb[b] = pb[SMEMC ? 0 : i][b]; }
-            }
-            int v[4];
-#pragma unroll
-            for (int b = 0; b < 4; ++b) {
-              // byte b, sign-extended by one byte permute
-              int x;
-              asm("prmt.b32 %0, %1, %1, %2;" : "=r"(x) : "r"(w[r][i]), "r"(0x8880 + 0x1111 * b));
-              // (x - mu) * F, formed modulo 2^32 (the difference always fits: |y F| <= 2^(M_ln+1))
-              const int yF = (int)((unsigned)x * (unsigned)Fr - (unsigned)muFr);
-              if (fast) {
-                v[b] = (__mulhi(yF, cm[b]) + cb[b]) >> cs[b];
-              } else {
-                v[b] = rq(yF, cm[b], cs[b]) + cb[b];
-              }
-            }
-            unsigned t, d;
-            asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(t) : "r"(v[3]), "r"(v[2]), "r"(0));
-            asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(v[1]), "r"(v[0]), "r"(t));
-            dst[idx] = (int)d;
-          }
-        }
-      }
-    }
+  for (int64_t r0 = warp * R; r0 < rows; r0 += nwarps * R) {
+    const int nrows = (int)(rows - r0 < R ? rows - r0 : R);
+    layernorm_rows<WPL, R, false>(in + r0 * ldin, ldin, nrows, C, M_ln, mean_magic, k, out + r0 * ldout, ldout, lane);
   }
 }
 
@@ -386,9 +243,7 @@ int launch_layernorm(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, 
   const int8_t* x = (const int8_t*)in;
   const int wpl = (int)((C / 4 + 31) / 32);
   if (wpl <= 8) {
-    // batched kernel: 16 to 2 rows per warp, fewer for wider rows, amortise the per-row scalar work and the
-    // per-channel constants (in registers up to 512 channels, in shared memory up to 1024); 128-thread blocks
-    const int rpw = wpl <= 1 ? 16 : (wpl <= 2 ? 8 : (wpl <= 4 ? 4 : 2)), tb = 128;
+    const int rpw = wpl <= 4 ? 8 : 4, tb = 128;
     const int64_t warps = (rows + rpw - 1) / rpw;
     const int64_t wantb = (warps + tb / 32 - 1) / (tb / 32);
     const int gridb = (int)(wantb < (int64_t)ctx->sm_count * 12 ? wantb : (int64_t)ctx->sm_count * 12);
@@ -396,17 +251,15 @@ int launch_layernorm(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, 
     const int vec = gs.mult_c && gs.shift_c && !(reinterpret_cast<uintptr_t>(gs.mult_c) & 15) && !(reinterpret_cast<uintptr_t>(gs.shift_c) & 3) &&
                     !(reinterpret_cast<uintptr_t>(beta) & 15);
     const size_t cbytes = (size_t)(C / 4) * 3 * sizeof(int4);
-    if (wpl <= 1) launch_k(layernorm_i8_batched_kernel<1, 16, false>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
-    else if (wpl <= 2) launch_k(layernorm_i8_batched_kernel<2, 8, false>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
-    else if (wpl <= 3) launch_k(layernorm_i8_batched_kernel<3, 4, false>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
-    else if (wpl <= 4) launch_k(layernorm_i8_batched_kernel<4, 4, false>, dim3(gridb), dim3(tb), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
-    else if (wpl <= 6) launch_k(layernorm_i8_batched_kernel<6, 2, true>, dim3(gridb), dim3(tb), cbytes, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
-    else launch_k(layernorm_i8_batched_kernel<8, 2, true>, dim3(gridb), dim3(tb), cbytes, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
+    if (wpl <= 1) launch_k(layernorm_rows_kernel<1, 8>, dim3(gridb), dim3(tb), cbytes, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
+    else if (wpl <= 2) launch_k(layernorm_rows_kernel<2, 8>, dim3(gridb), dim3(tb), cbytes, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
+    else if (wpl <= 3) launch_k(layernorm_rows_kernel<3, 8>, dim3(gridb), dim3(tb), cbytes, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
+    else if (wpl <= 4) launch_k(layernorm_rows_kernel<4, 8>, dim3(gridb), dim3(tb), cbytes, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
+    else if (wpl <= 6) launch_k(layernorm_rows_kernel<6, 4>, dim3(gridb), dim3(tb), cbytes, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
+    else launch_k(layernorm_rows_kernel<8, 4>, dim3(gridb), dim3(tb), cbytes, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
     return ls.done();
   }
-  if (wpl <= 6) launch_k(layernorm_i8_kernel<6>, dim3(grid), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-  else if (wpl <= 8) launch_k(layernorm_i8_kernel<8>, dim3(grid), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
-  else if (wpl <= 12) launch_k(layernorm_i8_kernel<12>, dim3(grid), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
+  if (wpl <= 12) launch_k(layernorm_i8_kernel<12>, dim3(grid), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
   else launch_k(layernorm_i8_long_kernel, dim3(grid), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
   return ls.done();
 }
@@ -759,31 +612,38 @@ __global__ void shiftgelu_table_kernel(ivit_exp_params p, int post_m, int post_s
   table[m * 256 + threadIdx.x] = (int8_t)out;
 }
 
-template <int WPL>
+// WPL > 0: rows of up to 512 * WPL values, R rows per warp at a time, kept in registers between the maximum and
+// the look-ups (shiftgelu_rows).  WPL == 0: any width; the row is read twice.
+template <int WPL, int R>
 __global__ void __launch_bounds__(256) shiftgelu_kernel(const int8_t* __restrict__ in, int64_t ldin,
                                                         const int8_t* __restrict__ table,
                                                         int8_t* __restrict__ out, int64_t ldout,
                                                         int64_t rows, int cols, int fixed_max) {
   pdl_trigger();
   pdl_wait();
-  __shared__ unsigned tab[8][64];  // one 256-byte table row per warp
+  __shared__ __align__(256) unsigned tab[8][(WPL > 0 ? R : 1) * 64];  // 256-byte table rows, per warp
   const int lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
   const int64_t warp = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int64_t nwarps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+  if (WPL > 0) {
+    constexpr int W = WPL > 0 ? WPL : 1;
+    for (int64_t r0 = warp * R; r0 < rows; r0 += nwarps * R) {
+      const int nrows = (int)(rows - r0 < R ? rows - r0 : R);
+      shiftgelu_rows<W, R, false>(in + r0 * ldin, ldin, nrows, cols, table, tab[wib], out + r0 * ldout, ldout, lane, fixed_max);
+      __syncwarp();
+    }
+    return;
+  }
   const int nvec = cols >> 4;  // 16-byte vectors per row
-  constexpr int W = WPL > 0 ? WPL : 1;
-  const int iters = WPL > 0 ? WPL : (nvec + 31) / 32;
+  const int iters = (nvec + 31) / 32;
   const unsigned char* t8 = reinterpret_cast<const unsigned char*>(tab[wib]);
   for (int64_t r = warp; r < rows; r += nwarps) {
     const int4* src = reinterpret_cast<const int4*>(in + r * ldin);
-    int4 w[W];
     int mx4 = (int)0x80808080;
-#pragma unroll
     for (int i = 0; i < iters; ++i) {
       const int idx = lane + 32 * i;
       int4 v = make_int4((int)0x80808080, (int)0x80808080, (int)0x80808080, (int)0x80808080);
       if (idx < nvec) v = __ldg(src + idx);
-      if (WPL > 0) w[i] = v;
       mx4 = (int)__vmaxs4(__vmaxs4((unsigned)v.x, (unsigned)v.y), __vmaxs4(__vmaxs4((unsigned)v.z, (unsigned)v.w), (unsigned)mx4));
     }
     int mx = max(max((int)(int8_t)mx4, (int)(int8_t)(mx4 >> 8)), max((int)(int8_t)(mx4 >> 16), (int)(int8_t)(mx4 >> 24)));
@@ -794,12 +654,10 @@ __global__ void __launch_bounds__(256) shiftgelu_kernel(const int8_t* __restrict
     tab[wib][lane + 32] = __ldg(trow + lane + 32);
     __syncwarp();
     int4* dst = reinterpret_cast<int4*>(out + r * ldout);
-#pragma unroll
     for (int i = 0; i < iters; ++i) {
       const int idx = lane + 32 * i;
       if (idx < nvec) {
-        const int4 v = WPL > 0 ? w[i] : __ldg(src + idx);
-        int4 o;
+        const int4 v = __ldg(src + idx);
         const int vin[4] = {v.x, v.y, v.z, v.w};
         int vout[4];
 #pragma unroll
@@ -811,8 +669,7 @@ __global__ void __launch_bounds__(256) shiftgelu_kernel(const int8_t* __restrict
           pk |= (unsigned)t8[u >> 24] << 24;
           vout[k] = (int)pk;
         }
-        o = make_int4(vout[0], vout[1], vout[2], vout[3]);
-        dst[idx] = o;
+        dst[idx] = make_int4(vout[0], vout[1], vout[2], vout[3]);
       }
     }
   }
@@ -843,6 +700,10 @@ static int gelu_table(ivit_ctx* ctx, ivit_exp_params p, ivit_scale post, const i
   return IVIT_OK;
 }
 
+int gelu_table_for(ivit_ctx* ctx, ivit_exp_params p, ivit_scale post, const int8_t** table) {
+  return gelu_table(ctx, p, post, table);
+}
+
 int gelu_static_row(ivit_ctx* ctx, ivit_exp_params p, ivit_scale post, const int8_t** row) {
   const int8_t* table = nullptr;
   const int rc = gelu_table(ctx, p, post, &table);
@@ -857,18 +718,19 @@ static int shiftgelu_rows(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_ex
   const int8_t* table = nullptr;
   int rc = gelu_table(ctx, p, post, &table);
   if (rc) return rc;
-  const int64_t want = (rows + 7) / 8;
-  const int grid = (int)(want < (int64_t)ctx->sm_count * 8 ? want : (int64_t)ctx->sm_count * 8);
   const int wpl = (int)((cols / 16 + 31) / 32);
+  const int rpw = wpl <= 2 ? 4 : (wpl <= 4 ? 2 : 1);            // rows a warp takes at a time
+  const int64_t want = ((rows + rpw - 1) / rpw + 7) / 8;
+  const int grid = (int)(want < (int64_t)ctx->sm_count * 8 ? want : (int64_t)ctx->sm_count * 8);
   cudaStream_t st = ctx->stream;
   LaunchScope ls(ctx, KIND_SHIFTGELU, 2.0 * (double)rows * (double)cols);
-  if (wpl <= 1) launch_k(shiftgelu_kernel<1>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
-  else if (wpl <= 2) launch_k(shiftgelu_kernel<2>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
-  else if (wpl <= 3) launch_k(shiftgelu_kernel<3>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
-  else if (wpl <= 4) launch_k(shiftgelu_kernel<4>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
-  else if (wpl <= 6) launch_k(shiftgelu_kernel<6>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
-  else if (wpl <= 8) launch_k(shiftgelu_kernel<8>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
-  else launch_k(shiftgelu_kernel<0>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
+  if (wpl <= 1) launch_k(shiftgelu_kernel<1, 4>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
+  else if (wpl <= 2) launch_k(shiftgelu_kernel<2, 4>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
+  else if (wpl <= 3) launch_k(shiftgelu_kernel<3, 2>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
+  else if (wpl <= 4) launch_k(shiftgelu_kernel<4, 2>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
+  else if (wpl <= 6) launch_k(shiftgelu_kernel<6, 1>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
+  else if (wpl <= 8) launch_k(shiftgelu_kernel<8, 1>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
+  else launch_k(shiftgelu_kernel<0, 1>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
   return ls.done();
 }
 
@@ -883,3 +745,20 @@ int launch_shiftgelu_static(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_
 }
 
 }  // namespace ivit
+
+// ---- verification aid: the square-root routine of the I-LayerNorm kernels over a range of radicands ----
+namespace ivit {
+__global__ void isqrt_range_kernel(unsigned n0, unsigned count, uint16_t* __restrict__ out) {
+  for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < count; i += gridDim.x * blockDim.x)
+    out[i] = (uint16_t)isqrt_bits26(n0 + i);
+}
+}  // namespace ivit
+
+extern "C" int ivit_isqrt_range(ivit_ctx* ctx, uint32_t n0, uint32_t count, uint16_t* out) {
+  if (!ctx || !out) return IVIT_ERR_INVALID_ARG;
+  if ((uint64_t)n0 + count > (1ull << 26)) return IVIT_ERR_RANGE;
+  if (count == 0) return IVIT_OK;
+  ivit::isqrt_range_kernel<<<ctx->sm_count * 8, 256, 0, ctx->stream>>>(n0, count, out);
+  ctx->launches += 1;
+  return cudaGetLastError() == cudaSuccess ? IVIT_OK : IVIT_ERR_CUDA;
+}

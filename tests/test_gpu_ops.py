@@ -457,3 +457,18 @@ def test_tensor_core_engine_takes_the_model_shapes():
     kinds = [k for k, _, _ in c.profile_stop()]
     assert kinds == ["gemm_tcgen05"] * 3, kinds
     assert c.poll_status() == 0
+
+
+def test_layernorm_square_root_routine_equals_the_iteration_exhaustively():
+    """The I-LayerNorm kernels take floor(sqrt(V)) bit by bit; Sec. 3.5 prescribes Eq. (iterative).  Both are run
+    over EVERY radicand an int8 row of up to 1024 channels can produce (V < 2^26) and compared with the oracle's
+    iteration (which is pinned against floor(sqrt) on CPU)."""
+    g = _g()
+    c = g.ctx()
+    step = 1 << 23
+    for n0 in range(0, 1 << 26, step):
+        got = c.isqrt_range(n0, step).cpu().numpy().astype(np.int64)
+        want = O.isqrt_array(np.arange(n0, n0 + step, dtype=np.int64))
+        assert np.array_equal(got, want), f"first mismatch at n = {n0 + int(np.argmax(got != want))}"
+    with pytest.raises(g.binding.IvitError):
+        c.isqrt_range((1 << 26) - 4, 8)
