@@ -83,10 +83,11 @@ constexpr int kThreads = 32 * kFirstEpiWarp + kEpiThreads;
 
 struct TcArgs {
   GemmEpilogue epi;
-  int64_t P, Q, K;   // extents along TMEM lanes / TMEM columns / contraction
+  int P, Q, K;       // extents along TMEM lanes / TMEM columns / contraction (32-bit: the launcher checks the sizes)
   int64_t sCo, sCi;
-  int64_t batches_inner;
-  int64_t total_tiles;
+  int batches_inner;
+  int total_tiles;
+  int tiles_each, tiles_extra;   // every CTA walks tiles_each tiles, the first tiles_extra CTAs one more
   int tiles_p, tiles_q;
   int BN;            // columns of the tile (multiple of 32, <= 256)
   int stages;
@@ -106,29 +107,29 @@ struct TcArgs {
 
 
 struct TileCoord {
-  int64_t batch;
+  int batch;
   int bo, bi, p0, q0;
 };
 
 // Tiles are ordered p-block fastest and every CTA owns a contiguous range of them, so that the tiles a
 // CTA works on in a row share their Q operand (the activation rows of a Dense layer).
-__device__ __forceinline__ TileCoord tile_coord(const TcArgs& a, int64_t t) {
+__device__ __forceinline__ TileCoord tile_coord(const TcArgs& a, int t) {
   TileCoord c;
   const uint32_t per_batch = (uint32_t)a.tiles_p * (uint32_t)a.tiles_q;
-  c.batch = t / per_batch;
-  const uint32_t t2 = (uint32_t)(t - c.batch * per_batch);
+  c.batch = (uint32_t)t < per_batch ? 0 : (int)((uint32_t)t / per_batch);     // a Dense layer is one batch
+  const uint32_t t2 = (uint32_t)t - (uint32_t)c.batch * per_batch;
   c.q0 = (int)(t2 / (uint32_t)a.tiles_p) * a.BN;
   c.p0 = (int)(t2 % (uint32_t)a.tiles_p) * BM;
-  c.bo = (int)(c.batch / a.batches_inner);
-  c.bi = (int)(c.batch - (int64_t)c.bo * a.batches_inner);
+  c.bo = c.batch == 0 ? 0 : c.batch / a.batches_inner;
+  c.bi = c.batch - c.bo * a.batches_inner;
   return c;
 }
 
 // Walks a contiguous range of tiles without divisions: p-block fastest, then q-block, then batch.
 struct TileIter {
   int p, q, bi, bo;       // block indices
-  long long batch;
-  __device__ __forceinline__ void init(const TcArgs& a, int64_t t) {
+  int batch;
+  __device__ __forceinline__ void init(const TcArgs& a, int t) {
     const TileCoord c = tile_coord(a, t);
     p = c.p0 / BM; q = c.q0 / a.BN; bi = c.bi; bo = c.bo; batch = c.batch;
   }
@@ -138,7 +139,7 @@ struct TileIter {
       if (++q == a.tiles_q) {
         q = 0;
         ++batch;
-        if (++bi == (int)a.batches_inner) { bi = 0; ++bo; }
+        if (++bi == a.batches_inner) { bi = 0; ++bo; }
       }
     }
   }
@@ -169,7 +170,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gen_base = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t stage_bytes = BM * BK + (a.q_resident ? 0 : a.q_stage_bytes);
-  const int kblocks = (int)((a.K + BK - 1) / BK);
+  const int kblocks = (a.K + BK - 1) / BK;
   const uint32_t qres_bytes = a.q_resident ? kblocks * a.q_stage_bytes : 0;
   const uint32_t qres = base + a.stages * stage_bytes;         // resident Q tile: kblocks x [BN rows x 128 B]
   const uint32_t stage_out = qres + qres_bytes;                // output slots: 2 x [32 rows][32 channels] int8 per epilogue warp
@@ -187,7 +188,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // this CTA's contiguous range of tiles
-  const int64_t t_begin = a.total_tiles * blockIdx.x / gridDim.x, t_end = a.total_tiles * (blockIdx.x + 1) / gridDim.x;
+  const int t_begin = (int)blockIdx.x * a.tiles_each + min((int)blockIdx.x, a.tiles_extra);
+  const int t_end = t_begin + a.tiles_each + ((int)blockIdx.x < a.tiles_extra ? 1 : 0);
 
   // set-up, spread over the epilogue threads: one barrier (or descriptor prefetch) each
   {
@@ -232,7 +234,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
   if (ROP == 1 && warp >= kFirstEpiWarp) {
     // I-LayerNorm constants of all channels into shared memory: parameters, read before the wait for the previous
     // kernel.  The form (fast / general, see LnConsts) is agreed on by all epilogue threads.
-    const int et0 = (int)threadIdx.x - 32 * kFirstEpiWarp, nwords = (int)(a.P >> 2);
+    const int et0 = (int)threadIdx.x - 32 * kFirstEpiWarp, nwords = a.P >> 2;
     int4* sm_m = reinterpret_cast<int4*>(rop_smem);
     if (!ln_stage_consts(a.rop.gs, a.rop.beta, nwords, a.rop.vec, sm_m, sm_m + nwords, sm_m + 2 * nwords, et0, kEpiThreads))
       atomicAnd(const_cast<uint32_t*>(rop_flag), 0u);
@@ -266,7 +268,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         }
       }
       pdl_wait();
-      for (int64_t t = t_begin; ok && t < t_end; ++t, ++pit, ti.next(a)) {
+      for (int t = t_begin; ok && t < t_end; ++t, ++pit, ti.next(a)) {
         const int p0 = ti.p0(), q0 = ti.q0(a);
         const int pc1 = pr == 1 ? p0 : (pbi == 1 ? ti.bi : ti.bo), pc2 = pr == 2 ? p0 : (pbi == 2 ? ti.bi : ti.bo),
                   pc3 = pr == 3 ? p0 : (pbi == 3 ? ti.bi : ti.bo);
@@ -314,12 +316,15 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       const uint32_t q_kstep16 = (!a.q_mn ? UMMA_K : UMMA_K * a.q_row_bytes) >> 4;
       const int k_tail = (int)(a.K - (int64_t)(kblocks - 1) * BK);            // bytes of K in the last k-block
       const int tail_steps = k_tail >= BK ? BK / UMMA_K : (k_tail + UMMA_K - 1) / UMMA_K;
+      // descriptor low words: the start-address field counts 16-byte units, so stages and k-blocks are plain adds
+      const uint32_t p_lo0 = desc_lo(base, 16), q_lo0 = desc_lo(qres, 16);
+      const uint32_t stage16 = stage_bytes >> 4, qstage16 = (uint32_t)a.q_stage_bytes >> 4;
       int consumed = 0, s = 0, wrap = 0, it = 0;
       bool ok = true;
       int cur_q = -1;
       TileIter ti;
       ti.init(a, t_begin);
-      for (int64_t t = t_begin; ok && t < t_end; ++t, ++it) {
+      for (int t = t_begin; ok && t < t_end; ++t, ++it) {
         const int buf = it & 1;
         bool last_of_q = false;
         if (a.q_resident) {
@@ -335,13 +340,18 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!mbar_wait(full0 + 8 * s, wrap & 1, a.status)) { ok = false; break; }
           tc_fence_after();
-          const uint32_t sp = base + s * stage_bytes, sq = a.q_resident ? qres + kb * a.q_stage_bytes : sp + BM * BK;
-          uint32_t p_lo = desc_lo(sp, 16), q_lo = desc_lo(sq, 16);
-          const int ksteps = kb == kblocks - 1 ? tail_steps : BK / UMMA_K;
-          for (int k = 0; k < ksteps; ++k) {
-            umma_i8_lohi(d_tmem, p_lo, p_hi, q_lo, q_hi, idesc, (kb | k) != 0);
-            p_lo += UMMA_K >> 4;
-            q_lo += q_kstep16;
+          // low descriptor words of this stage's P tile and of the Q tile (resident, or behind P in the stage)
+          const uint32_t p_lo = p_lo0 + (uint32_t)s * stage16;
+          const uint32_t q_lo = a.q_resident ? q_lo0 + (uint32_t)kb * qstage16 : p_lo + ((BM * BK) >> 4);
+          if (kb != kblocks - 1 || tail_steps == BK / UMMA_K) {
+            umma_i8_x4(d_tmem, p_lo, p_hi, q_lo, q_hi, idesc, kb != 0, UMMA_K >> 4, q_kstep16);
+          } else {
+            uint32_t pl = p_lo, ql = q_lo;
+            for (int k = 0; k < tail_steps; ++k) {
+              umma_i8_lohi(d_tmem, pl, p_hi, ql, q_hi, idesc, (kb | k) != 0);
+              pl += UMMA_K >> 4;
+              ql += q_kstep16;
+            }
           }
           umma_commit(empty0 + 8 * s);   // the stage may be refilled once these MMAs have read it
           ++consumed;
@@ -395,7 +405,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         if (e.bias) nb = __ldg(e.bias + c);
       }
     };
-    if (dense && t_begin < t_end) fetch_channel(tile_coord(a, t_begin).p0);
+    // the first tile's coordinates, computed once (they cost integer divisions)
+    TileIter ti_first;
+    ti_first.init(a, t_begin);
+    if (dense && t_begin < t_end) fetch_channel(ti_first.p0());
     // MatMul orientation: one per-tensor constant set
     const int um = e.scale.mult, us = clamp_shift(e.scale.shift);
     const long long uc = 1ll << (us - 1);
@@ -411,13 +424,13 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     uint32_t rpar = 0, rpend = 0;       // per residual slot (bit 0 / 1): parity of its next arrival; a fetch in flight
     // the warp's chunk sequence two chunks ahead: tile by tile, chunks part, part + kParts, ...
     TileIter pf_ti;
-    int64_t pf_t = t_begin;
+    int pf_t = t_begin;
     int pf_ck = part;
     uint32_t pf_g = 0;
     auto pf_settle = [&]() {
       while (pf_t < t_end) {
-        const int64_t left = a.Q - pf_ti.q0(a);
-        const int nck = (int)((left < a.BN ? left : a.BN) + 31) >> 5;
+        const int left = a.Q - pf_ti.q0(a);
+        const int nck = ((left < a.BN ? left : a.BN) + 31) >> 5;
         if (pf_ck < nck) break;
         pf_ti.next(a);
         ++pf_t;
@@ -442,7 +455,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       }
     };
     if (tma_res && t_begin < t_end) {
-      pf_ti.init(a, t_begin);
+      pf_ti = ti_first;
       pf_settle();
       pf_fetch();
       pf_fetch();
@@ -450,9 +463,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
 
     int it = 0;
     int tiles_in_q = 0;   // ROP: tiles of the current block of output rows that this CTA has finished
-    TileIter ti;
-    ti.init(a, t_begin);
-    for (int64_t t = t_begin; t < t_end; ++t, ++it) {
+    TileIter ti = ti_first;
+    for (int t = t_begin; t < t_end; ++t, ++it) {
       TileCoord tc;
       tc.batch = ti.batch; tc.bo = ti.bo; tc.bi = ti.bi; tc.p0 = ti.p0(); tc.q0 = ti.q0(a);
       ti.next(a);   // ti now describes the next tile
@@ -470,8 +482,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       if (ok) ok = mbar_wait(accf0 + 8 * buf, (it >> 1) & 1, a.status);
       tc_fence_after();
       const uint32_t t_row = tmem_base + ((uint32_t)(qd * 32) << 16) + (uint32_t)(buf * a.BN);
-      const int64_t cols_left = a.Q - tc.q0;
-      const int nck = (int)((cols_left < a.BN ? cols_left : a.BN) + 31) >> 5;   // chunks that hold output
+      const int cols_left = a.Q - tc.q0;
+      const int nck = ((cols_left < a.BN ? cols_left : a.BN) + 31) >> 5;   // chunks that hold output
 
       if (dense) {
         // lane = output channel c, TMEM column = output row
@@ -488,8 +500,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         // that hides the latencies of the shuffles, the shared-memory traffic and the barrier operations.
         auto half = [&](int (&v)[16], int ck, int h, uint8_t* pe) {
           const int j0 = ck * 32 + h * 16;
-          const int64_t r0 = (int64_t)tc.q0 + j0;
-          const int nrow = (int)min((int64_t)16, a.Q - r0);
+          const int r0 = tc.q0 + j0;
+          const int nrow = min(16, a.Q - r0);
           if (hi_only) {
 #pragma unroll
             for (int j = 0; j < 16; ++j) v[j] = mad_hi(v[j] + cbias, cm, rnd_hi) >> sh_hi;
@@ -526,7 +538,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
           if (out_i32) {
 #pragma unroll
             for (int j = 0; j < 16; ++j)
-              if (j < nrow && c_ok) reinterpret_cast<int32_t*>(e.out)[(r0 + j) * e.ldo + c] = v[j];
+              if (j < nrow && c_ok) reinterpret_cast<int32_t*>(e.out)[(int64_t)(r0 + j) * e.ldo + c] = v[j];
             return;
           }
           if (act) {
@@ -553,7 +565,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
             for (int k = 0; k < 4; ++k) *reinterpret_cast<uint32_t*>(pe + 512 * h + 128 * k) = w[k];
           } else {
             // direct stores (grouped output rows): this lane's first word is row r0 + li, then + 4 per word
-            int64_t row = r0 + li, ro = row, grem = 0;
+            int64_t row = (int64_t)r0 + li, ro = row, grem = 0;
             if (e.group_rows > 0) {
               grem = (int64_t)((uint64_t)row % (uint64_t)e.group_rows);
               ro = (int64_t)((uint64_t)row / (uint64_t)e.group_rows) * e.group_stride + grem;
@@ -604,17 +616,17 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         }
       } else {
         // lane = output row, TMEM column = output column
-        const int64_t r = (int64_t)tc.p0 + qd * 32 + lane;
+        const int r = tc.p0 + qd * 32 + lane;
         const bool row_ok = r < a.P;
-        const int64_t out_row = tc.bo * a.sCo + tc.bi * a.sCi + r * e.ldo;
-        const int32_t* bias_row = e.bias32 ? e.bias32 + ((tc.batch % e.bias_batches) * a.P + r) * e.ldbias : nullptr;
+        const int64_t out_row = tc.bo * a.sCo + tc.bi * a.sCi + (int64_t)r * e.ldo;
+        const int32_t* bias_row = e.bias32 ? e.bias32 + ((tc.batch % e.bias_batches) * (int64_t)a.P + r) * e.ldbias : nullptr;
         for (int ck = part; ck < nck; ck += kParts) {
           const int j0 = ck * 32;
           const int c0 = tc.q0 + j0;
           int v[32];
           tmem_ld32(t_row + (uint32_t)j0, v);
           if (!row_ok) continue;
-          const int ncol = (int)min((int64_t)32, a.Q - c0);
+          const int ncol = min(32, a.Q - c0);
           if (bias_row) {
 #pragma unroll
             for (int j = 0; j < 32; ++j)
@@ -677,16 +689,16 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       const unsigned spb = (unsigned)(a.BN + kSlice - 1) / kSlice;   // slices per row block
       const unsigned total = (unsigned)a.tiles_q * spb;
       const unsigned nwarps = gridDim.x * kEpiWarps;
-      const int C = (int)a.P;
+      const int C = a.P;
       const int nwords = C >> 2;
       const int4* sm_m = reinterpret_cast<const int4*>(rop_smem);
       const LnConsts lk{sm_m, sm_m + nwords, sm_m + 2 * nwords, *rop_flag != 0u};
       unsigned* tab = reinterpret_cast<unsigned*>(rop_smem) + ew * (kGeluTailRows * 64);
       for (unsigned sl = (unsigned)ew * gridDim.x + blockIdx.x; sl < total; sl += nwarps) {
         const unsigned blk = sl / spb, j = sl - blk * spb;
-        const int64_t q0 = (int64_t)blk * a.BN;
-        const int64_t left = a.Q - q0;
-        const int in_blk = (int)(left < a.BN ? left : a.BN);
+        const int q0 = (int)blk * a.BN;
+        const int left = a.Q - q0;
+        const int in_blk = left < a.BN ? left : a.BN;
         const int r0 = (int)j * kSlice;
         if (r0 >= in_blk) continue;
         unsigned rdy = 0;
@@ -708,9 +720,9 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         rdy = __shfl_sync(0xffffffffu, rdy, 0);
         if (!rdy) break;
         const int nrows = in_blk - r0 < kSlice ? in_blk - r0 : kSlice;
-        int8_t* rows0 = reinterpret_cast<int8_t*>(e.out) + (q0 + r0) * e.ldo;
+        int8_t* rows0 = reinterpret_cast<int8_t*>(e.out) + (int64_t)(q0 + r0) * e.ldo;
         if (ROP == 1) {
-          int8_t* dst = a.rop.ln_out + (q0 + r0) * a.rop.ld_ln;
+          int8_t* dst = a.rop.ln_out + (int64_t)(q0 + r0) * a.rop.ld_ln;
           if (C <= 384) {
             layernorm_rows<3, 8, true>(rows0, e.ldo, nrows, C, a.rop.M_ln, a.rop.mean_magic, lk, dst, a.rop.ld_ln, lane);
           } else if (C <= 512) {
@@ -815,13 +827,13 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
   if (!ctx->tmap_encode) return IVIT_ERR_UNSUPPORTED;
   const int64_t batches = g.batches_outer * g.batches_inner;
   if (batches == 0 || g.M == 0 || g.N == 0) return IVIT_OK;
-  if (g.M > 2147483647LL || g.N > 2147483647LL || g.K > 65536 || batches > 2147483647LL) return IVIT_ERR_UNSUPPORTED;
+  if (g.M > 2147483647LL - 512 || g.N > 2147483647LL - 512 || g.K > 65536 || batches > 2147483647LL) return IVIT_ERR_UNSUPPORTED;
   const GemmEpilogue& e = g.epi;
   if (g.lda % 16 || g.ldb % 16 || g.sAo % 16 || g.sAi % 16 || g.sBo % 16 || g.sBi % 16) return IVIT_ERR_UNSUPPORTED;
 
   TcArgs a{};
   a.epi = e;
-  a.K = g.K; a.sCo = g.sCo; a.sCi = g.sCi; a.batches_inner = g.batches_inner;
+  a.K = (int)g.K; a.sCo = g.sCo; a.sCi = g.sCi; a.batches_inner = (int)g.batches_inner;
   a.status = ctx->status_dev;
   CUtensorMap tmP, tmQ;
   const bool dense = g.transB && batches == 1 && !e.bias32;
@@ -829,7 +841,7 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
     if (g.N % 4 || e.ldo % 4 || (reinterpret_cast<uintptr_t>(e.out) & 3)) return IVIT_ERR_UNSUPPORTED;
     // Dense orientation: lanes = output channels (rows of W), columns = output rows (rows of A)
     a.lanes_are_channels = 1;
-    a.P = g.N; a.Q = g.M;
+    a.P = (int)g.N; a.Q = (int)g.M;
     a.tiles_p = (int)((a.P + BM - 1) / BM);
     a.BN = pick_bn(a.Q, a.tiles_p, g.K, ctx->sm_count);
     a.q_stage_bytes = a.BN * BK;
@@ -840,7 +852,7 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
     // MatMul orientation: lanes = rows of A; the epilogue's 16-byte stores need aligned output rows
     if (e.out_dtype != IVIT_I8 || e.bias || e.res || e.scale.mult_c || e.group_rows > 0 || e.act_table) return IVIT_ERR_UNSUPPORTED;
     if ((reinterpret_cast<uintptr_t>(e.out) & 15) || e.ldo % 16 || g.sCo % 16 || g.sCi % 16) return IVIT_ERR_UNSUPPORTED;
-    a.P = g.M; a.Q = g.N;
+    a.P = (int)g.M; a.Q = (int)g.N;
     a.tiles_p = (int)((a.P + BM - 1) / BM);
     a.q_mn = g.transB ? 0 : 1;
     if (!make_tensor_map(ctx, &tmP, g.A, g.K, g.M, g.batches_inner, g.batches_outer, g.lda, g.sAi, g.sAo, BK, BM,
@@ -904,10 +916,14 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
   if (a.stages < 2) return IVIT_ERR_UNSUPPORTED;
   a.tmem_cols = pow2_at_least(2 * a.BN);
   a.tiles_q = (int)((a.Q + a.BN - 1) / a.BN);
-  a.total_tiles = (int64_t)a.tiles_p * a.tiles_q * batches;
+  const int64_t total_tiles = (int64_t)a.tiles_p * a.tiles_q * batches;
+  if (total_tiles > 2147483647LL) return IVIT_ERR_UNSUPPORTED;
+  a.total_tiles = (int)total_tiles;
 
   const size_t smem = kSmemFixed + rop_bytes + (size_t)a.stages * stage + fixed;
   const unsigned grid = (unsigned)(a.total_tiles < ctx->sm_count ? a.total_tiles : ctx->sm_count);
+  a.tiles_each = a.total_tiles / (int)grid;
+  a.tiles_extra = a.total_tiles % (int)grid;
   LaunchScope ls(ctx, KIND_GEMM_TC, 2.0 * (double)batches * (double)g.M * (double)g.N * (double)g.K);
   // the encoder block's Dense layers take the specialised instantiations
   int mode = (a.lanes_are_channels && a.tma_out && (!e.res || a.tma_res)) ? (a.tma_res ? 2 : 1) : 0;

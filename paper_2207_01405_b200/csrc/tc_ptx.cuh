@@ -118,6 +118,37 @@ __device__ __forceinline__ void umma_i8_lohi(uint32_t d_tmem, uint32_t a_lo, uin
       "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %5, p;\n\t}"
       ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
 }
+// Four MMAs of one 128-byte k-block in one go: the descriptors advance along K by a_step / b_step (units of 16
+// bytes, added to the low words); the first MMA accumulates only if `accumulate`, the others always.  The issuing
+// thread shares its scheduler with busy epilogue warps, so every instruction it saves shortens the time until the
+// tensor core has its work.
+__device__ __forceinline__ void umma_i8_x4(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                           uint32_t idesc, uint32_t accumulate, uint32_t a_step, uint32_t b_step) {
+  asm volatile(
+      "{\n\t.reg .pred p, pt;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "setp.eq.b32 pt, 0, 0;\n\t"
+      "mov.b64 da, {%1, %2};\n\t"
+      "mov.b64 db, {%3, %4};\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %5, p;\n\t"
+      "add.u32 al, %1, %7;\n\t"
+      "add.u32 bl, %3, %8;\n\t"
+      "mov.b64 da, {al, %2};\n\t"
+      "mov.b64 db, {bl, %4};\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %5, pt;\n\t"
+      "add.u32 al, al, %7;\n\t"
+      "add.u32 bl, bl, %8;\n\t"
+      "mov.b64 da, {al, %2};\n\t"
+      "mov.b64 db, {bl, %4};\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %5, pt;\n\t"
+      "add.u32 al, al, %7;\n\t"
+      "add.u32 bl, bl, %8;\n\t"
+      "mov.b64 da, {al, %2};\n\t"
+      "mov.b64 db, {bl, %4};\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %5, pt;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate), "r"(a_step), "r"(b_step)
+      : "memory");
+}
 // Low / high words of a shared-memory matrix descriptor (see smem_desc).
 __device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
   return ((addr >> 4) & 0x3FFF) | (((lbo_bytes >> 4) & 0x3FFF) << 16);
