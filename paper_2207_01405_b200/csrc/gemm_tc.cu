@@ -801,7 +801,9 @@ int pick_bn(int64_t extent, int64_t tiles_other, int64_t K, int sm_count) {
     const int64_t tiles = tiles_other * ((extent + bn - 1) / bn);
     const double rounds = (double)((tiles + sm_count - 1) / sm_count);
     const double feed = (double)K * (128.0 + bn) / 46.0;
-    const double epilogue = 2000.0 * ((bn + 127) / 128);
+    // the epilogue works in rounds of four 32-row chunks; the small term in bn makes the narrower of two tiles
+    // with the same number of rounds win (its MMAs, loads and stores are shorter)
+    const double epilogue = 2000.0 * ((bn + 127) / 128) + 3.0 * bn;
     const double cost = rounds * ((feed > epilogue ? feed : epilogue) + 1200.0);
     if (!best || cost < best_cost) { best = bn; best_cost = cost; }
   }
