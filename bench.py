@@ -504,7 +504,12 @@ def run_gpu(args):
     ctx.set_stream(side)
 
     # every rank serves its own batch of the same synthetic workload (weak scaling, no exchange step)
-    model, image = make_config(CONFIG_INDEX)
+    from ivit_inputs.gen import CONFIGS
+    model, image = make_config(args.config)
+    workload = CONFIGS[args.config]["name"]
+    metric = METRIC if args.config == CONFIG_INDEX else f"int-only ViT images/s ({workload})"
+    if args.config != CONFIG_INDEX:
+        args.headline_only = True
     dm = binding.DeviceVit(model, dev)
     B = model.B
     ws = dm.host_workspace()
@@ -548,7 +553,8 @@ def run_gpu(args):
     except Exception as exc:   # noqa: BLE001
         print(f"graph capture unavailable ({exc}); timing stream launches", file=sys.stderr)
     t_begin = time.time()
-    ms_total, repeats = time_loop(torch, step_timed, args.steps, flush, barrier, MIN_TIMED_SECONDS)
+    min_s = 0.0 if args.headline_only else MIN_TIMED_SECONDS
+    ms_total, repeats = time_loop(torch, step_timed, args.steps, flush, barrier, min_s)
     t_end = time.time()
     launches = launches_per_step * args.steps
     clocks = sampler.stop(t_begin, t_end)
@@ -559,7 +565,7 @@ def run_gpu(args):
     for _ in range(8):
         step_e2e()
     torch.cuda.synchronize()
-    ms_e2e, _ = time_loop(torch, step_e2e, args.steps, flush, barrier, MIN_TIMED_SECONDS / 2)
+    ms_e2e, _ = time_loop(torch, step_e2e, args.steps, flush, barrier, min_s / 2)
     ctx.set_host_graph(False)
     status = ctx.poll_status()
     if status != 0:
@@ -617,7 +623,8 @@ def run_gpu(args):
         achieved = dk["work"] / (dk["ms"] * 1e-3) / 1e12
         in_step = dk["work"] / prof_steps / (ms_total / args.steps * 1e-3 * dk["ms"] / total_kernel_ms) / 1e12
         roofline = {"kernel": dom, "bound": "tensor", "achieved": round(achieved, 2), "peak": int8_peak, "unit": "TOP/s",
-                    "frac": round(achieved / int8_peak, 4), "traffic": GEMM_DRAM_BYTES_PER_LAUNCH,
+                    "frac": round(achieved / int8_peak, 4),
+                    "traffic": GEMM_DRAM_BYTES_PER_LAUNCH if args.config == CONFIG_INDEX else None,
                     # the event pair around every launch costs a few microseconds and stops the overlap of one kernel's
                     # set-up with its predecessor's tail; the same work over (un-bracketed step time x this kernel's share)
                     "achieved_in_step": round(in_step, 2),
@@ -629,52 +636,62 @@ def run_gpu(args):
         roofline = {"kernel": dom, "bound": "hbm", "achieved": round(achieved, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": round(achieved / peaks["hbm_gbs"], 4), "traffic": None, "peak_source": f"{peak_src} copy bandwidth"}
 
-    probe = gemm_probe(ctx, binding, peaks, dev)
-    for pr in probe:
-        pr["frac_of_mma_issue_probe"] = round(pr["TOPS"] / int8_probe, 4)
-    # the same forward with the static-maximum ShiftGELU variant (a different function from the paper's Algorithm 2,
-    # applied inside the FC1 epilogue): reported beside the headline, never as the headline
-    import copy
-    vmodel = copy.copy(model)
-    vmodel.blocks = [copy.copy(b) for b in model.blocks]
-    for b in vmodel.blocks:
-        b.gelu_static_max = True
-    vdm = binding.DeviceVit(vmodel, dev)
-    for _ in range(3):
-        ctx.vit_forward(vdm, d_image, logits=d_logits, workspace=ws)
-    vsteps = min(args.steps, 50)
-    ms_variant, _ = time_loop(torch, lambda: ctx.vit_forward(vdm, d_image, logits=d_logits, workspace=ws), vsteps, flush, barrier, 0.0)
-    variant = {"images_per_s": round(B * vsteps / (ms_variant * 1e-3), 1),
-               "note": "ShiftGELU with I_max fixed at I_p(127), fused into the FC1 epilogue; not Algorithm 2"}
-    del vdm
-    # the same forward with LayerNorm / ShiftGELU run inside the Dense kernels that produce their rows (off by default)
-    ctx.set_row_fusion(True)
-    l0 = ctx.launch_count()
-    for _ in range(3):
-        step_resident()
-    fused_launches = (ctx.launch_count() - l0) // 3
-    ms_fused, _ = time_loop(torch, step_resident, vsteps, flush, barrier, 0.0)
-    ctx.set_row_fusion(False)
-    fused = {"images_per_s": round(B * vsteps / (ms_fused * 1e-3), 1), "kernels_per_forward": int(fused_launches),
-             "note": "ivit_ctx_set_row_fusion(1): same bytes, row operators inside the Dense kernels; stream launches"}
-    in_flight = two_in_flight(binding, model, image, dev, dm, min(args.steps, 100))
-    cpu_rate, cpu_n, cpu_s, cpu_threads = time_oracle(model, image)
-    # the timed steps really computed the forward: spot-check one image against the oracle
-    from oracle import api as O
-    ok = bool(np.array_equal(h_logits[:1].numpy(), O.vit_forward(model, image[:1])))
-    ops_standalone = standalone_ops(ctx, binding, torch, np, peaks, dev)
-    configs = other_configs(ctx, binding, torch, np, flush, dev)
-    b8 = batch8_latencies(ctx, binding, torch, flush, dev)
+    extras = {}
+    if not args.headline_only:
+        probe = gemm_probe(ctx, binding, peaks, dev)
+        for pr in probe:
+            pr["frac_of_mma_issue_probe"] = round(pr["TOPS"] / int8_probe, 4)
+        # the same forward with the static-maximum ShiftGELU variant (a different function from the paper's Algorithm 2,
+        # applied inside the FC1 epilogue): reported beside the headline, never as the headline
+        import copy
+        vmodel = copy.copy(model)
+        vmodel.blocks = [copy.copy(b) for b in model.blocks]
+        for b in vmodel.blocks:
+            b.gelu_static_max = True
+        vdm = binding.DeviceVit(vmodel, dev)
+        for _ in range(3):
+            ctx.vit_forward(vdm, d_image, logits=d_logits, workspace=ws)
+        vsteps = min(args.steps, 50)
+        ms_variant, _ = time_loop(torch, lambda: ctx.vit_forward(vdm, d_image, logits=d_logits, workspace=ws), vsteps, flush, barrier, 0.0)
+        variant = {"images_per_s": round(B * vsteps / (ms_variant * 1e-3), 1),
+                   "note": "ShiftGELU with I_max fixed at I_p(127), fused into the FC1 epilogue; not Algorithm 2"}
+        del vdm
+        # the same forward with LayerNorm / ShiftGELU run inside the Dense kernels that produce their rows (off by default)
+        ctx.set_row_fusion(True)
+        l0 = ctx.launch_count()
+        for _ in range(3):
+            step_resident()
+        fused_launches = (ctx.launch_count() - l0) // 3
+        ms_fused, _ = time_loop(torch, step_resident, vsteps, flush, barrier, 0.0)
+        ctx.set_row_fusion(False)
+        fused = {"images_per_s": round(B * vsteps / (ms_fused * 1e-3), 1), "kernels_per_forward": int(fused_launches),
+                 "note": "ivit_ctx_set_row_fusion(1): same bytes, row operators inside the Dense kernels; stream launches"}
+        in_flight = two_in_flight(binding, model, image, dev, dm, min(args.steps, 100))
+        cpu_rate, cpu_n, cpu_s, cpu_threads = time_oracle(model, image)
+        # the timed steps really computed the forward: spot-check one image against the oracle
+        from oracle import api as O
+        ok = bool(np.array_equal(h_logits[:1].numpy(), O.vit_forward(model, image[:1])))
+        ops_standalone = standalone_ops(ctx, binding, torch, np, peaks, dev)
+        configs = other_configs(ctx, binding, torch, np, flush, dev)
+        b8 = batch8_latencies(ctx, binding, torch, flush, dev)
+        extras = {
+            "gemm_probe": probe, "static_gelu_variant": variant, "row_fusion_variant": fused, "two_forwards_in_flight": in_flight,
+            "cpu_baseline": {"value": cpu_rate, "unit": "images/s", "cores": cpu_threads, "kind": "oracle",
+                             "sample": f"{cpu_n} of {B} images ({cpu_s:.1f} s; images are independent)"},
+            "nonlinear_standalone": {k: v for k, v in ops_standalone.items() if k not in ("linear_qkv", "matmul_qk")},
+            "per_op_gpu_vs_oracle": {k: v for k, v in ops_standalone.items() if k in ("linear_qkv", "matmul_qk")},
+            "configs": configs, "batch8_latency_ms": b8, "parity_spot_check": ok,
+        }
     status = ctx.poll_status()
     if status != 0:
         raise RuntimeError(f"device-side error {status}")
 
     ops = vit_int8_ops(model)
     line = {
-        "metric": METRIC, "value": whole_job_rate(B, world, args.steps, ms_total), "unit": "images/s", "n_gpus": world, "steps": args.steps,
+        "metric": metric, "value": whole_job_rate(B, world, args.steps, ms_total), "unit": "images/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_total / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int8 x int8 -> int32",
-        "data": "synthetic", "config": {"workload": WORKLOAD, "batch_per_gpu": B, "tokens": model.T, "embed": model.D,
+        "data": "synthetic", "config": {"workload": workload, "batch_per_gpu": B, "tokens": model.T, "embed": model.D,
                                         "heads": model.heads, "mlp": model.H, "blocks": model.depth,
                                         "l2": "256 MB buffer written between steps, outside the per-step event pairs",
                                         "timed_region": f"the {args.steps}-step loop repeated {repeats} times "
@@ -686,25 +703,15 @@ def run_gpu(args):
         "gpu_launches": int(launches),
         "clocks": clocks,
         "roofline": roofline,
-        "cpu_baseline": {"value": cpu_rate, "unit": "images/s", "cores": cpu_threads, "kind": "oracle",
-                         "sample": f"{cpu_n} of {B} images ({cpu_s:.1f} s; images are independent)"},
         "launch": {"mode": launch_mode, "kernels_per_forward": int(launches_per_step),
                    "stream_launch_images_per_s": round(B * world * min(args.steps, 50) / (ms_eager * 1e-3), 1)},
         "int8_peak_probe": {"TOPS": round(int8_probe, 1), "ms": round(probe_ms, 4),
                             "what": "tcgen05.mma.kind::i8 M128 N256 K32, issue-only, operands fixed in shared memory, one CTA per SM",
                             "spec_TOPS": 4500.0, "twice_bf16_sustained": int8_peak, "twice_bf16_burst": 2.0 * peaks["bf16_tflops"]},
-        "gemm_probe": probe,
-        "static_gelu_variant": variant,
-        "row_fusion_variant": fused,
-        "two_forwards_in_flight": in_flight,
         "int8_tops_whole_step": round(ops / (ms_total / args.steps * 1e-3) / 1e12, 2),
         "kernels": kernels,
-        "nonlinear_standalone": {k: v for k, v in ops_standalone.items() if k in ("layernorm", "shiftmax", "shiftgelu", "l2_bytes", "shapes", "hbm_peak_gbs_measured", "hbm_peak_gbs_spec")},
-        "per_op_gpu_vs_oracle": {k: v for k, v in ops_standalone.items() if k in ("linear_qkv", "matmul_qk")},
-        "configs": configs,
-        "batch8_latency_ms": b8,
-        "parity_spot_check": ok,
     }
+    line.update(extras)
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -717,6 +724,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ivit", choices=["ivit", "reference"])
     ap.add_argument("--detail", action="store_true", help="print per-shape kernel times to stderr")
+    ap.add_argument("--config", type=int, default=CONFIG_INDEX, choices=[1, 2, 4],
+                    help="ViT-family configuration to time (default 1, the headline; 2 and 4 print the same line for that workload, without the extra sections)")
+    ap.add_argument("--headline-only", action="store_true",
+                    help="time the headline workload only (K steps once, no extra sections): the command the ncu captures run")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
