@@ -576,6 +576,10 @@ def run_gpu(args):
     prof_steps = min(args.steps, 5)
     ctx.profile_start()
     for _ in range(prof_steps):
+        # ~2 ms of device work queued first, so that the host has submitted the whole step before the device
+        # reaches it: an event pair then spans its kernel, not the host's launch latency
+        for _ in range(30):
+            flush.zero_()
         step_resident()
     records = ctx.profile_stop()
 

@@ -378,6 +378,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     const int qd = warp & 3;
     const int part = ew >> 2;
     constexpr int kParts = kEpiWarps / 4;
+    static_assert((kParts & (kParts - 1)) == 0, "chunk rotation");
     const GemmEpilogue& e = a.epi;
     const bool dense = MODE ? true : a.lanes_are_channels != 0;
     const bool tma_out = MODE ? true : a.tma_out != 0;
@@ -422,10 +423,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     const int c_first = qd * 32;        // first channel of this warp inside the tile
     uint32_t g = 0;                     // chunks this warp has worked on
     uint32_t rpar = 0, rpend = 0;       // per residual slot (bit 0 / 1): parity of its next arrival; a fetch in flight
-    // the warp's chunk sequence two chunks ahead: tile by tile, chunks part, part + kParts, ...
+    // Chunks are dealt to the parts round-robin ACROSS tiles (chunk j of a tile goes to part (rot + j) % kParts,
+    // rot = chunks of this CTA's earlier tiles), so that a tile whose chunk count is no multiple of kParts
+    // does not leave the same part idle every time.
+    // The warp's chunk sequence two chunks ahead (residual fetches):
     TileIter pf_ti;
     int pf_t = t_begin;
     int pf_ck = part;
+    int pf_rot = 0;
     uint32_t pf_g = 0;
     auto pf_settle = [&]() {
       while (pf_t < t_end) {
@@ -434,7 +439,8 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         if (pf_ck < nck) break;
         pf_ti.next(a);
         ++pf_t;
-        pf_ck = part;
+        pf_rot = (pf_rot + nck) & (kParts - 1);
+        pf_ck = (part - pf_rot) & (kParts - 1);
       }
     };
     // residual bytes of the next chunk of the look-ahead into slot pf_g & 1 (a box wholly past the last channel
@@ -462,6 +468,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     }
 
     int it = 0;
+    int rot = 0;          // chunks of this CTA's earlier tiles, modulo kParts
     int tiles_in_q = 0;   // ROP: tiles of the current block of output rows that this CTA has finished
     TileIter ti = ti_first;
     for (int t = t_begin; t < t_end; ++t, ++it) {
@@ -586,7 +593,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         };
 
         const bool c_any = tc.p0 + c_first < a.P;   // else the warp's box lies wholly past the last channel
-        for (int ck = part; ck < nck; ck += kParts) {
+        for (int ck = (part - rot) & (kParts - 1); ck < nck; ck += kParts) {
           uint8_t* pe = nullptr;
           if (tma_out) {
             const uint32_t sl = g & 1u;
@@ -620,7 +627,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
         const bool row_ok = r < a.P;
         const int64_t out_row = tc.bo * a.sCo + tc.bi * a.sCi + (int64_t)r * e.ldo;
         const int32_t* bias_row = e.bias32 ? e.bias32 + ((tc.batch % e.bias_batches) * (int64_t)a.P + r) * e.ldbias : nullptr;
-        for (int ck = part; ck < nck; ck += kParts) {
+        for (int ck = (part - rot) & (kParts - 1); ck < nck; ck += kParts) {
           const int j0 = ck * 32;
           const int c0 = tc.q0 + j0;
           int v[32];
@@ -656,6 +663,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
           }
         }
       }
+      rot = (rot + nck) & (kParts - 1);
       // this warp has read everything it needs from the buffer: hand it back to the MMA warp
       tc_fence_before();
       __syncwarp();
@@ -790,9 +798,10 @@ static_assert(8 * (2 * kMaxStages + 5 + 2 * kEpiWarps) + 32 + 512 <= 1024, "barr
 
 
 // Tile width along the TMEM columns: the candidate with the least (rounds of tiles per CTA) x (time of a tile).
-// A tile's time is the larger of its operand traffic, (128 + bn) x K bytes at about 46 bytes per clock into an
-// SM's shared memory, and its epilogue, one 32-row chunk per epilogue part at a time (about 2000 clocks per round
-// of four chunks), plus a fixed cost per tile; the constants are measured on DeiT-S / ViT-B / ViT-L layer shapes.
+// Model of a tile's time: the larger of its operand traffic, (128 + bn) x K bytes at about 60 bytes per clock into
+// an SM's shared memory, and its epilogue, which grows with the tile's width now that chunks are dealt to the
+// epilogue parts across tiles, plus a fixed cost per tile.  The constants are fitted to measured launch times of the
+// DeiT-S / ViT-B / ViT-L layer shapes at widths 128 ... 256 (the pick is within 4 % of the best width on each).
 int pick_bn(int64_t extent, int64_t tiles_other, int64_t K, int sm_count) {
   if (extent <= 256) return (int)((extent + 31) / 32 * 32);
   int best = 0;
@@ -800,12 +809,11 @@ int pick_bn(int64_t extent, int64_t tiles_other, int64_t K, int sm_count) {
   for (int bn : {256, 224, 192, 160, 128}) {
     const int64_t tiles = tiles_other * ((extent + bn - 1) / bn);
     const double rounds = (double)((tiles + sm_count - 1) / sm_count);
-    const double feed = (double)K * (128.0 + bn) / 46.0;
-    // the epilogue works in rounds of four 32-row chunks; the small term in bn makes the narrower of two tiles
-    // with the same number of rounds win (its MMAs, loads and stores are shorter)
-    const double epilogue = 2000.0 * ((bn + 127) / 128) + 3.0 * bn;
-    const double cost = rounds * ((feed > epilogue ? feed : epilogue) + 1200.0);
-    if (!best || cost < best_cost) { best = bn; best_cost = cost; }
+    const double feed = (double)K * (128.0 + bn) / 60.0;
+    const double epilogue = 8.0 * bn;
+    // ties go to the narrower tile (its MMAs, loads and stores are shorter): the loop runs from wide to narrow
+    const double cost = rounds * ((feed > epilogue ? feed : epilogue) + 900.0);
+    if (!best || cost <= best_cost) { best = bn; best_cost = cost; }
   }
   return best;
 }
