@@ -388,6 +388,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     const int8_t* res_tab0 = res_tab + 128;   // entry of residual byte 0
     const int8_t* act_tab0 = res_tab + 256 + 128;   // entry of value 0 of the activation table
     const bool act = MODE == 3 ? true : (MODE ? false : e.act_table != nullptr);
+    constexpr bool kFrag = MODE == 1 || MODE == 3;
     if (act) {
       // the table may come from an earlier kernel of the stream: read it after the dependency wait above
       if (et < 256) res_tab[256 + et] = e.act_table[et];
@@ -484,6 +485,20 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       const int cbias = nb;
       const bool hi_only = __all_sync(0xffffffffu, cs >= 33 && nb > -(1 << 30) && nb < (1 << 30));
       const int rnd_hi = cs >= 33 ? 1 << (cs - 33) : 0;
+      // The kernels without a residual port (MODE 1, 3) read the accumulators as fragments (tmem_ld_frag16): thread l
+      // then works on the four channels (l >> 2) + 8 j of its warp, whose constants it takes from the lanes that
+      // fetched them.  (With the residual port the fragment form is slower: its byte look-ups lose more to bank
+      // conflicts than the transposes cost.)
+      int km[4], ks[4], kb[4];
+      if (kFrag) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int src = (lane >> 2) + 8 * j;
+          km[j] = __shfl_sync(0xffffffffu, cm, src);
+          ks[j] = __shfl_sync(0xffffffffu, cs, src);
+          kb[j] = __shfl_sync(0xffffffffu, cbias, src);
+        }
+      }
       if (dense && t + 1 < t_end) fetch_channel(ti.p0());
 
       if (ok) ok = mbar_wait(accf0 + 8 * buf, (it >> 1) & 1, a.status);
@@ -607,11 +622,61 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
             // after the transposes a lane holds 4 consecutive channels (lane >> 2) of slot row li + 4k
             pe = gen_base + (my_out - base) + sl * 1024 + li * 32 + (lane >> 2) * 4;
           }
-          int v[16];
-          tmem_ld16(t_row + (uint32_t)(32 * ck), v);
-          half(v, ck, 0, pe);
-          tmem_ld16(t_row + (uint32_t)(32 * ck + 16), v);
-          half(v, ck, 1, pe);
+          if constexpr (kFrag) {
+            // fragment form: 16 channels x 32 rows per step; the packed words are the fragment that one stmatrix
+            // stores transposed, i.e. as rows of 16 consecutive channels, into the [32 rows][32 channels] slot
+            const uint32_t out_slot = my_out + 1024u * (g & 1u) + (uint32_t)lane * 32u;
+            const uint8_t* res_slot = gen_base + (my_res - base) + (g & 1u) * 1024 + (2 * (lane & 3)) * 32 + (lane >> 2);
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              int v[16];
+              tmem_ld_frag16(t_row + ((uint32_t)(16 * h) << 16) + (uint32_t)(32 * ck), v);
+#pragma unroll
+              for (int u = 0; u < 2; ++u) {       // u = 0: channel (l >> 2) + 16 h, u = 1: eight channels on
+                const int m = km[2 * h + u], sft = ks[2 * h + u], bia = kb[2 * h + u];
+                if (hi_only) {
+                  const int add = 1 << (sft - 33), sh = sft - 32;
+#pragma unroll
+                  for (int i = 0; i < 4; ++i) {
+                    v[4 * i + 2 * u] = mad_hi(v[4 * i + 2 * u] + bia, m, add) >> sh;
+                    v[4 * i + 2 * u + 1] = mad_hi(v[4 * i + 2 * u + 1] + bia, m, add) >> sh;
+                  }
+                } else {
+                  const long long c64 = (long long)bia * m + (1ll << (sft - 1));
+#pragma unroll
+                  for (int i = 0; i < 4; ++i) {
+                    v[4 * i + 2 * u] = (int)(mad_wide(v[4 * i + 2 * u], m, c64) >> sft);
+                    v[4 * i + 2 * u + 1] = (int)(mad_wide(v[4 * i + 2 * u + 1], m, c64) >> sft);
+                  }
+                }
+              }
+              if (tma_res) {
+                // residual bytes [row][32 channels]: rows 8 i + 2 (l & 3) + {0, 1}, channels 16 h + (l >> 2) + {0, 8}
+                const uint8_t* rt = res_slot + 16 * h;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  v[4 * i] += (int)res_tab0[(int)*reinterpret_cast<const int8_t*>(rt + i * 256)];
+                  v[4 * i + 1] += (int)res_tab0[(int)*reinterpret_cast<const int8_t*>(rt + i * 256 + 32)];
+                  v[4 * i + 2] += (int)res_tab0[(int)*reinterpret_cast<const int8_t*>(rt + i * 256 + 8)];
+                  v[4 * i + 3] += (int)res_tab0[(int)*reinterpret_cast<const int8_t*>(rt + i * 256 + 40)];
+                }
+              }
+              if (act) {
+#pragma unroll
+                for (int j = 0; j < 16; ++j) v[j] = (int)act_tab0[max(-128, min(127, v[j]))];
+              }
+              uint32_t w[4];
+#pragma unroll
+              for (int i = 0; i < 4; ++i) w[i] = pack_sat8(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+              stmatrix_x4_trans_b8(out_slot + 16u * (uint32_t)h, w[0], w[1], w[2], w[3]);
+            }
+          } else {
+            int v[16];
+            tmem_ld16(t_row + (uint32_t)(32 * ck), v);
+            half(v, ck, 0, pe);
+            tmem_ld16(t_row + (uint32_t)(32 * ck + 16), v);
+            half(v, ck, 1, pe);
+          }
           if (tma_out) {
             fence_async_smem();
             __syncwarp();

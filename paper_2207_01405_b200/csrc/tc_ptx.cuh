@@ -242,6 +242,27 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const int (&v)[16]) {
       :: "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(taddr) : "memory");
 }
+// Accumulator-fragment load: 16 TMEM lanes x 32 columns per warp.  Thread l receives, for i = 0..3,
+//   v[4i], v[4i+1] = lane (l >> 2),     columns 8i + 2 (l & 3), + 1
+//   v[4i+2], v[4i+3] = lane (l >> 2) + 8, the same two columns
+// (lanes counted from the lane field of taddr, which may be the warp's quarter or its upper half).  Packed four to
+// a word this is the fragment that stmatrix_x4_trans_b8 stores transposed.
+__device__ __forceinline__ void tmem_ld_frag16(uint32_t taddr, int (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];\n\t"
+      "tcgen05.wait::ld.sync.aligned;"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr) : "memory");
+}
+// Four 16 x 8 byte matrices, stored transposed: matrix i (word w_i of every thread, bytes = the fragment above) becomes
+// 8 rows of 16 bytes; row r of matrix i goes to the shared-memory address that lane 8 i + r passes in `row_addr`
+// (16-byte aligned).  Byte c of such a row comes from thread 4 (c & 7) + (r >> 1), byte (r & 1) + 2 (c >> 3).
+__device__ __forceinline__ void stmatrix_x4_trans_b8(uint32_t row_addr, uint32_t w0, uint32_t w1, uint32_t w2, uint32_t w3) {
+  asm volatile("stmatrix.sync.aligned.m16n8.x4.trans.shared.b8 [%0], {%1, %2, %3, %4};"
+               ::"r"(row_addr), "r"(w0), "r"(w1), "r"(w2), "r"(w3) : "memory");
+}
 __device__ __forceinline__ void tmem_st4(uint32_t taddr, const uint32_t (&v)[4]) {
   asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%4], {%0, %1, %2, %3};"
                :: "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(taddr) : "memory");
