@@ -627,10 +627,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
             // stores transposed, i.e. as rows of 16 consecutive channels, into the [32 rows][32 channels] slot
             const uint32_t out_slot = my_out + 1024u * (g & 1u) + (uint32_t)lane * 32u;
             const uint8_t* res_slot = gen_base + (my_res - base) + (g & 1u) * 1024 + (2 * (lane & 3)) * 32 + (lane >> 2);
+            // both halves are requested before the arithmetic on the first begins
+            int vv[32];
+            tmem_ld_frag16_issue<0>(t_row + (uint32_t)(32 * ck), vv);
+            tmem_ld_frag16_issue<16>(t_row + (16u << 16) + (uint32_t)(32 * ck), vv);
+            tmem_ld_wait(vv);
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-              int v[16];
-              tmem_ld_frag16(t_row + ((uint32_t)(16 * h) << 16) + (uint32_t)(32 * ck), v);
+              int (&v)[16] = *reinterpret_cast<int (*)[16]>(&vv[16 * h]);
 #pragma unroll
               for (int u = 0; u < 2; ++u) {       // u = 0: channel (l >> 2) + 16 h, u = 1: eight channels on
                 const int m = km[2 * h + u], sft = ks[2 * h + u], bia = kb[2 * h + u];

@@ -256,6 +256,16 @@ __device__ __forceinline__ void tmem_ld_frag16(uint32_t taddr, int (&v)[16]) {
         "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
       : "r"(taddr) : "memory");
 }
+// The same load without the wait: into v[O .. O + 15]; valid after tmem_ld_wait(v).
+template <int O>
+__device__ __forceinline__ void tmem_ld_frag16_issue(uint32_t taddr, int (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.16x256b.x4.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(v[O + 0]), "=r"(v[O + 1]), "=r"(v[O + 2]), "=r"(v[O + 3]), "=r"(v[O + 4]), "=r"(v[O + 5]), "=r"(v[O + 6]), "=r"(v[O + 7]),
+        "=r"(v[O + 8]), "=r"(v[O + 9]), "=r"(v[O + 10]), "=r"(v[O + 11]), "=r"(v[O + 12]), "=r"(v[O + 13]), "=r"(v[O + 14]), "=r"(v[O + 15])
+      : "r"(taddr) : "memory");
+}
 // Four 16 x 8 byte matrices, stored transposed: matrix i (word w_i of every thread, bytes = the fragment above) becomes
 // 8 rows of 16 bytes; row r of matrix i goes to the shared-memory address that lane 8 i + r passes in `row_addr`
 // (16-byte aligned).  Byte c of such a row comes from thread 4 (c & 7) + (r >> 1), byte (r & 1) + 2 (c >> 3).
