@@ -243,7 +243,9 @@ int launch_layernorm(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, 
   const int8_t* x = (const int8_t*)in;
   const int wpl = (int)((C / 4 + 31) / 32);
   if (wpl <= 8) {
-    const int rpw = wpl <= 4 ? 8 : 4, tb = 128;
+    // four rows per warp (eight for rows of at most 128 channels, two above 512): short per-warp work lets the blocks of this
+    // kernel slip into the tail of the kernel before it and out of the way of the one after it
+    const int rpw = wpl <= 1 ? 8 : (wpl <= 4 ? 4 : 2), tb = 128;
     const int64_t warps = (rows + rpw - 1) / rpw;
     const int64_t wantb = (warps + tb / 32 - 1) / (tb / 32);
     const int gridb = (int)(wantb < (int64_t)ctx->sm_count * 12 ? wantb : (int64_t)ctx->sm_count * 12);
@@ -252,11 +254,11 @@ int launch_layernorm(ivit_ctx* ctx, const void* in, int in_dtype, int64_t ldin, 
                     !(reinterpret_cast<uintptr_t>(beta) & 15);
     const size_t cbytes = (size_t)(C / 4) * 3 * sizeof(int4);
     if (wpl <= 1) launch_k(layernorm_rows_kernel<1, 8>, dim3(gridb), dim3(tb), cbytes, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
-    else if (wpl <= 2) launch_k(layernorm_rows_kernel<2, 8>, dim3(gridb), dim3(tb), cbytes, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
-    else if (wpl <= 3) launch_k(layernorm_rows_kernel<3, 8>, dim3(gridb), dim3(tb), cbytes, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
-    else if (wpl <= 4) launch_k(layernorm_rows_kernel<4, 8>, dim3(gridb), dim3(tb), cbytes, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
-    else if (wpl <= 6) launch_k(layernorm_rows_kernel<6, 4>, dim3(gridb), dim3(tb), cbytes, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
-    else launch_k(layernorm_rows_kernel<8, 4>, dim3(gridb), dim3(tb), cbytes, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
+    else if (wpl <= 2) launch_k(layernorm_rows_kernel<2, 4>, dim3(gridb), dim3(tb), cbytes, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
+    else if (wpl <= 3) launch_k(layernorm_rows_kernel<3, 4>, dim3(gridb), dim3(tb), cbytes, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
+    else if (wpl <= 4) launch_k(layernorm_rows_kernel<4, 4>, dim3(gridb), dim3(tb), cbytes, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
+    else if (wpl <= 6) launch_k(layernorm_rows_kernel<6, 2>, dim3(gridb), dim3(tb), cbytes, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
+    else launch_k(layernorm_rows_kernel<8, 2>, dim3(gridb), dim3(tb), cbytes, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C, magic, vec);
     return ls.done();
   }
   if (wpl <= 12) launch_k(layernorm_i8_kernel<12>, dim3(grid), dim3(threads), 0, st, x, ldin, gs, beta, M_ln, out, ldout, rows, (int)C);
@@ -719,14 +721,14 @@ static int shiftgelu_rows(ivit_ctx* ctx, const int8_t* in, int64_t ldin, ivit_ex
   int rc = gelu_table(ctx, p, post, &table);
   if (rc) return rc;
   const int wpl = (int)((cols / 16 + 31) / 32);
-  const int rpw = wpl <= 2 ? 4 : (wpl <= 4 ? 2 : 1);            // rows a warp takes at a time
+  const int rpw = wpl <= 1 ? 4 : (wpl == 2 || wpl == 4 ? 2 : 1);            // rows a warp takes at a time
   const int64_t want = ((rows + rpw - 1) / rpw + 7) / 8;
-  const int grid = (int)(want < (int64_t)ctx->sm_count * 8 ? want : (int64_t)ctx->sm_count * 8);
+  const int grid = (int)(want < (int64_t)ctx->sm_count * 12 ? want : (int64_t)ctx->sm_count * 12);
   cudaStream_t st = ctx->stream;
   LaunchScope ls(ctx, KIND_SHIFTGELU, 2.0 * (double)rows * (double)cols);
   if (wpl <= 1) launch_k(shiftgelu_kernel<1, 4>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
-  else if (wpl <= 2) launch_k(shiftgelu_kernel<2, 4>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
-  else if (wpl <= 3) launch_k(shiftgelu_kernel<3, 2>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
+  else if (wpl <= 2) launch_k(shiftgelu_kernel<2, 2>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
+  else if (wpl <= 3) launch_k(shiftgelu_kernel<3, 1>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
   else if (wpl <= 4) launch_k(shiftgelu_kernel<4, 2>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
   else if (wpl <= 6) launch_k(shiftgelu_kernel<6, 1>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
   else if (wpl <= 8) launch_k(shiftgelu_kernel<8, 1>, dim3(grid), dim3(256), 0, st, in, ldin, table, out, ldout, rows, (int)cols, fixed_max);
