@@ -87,7 +87,9 @@ struct TcArgs {
   int64_t sCo, sCi;
   int batches_inner;
   int total_tiles;
-  int tiles_each, tiles_extra;   // every CTA walks tiles_each tiles, the first tiles_extra CTAs one more
+  int tiles_each, tiles_extra;   // every CTA walks tiles_each tiles, tiles_extra CTAs one more: the first ones, or
+  int long_last;                 // (long_last) the last ones, when the short tiles of a ragged last row block, which
+                                 // end the tile order, can make up for the extra tile
   int tiles_p, tiles_q;
   int BN;            // columns of the tile (multiple of 32, <= 256)
   int stages;
@@ -188,8 +190,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   // this CTA's contiguous range of tiles
-  const int t_begin = (int)blockIdx.x * a.tiles_each + min((int)blockIdx.x, a.tiles_extra);
-  const int t_end = t_begin + a.tiles_each + ((int)blockIdx.x < a.tiles_extra ? 1 : 0);
+  const int first_long = a.long_last ? (int)gridDim.x - a.tiles_extra : 0;   // first CTA with one tile more
+  const int n_long = (int)blockIdx.x - first_long;                            // long CTAs before this one
+  const int t_begin = (int)blockIdx.x * a.tiles_each + min(max(n_long, 0), a.tiles_extra);
+  const int t_end = t_begin + a.tiles_each + ((n_long >= 0 && n_long < a.tiles_extra) ? 1 : 0);
 
   // set-up, spread over the epilogue threads: one barrier (or descriptor prefetch) each
   {
@@ -871,13 +875,19 @@ static_assert(8 * (2 * kMaxStages + 5 + 2 * kEpiWarps) + 32 + 512 <= 1024, "barr
 // an SM's shared memory, and its epilogue, which grows with the tile's width now that chunks are dealt to the
 // epilogue parts across tiles, plus a fixed cost per tile.  The constants are fitted to measured launch times of the
 // DeiT-S / ViT-B / ViT-L layer shapes at widths 128 ... 256 (the pick is within 4 % of the best width on each).
-int pick_bn(int64_t extent, int64_t tiles_other, int64_t K, int sm_count) {
+int pick_bn(int64_t extent, int64_t tiles_other, int64_t K, int sm_count, bool single_batch) {
   if (extent <= 256) return (int)((extent + 31) / 32 * 32);
   int best = 0;
   double best_cost = 0;
   for (int bn : {256, 224, 192, 160, 128}) {
     const int64_t tiles = tiles_other * ((extent + bn - 1) / bn);
-    const double rounds = (double)((tiles + sm_count - 1) / sm_count);
+    double rounds = (double)((tiles + sm_count - 1) / sm_count);
+    // a ragged last block of at most half a tile: if every CTA that needs an extra tile gets one of its short tiles
+    // (long_last in the launcher), the extra tile costs about half a round
+    const int64_t ragged = extent % bn, extra = tiles % sm_count, each = tiles / sm_count;
+    // (only from two full rounds on: measured inside an encoder block, a launch of one round and a half
+    // of wide tiles loses to two rounds of narrow ones although it wins when timed alone)
+    if (single_batch && each >= 2 && ragged != 0 && ragged <= bn / 2 && extra != 0 && (extra - 1) * (each + 1) < tiles_other) rounds -= 0.5;
     const double feed = (double)K * (128.0 + bn) / 60.0;
     const double epilogue = 8.0 * bn;
     // ties go to the narrower tile (its MMAs, loads and stores are shorter): the loop runs from wide to narrow
@@ -922,7 +932,7 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
     a.lanes_are_channels = 1;
     a.P = (int)g.N; a.Q = (int)g.M;
     a.tiles_p = (int)((a.P + BM - 1) / BM);
-    a.BN = pick_bn(a.Q, a.tiles_p, g.K, ctx->sm_count);
+    a.BN = pick_bn(a.Q, a.tiles_p, g.K, ctx->sm_count, batches == 1);
     a.q_stage_bytes = a.BN * BK;
     if (!make_tensor_map(ctx, &tmP, g.B, g.K, g.N, 1, 1, g.ldb, 0, 0, BK, BM, CU_TENSOR_MAP_SWIZZLE_128B, a.p_pos) ||
         !make_tensor_map(ctx, &tmQ, g.A, g.K, g.M, 1, 1, g.lda, 0, 0, BK, a.BN, CU_TENSOR_MAP_SWIZZLE_128B, a.q_pos))
@@ -949,7 +959,7 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
                     swz, a.q_pos))
         return IVIT_ERR_UNSUPPORTED;
     } else {
-      a.BN = pick_bn(a.Q, (int64_t)a.tiles_p * batches, g.K, ctx->sm_count);
+      a.BN = pick_bn(a.Q, (int64_t)a.tiles_p * batches, g.K, ctx->sm_count, false);
       a.q_stage_bytes = a.BN * BK;
       if (!make_tensor_map(ctx, &tmQ, g.B, g.K, g.N, g.batches_inner, g.batches_outer, g.ldb, g.sBi, g.sBo, BK, a.BN,
                     CU_TENSOR_MAP_SWIZZLE_128B, a.q_pos))
@@ -1003,6 +1013,9 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
   const unsigned grid = (unsigned)(a.total_tiles < ctx->sm_count ? a.total_tiles : ctx->sm_count);
   a.tiles_each = a.total_tiles / (int)grid;
   a.tiles_extra = a.total_tiles % (int)grid;
+  // ... which needs a short tile in the range of every long CTA
+  a.long_last = (a.Q % a.BN != 0 && a.Q % a.BN <= a.BN / 2 && batches == 1 && a.tiles_extra > 0 &&
+                 (int64_t)(a.tiles_extra - 1) * (a.tiles_each + 1) < a.tiles_p) ? 1 : 0;
   LaunchScope ls(ctx, KIND_GEMM_TC, 2.0 * (double)batches * (double)g.M * (double)g.N * (double)g.K);
   // the encoder block's Dense layers take the specialised instantiations
   int mode = (a.lanes_are_channels && a.tma_out && (!e.res || a.tma_res)) ? (a.tma_res ? 2 : 1) : 0;
