@@ -47,6 +47,7 @@ struct ivit_ctx {
   int gemm_engine;
   int sm_count;
   void* tmap_encode;  // cuTensorMapEncodeTiled, resolved at context creation
+  void* tmap_cache;   // encoded tensor maps by (address, extents, strides, box, swizzle); see make_tensor_map
   // ivit_vit_forward_host: input copies run on their own stream into two staging buffers (created on first use)
   cudaStream_t copy_stream;
   cudaEvent_t img_ready[2], img_free[2];
@@ -221,6 +222,7 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g);
 int launch_gemm(ivit_ctx* ctx, const GemmProblem& g);
 // Per-device kernel attributes (shared-memory limits) of the tensor-core kernels, for the current device.
 int gemm_tc_prepare_device();
+void tmap_cache_free(ivit_ctx* ctx);
 int attention_prepare_device();
 // Fused Q K^T -> requant -> Shiftmax -> P V -> requant; IVIT_ERR_UNSUPPORTED when the shape does not qualify.
 int launch_attention_fused(ivit_ctx* ctx, const ivit_block_params* p, const int8_t* QKV, int8_t* O);

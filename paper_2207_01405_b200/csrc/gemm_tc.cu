@@ -27,6 +27,8 @@
 // context's status word, carries on without further waits, drains its outstanding copies, and the
 // CTA frees its tensor memory and returns.
 #include "tc_ptx.cuh"
+#include <cstring>
+#include <new>
 #include "rowops.cuh"
 
 namespace ivit {
@@ -39,6 +41,21 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 // ordered by ascending byte stride (a head inside a token row has a smaller stride than the row);
 // pos[0..2] receive the tensor-map dimension that holds the row, inner-batch and outer-batch
 // coordinate.  Byte strides must be multiples of 16.
+namespace {
+struct TmapKey {
+  const void* ptr;
+  uint64_t dims[4], strides[3];
+  uint32_t box[4];
+  int64_t swz;   // (64 bits: the key has no padding, it is compared bytewise)
+};
+struct TmapSlot {
+  TmapKey key;
+  CUtensorMap map;
+  bool used;
+};
+constexpr int kTmapSlots = 512;
+}  // namespace
+
 bool make_tensor_map(ivit_ctx* ctx, CUtensorMap* map, const int8_t* ptr, int64_t inner, int64_t rows, int64_t bi, int64_t bo,
               int64_t row_stride, int64_t si, int64_t so, int box_inner, int box_rows, CUtensorMapSwizzle swz,
               int pos[3], int box_bo) {
@@ -64,10 +81,40 @@ bool make_tensor_map(ivit_ctx* ctx, CUtensorMap* map, const int8_t* ptr, int64_t
     pos[d[i].which] = i + 1;
   }
   const cuuint32_t estr[4] = {1, 1, 1, 1};
+  // An encoded map depends on nothing but these values: a forward pass asks for the same few dozen maps again and
+  // again, so they are kept (direct-mapped, the newer entry wins a slot).
+  TmapKey key{};
+  key.ptr = ptr;
+  for (int i = 0; i < 4; ++i) { key.dims[i] = dims[i]; key.box[i] = box[i]; }
+  for (int i = 0; i < 3; ++i) key.strides[i] = strides[i];
+  key.swz = (int64_t)swz;
+  if (!ctx->tmap_cache) ctx->tmap_cache = new (std::nothrow) TmapSlot[kTmapSlots]();
+  TmapSlot* slot = nullptr;
+  if (ctx->tmap_cache) {
+    uint64_t h = reinterpret_cast<uintptr_t>(ptr) * 0x9E3779B97F4A7C15ull;
+    h ^= (dims[1] + 31 * dims[2] + 131 * box[1] + 1031 * box[0] + 7 * (uint64_t)swz + 17 * strides[0]) * 0xC2B2AE3D27D4EB4Full;
+    slot = static_cast<TmapSlot*>(ctx->tmap_cache) + (h >> 40) % kTmapSlots;
+    if (slot->used && std::memcmp(&slot->key, &key, sizeof(key)) == 0) {
+      *map = slot->map;
+      return true;
+    }
+  }
   EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(ctx->tmap_encode);
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(ptr), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  if (fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(ptr), dims, strides, box, estr,
+         CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return false;
+  if (slot) {
+    slot->key = key;
+    slot->map = *map;
+    slot->used = true;
+  }
+  return true;
+}
+
+void tmap_cache_free(ivit_ctx* ctx) {
+  delete[] static_cast<TmapSlot*>(ctx->tmap_cache);
+  ctx->tmap_cache = nullptr;
 }
 
 namespace {

@@ -369,6 +369,7 @@ int ivit_ctx_destroy(ivit_ctx* ctx) {
   cudaStreamSynchronize(ctx->stream);
   cudaFree(ctx->gelu_tables);
   cudaFreeHost(ctx->status_host);
+  tmap_cache_free(ctx);
   if (ctx->copy_stream) {
     cudaStreamSynchronize(ctx->copy_stream);
     for (int i = 0; i < 2; ++i) {
