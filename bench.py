@@ -624,14 +624,18 @@ def run_gpu(args):
     dk = by_kind[dom]
     int8_peak = 2.0 * peaks["bf16_tflops_sustained"]      # int8 dense = 2 x bf16 (nominal ratio), sustained: timed inside a long step
     if dom.startswith("gemm") or dom.startswith("attention"):
-        achieved = dk["work"] / (dk["ms"] * 1e-3) / 1e12
-        in_step = dk["work"] / prof_steps / (ms_total / args.steps * 1e-3 * dk["ms"] / total_kernel_ms) / 1e12
+        # Average duration of this kernel's launches INSIDE the timed region: the timed step (CUDA events around the
+        # whole forward) x this kernel's share of the per-launch event times (the share agrees with ncu's launch
+        # list).  `achieved_alone` divides by the per-launch event times themselves: an event pair around every launch
+        # adds a few microseconds and stops the overlap of a kernel's set-up with its predecessor's tail.
+        alone = dk["work"] / (dk["ms"] * 1e-3) / 1e12
+        achieved = dk["work"] / prof_steps / (ms_total / args.steps * 1e-3 * dk["ms"] / total_kernel_ms) / 1e12
         roofline = {"kernel": dom, "bound": "tensor", "achieved": round(achieved, 2), "peak": int8_peak, "unit": "TOP/s",
                     "frac": round(achieved / int8_peak, 4),
                     "traffic": GEMM_DRAM_BYTES_PER_LAUNCH if args.config == CONFIG_INDEX else None,
-                    # the event pair around every launch costs a few microseconds and stops the overlap of one kernel's
-                    # set-up with its predecessor's tail; the same work over (un-bracketed step time x this kernel's share)
-                    "achieved_in_step": round(in_step, 2),
+                    "achieved_alone": round(alone, 2), "frac_alone": round(alone / int8_peak, 4),
+                    "us_per_launch_in_step": round(ms_total / args.steps * 1e3 * dk["ms"] / total_kernel_ms / (dk["launches"] / prof_steps), 2),
+                    "us_per_launch_alone": round(dk["ms"] * 1e3 / dk["launches"], 2),
                     "frac_of_mma_issue_probe": round(achieved / int8_probe, 4),
                     "frac_of_spec_4500": round(achieved / 4500.0, 4),
                     "peak_source": f"2 x {peak_src} sustained bf16 cuBLAS ({peaks['bf16_tflops_sustained']} TFLOP/s)"}
