@@ -91,6 +91,13 @@ typedef struct {
 
 /* ---- context ---- */
 
+/* Dense layers with a long contraction (K >= 1024, output channels a multiple of 256, at least 256 rows, int8 output
+ * in one of the staged forms) run on pairs of CTAs: two SMs share a tile of 256 channels x 256 rows (tcgen05
+ * cta_group::2; a CUDA implementation choice, the paper has no counterpart), each loading its own 128 weight rows and
+ * half of the activation rows.  On by default; results are identical in both modes.  enable: 0 = off, non-zero = on.
+ * Host graphs kept by the context are dropped.  Returns IVIT_OK, or IVIT_ERR_INVALID_ARG for a null context. */
+int ivit_ctx_set_gemm_pairs(ivit_ctx* ctx, int enable);
+
 /* Creates a context on `device` that enqueues on `cuda_stream` (a
  * cudaStream_t; NULL = the legacy default stream).  Fails with IVIT_ERR_CUDA
  * when no usable sm_100 device is present: there is no CPU fallback. */

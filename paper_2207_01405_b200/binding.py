@@ -19,7 +19,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libivit.so")
 
 EXPORTS = [
-    "ivit_ctx_create", "ivit_ctx_destroy", "ivit_swin_workspace_bytes", "ivit_swin_forward", "ivit_swin_host_workspace_bytes", "ivit_swin_forward_host", "ivit_isqrt_range", "ivit_ctx_set_row_fusion", "ivit_probe_int8_mma", "ivit_ctx_table_generation", "ivit_vit_forward_tokens", "ivit_ctx_set_stream", "ivit_ctx_poll_status", "ivit_ctx_launch_count",
+    "ivit_ctx_create", "ivit_ctx_destroy", "ivit_swin_workspace_bytes", "ivit_swin_forward", "ivit_swin_host_workspace_bytes", "ivit_swin_forward_host", "ivit_isqrt_range", "ivit_ctx_set_row_fusion", "ivit_ctx_set_gemm_pairs", "ivit_probe_int8_mma", "ivit_ctx_table_generation", "ivit_vit_forward_tokens", "ivit_ctx_set_stream", "ivit_ctx_poll_status", "ivit_ctx_launch_count",
     "ivit_ctx_set_gemm_engine", "ivit_strerror", "ivit_linear", "ivit_matmul", "ivit_shiftmax", "ivit_shiftgelu",
     "ivit_shiftgelu_static",
     "ivit_shiftmax_direct", "ivit_ctx_set_host_graph", "ivit_ctx_host_graph_count",
@@ -109,6 +109,7 @@ def load_library():
     L.ivit_ctx_launch_count.restype = i64
     L.ivit_ctx_set_gemm_engine.argtypes = [vp, C.c_int]
     L.ivit_ctx_set_row_fusion.argtypes = [vp, C.c_int]
+    L.ivit_ctx_set_gemm_pairs.argtypes = [vp, C.c_int]
     L.ivit_ctx_table_generation.argtypes = [vp]
     L.ivit_ctx_table_generation.restype = C.c_uint64
     L.ivit_ctx_set_host_graph.argtypes = [vp, C.c_int]
@@ -245,6 +246,10 @@ class Context:
 
     def set_gemm_engine(self, engine: int):
         _chk(self.lib.ivit_ctx_set_gemm_engine(self.h, engine), "ivit_ctx_set_gemm_engine")
+
+    def set_gemm_pairs(self, enable: bool):
+        """CTA pairs (cta_group::2) for Dense layers with K >= 1536 and N % 256 == 0."""
+        _chk(self.lib.ivit_ctx_set_gemm_pairs(self.h, 1 if enable else 0), "ivit_ctx_set_gemm_pairs")
 
     def set_row_fusion(self, enable: bool):
         """ivit_ctx_set_row_fusion: LayerNorm / ShiftGELU in the tail of the producing Dense kernel (default) or alone."""

@@ -47,6 +47,7 @@ struct ivit_ctx {
   int gemm_engine;
   int sm_count;
   void* tmap_encode;  // cuTensorMapEncodeTiled, resolved at context creation
+  int gemm_pairs;     // CTA pairs (cta_group::2) for Dense layers with a long contraction (ivit_ctx_set_gemm_pairs)
   void* tmap_cache;   // encoded tensor maps by (address, extents, strides, box, swizzle); see make_tensor_map
   // ivit_vit_forward_host: input copies run on their own stream into two staging buffers (created on first use)
   cudaStream_t copy_stream;
@@ -167,6 +168,27 @@ inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
+// The same for a kernel whose CTAs work in pairs: clusters of two CTAs along x.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k_pair(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                                 Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = 2;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 

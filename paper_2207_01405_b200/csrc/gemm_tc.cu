@@ -148,6 +148,8 @@ struct TcArgs {
   int p_pos[3], q_pos[3];  // tensor-map dimension (1..3) that holds the row / inner-batch / outer-batch coordinate
   int tma_out;       // Dense orientation, int8: the output tile is staged in shared memory and stored by TMA
   int tma_res;       // ... and the residual tile of the same shape is fetched by TMA into shared memory
+  int pair;          // two CTAs (a cluster) per tile of 256 channels: cta_group::2 MMAs, each CTA loads its own 128
+                     // weight rows and half of the activation rows; tiles_p then counts channel PAIRS of tiles
   int q_resident;    // Dense orientation, short K: all k-blocks of the Q (activation row) tile stay in shared
                      // memory while the CTA walks the channel blocks; only weight tiles stream through the ring
   RowOpArgs rop;     // row operator on finished blocks of output rows (Dense orientation, staged int8 output)
@@ -178,9 +180,12 @@ __device__ __forceinline__ TileCoord tile_coord(const TcArgs& a, int t) {
 struct TileIter {
   int p, q, bi, bo;       // block indices
   int batch;
-  __device__ __forceinline__ void init(const TcArgs& a, int t) {
+  int pstep, poff;        // lanes between consecutive p-blocks (two tiles when a CTA pair shares them) and this CTA's offset
+  __device__ __forceinline__ void init(const TcArgs& a, int t, int poff_ = 0) {
     const TileCoord c = tile_coord(a, t);
     p = c.p0 / BM; q = c.q0 / a.BN; bi = c.bi; bo = c.bo; batch = c.batch;
+    pstep = a.pair ? 2 * BM : BM;
+    poff = poff_;
   }
   __device__ __forceinline__ void next(const TcArgs& a) {
     if (++p == a.tiles_p) {
@@ -192,7 +197,7 @@ struct TileIter {
       }
     }
   }
-  __device__ __forceinline__ int p0() const { return p * BM; }
+  __device__ __forceinline__ int p0() const { return p * pstep + poff; }
   __device__ __forceinline__ int q0(const TcArgs& a) const { return q * a.BN; }
 };
 
@@ -209,7 +214,7 @@ struct TileIter {
 // row routine each) that are dealt to all epilogue warps of the grid in a fixed order; a warp works on its slices
 // after its CTA's last tile, straight out of L2, waiting (bounded) only for the ready flag of the slice's block.
 // The last CTA to finish leaves counters and flags at zero for the next launch.
-template <int MODE, int ROP>
+template <int MODE, int ROP, bool PAIR = false>
 __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_constant__ CUtensorMap tmP,
                                                               const __grid_constant__ CUtensorMap tmQ,
                                                               const __grid_constant__ CUtensorMap tmO,
@@ -236,10 +241,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
   uint8_t* rop_smem = gen_base + bars_off + 1024;   // ROP == 1: LayerNorm constants; ROP == 2: table rows, per warp
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  // this CTA's contiguous range of tiles
-  const int first_long = a.long_last ? (int)gridDim.x - a.tiles_extra : 0;   // first CTA with one tile more
-  const int n_long = (int)blockIdx.x - first_long;                            // long CTAs before this one
-  const int t_begin = (int)blockIdx.x * a.tiles_each + min(max(n_long, 0), a.tiles_extra);
+  // this CTA's (with PAIR: this CTA pair's) contiguous range of tiles
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;      // PAIR: 0 = the CTA that issues the MMAs of the pair
+  const int poff = (int)rank * BM;                          // this CTA's 128 channels inside the pair's 256
+  const int worker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int workers = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+  const int first_long = a.long_last ? workers - a.tiles_extra : 0;   // first worker with one tile more
+  const int n_long = worker - first_long;                              // long workers before this one
+  const int t_begin = worker * a.tiles_each + min(max(n_long, 0), a.tiles_extra);
   const int t_end = t_begin + a.tiles_each + ((n_long >= 0 && n_long < a.tiles_extra) ? 1 : 0);
 
   // set-up, spread over the epilogue threads: one barrier (or descriptor prefetch) each
@@ -252,7 +261,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     } else if (i < 2 * kMaxStages + 2) {
       mbar_init(accf0 + 8 * (i - 2 * kMaxStages), 1);
     } else if (i < 2 * kMaxStages + 4) {
-      mbar_init(acce0 + 8 * (i - 2 * kMaxStages - 2), kEpiWarps);
+      mbar_init(acce0 + 8 * (i - 2 * kMaxStages - 2), PAIR ? 2 * kEpiWarps : kEpiWarps);   // PAIR: both CTAs' warps
     } else if (i < 2 * kMaxStages + 4 + 2 * kEpiWarps) {
       mbar_init(resf + 8 * (i - 2 * kMaxStages - 4), 1);   // residual slots: 2 per epilogue warp
     } else if (i == 2 * kMaxStages + 4 + 2 * kEpiWarps) {
@@ -274,9 +283,13 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     }
     if (i >= 0 && i < 256 && a.epi.res) res_tab[i] = (int8_t)rq(i - 128, a.epi.res_scale.mult, clamp_shift(a.epi.res_scale.shift));
   }
-  if (warp == 1) tmem_alloc(smem_u32(tmem_slot), (uint32_t)a.tmem_cols);
+  if (warp == 1) {
+    if (PAIR) tmem_alloc_pair(smem_u32(tmem_slot), (uint32_t)a.tmem_cols);
+    else tmem_alloc(smem_u32(tmem_slot), (uint32_t)a.tmem_cols);
+  }
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync_all();   // the other CTA's barriers are initialised before anything arrives on them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   // set-up done (barriers, tensor memory, descriptor prefetch): let the next kernel be scheduled, then wait
@@ -303,9 +316,19 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       bool ok = true;
       int pit = 0, qi = 0, cur_q = -1;
       TileIter ti;
-      ti.init(a, t_begin);
+      ti.init(a, t_begin, poff);
       // which tensor-map coordinate (1..3) carries the row / inner batch / outer batch index
       const int pr = a.p_pos[0], pbi = a.p_pos[1], qr = a.q_pos[0], qbi = a.q_pos[1];
+      // PAIR: both CTAs load (their 128 weight rows, their half of the activation rows); the bytes of both are
+      // counted by the stage barrier of CTA rank 0, which alone arms it
+      auto arm = [&](uint32_t bar, uint32_t bytes) {
+        if (!PAIR) mbar_expect_tx(bar, bytes);
+        else if (rank == 0) mbar_expect_tx(bar, 2u * bytes);
+      };
+      auto load = [&](uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3) {
+        if (PAIR) tma_load_4d_pair(dst, map, mapa_rank0(bar), c0, c1, c2, c3);
+        else tma_load_4d(dst, map, bar, c0, c1, c2, c3);
+      };
       // Dense orientation: the P operand is the weight matrix, which no kernel writes.  The weight k-blocks of the
       // first tile are requested before the wait for the previous kernel (whose last CTAs may still be running
       // elsewhere); the activation k-blocks that complete the same stage barriers follow after the wait.
@@ -313,14 +336,14 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       if (a.lanes_are_channels && t_begin < t_end) {
         pre = kblocks < a.stages ? kblocks : a.stages;
         for (int kb = 0; kb < pre; ++kb) {
-          mbar_expect_tx(full0 + 8 * kb, BM * BK + a.q_stage_bytes);
-          tma_load_4d(base + kb * stage_bytes, &tmP, full0 + 8 * kb, kb * BK, pr == 1 ? ti.p0() : 0, pr == 2 ? ti.p0() : 0,
-                      pr == 3 ? ti.p0() : 0);
+          arm(full0 + 8 * kb, BM * BK + a.q_stage_bytes);
+          load(base + kb * stage_bytes, &tmP, full0 + 8 * kb, kb * BK, pr == 1 ? ti.p0() : 0, pr == 2 ? ti.p0() : 0,
+               pr == 3 ? ti.p0() : 0);
         }
       }
       pdl_wait();
       for (int t = t_begin; ok && t < t_end; ++t, ++pit, ti.next(a)) {
-        const int p0 = ti.p0(), q0 = ti.q0(a);
+        const int p0 = ti.p0(), q0 = ti.q0(a) + (PAIR ? (int)rank * (a.BN >> 1) : 0);   // PAIR: this CTA's half of the rows
         const int pc1 = pr == 1 ? p0 : (pbi == 1 ? ti.bi : ti.bo), pc2 = pr == 2 ? p0 : (pbi == 2 ? ti.bi : ti.bo),
                   pc3 = pr == 3 ? p0 : (pbi == 3 ? ti.bi : ti.bo);
         bool bring_q = false;
@@ -336,16 +359,16 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
           if (wrap > 0 && !mbar_wait(empty0 + 8 * s, (wrap & 1) ^ 1, a.status)) { ok = false; break; }
           const uint32_t sp = base + s * stage_bytes, sq = sp + BM * BK;
           const bool early = t == t_begin && kb < pre;   // barrier armed and weights requested before the wait
-          if (!early) mbar_expect_tx(full0 + 8 * s, stage_bytes + (bring_q ? a.q_stage_bytes : 0));
+          if (!early) arm(full0 + 8 * s, stage_bytes + (bring_q ? a.q_stage_bytes : 0));
           if (bring_q)
-            tma_load_4d(qres + kb * a.q_stage_bytes, &tmQ, full0 + 8 * s, kb * BK, qr == 1 ? q0 : 0, qr == 2 ? q0 : 0,
-                        qr == 3 ? q0 : 0);
-          if (!early) tma_load_4d(sp, &tmP, full0 + 8 * s, kb * BK, pc1, pc2, pc3);
+            load(qres + kb * a.q_stage_bytes, &tmQ, full0 + 8 * s, kb * BK, qr == 1 ? q0 : 0, qr == 2 ? q0 : 0,
+                 qr == 3 ? q0 : 0);
+          if (!early) load(sp, &tmP, full0 + 8 * s, kb * BK, pc1, pc2, pc3);
           if (!a.q_resident) {
             const int qrow = a.q_mn ? kb * BK : q0;     // MN-major: rows of the map are k, the inner index is n
             const int qc0 = a.q_mn ? q0 : kb * BK;
-            tma_load_4d(sq, &tmQ, full0 + 8 * s, qc0, qr == 1 ? qrow : (qbi == 1 ? ti.bi : ti.bo),
-                        qr == 2 ? qrow : (qbi == 2 ? ti.bi : ti.bo), qr == 3 ? qrow : (qbi == 3 ? ti.bi : ti.bo));
+            load(sq, &tmQ, full0 + 8 * s, qc0, qr == 1 ? qrow : (qbi == 1 ? ti.bi : ti.bo),
+                 qr == 2 ? qrow : (qbi == 2 ? ti.bi : ti.bo), qr == 3 ? qrow : (qbi == 3 ? ti.bi : ti.bo));
           }
           *issued_slot = ++issued;
           if (++s == a.stages) { s = 0; ++wrap; }
@@ -354,10 +377,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     }
   } else if (warp == 1) {
     // ---------------- MMA issuer ----------------
-    if (lane == 0) {
-      // instruction descriptor: D = S32, A = B = signed 8 bit, A K-major, M = 128, N = BN, no saturation
+    if (lane == 0 && rank == 0) {   // PAIR: CTA rank 0 issues for both CTAs
+      // instruction descriptor: D = S32, A = B = signed 8 bit, A K-major, M = 128 (PAIR: 256 over both CTAs), N = BN,
+      // no saturation
       const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a.q_mn << 16) |
-                             ((uint32_t)(a.BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+                             ((uint32_t)(a.BN >> 3) << 17) | ((uint32_t)((PAIR ? 2 * BM : BM) >> 4) << 24);
       // P descriptors: K-major rows of 128 bytes (128B swizzle, 1024 bytes per 8 rows).  Q: the same,
       // or MN-major rows of q_row_bytes (swizzle = row width, 8 rows per group).  Along K a descriptor
       // advances by 32 bytes (K-major) or 32 rows (MN-major): an add on the low word.
@@ -374,7 +398,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       bool ok = true;
       int cur_q = -1;
       TileIter ti;
-      ti.init(a, t_begin);
+      ti.init(a, t_begin, poff);
       for (int t = t_begin; ok && t < t_end; ++t, ++it) {
         const int buf = it & 1;
         bool last_of_q = false;
@@ -395,20 +419,27 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
           const uint32_t p_lo = p_lo0 + (uint32_t)s * stage16;
           const uint32_t q_lo = a.q_resident ? q_lo0 + (uint32_t)kb * qstage16 : p_lo + ((BM * BK) >> 4);
           if (kb != kblocks - 1 || tail_steps == BK / UMMA_K) {
-            umma_i8_x4(d_tmem, p_lo, p_hi, q_lo, q_hi, idesc, kb != 0, UMMA_K >> 4, q_kstep16);
+            if (PAIR) umma_i8_x4_pair(d_tmem, p_lo, p_hi, q_lo, q_hi, idesc, kb != 0, UMMA_K >> 4, q_kstep16);
+            else umma_i8_x4(d_tmem, p_lo, p_hi, q_lo, q_hi, idesc, kb != 0, UMMA_K >> 4, q_kstep16);
           } else {
             uint32_t pl = p_lo, ql = q_lo;
             for (int k = 0; k < tail_steps; ++k) {
-              umma_i8_lohi(d_tmem, pl, p_hi, ql, q_hi, idesc, (kb | k) != 0);
+              if (PAIR) umma_i8_pair(d_tmem, pl, p_hi, ql, q_hi, idesc, (kb | k) != 0);
+              else umma_i8_lohi(d_tmem, pl, p_hi, ql, q_hi, idesc, (kb | k) != 0);
               pl += UMMA_K >> 4;
               ql += q_kstep16;
             }
           }
-          umma_commit(empty0 + 8 * s);   // the stage may be refilled once these MMAs have read it
+          // the stage may be refilled once these MMAs have read it (PAIR: in both CTAs)
+          if (PAIR) umma_commit_pair(empty0 + 8 * s);
+          else umma_commit(empty0 + 8 * s);
           ++consumed;
           if (++s == a.stages) { s = 0; ++wrap; }
         }
-        if (ok) umma_commit(accf0 + 8 * buf);  // accumulator of this tile complete
+        if (ok) {   // accumulator of this tile complete (PAIR: told to the epilogue warps of both CTAs)
+          if (PAIR) umma_commit_pair(accf0 + 8 * buf);
+          else umma_commit(accf0 + 8 * buf);
+        }
         if (ok && last_of_q) umma_commit(qrese);   // the resident tile may be replaced once these MMAs are done
       }
       if (!ok) {
@@ -460,7 +491,7 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
     };
     // the first tile's coordinates, computed once (they cost integer divisions)
     TileIter ti_first;
-    ti_first.init(a, t_begin);
+    ti_first.init(a, t_begin, poff);
     if (dense && t_begin < t_end) fetch_channel(ti_first.p0());
     // MatMul orientation: one per-tensor constant set
     const int um = e.scale.mult, us = clamp_shift(e.scale.shift);
@@ -787,7 +818,10 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
       // this warp has read everything it needs from the buffer: hand it back to the MMA warp
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(acce0 + 8 * buf);
+      if (lane == 0) {
+        if (PAIR) mbar_arrive_cluster(mapa_rank0(acce0 + 8 * buf));   // the issuing CTA waits for both CTAs' warps
+        else mbar_arrive(acce0 + 8 * buf);
+      }
       if (ROP) {
         ++tiles_in_q;
         if (t + 1 >= t_end || ti.q0(a) != tc.q0) {
@@ -882,9 +916,11 @@ __global__ void __launch_bounds__(kThreads, 1) gemm_tc_kernel(const __grid_const
   }
   tc_fence_before();
   __syncthreads();
+  if (PAIR) cluster_sync_all();   // neither CTA leaves (or frees tensor memory) while the other may still use it
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, (uint32_t)a.tmem_cols);
+    if (PAIR) tmem_dealloc_pair(tmem_base, (uint32_t)a.tmem_cols);
+    else tmem_dealloc(tmem_base, (uint32_t)a.tmem_cols);
   }
   if (ROP) {
     // the last CTA to get here finds every other CTA out of the queue: it leaves the queue state at zero
@@ -911,6 +947,7 @@ int pow2_at_least(int v) {
 }
 
 constexpr size_t kSmemBudget = 227 * 1024;
+constexpr int64_t kPairMinK = 1024;   // contraction length from which a CTA pair per tile pays (measured)
 // alignment slack + one KB of barriers, tensor-memory slot, flags and the two 256-entry tables of the residual /
 // activation port; a row operator's shared memory follows it
 constexpr size_t kSmemFixed = 1024 + 1024;
@@ -954,7 +991,9 @@ int gemm_tc_prepare_device() {
       cudaFuncSetAttribute(gemm_tc_kernel<3, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
       cudaFuncSetAttribute(gemm_tc_kernel<1, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
       cudaFuncSetAttribute(gemm_tc_kernel<2, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
-      cudaFuncSetAttribute(gemm_tc_kernel<1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess)
+      cudaFuncSetAttribute(gemm_tc_kernel<1, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
+      cudaFuncSetAttribute(gemm_tc_kernel<1, 0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess ||
+      cudaFuncSetAttribute(gemm_tc_kernel<2, 0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget) != cudaSuccess)
     return IVIT_ERR_CUDA;
   return IVIT_OK;
 }
@@ -979,10 +1018,24 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
     a.lanes_are_channels = 1;
     a.P = (int)g.N; a.Q = (int)g.M;
     a.tiles_p = (int)((a.P + BM - 1) / BM);
-    a.BN = pick_bn(a.Q, a.tiles_p, g.K, ctx->sm_count, batches == 1);
-    a.q_stage_bytes = a.BN * BK;
+    // Long contractions are bound by the operand feed from L2 and by the issuing thread's loop: a pair of CTAs per
+    // tile of 256 channels (cta_group::2) halves the activation bytes per SM and the MMAs issued per SM.  Taken
+    // when the layer has whole pairs of channel tiles and the epilogue is one of the specialised forms.
+    a.pair = (ctx->gemm_pairs && g.K >= kPairMinK && g.N % (2 * BM) == 0 && ctx->sm_count % 2 == 0 && g.M >= 256 &&
+              e.out_dtype == IVIT_I8 && e.group_rows <= 0 && !(reinterpret_cast<uintptr_t>(e.out) & 15) && e.ldo % 16 == 0 &&
+              (!e.res || (e.res_rows >= g.M && !(reinterpret_cast<uintptr_t>(e.res) & 15) && e.ldres % 16 == 0)) &&
+              !e.act_table && !(e.rop.kind && ctx->row_fusion)) ? 1 : 0;
+    if (a.pair) {
+      a.tiles_p = (int)(g.N / (2 * BM));   // pairs of channel tiles
+      a.BN = 256;
+      a.q_stage_bytes = (a.BN / 2) * BK;   // every CTA of a pair loads half of the activation rows
+    } else {
+      a.BN = pick_bn(a.Q, a.tiles_p, g.K, ctx->sm_count, batches == 1);
+      a.q_stage_bytes = a.BN * BK;
+    }
     if (!make_tensor_map(ctx, &tmP, g.B, g.K, g.N, 1, 1, g.ldb, 0, 0, BK, BM, CU_TENSOR_MAP_SWIZZLE_128B, a.p_pos) ||
-        !make_tensor_map(ctx, &tmQ, g.A, g.K, g.M, 1, 1, g.lda, 0, 0, BK, a.BN, CU_TENSOR_MAP_SWIZZLE_128B, a.q_pos))
+        !make_tensor_map(ctx, &tmQ, g.A, g.K, g.M, 1, 1, g.lda, 0, 0, BK, a.pair ? a.BN / 2 : a.BN, CU_TENSOR_MAP_SWIZZLE_128B,
+                         a.q_pos))
       return IVIT_ERR_UNSUPPORTED;
   } else {
     // MatMul orientation: lanes = rows of A; the epilogue's 16-byte stores need aligned output rows
@@ -1044,7 +1097,7 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
   // short K: keep the activation tile resident if that still leaves four weight stages
   const size_t kblocks = (size_t)((g.K + BK - 1) / BK);
   const size_t qres_bytes = kblocks * a.q_stage_bytes;
-  a.q_resident = (dense && kSmemFixed + rop_bytes + out_stage + qres_bytes + 4 * (size_t)BM * BK <= kSmemBudget) ? 1 : 0;
+  a.q_resident = (dense && !a.pair && kSmemFixed + rop_bytes + out_stage + qres_bytes + 4 * (size_t)BM * BK <= kSmemBudget) ? 1 : 0;
   const size_t stage = (size_t)BM * BK + (a.q_resident ? 0 : a.q_stage_bytes);
   const size_t fixed = out_stage + (a.q_resident ? qres_bytes : 0);
   int stages = (int)((kSmemBudget - kSmemFixed - rop_bytes - fixed) / stage);
@@ -1057,9 +1110,11 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
   a.total_tiles = (int)total_tiles;
 
   const size_t smem = kSmemFixed + rop_bytes + (size_t)a.stages * stage + fixed;
-  const unsigned grid = (unsigned)(a.total_tiles < ctx->sm_count ? a.total_tiles : ctx->sm_count);
-  a.tiles_each = a.total_tiles / (int)grid;
-  a.tiles_extra = a.total_tiles % (int)grid;
+  const int workers_max = a.pair ? ctx->sm_count / 2 : ctx->sm_count;   // CTAs, or CTA pairs
+  const int workers = a.total_tiles < workers_max ? a.total_tiles : workers_max;
+  const unsigned grid = (unsigned)(a.pair ? 2 * workers : workers);
+  a.tiles_each = a.total_tiles / workers;
+  a.tiles_extra = a.total_tiles % workers;
   // ... which needs a short tile in the range of every long CTA
   a.long_last = (a.Q % a.BN != 0 && a.Q % a.BN <= a.BN / 2 && batches == 1 && a.tiles_extra > 0 &&
                  (int64_t)(a.tiles_extra - 1) * (a.tiles_each + 1) < a.tiles_p) ? 1 : 0;
@@ -1067,7 +1122,10 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
   // the encoder block's Dense layers take the specialised instantiations
   int mode = (a.lanes_are_channels && a.tma_out && (!e.res || a.tma_res)) ? (a.tma_res ? 2 : 1) : 0;
   if (e.act_table) mode = mode == 1 ? 3 : 0;
-  if (rop == 1 && mode == 2) launch_k(gemm_tc_kernel<2, 1>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
+  if (a.pair && (mode != 1 && mode != 2)) return IVIT_ERR_UNSUPPORTED;   // (the conditions above imply mode 1 or 2)
+  if (a.pair && mode == 2) launch_k_pair(gemm_tc_kernel<2, 0, true>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
+  else if (a.pair) launch_k_pair(gemm_tc_kernel<1, 0, true>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
+  else if (rop == 1 && mode == 2) launch_k(gemm_tc_kernel<2, 1>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
   else if (rop == 1 && mode == 1) launch_k(gemm_tc_kernel<1, 1>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
   else if (rop == 2 && mode == 1) launch_k(gemm_tc_kernel<1, 2>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
   else if (mode == 3) launch_k(gemm_tc_kernel<3, 0>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);

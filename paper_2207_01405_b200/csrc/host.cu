@@ -353,6 +353,7 @@ int ivit_ctx_create(ivit_ctx** out, int device, void* cuda_stream) {
   c->sched_dev = reinterpret_cast<unsigned*>(c->gelu_tables + (size_t)kGeluTableSlots * kGeluTableBytes);
   c->rowblk_dev = c->sched_dev + 32;
   c->row_fusion = 0;
+  c->gemm_pairs = 1;
   *out = c;
   return IVIT_OK;
 }
@@ -419,6 +420,13 @@ int ivit_ctx_set_row_fusion(ivit_ctx* ctx, int enable) {
   if (!ctx) return IVIT_ERR_INVALID_ARG;
   // 1: every row operator; 2: I-LayerNorm only, 4: ShiftGELU only (for measurements)
   ctx->row_fusion = enable == 1 ? 3 : (enable == 2 ? 1 : (enable == 4 ? 2 : 0));
+  for (int i = 0; i < 2; ++i) host_graph_drop(ctx, i);
+  return IVIT_OK;
+}
+
+int ivit_ctx_set_gemm_pairs(ivit_ctx* ctx, int enable) {
+  if (!ctx) return IVIT_ERR_INVALID_ARG;
+  ctx->gemm_pairs = enable ? 1 : 0;
   for (int i = 0; i < 2; ++i) host_graph_drop(ctx, i);
   return IVIT_OK;
 }

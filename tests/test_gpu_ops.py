@@ -99,6 +99,36 @@ def test_linear_residual_full_rows(M, N, K):
     assert c.poll_status() == 0
 
 
+@pytest.mark.parametrize("M,N,K,with_res", [(256, 256, 1024, False), (300, 256, 1536, True), (777, 512, 1600, True),
+                                            (1300, 768, 1024, False), (521, 512, 3072, True)])
+def test_linear_cta_pairs(M, N, K, with_res):
+    """Dense layers with K >= 1024 and N % 256 == 0 on pairs of CTAs (cta_group::2): against the oracle and against
+    the one-CTA form; ragged last row block (the second CTA's half may lie past the last row), contraction tail."""
+    g = _g()
+    c = g.ctx()
+    rng = np.random.default_rng(M * 13 + N * 7 + K)
+    A, W = rand_i8(rng, (M, K)), rand_i8(rng, (N, K))
+    bias = rng.integers(-20000, 20000, N).astype(np.int32)
+    acc_std = np.sqrt(K) * 40 * 40
+    scale = scale_channels(rng.uniform(20, 60, N) / acc_std)
+    res = rand_i8(rng, (M, N)) if with_res else None
+    rs = Scale(*dyadic(0.9))
+    want = O.linear(A, W, bias, scale, res=res, res_scale=rs if with_res else None)
+    try:
+        for pairs in (True, False):
+            c.set_gemm_pairs(pairs)
+            n0 = c.launch_count()
+            got = c.linear(g.dev(A), g.dev(W), torch.from_numpy(bias).cuda(), g.binding.DevScale(scale, "cuda"),
+                           res=None if res is None else g.dev(res),
+                           res_scale=g.binding.DevScale(rs, "cuda") if with_res else None,
+                           out=g.dev(np.full((M, N), 77, np.int8)))
+            g.assert_equal(g.host(got), want, f"linear pairs={pairs}")
+            assert c.launch_count() - n0 == 1
+            assert c.poll_status() == 0
+    finally:
+        c.set_gemm_pairs(True)
+
+
 @pytest.mark.parametrize("M,N,K", [(130, 200, 16), (260, 128, 32)])
 def test_linear_low_shifts(M, N, K):
     """Per-channel shifts of 31 and 32 next to larger ones: the requantisation leaves its high-word form."""
