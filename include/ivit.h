@@ -91,8 +91,8 @@ typedef struct {
 
 /* ---- context ---- */
 
-/* Dense layers with a long contraction (K >= 1024, output channels a multiple of 256, at least 256 rows, int8 output
- * in one of the staged forms) run on pairs of CTAs: two SMs share a tile of 256 channels x 256 rows (tcgen05
+/* Dense layers with a long contraction (K >= 1024, output channels a multiple of 256, enough rows to give every pair of
+ * SMs a tile of 256 x 256, int8 output in one of the staged forms) run on pairs of CTAs: two SMs share a tile of 256 channels x 256 rows (tcgen05
  * cta_group::2; a CUDA implementation choice, the paper has no counterpart), each loading its own 128 weight rows and
  * half of the activation rows.  On by default; results are identical in both modes.  enable: 0 = off, non-zero = on.
  * Host graphs kept by the context are dropped.  Returns IVIT_OK, or IVIT_ERR_INVALID_ARG for a null context. */
@@ -109,6 +109,8 @@ int ivit_ctx_set_stream(ivit_ctx* ctx, void* cuda_stream);
 int ivit_ctx_poll_status(ivit_ctx* ctx);
 /* Number of kernels this context has launched since creation. */
 int64_t ivit_ctx_launch_count(const ivit_ctx* ctx);
+/* How many of those were Dense launches on CTA pairs (ivit_ctx_set_gemm_pairs); 0 for a null context. */
+int64_t ivit_ctx_pair_launch_count(const ivit_ctx* ctx);
 /* ShiftGELU look-up tables (one per parameter set: I0, N, M, k_out, post) are built on first use and cached in
  * the context, 16 sets at a time, the oldest slot being rebuilt for a 17th.  This counter changes whenever a slot
  * is built or rebuilt.  A CUDA graph that the CALLER captured around library calls holds the addresses of the

@@ -19,7 +19,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libivit.so")
 
 EXPORTS = [
-    "ivit_ctx_create", "ivit_ctx_destroy", "ivit_swin_workspace_bytes", "ivit_swin_forward", "ivit_swin_host_workspace_bytes", "ivit_swin_forward_host", "ivit_isqrt_range", "ivit_ctx_set_row_fusion", "ivit_ctx_set_gemm_pairs", "ivit_probe_int8_mma", "ivit_ctx_table_generation", "ivit_vit_forward_tokens", "ivit_ctx_set_stream", "ivit_ctx_poll_status", "ivit_ctx_launch_count",
+    "ivit_ctx_create", "ivit_ctx_destroy", "ivit_swin_workspace_bytes", "ivit_swin_forward", "ivit_swin_host_workspace_bytes", "ivit_swin_forward_host", "ivit_isqrt_range", "ivit_ctx_set_row_fusion", "ivit_ctx_set_gemm_pairs", "ivit_probe_int8_mma", "ivit_ctx_table_generation", "ivit_vit_forward_tokens", "ivit_ctx_set_stream", "ivit_ctx_poll_status", "ivit_ctx_launch_count", "ivit_ctx_pair_launch_count",
     "ivit_ctx_set_gemm_engine", "ivit_strerror", "ivit_linear", "ivit_matmul", "ivit_shiftmax", "ivit_shiftgelu",
     "ivit_shiftgelu_static",
     "ivit_shiftmax_direct", "ivit_ctx_set_host_graph", "ivit_ctx_host_graph_count",
@@ -107,6 +107,8 @@ def load_library():
     L.ivit_ctx_poll_status.argtypes = [vp]
     L.ivit_ctx_launch_count.argtypes = [vp]
     L.ivit_ctx_launch_count.restype = i64
+    L.ivit_ctx_pair_launch_count.argtypes = [vp]
+    L.ivit_ctx_pair_launch_count.restype = i64
     L.ivit_ctx_set_gemm_engine.argtypes = [vp, C.c_int]
     L.ivit_ctx_set_row_fusion.argtypes = [vp, C.c_int]
     L.ivit_ctx_set_gemm_pairs.argtypes = [vp, C.c_int]
@@ -267,6 +269,9 @@ class Context:
 
     def launch_count(self) -> int:
         return int(self.lib.ivit_ctx_launch_count(self.h))
+
+    def pair_launch_count(self) -> int:
+        return int(self.lib.ivit_ctx_pair_launch_count(self.h))
 
     def probe_int8_mma(self, iters: int = 4096):
         """ivit_probe_int8_mma: (milliseconds, int8 operations) of the issue-only tensor-core loop."""

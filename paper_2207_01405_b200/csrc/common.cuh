@@ -44,6 +44,7 @@ struct ivit_ctx {
   int gelu_next;
   uint64_t gelu_gen;    // bumped whenever a table slot is (re)built: graphs that point at the tables check it
   int64_t launches;
+  int64_t pair_launches;   // Dense launches that ran on CTA pairs (ivit_ctx_pair_launch_count)
   int gemm_engine;
   int sm_count;
   void* tmap_encode;  // cuTensorMapEncodeTiled, resolved at context creation

@@ -1021,7 +1021,9 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
     // Long contractions are bound by the operand feed from L2 and by the issuing thread's loop: a pair of CTAs per
     // tile of 256 channels (cta_group::2) halves the activation bytes per SM and the MMAs issued per SM.  Taken
     // when the layer has whole pairs of channel tiles and the epilogue is one of the specialised forms.
-    a.pair = (ctx->gemm_pairs && g.K >= kPairMinK && g.N % (2 * BM) == 0 && ctx->sm_count % 2 == 0 && g.M >= 256 &&
+    a.pair = (ctx->gemm_pairs && g.K >= kPairMinK && g.N % (2 * BM) == 0 && ctx->sm_count % 2 == 0 &&
+              (g.N / (2 * BM)) * ((g.M + 255) / 256) >= ctx->sm_count / 2 &&   // a pair-tile for every pair of SMs
+             
               e.out_dtype == IVIT_I8 && e.group_rows <= 0 && !(reinterpret_cast<uintptr_t>(e.out) & 15) && e.ldo % 16 == 0 &&
               (!e.res || (e.res_rows >= g.M && !(reinterpret_cast<uintptr_t>(e.res) & 15) && e.ldres % 16 == 0)) &&
               !e.act_table && !(e.rop.kind && ctx->row_fusion)) ? 1 : 0;
@@ -1123,6 +1125,7 @@ int launch_gemm_tc(ivit_ctx* ctx, const GemmProblem& g) {
   int mode = (a.lanes_are_channels && a.tma_out && (!e.res || a.tma_res)) ? (a.tma_res ? 2 : 1) : 0;
   if (e.act_table) mode = mode == 1 ? 3 : 0;
   if (a.pair && (mode != 1 && mode != 2)) return IVIT_ERR_UNSUPPORTED;   // (the conditions above imply mode 1 or 2)
+  if (a.pair) ++ctx->pair_launches;
   if (a.pair && mode == 2) launch_k_pair(gemm_tc_kernel<2, 0, true>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
   else if (a.pair) launch_k_pair(gemm_tc_kernel<1, 0, true>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);
   else if (rop == 1 && mode == 2) launch_k(gemm_tc_kernel<2, 1>, dim3(grid), dim3(kThreads), smem, ctx->stream, tmP, tmQ, tmO, tmR, a);

@@ -413,6 +413,7 @@ int ivit_ctx_poll_status(ivit_ctx* ctx) {
 }
 
 int64_t ivit_ctx_launch_count(const ivit_ctx* ctx) { return ctx ? ctx->launches : 0; }
+int64_t ivit_ctx_pair_launch_count(const ivit_ctx* ctx) { return ctx ? ctx->pair_launches : 0; }
 
 uint64_t ivit_ctx_table_generation(const ivit_ctx* ctx) { return ctx ? ctx->gelu_gen : 0; }
 

@@ -99,8 +99,8 @@ def test_linear_residual_full_rows(M, N, K):
     assert c.poll_status() == 0
 
 
-@pytest.mark.parametrize("M,N,K,with_res", [(256, 256, 1024, False), (300, 256, 1536, True), (777, 512, 1600, True),
-                                            (1300, 768, 1024, False), (521, 512, 3072, True)])
+@pytest.mark.parametrize("M,N,K,with_res", [(9500, 512, 1024, False), (19000, 256, 1536, True), (9477, 512, 1600, True),
+                                            (6400, 768, 1024, False), (4800, 1024, 3072, True)])
 def test_linear_cta_pairs(M, N, K, with_res):
     """Dense layers with K >= 1024 and N % 256 == 0 on pairs of CTAs (cta_group::2): against the oracle and against
     the one-CTA form; ragged last row block (the second CTA's half may lie past the last row), contraction tail."""
@@ -117,13 +117,14 @@ def test_linear_cta_pairs(M, N, K, with_res):
     try:
         for pairs in (True, False):
             c.set_gemm_pairs(pairs)
-            n0 = c.launch_count()
+            n0, p0 = c.launch_count(), c.pair_launch_count()
             got = c.linear(g.dev(A), g.dev(W), torch.from_numpy(bias).cuda(), g.binding.DevScale(scale, "cuda"),
                            res=None if res is None else g.dev(res),
                            res_scale=g.binding.DevScale(rs, "cuda") if with_res else None,
                            out=g.dev(np.full((M, N), 77, np.int8)))
             g.assert_equal(g.host(got), want, f"linear pairs={pairs}")
             assert c.launch_count() - n0 == 1
+            assert c.pair_launch_count() - p0 == (1 if pairs else 0)   # the pair form really ran (needs >= 74 pair tiles)
             assert c.poll_status() == 0
     finally:
         c.set_gemm_pairs(True)
