@@ -237,6 +237,13 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
       const bool row_ok = r < a.T && (!kPack || b < a.Btot);
       const bool warp_ok = m0 + qd * 32 - col0 < a.T && (!kPack || b < a.Btot);   // warps whose 32 rows all lie past T only keep the barriers
       const int c_lo = col0 >> 4, c_hi = kPack ? c_lo + (a.R >> 4) : nch;   // this row's 16-column chunks
+      // Plain form: the passes work on the chunks that hold columns; when the last of them holds at most eight, it is
+      // taken as one 8-column piece by the second thread of the row (whose share of full chunks is never the larger
+      // one), and chunks wholly past T only get their zero probabilities written.
+      const int c_real = kPack ? c_hi : (a.T + 15) >> 4;
+      const bool tail8 = !kPack && (a.T & 15) != 0 && (a.T & 15) <= 8;
+      const int c_end = tail8 ? c_real - 1 : c_real;   // chunks worked on sixteen columns at a time
+      const int ct = c_end * 16;                       // first column of the 8-column piece
       const int32_t* brow = a.bias ? a.bias + ((((int64_t)b * a.heads + h) % a.bias_batches) * a.T + (row_ok ? r : 0)) * (int64_t)a.T - col0 : nullptr;
 
       int mx = -128;
@@ -249,7 +256,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
         // code stays within the instruction cache); what a later pass needs of a chunk waits in the chunk's own
         // tensor-memory columns.
 #pragma unroll 1
-        for (int c = c_lo + half; c < c_hi; c += 2) {
+        for (int c = c_lo + half; c < c_end; c += 2) {
           int v[16];
           tmem_ld16(t_row + c * 16, v);
           if (brow) {
@@ -265,7 +272,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
             for (int j = 0; j < 16; ++j) v[j] = (int)(((long long)v[j] * a.qk_m + qk_c) >> a.qk_s);
           }
           // columns past T (only in the last two chunks) never win the maximum and look up a valid table entry
-          if (c >= c_hi - 2) {
+          if (c >= c_end - 2) {
 #pragma unroll
             for (int j = 0; j < 16; ++j)
               if (c * 16 + j - col0 >= a.T) v[j] = -128;
@@ -283,6 +290,24 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
             xs[k] = pack_sat8(v[4 * k], v[4 * k + 1], v[4 * k + 2], v[4 * k + 3]) ^ 0x80808080u;
           tmem_st4(t_row + c * 16, xs);
         }
+        if (tail8 && half == 1) {
+          int v[8];
+          tmem_ld8(t_row + ct, v);
+          if (brow) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              if (ct + j < a.T) v[j] += __ldg(brow + ct + j);
+          }
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            v[j] = qk_hi ? mad_hi(v[j], a.qk_m, qk_rnd) >> qk_sh : (int)(((long long)v[j] * a.qk_m + qk_c) >> a.qk_s);
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            if (ct + j >= a.T) v[j] = -128;
+          mx = max(mx, max(max(max(v[0], v[1]), max(v[2], v[3])), max(max(v[4], v[5]), max(v[6], v[7]))));
+          const uint32_t xs2[2] = {pack_sat8(v[0], v[1], v[2], v[3]) ^ 0x80808080u, pack_sat8(v[4], v[5], v[6], v[7]) ^ 0x80808080u};
+          tmem_st2(t_row + ct, xs2);
+        }
         tmem_st_wait();
         mx = max(-128, min(127, mx));
         part_max[half * 128 + trow] = mx;
@@ -296,7 +321,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
         // entry (I_max - I) of the table = word at tab + 4*(I_max + 128) - 4*(I + 128)
         const uint8_t* tmx = reinterpret_cast<const uint8_t*>(tab) + 4 * (mx + 128);
 #pragma unroll 1
-        for (int c = c_lo + half; c < c_hi; c += 2) {
+        for (int c = c_lo + half; c < c_end; c += 2) {
           int ev[16];
           uint32_t xs[4];
           tmem_ld4(t_row + c * 16, xs);
@@ -307,7 +332,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
             for (int bb = 0; bb < 4; ++bb)
               ev[4 * k + bb] = (int)*reinterpret_cast<const unsigned*>(tmx - 4 * (int)__byte_perm(w, 0, 0x4440 + bb));
           }
-          if (c >= c_hi - 2) {   // columns past T contribute nothing
+          if (c >= c_end - 2) {   // columns past T contribute nothing
 #pragma unroll
             for (int j = 0; j < 16; ++j)
               if (c * 16 + j - col0 >= a.T) ev[j] = 0;
@@ -315,6 +340,22 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
 #pragma unroll
           for (int j = 0; j < 16; ++j) sum += (unsigned)ev[j];
           tmem_st16(t_row + c * 16, ev);
+        }
+        if (tail8 && half == 1) {
+          int ev[8];
+          uint32_t xs2[2];
+          tmem_ld2(t_row + ct, xs2);
+#pragma unroll
+          for (int k = 0; k < 2; ++k)
+#pragma unroll
+            for (int bb = 0; bb < 4; ++bb)
+              ev[4 * k + bb] = (int)*reinterpret_cast<const unsigned*>(tmx - 4 * (int)__byte_perm(xs2[k], 0, 0x4440 + bb));
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            if (ct + j >= a.T) ev[j] = 0;
+            sum += (unsigned)ev[j];
+          }
+          tmem_st8(t_row + ct, ev);
         }
         tmem_st_wait();
         part_sum[half * 128 + trow] = sum;
@@ -325,7 +366,7 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
         // pass C: Eq. (IntDiv) with M = 45 (prob_word)
         const unsigned factor = (unsigned)((1ull << 45) / (unsigned long long)(sum ? sum : 1u));
 #pragma unroll 1
-        for (int c = c_lo + half; c < c_hi; c += 2) {
+        for (int c = c_lo + half; c < c_end; c += 2) {
           int ev[16];
           tmem_ld16(t_row + c * 16, ev);
           uint32_t w[4];
@@ -335,6 +376,21 @@ __global__ void __launch_bounds__(kAttnThreads, 2) attention_kernel(const __grid
           // A operand of P V: row = tile row, k-block = 128 columns, 16-byte pieces XOR (row & 7)
           uint8_t* prow = gen + p_off + (c >> 3) * (128 * 128) + trow * 128;
           *reinterpret_cast<uint4*>(prow + ((((c & 7)) ^ (trow & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+        if (!kPack) {
+          if (tail8 && half == 1) {   // the 8-column piece and eight zeros
+            int ev[8];
+            tmem_ld8(t_row + ct, ev);
+            const uint32_t w0 = prob_word<K8>(factor, ev[0], ev[1], ev[2], ev[3], 14 - a.smax.k_out, (1 << (a.smax.k_out - 1)) - 1);
+            const uint32_t w1 = prob_word<K8>(factor, ev[4], ev[5], ev[6], ev[7], 14 - a.smax.k_out, (1 << (a.smax.k_out - 1)) - 1);
+            uint8_t* prow = gen + p_off + (c_end >> 3) * (128 * 128) + trow * 128;
+            *reinterpret_cast<uint4*>(prow + ((((c_end & 7)) ^ (trow & 7)) << 4)) = make_uint4(w0, w1, 0u, 0u);
+          }
+          // chunks wholly past T: probability 0 (the contraction of P V runs over Npad columns)
+          for (int c = c_real + half; c < nch; c += 2) {
+            uint8_t* prow = gen + p_off + (c >> 3) * (128 * 128) + trow * 128;
+            *reinterpret_cast<uint4*>(prow + ((((c & 7)) ^ (trow & 7)) << 4)) = make_uint4(0u, 0u, 0u, 0u);
+          }
         }
         if (kPack) {   // the other windows' columns of this row: probability 0, so that P V stays inside the window
           for (int c = half; c < nch; c += 2)

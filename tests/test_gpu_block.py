@@ -172,6 +172,30 @@ def test_long_row_attention_bit_exact(B, T, D, heads, bias):
     assert c.poll_status() == 0
 
 
+@pytest.mark.parametrize("bias", [False, True])
+def test_attention_row_lengths_around_chunk_boundaries(bias):
+    """The short-row kernel walks a row of scores in 16-column chunks and takes a remainder of at most eight columns
+    as one 8-column piece: row lengths on both sides of every such boundary, with and without a score bias, and with a
+    narrower Shiftmax output."""
+    import dataclasses
+    from ivit_inputs import ExpParams, Scale
+    g = _g()
+    c = g.ctx()
+    rng = np.random.default_rng(5)
+    for i, T in enumerate([1, 5, 8, 9, 16, 17, 24, 25, 40, 72, 129, 136, 137, 197, 200, 201, 248, 249, 256]):
+        heads, d, B = 2, 32, 3
+        D = heads * d
+        blk = make_block(_Ids(3000 + T), 1, B, T, D, heads, 2 * D, attn_bias_batches=heads if bias else 0)
+        if i % 3 == 2:
+            blk = dataclasses.replace(blk, smax=ExpParams(blk.smax.I0, blk.smax.N, 45, 5),
+                                      pv_scale=Scale(blk.pv_scale.mult, max(31, blk.pv_scale.shift - 3)))
+        dblk = g.binding.DeviceBlock(blk, "cuda")
+        QKV = np.clip(np.rint(rng.standard_normal((B * T, 3 * D)) * 32), -128, 127).astype(np.int8)
+        got = g.host(c.attention(dblk, torch.from_numpy(QKV).cuda()))
+        g.assert_equal(got, O.attention(blk, QKV), f"T={T} bias={bias}")
+    assert c.poll_status() == 0
+
+
 def test_attention_random_shapes():
     """Thirty seeded random attention problems (fused short-row, window-packed and key-block kernels, and the composed
     path for head dimensions the fused kernels do not take): random batch, row length, heads and head dimension, with
