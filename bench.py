@@ -320,7 +320,11 @@ def other_configs(ctx, binding, torch, np, flush, dev):
     ms = time_steps(lambda: binding.swin_forward(ctx, dm, d_img, logits=d_out, workspace=wsw), 20)
     h_img = torch.from_numpy(image).pin_memory()
     h_out = torch.empty((model.B, model.classes), dtype=torch.int32).pin_memory()
+    ctx.set_host_graph(True)   # the host entry replays its own captured graph from the third call on
+    for _ in range(4):
+        binding.swin_forward_host(ctx, dm, h_img, h_out, wsw)
     ms_e2e = time_steps(lambda: binding.swin_forward_host(ctx, dm, h_img, h_out, wsw), 20)
+    ctx.set_host_graph(False)
     torch.cuda.synchronize()
     one, _ = make_config(3, batch=1)
     want = O.swin_forward(one, image[63:])
@@ -329,7 +333,7 @@ def other_configs(ctx, binding, torch, np, flush, dev):
                                "int8_TOPS": round(574.8e9 / (ms * 1e-3) / 1e12, 1), "oracle_check": ok, "image_checked": 63,
                                "e2e": {"images_per_s": round(model.B / (ms_e2e * 1e-3), 1), "ms_per_forward": round(ms_e2e, 4),
                                        "h2d_bytes": int(h_img.numel()), "d2h_bytes": int(h_out.numel() * 4),
-                                       "entry": "ivit_swin_forward_host"}}
+                                       "entry": "ivit_swin_forward_host with ivit_ctx_set_host_graph(1)"}}
     del dm, d_img, wsw
     return out
 

@@ -363,8 +363,8 @@ size_t ivit_swin_host_workspace_bytes(const ivit_swin_params* p);
 int ivit_swin_forward_host(ivit_ctx* ctx, const ivit_swin_params* p, const int8_t* image_host,
                            int32_t* logits_host, void* workspace, size_t workspace_bytes);
 
-/* Graph replay for ivit_vit_forward_host (off by default).  When enabled, the third call in a row that repeats
- * the same model description (every field of p and of its blocks), workspace and stream captures the device part
+/* Graph replay for ivit_vit_forward_host and ivit_swin_forward_host (off by default).  When enabled, the third call in a row that repeats
+ * the same model description (every field of p, of its stages and of its blocks), workspace and stream captures the device part
  * of the forward into a CUDA graph, and later calls launch that graph instead of about a hundred kernels; any
  * change of those arguments, a new stream, or switching the mode off drops the graph.  Needs a stream other than
  * the legacy default stream (with the default stream the kernels keep being launched one by one).  Tensors the

@@ -209,19 +209,11 @@ bool grow(char*& buf, size_t& cap, size_t need) {
 // generation of the context is the one it was captured at (another call that rebuilds a table slot makes the
 // next call fall back to kernels and capture again), and a capture during which a table had to be built is thrown
 // away.  A capture that fails leaves the kernel-by-kernel path in place.
-int forward_or_replay(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* img_dev, int32_t* lg_dev, void* workspace,
-                      size_t inner, int slot) {
-  if (!ctx->host_graph || ctx->profiling || ctx->stream == nullptr)
-    return ivit_vit_forward(ctx, p, img_dev, lg_dev, workspace, inner);
-  const size_t nb = (size_t)p->depth * sizeof(ivit_block_params);
-  const void* tail[4] = {img_dev, lg_dev, workspace, (const void*)ctx->stream};
-  const size_t key_bytes = sizeof(*p) + nb + sizeof(tail) + sizeof(int);
-  if (!grow(ctx->hg_scratch, ctx->hg_scratch_cap, key_bytes)) return IVIT_ERR_CUDA;
-  char* key = ctx->hg_scratch;
-  std::memcpy(key, p, sizeof(*p));
-  std::memcpy(key + sizeof(*p), p->blocks, nb);
-  std::memcpy(key + sizeof(*p) + nb, tail, sizeof(tail));
-  std::memcpy(key + sizeof(*p) + nb + sizeof(tail), &ctx->gemm_engine, sizeof(int));
+// `run` enqueues the forward kernel by kernel; ctx->hg_scratch holds key_bytes bytes that describe the call (model
+// description, buffers, stream, engine).
+template <class Run>
+int replay_or_run(ivit_ctx* ctx, int slot, size_t key_bytes, Run run) {
+  const char* key = ctx->hg_scratch;
   const bool same = ctx->hg_key_bytes[slot] == key_bytes && std::memcmp(ctx->hg_key[slot], key, key_bytes) == 0;
   if (!same) {
     host_graph_drop(ctx, slot);
@@ -229,7 +221,7 @@ int forward_or_replay(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* img
     std::memcpy(ctx->hg_key[slot], key, key_bytes);
     ctx->hg_key_bytes[slot] = key_bytes;
     ctx->hg_seen[slot] = 1;
-    return ivit_vit_forward(ctx, p, img_dev, lg_dev, workspace, inner);
+    return run();
   }
   if (ctx->hg_exec[slot]) {
     if (ctx->hg_gen[slot] == ctx->gelu_gen) {
@@ -241,9 +233,9 @@ int forward_or_replay(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* img
     cudaGraphExecDestroy(ctx->hg_exec[slot]);
     ctx->hg_exec[slot] = nullptr;
     ctx->hg_seen[slot] = 1;
-    return ivit_vit_forward(ctx, p, img_dev, lg_dev, workspace, inner);
+    return run();
   }
-  if (ctx->hg_seen[slot] < 0 || ++ctx->hg_seen[slot] < 3) return ivit_vit_forward(ctx, p, img_dev, lg_dev, workspace, inner);
+  if (ctx->hg_seen[slot] < 0 || ++ctx->hg_seen[slot] < 3) return run();
   const int64_t before = ctx->launches;
   // state of the table cache, put back if the capture is not kept (kernels recorded in a discarded capture never ran)
   GeluKey keys_before[kGeluTableSlots];
@@ -260,9 +252,9 @@ int forward_or_replay(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* img
   if (cudaStreamBeginCapture(ctx->stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
     cudaGetLastError();
     ctx->hg_seen[slot] = -1;
-    return ivit_vit_forward(ctx, p, img_dev, lg_dev, workspace, inner);
+    return run();
   }
-  const int rc = ivit_vit_forward(ctx, p, img_dev, lg_dev, workspace, inner);
+  const int rc = run();
   cudaGraph_t graph = nullptr;
   const cudaError_t end = cudaStreamEndCapture(ctx->stream, &graph);
   cudaGraphExec_t exec = nullptr;
@@ -282,7 +274,55 @@ int forward_or_replay(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* img
   // a model with more parameter sets than table slots rebuilds tables on every call: try again later, not never
   ctx->hg_seen[slot] = tables_stable ? -1 : 1;
   if (rc) return rc;
-  return ivit_vit_forward(ctx, p, img_dev, lg_dev, workspace, inner);   // nothing ran during the discarded capture
+  return run();   // nothing ran during the discarded capture
+}
+
+
+int forward_or_replay(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* img_dev, int32_t* lg_dev, void* workspace,
+                      size_t inner, int slot) {
+  auto run = [&]() { return ivit_vit_forward(ctx, p, img_dev, lg_dev, workspace, inner); };
+  if (!ctx->host_graph || ctx->profiling || ctx->stream == nullptr) return run();
+  const size_t nb = (size_t)p->depth * sizeof(ivit_block_params);
+  const void* tail[4] = {img_dev, lg_dev, workspace, (const void*)ctx->stream};
+  const size_t key_bytes = sizeof(*p) + nb + sizeof(tail) + 2 * sizeof(int);
+  if (!grow(ctx->hg_scratch, ctx->hg_scratch_cap, key_bytes)) return IVIT_ERR_CUDA;
+  char* key = ctx->hg_scratch;
+  std::memcpy(key, p, sizeof(*p));
+  std::memcpy(key + sizeof(*p), p->blocks, nb);
+  std::memcpy(key + sizeof(*p) + nb, tail, sizeof(tail));
+  const int modes[2] = {ctx->gemm_engine, 0};   // second word: which forward (0 = ViT)
+  std::memcpy(key + sizeof(*p) + nb + sizeof(tail), modes, sizeof(modes));
+  return replay_or_run(ctx, slot, key_bytes, run);
+}
+
+// The same for the Swin-shaped forward: the description also covers the stages, their blocks and shift flags.
+int swin_forward_or_replay(ivit_ctx* ctx, const ivit_swin_params* p, const int8_t* img_dev, int32_t* lg_dev, void* workspace,
+                           size_t inner) {
+  auto run = [&]() { return ivit_swin_forward(ctx, p, img_dev, lg_dev, nullptr, workspace, inner); };
+  if (!ctx->host_graph || ctx->profiling || ctx->stream == nullptr) return run();
+  size_t key_bytes = sizeof(*p) + (size_t)p->n_stages * sizeof(ivit_swin_stage);
+  for (int64_t i = 0; i < p->n_stages; ++i)
+    key_bytes += (size_t)p->stages[i].depth * (sizeof(ivit_block_params) + 1);
+  const void* tail[4] = {img_dev, lg_dev, workspace, (const void*)ctx->stream};
+  key_bytes += sizeof(tail) + 2 * sizeof(int);
+  if (!grow(ctx->hg_scratch, ctx->hg_scratch_cap, key_bytes)) return IVIT_ERR_CUDA;
+  char* key = ctx->hg_scratch;
+  size_t off = 0;
+  auto put = [&](const void* src, size_t n) { std::memcpy(key + off, src, n); off += n; };
+  put(p, sizeof(*p));
+  put(p->stages, (size_t)p->n_stages * sizeof(ivit_swin_stage));
+  for (int64_t i = 0; i < p->n_stages; ++i) {
+    const ivit_swin_stage& st = p->stages[i];
+    put(st.blocks, (size_t)st.depth * sizeof(ivit_block_params));
+    for (int64_t b = 0; b < st.depth; ++b) {
+      const uint8_t f = st.shifted ? st.shifted[b] : 0;
+      put(&f, 1);
+    }
+  }
+  put(tail, sizeof(tail));
+  const int modes[2] = {ctx->gemm_engine, 1};   // 1 = Swin-shaped forward
+  put(modes, sizeof(modes));
+  return replay_or_run(ctx, 0, key_bytes, run);
 }
 
 }  // namespace
@@ -864,8 +904,8 @@ int ivit_swin_forward_host(ivit_ctx* ctx, const ivit_swin_params* p, const int8_
     return IVIT_ERR_WORKSPACE;
   char* ws = static_cast<char*>(workspace);
   if (cudaMemcpyAsync(ws + inner, image_host, img_bytes, cudaMemcpyHostToDevice, ctx->stream) != cudaSuccess) return IVIT_ERR_CUDA;
-  if ((rc = ivit_swin_forward(ctx, p, reinterpret_cast<const int8_t*>(ws + inner), reinterpret_cast<int32_t*>(ws + lg_off), nullptr,
-                              workspace, inner))) return rc;
+  if ((rc = swin_forward_or_replay(ctx, p, reinterpret_cast<const int8_t*>(ws + inner), reinterpret_cast<int32_t*>(ws + lg_off),
+                                   workspace, inner))) return rc;
   if (cudaMemcpyAsync(logits_host, ws + lg_off, lg_bytes, cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess) return IVIT_ERR_CUDA;
   return IVIT_OK;
 }

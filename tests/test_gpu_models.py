@@ -164,6 +164,45 @@ def test_host_forward_graph_replay_mode():
 
 
 
+def test_swin_host_forward_graph_replay_mode():
+    """The Swin-shaped host-buffer forward under ivit_ctx_set_host_graph: captured at the third repeat (shifted-window
+    blocks with their row gathers included), replayed afterwards; every call gives the oracle's logits, and far fewer
+    launches reach the stream once it replays."""
+    import gpu_util as g
+    dev = torch.device("cuda", 0)
+    c = g.binding.Context(0)
+    side = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(side):
+        c.set_stream(side)
+        c.set_host_graph(True)
+        model, image = make_config(3, batch=2, shifted=True)
+        dm = g.binding.DeviceSwin(model, dev)
+        ws = dm.host_workspace()
+        rng = np.random.default_rng(19)
+        images = [np.clip(image.astype(np.int32) + rng.integers(-30, 30, image.shape), -128, 127).astype(np.int8)
+                  for _ in range(6)]
+        h_img = [torch.from_numpy(x).pin_memory() for x in images]
+        h_out = [torch.empty((2, model.classes), dtype=torch.int32).pin_memory() for _ in images]
+        counts = []
+        for x, y in zip(h_img, h_out):
+            n0 = c.launch_count()
+            g.binding.swin_forward_host(c, dm, x, y, ws)
+            side.synchronize()
+            counts.append(c.launch_count() - n0)
+        for k, (x, y) in enumerate(zip(images, h_out)):
+            g.assert_equal(y.numpy(), O.swin_forward(model, x), f"call {k}")
+        assert c.host_graph_count() == 1
+        # the launch counter counts the kernels of a replayed graph as well (the first call also builds tables)
+        assert len(set(counts[1:])) == 1 and counts[0] >= counts[1]
+        c.set_host_graph(False)
+        assert c.host_graph_count() == 0
+        y = torch.empty((2, model.classes), dtype=torch.int32).pin_memory()
+        g.binding.swin_forward_host(c, dm, h_img[0], y, ws)
+        side.synchronize()
+        g.assert_equal(y.numpy(), O.swin_forward(model, images[0]), "mode off")
+    assert c.poll_status() == 0
+
+
 def test_host_graph_survives_table_cache_eviction():
     """The graphs of ivit_vit_forward_host point at cached ShiftGELU tables.  Seventeen ivit_shiftgelu calls with
     distinct parameter sets between two forwards rebuild every slot of the 16-entry cache; the next forward must
