@@ -355,8 +355,9 @@ size_t ivit_swin_workspace_bytes(const ivit_swin_params* p);
  * at least ivit_swin_workspace_bytes(p)). */
 int ivit_swin_forward(ivit_ctx* ctx, const ivit_swin_params* p, const int8_t* image, int32_t* logits,
                       int8_t* tokens, void* workspace, size_t workspace_bytes);
-/* The same with HOST buffers: image_host is copied to a staging area of the workspace on the context's stream,
- * the forward runs, the logits are copied back to logits_host; the call only enqueues (synchronise the stream
+/* The same with HOST buffers: image_host is copied to one of two staging areas of the workspace (on a copy stream of
+ * the context, so that the copy overlaps the previous call's compute), the forward runs, the logits are copied back
+ * to logits_host; the call only enqueues (synchronise the stream
  * before reading logits_host; keep both host buffers valid until then; pinned memory makes the copies
  * asynchronous).  workspace must hold ivit_swin_host_workspace_bytes(p). */
 size_t ivit_swin_host_workspace_bytes(const ivit_swin_params* p);

@@ -297,7 +297,7 @@ int forward_or_replay(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* img
 
 // The same for the Swin-shaped forward: the description also covers the stages, their blocks and shift flags.
 int swin_forward_or_replay(ivit_ctx* ctx, const ivit_swin_params* p, const int8_t* img_dev, int32_t* lg_dev, void* workspace,
-                           size_t inner) {
+                           size_t inner, int slot) {
   auto run = [&]() { return ivit_swin_forward(ctx, p, img_dev, lg_dev, nullptr, workspace, inner); };
   if (!ctx->host_graph || ctx->profiling || ctx->stream == nullptr) return run();
   size_t key_bytes = sizeof(*p) + (size_t)p->n_stages * sizeof(ivit_swin_stage);
@@ -322,8 +322,49 @@ int swin_forward_or_replay(ivit_ctx* ctx, const ivit_swin_params* p, const int8_
   put(tail, sizeof(tail));
   const int modes[2] = {ctx->gemm_engine, 1};   // 1 = Swin-shaped forward
   put(modes, sizeof(modes));
-  return replay_or_run(ctx, 0, key_bytes, run);
+  return replay_or_run(ctx, slot, key_bytes, run);
 }
+
+// The host-buffer forwards: [inner workspace | two image staging buffers | logits].  The buffers are used alternately:
+// the copy of this call's image runs on a copy stream of the context while the compute stream still works on the
+// previous call; it only waits for the call before that to have finished with the buffer.  `run(img_dev, lg_dev,
+// slot)` enqueues the device part on the compute stream.
+template <class Run>
+int host_forward(ivit_ctx* ctx, const int8_t* image_host, int32_t* logits_host, size_t img_bytes, size_t lg_bytes,
+                        size_t inner, void* workspace, size_t workspace_bytes, Run run) {
+  const size_t img_slot = align_up(img_bytes, 256);
+  const size_t img_off = inner, lg_off = inner + 2 * img_slot;
+  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < lg_off + align_up(lg_bytes, 256))
+    return IVIT_ERR_WORKSPACE;
+  if (!ctx->copy_stream) {
+    // first use: a stream of its own for the input copies, and the events that order it with the compute stream
+    if (cudaSetDevice(ctx->device) != cudaSuccess ||
+        cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess)
+      return IVIT_ERR_CUDA;
+    for (int i = 0; i < 2; ++i)
+      if (cudaEventCreateWithFlags(&ctx->img_ready[i], cudaEventDisableTiming) != cudaSuccess ||
+          cudaEventCreateWithFlags(&ctx->img_free[i], cudaEventDisableTiming) != cudaSuccess)
+        return IVIT_ERR_CUDA;
+    ctx->host_calls = 0;
+  }
+  const int slot = (int)(ctx->host_calls & 1);
+  char* ws = static_cast<char*>(workspace);
+  char* img_dev = ws + img_off + (size_t)slot * img_slot;
+  if (ctx->host_calls >= 2 && cudaStreamWaitEvent(ctx->copy_stream, ctx->img_free[slot], 0) != cudaSuccess) return IVIT_ERR_CUDA;
+  if (cudaMemcpyAsync(img_dev, image_host, img_bytes, cudaMemcpyHostToDevice, ctx->copy_stream) != cudaSuccess ||
+      cudaEventRecord(ctx->img_ready[slot], ctx->copy_stream) != cudaSuccess ||
+      cudaStreamWaitEvent(ctx->stream, ctx->img_ready[slot], 0) != cudaSuccess)
+    return IVIT_ERR_CUDA;
+  ++ctx->host_calls;
+  const int rc = run(reinterpret_cast<const int8_t*>(img_dev), reinterpret_cast<int32_t*>(ws + lg_off), slot);
+  // recorded even after an error: a later copy into this buffer waits for it
+  if (cudaEventRecord(ctx->img_free[slot], ctx->stream) != cudaSuccess) return IVIT_ERR_CUDA;
+  if (rc) return rc;
+  if (cudaMemcpyAsync(logits_host, ws + lg_off, lg_bytes, cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess)
+    return IVIT_ERR_CUDA;
+  return IVIT_OK;
+}
+
 
 }  // namespace
 
@@ -890,24 +931,19 @@ int ivit_swin_forward(ivit_ctx* ctx, const ivit_swin_params* p, const int8_t* im
 
 size_t ivit_swin_host_workspace_bytes(const ivit_swin_params* p) {
   if (check_swin(p) != IVIT_OK) return 0;
-  return swin_ws(p).total + align_up((size_t)(p->B * 3 * p->img * p->img), 256) + align_up((size_t)(p->B * p->classes) * 4, 256);
+  return swin_ws(p).total + 2 * align_up((size_t)(p->B * 3 * p->img * p->img), 256) + align_up((size_t)(p->B * p->classes) * 4, 256);
 }
 
 int ivit_swin_forward_host(ivit_ctx* ctx, const ivit_swin_params* p, const int8_t* image_host, int32_t* logits_host,
                            void* workspace, size_t workspace_bytes) {
   if (!ctx || !image_host || !logits_host) return IVIT_ERR_INVALID_ARG;
-  int rc = check_swin(p);
+  const int rc = check_swin(p);
   if (rc) return rc;
-  const size_t img_bytes = (size_t)(p->B * 3 * p->img * p->img), lg_bytes = (size_t)(p->B * p->classes) * 4;
-  const size_t inner = swin_ws(p).total, lg_off = inner + align_up(img_bytes, 256);
-  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < lg_off + align_up(lg_bytes, 256))
-    return IVIT_ERR_WORKSPACE;
-  char* ws = static_cast<char*>(workspace);
-  if (cudaMemcpyAsync(ws + inner, image_host, img_bytes, cudaMemcpyHostToDevice, ctx->stream) != cudaSuccess) return IVIT_ERR_CUDA;
-  if ((rc = swin_forward_or_replay(ctx, p, reinterpret_cast<const int8_t*>(ws + inner), reinterpret_cast<int32_t*>(ws + lg_off),
-                                   workspace, inner))) return rc;
-  if (cudaMemcpyAsync(logits_host, ws + lg_off, lg_bytes, cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess) return IVIT_ERR_CUDA;
-  return IVIT_OK;
+  const size_t inner = swin_ws(p).total;
+  return host_forward(ctx, image_host, logits_host, (size_t)(p->B * 3 * p->img * p->img), (size_t)(p->B * p->classes) * 4, inner,
+                      workspace, workspace_bytes, [&](const int8_t* img_dev, int32_t* lg_dev, int slot) {
+                        return swin_forward_or_replay(ctx, p, img_dev, lg_dev, workspace, inner, slot);
+                      });
 }
 
 int ivit_ctx_set_host_graph(ivit_ctx* ctx, int enable) {
@@ -926,43 +962,13 @@ int ivit_ctx_host_graph_count(ivit_ctx* ctx) {
 int ivit_vit_forward_host(ivit_ctx* ctx, const ivit_vit_params* p, const int8_t* image_host,
                           int32_t* logits_host, void* workspace, size_t workspace_bytes) {
   if (!ctx || !image_host || !logits_host) return IVIT_ERR_INVALID_ARG;
-  int rc = check_vit(p);
+  const int rc = check_vit(p);
   if (rc) return rc;
-  const size_t img_bytes = (size_t)(p->B * 3 * p->img * p->img), lg_bytes = (size_t)(p->B * p->classes) * 4;
-  const size_t img_slot = align_up(img_bytes, 256);
-  const size_t inner = vit_ws(p).total, img_off = inner, lg_off = inner + 2 * img_slot;
-  if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255) || workspace_bytes < lg_off + align_up(lg_bytes, 256))
-    return IVIT_ERR_WORKSPACE;
-  if (!ctx->copy_stream) {
-    // first use: a stream of its own for the input copies, and the events that order it with the compute stream
-    if (cudaSetDevice(ctx->device) != cudaSuccess ||
-        cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess)
-      return IVIT_ERR_CUDA;
-    for (int i = 0; i < 2; ++i)
-      if (cudaEventCreateWithFlags(&ctx->img_ready[i], cudaEventDisableTiming) != cudaSuccess ||
-          cudaEventCreateWithFlags(&ctx->img_free[i], cudaEventDisableTiming) != cudaSuccess)
-        return IVIT_ERR_CUDA;
-    ctx->host_calls = 0;
-  }
-  // Two staging buffers used alternately: the copy of this call's image runs on the copy stream while the
-  // compute stream still works on the previous call; it only waits for the call before that to have finished
-  // with the buffer.
-  const int slot = (int)(ctx->host_calls & 1);
-  char* ws = static_cast<char*>(workspace);
-  char* img_dev = ws + img_off + (size_t)slot * img_slot;
-  if (ctx->host_calls >= 2 && cudaStreamWaitEvent(ctx->copy_stream, ctx->img_free[slot], 0) != cudaSuccess) return IVIT_ERR_CUDA;
-  if (cudaMemcpyAsync(img_dev, image_host, img_bytes, cudaMemcpyHostToDevice, ctx->copy_stream) != cudaSuccess ||
-      cudaEventRecord(ctx->img_ready[slot], ctx->copy_stream) != cudaSuccess ||
-      cudaStreamWaitEvent(ctx->stream, ctx->img_ready[slot], 0) != cudaSuccess)
-    return IVIT_ERR_CUDA;
-  ++ctx->host_calls;
-  rc = forward_or_replay(ctx, p, reinterpret_cast<const int8_t*>(img_dev), reinterpret_cast<int32_t*>(ws + lg_off), workspace, inner, slot);
-  // recorded even after an error: a later copy into this buffer waits for it
-  if (cudaEventRecord(ctx->img_free[slot], ctx->stream) != cudaSuccess) return IVIT_ERR_CUDA;
-  if (rc) return rc;
-  if (cudaMemcpyAsync(logits_host, ws + lg_off, lg_bytes, cudaMemcpyDeviceToHost, ctx->stream) != cudaSuccess)
-    return IVIT_ERR_CUDA;
-  return IVIT_OK;
+  const size_t inner = vit_ws(p).total;
+  return host_forward(ctx, image_host, logits_host, (size_t)(p->B * 3 * p->img * p->img), (size_t)(p->B * p->classes) * 4, inner,
+                      workspace, workspace_bytes, [&](const int8_t* img_dev, int32_t* lg_dev, int slot) {
+                        return forward_or_replay(ctx, p, img_dev, lg_dev, workspace, inner, slot);
+                      });
 }
 
 int ivit_ctx_profile_start(ivit_ctx* ctx) {

@@ -191,7 +191,7 @@ def test_swin_host_forward_graph_replay_mode():
             counts.append(c.launch_count() - n0)
         for k, (x, y) in enumerate(zip(images, h_out)):
             g.assert_equal(y.numpy(), O.swin_forward(model, x), f"call {k}")
-        assert c.host_graph_count() == 1
+        assert c.host_graph_count() == 2          # one graph per staging buffer
         # the launch counter counts the kernels of a replayed graph as well (the first call also builds tables)
         assert len(set(counts[1:])) == 1 and counts[0] >= counts[1]
         c.set_host_graph(False)
