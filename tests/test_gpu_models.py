@@ -164,6 +164,36 @@ def test_host_forward_graph_replay_mode():
 
 
 
+def test_cta_pair_launches_inside_a_replayed_graph():
+    """ViT-B shapes at batch 64 (one block): FC2 runs on CTA pairs (a cluster launch).  The host-buffer forward captures
+    it into a CUDA graph at the third call; calls before and after the capture give the oracle's logits."""
+    import gpu_util as g
+    dev = torch.device("cuda", 0)
+    c = g.binding.Context(0)
+    side = torch.cuda.Stream(device=dev)
+    with torch.cuda.stream(side):
+        c.set_stream(side)
+        c.set_host_graph(True)
+        model, image = make_config(2, batch=64, depth=1)
+        dm = g.binding.DeviceVit(model, dev)
+        ws = dm.host_workspace()
+        h_img = torch.from_numpy(image).pin_memory()
+        outs = [torch.empty((64, model.classes), dtype=torch.int32).pin_memory() for _ in range(6)]
+        p0 = c.pair_launch_count()
+        for y in outs[:2]:
+            g.binding.vit_forward_host(c, dm, h_img, y, ws)
+        side.synchronize()
+        assert c.pair_launch_count() - p0 == 2      # one FC2 per forward ran on CTA pairs
+        for y in outs[2:]:
+            g.binding.vit_forward_host(c, dm, h_img, y, ws)
+        side.synchronize()
+        assert c.host_graph_count() == 2
+        want = O.vit_forward(model, image)
+        for k, y in enumerate(outs):
+            g.assert_equal(y.numpy(), want, f"call {k}")
+    assert c.poll_status() == 0
+
+
 def test_swin_host_forward_graph_replay_mode():
     """The Swin-shaped host-buffer forward under ivit_ctx_set_host_graph: captured at the third repeat (shifted-window
     blocks with their row gathers included), replayed afterwards; every call gives the oracle's logits, and far fewer
